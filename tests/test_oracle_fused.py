@@ -1,0 +1,88 @@
+"""Pins for the oracle's fused LM-head variant: logits are the contraction H W^T (the policy head
+behind pi_theta of Sec. 2.2), the loss is the same, gradients follow by the chain rule."""
+import numpy as np
+import torch
+
+from oracle import rlf_oracle as orc
+
+
+def _bf16(x):
+    t = torch.tensor(x, dtype=torch.float32).to(torch.bfloat16)
+    return t.view(torch.int16).numpy().view(np.uint16), t.double().numpy()
+
+
+def _problem(seed, T=10, D=12, V=17, B=3):
+    rng = np.random.default_rng(seed)
+    Hb, H = _bf16(rng.normal(size=(T, D)))
+    Wb, W = _bf16(rng.normal(size=(V, D)) * 0.5)
+    ids = rng.integers(0, V, size=T).astype(np.int32)
+    seq = np.sort(rng.integers(0, B, size=T)).astype(np.int32)
+    adv = rng.normal(size=B).astype(np.float32)
+    mask = (rng.random(T) < 0.7).astype(np.uint8)
+    z = H @ W.T
+    new = orc.grpo_loss(z, ids, seq, adv, np.zeros(T), np.zeros(T), mask, 0.2, 0.0, want_grad=False)["logp"]
+    old = (new + rng.normal(0, 0.3, size=T)).astype(np.float32)
+    ref = (new + rng.normal(0, 0.3, size=T)).astype(np.float32)
+    return Hb, H, Wb, W, ids, seq, adv, old, ref, mask
+
+
+def test_logits_are_the_fp64_contraction_with_untransposed_layouts():
+    Hb, H, Wb, W, ids, seq, adv, old, ref, mask = _problem(0)
+    r = orc.fused_lmhead_grpo(Hb, Wb, ids, seq, adv, old, ref, mask, 0.2, 0.1, want_z=True)
+    assert np.abs(r["z"] - H @ W.T).max() < 1e-13          # numpy matmul: library contraction
+    same = orc.grpo_loss(H @ W.T, ids, seq, adv, old, ref, mask, 0.2, 0.1)
+    assert np.allclose(r["logp"], same["logp"], atol=1e-13) and np.allclose(r["loss"], same["loss"], atol=1e-13)
+    assert np.allclose(r["grad_hidden"], same["grad"] @ W, atol=1e-14)
+    assert np.allclose(r["grad_W"], same["grad"].T @ H, atol=1e-14)
+
+
+def test_gradients_match_torch_autograd_fp64():
+    Hb, H, Wb, W, ids, seq, adv, old, ref, mask = _problem(1)
+    r = orc.fused_lmhead_grpo(Hb, Wb, ids, seq, adv, old, ref, mask, 0.2, 0.05)
+    Ht = torch.tensor(H, requires_grad=True)
+    Wt = torch.tensor(W, requires_grad=True)
+    z = Ht @ Wt.t()
+    logp = torch.log_softmax(z, -1).gather(1, torch.tensor(ids, dtype=torch.int64)[:, None])[:, 0]
+    A = torch.tensor(adv, dtype=torch.float64)[torch.tensor(seq, dtype=torch.int64)]
+    rho = torch.exp(logp - torch.tensor(old, dtype=torch.float64))
+    pg = -torch.minimum(rho * A, torch.clamp(rho, 0.8, 1.2) * A)
+    d = torch.tensor(ref, dtype=torch.float64) - logp
+    m = torch.tensor(mask, dtype=torch.float64)
+    L = (m * (pg + 0.05 * (torch.exp(d) - d - 1))).sum() / m.sum()
+    L.backward()
+    assert abs(r["loss"][0] - L.item()) < 1e-13
+    assert np.abs(r["grad_hidden"] - Ht.grad.numpy()).max() < 1e-14
+    assert np.abs(r["grad_W"] - Wt.grad.numpy()).max() < 1e-14
+
+
+def test_invariants_of_the_head_gradients():
+    Hb, H, Wb, W, ids, seq, adv, old, ref, mask = _problem(2, T=14, D=9, V=21)
+    r = orc.fused_lmhead_grpo(Hb, Wb, ids, seq, adv, old, ref, mask, 0.2, 0.05)
+    # every row of grad_z sums to zero, so the columns of grad_W sum to zero over the vocabulary
+    assert np.abs(r["grad_W"].sum(axis=0)).max() < 1e-14
+    assert (r["grad_hidden"][mask == 0] == 0).all()
+    # grad_hidden[t] = coef_t (E_p[W] - W_y)
+    z = H @ W.T
+    g = orc.grpo_loss(z, ids, seq, adv, old, ref, mask, 0.2, 0.05, want_coef=True)
+    p = np.exp(z - z.max(1, keepdims=True)); p /= p.sum(1, keepdims=True)
+    want = g["coef"][:, None] * (p @ W - W[ids])
+    assert np.allclose(r["grad_hidden"], want, atol=1e-14)
+
+
+def test_finite_differences_through_the_head():
+    """bf16 inputs cannot be perturbed by 1e-6, so the check differentiates the fp64 logits path
+    composed with the contraction: dL/dH[t,k] ~ (L(H + h e_tk) - L(H - h e_tk)) / 2h."""
+    Hb, H, Wb, W, ids, seq, adv, old, ref, mask = _problem(3, T=5, D=4, V=7)
+    r = orc.fused_lmhead_grpo(Hb, Wb, ids, seq, adv, old, ref, mask, 0.2, 0.2)
+
+    def L(Hx, Wx):
+        return orc.grpo_loss(Hx @ Wx.T, ids, seq, adv, old, ref, mask, 0.2, 0.2, want_grad=False)["loss"][0]
+    h = 1e-6
+    for (t, k) in [(0, 0), (1, 3), (4, 2), (2, 1)]:
+        Hp, Hm = H.copy(), H.copy()
+        Hp[t, k] += h; Hm[t, k] -= h
+        assert abs((L(Hp, W) - L(Hm, W)) / (2 * h) - r["grad_hidden"][t, k]) < 1e-8
+    for (v, k) in [(0, 0), (6, 3), (3, 1), (int(ids[0]), 2)]:
+        Wp, Wm = W.copy(), W.copy()
+        Wp[v, k] += h; Wm[v, k] -= h
+        assert abs((L(H, Wp) - L(H, Wm)) / (2 * h) - r["grad_W"][v, k]) < 1e-8
