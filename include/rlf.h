@@ -1,0 +1,213 @@
+/*
+ * rlf.h -- C ABI of the B200 (sm_100a) GRPO policy-update loss path.
+ *
+ * The path, in call order for one training micro-batch of packed multi-turn
+ * tool-use responses:
+ *     rlf_build_loss_mask  ->  rlf_group_advantage  ->
+ *     rlf_grpo_logp_loss_fwd_bwd   (logits materialised by the caller)   or
+ *     rlf_fused_lmhead_grpo        (logits formed on the fly from hidden states)
+ *
+ * Conventions that hold for every entry point unless stated otherwise:
+ *   - Every pointer is DEVICE memory owned by the caller and valid on the
+ *     current device until the work queued on `stream` has finished.  The
+ *     library allocates nothing, keeps no state between calls and never
+ *     synchronises: it validates arguments on the host, queues kernels (and
+ *     small memsets) on `stream`, and returns.
+ *   - `stream` is a CUDA stream handle (cudaStream_t); NULL is the default stream.
+ *   - Host-detectable problems return a negative rlf_status before anything is
+ *     queued.  Problems only visible on the device (a target id outside the
+ *     vocabulary, a malformed cu_seqlens, a non-finite row) OR a bit into
+ *     *dev_status (caller-owned int32 on the device, may be NULL; never
+ *     cleared by the library) and neutralise the offending row: it gets loss
+ *     weight 0 and an all-zero gradient.  Kernels never trap or assert.
+ *   - Row r of logits / hidden predicts token ids[r]; the caller has already
+ *     applied the next-token shift.  Rows [cu_seqlens[b], cu_seqlens[b+1]) belong to response b.
+ *   - There is no CPU fallback: on a device that is not compute capability
+ *     10.x every compute entry point returns RLF_ERR_ARCH.
+ */
+#ifndef RLF_H_
+#define RLF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RLF_OK = 0,
+    RLF_ERR_NULL = -1,      /* a required pointer is NULL */
+    RLF_ERR_SHAPE = -2,     /* a size is negative / zero where it may not be / inconsistent */
+    RLF_ERR_ALIGN = -3,     /* a pointer or stride violates the stated alignment */
+    RLF_ERR_DTYPE = -4,     /* unknown rlf_dtype */
+    RLF_ERR_WORKSPACE = -5, /* workspace NULL, misaligned or smaller than rlf_workspace_bytes() */
+    RLF_ERR_ARCH = -6,      /* current device is not sm_100 */
+    RLF_ERR_CUDA = -7,      /* a CUDA runtime call failed (launch, memset, copy) */
+    RLF_ERR_UNSUPPORTED = -8 /* valid request outside what this build implements */
+} rlf_status;
+
+typedef enum { RLF_BF16 = 0, RLF_F32 = 1 } rlf_dtype;
+
+/* bits OR-ed into *dev_status by kernels */
+#define RLF_DEV_BAD_TARGET 1   /* ids[r] outside [0, V) */
+#define RLF_DEV_BAD_SEQ 2      /* cu_seqlens not monotone / outside [0, T], or seq_id outside [0, B) */
+#define RLF_DEV_NONFINITE 4    /* a row's log-sum-exp or log-prob is not finite */
+#define RLF_DEV_TIMEOUT 8      /* a bounded device-side wait gave up */
+
+/* selectors for rlf_workspace_bytes */
+#define RLF_FN_LOGP_LOSS 3
+#define RLF_FN_FUSED_LMHEAD 4
+
+typedef struct CUstream_st *rlf_stream_t;
+
+/*
+ * Loss mask from observation markers.  (Paper Sec. 2.2: observation tokens are
+ * tool output appended to the trajectory and take no part in the loss; Sec.
+ * 2.3.2: a loss mask is set over tool results.)
+ *
+ * A span runs from a token equal to `open_id` to the next token equal to
+ * `close_id` in the same response, both markers included; every token of a
+ * span gets mask 0, every other token 1.  A close marker outside a span is an
+ * ordinary token, an open marker inside a span changes nothing, a span that is
+ * not closed runs to the end of its response, and the state resets at every
+ * response start.  If `valid` is given the result is AND-ed with valid[t] != 0.
+ *
+ *   ids         [T] int32   target token ids (packed responses)
+ *   cu_seqlens  [B+1] int32 response boundaries, cu_seqlens[0] = 0, cu_seqlens[B] = T
+ *   valid       [T] uint8 or NULL
+ *   mask_out    [T] uint8   written for every t (tokens outside every response get 0)
+ *   seq_id_out  [T] int32 or NULL: response index of each token (-1 outside every response)
+ *   n_out       [1] int64   number of tokens with mask 1 (overwritten)
+ * T = 0 and B = 0 are valid.  A non-monotone or out-of-range cu_seqlens sets RLF_DEV_BAD_SEQ and
+ * the affected response is clipped to [0, T).
+ */
+rlf_status rlf_build_loss_mask(const int32_t *ids, const int32_t *cu_seqlens, int32_t B, int64_t T,
+                               int32_t open_id, int32_t close_id, const uint8_t *valid,
+                               uint8_t *mask_out, int32_t *seq_id_out, int64_t *n_out,
+                               int32_t *dev_status, rlf_stream_t stream);
+
+/*
+ * Group-relative outcome advantage.  (Paper Sec. 2.3.2 / Fig. 4 name GRPO as
+ * the algorithm; the formula is the standard group normalisation.)
+ *     A_i = (r_i - mean_g) / (std_g + eps),  g = group of response i
+ * std_g divides by n-1 if `unbiased_std` else by n; a group with one member or
+ * zero spread gets A = 0.  Sums are accumulated in fp64 in index order.
+ *
+ *   rewards   [B] fp32
+ *   group_id  [B] int32 in [0, g_or_num_groups), or NULL: response i is in group i / g_or_num_groups
+ *   g_or_num_groups  number of groups if group_id is given, else the group size G
+ *   adv_out   [B] fp32
+ * A group_id outside its range sets RLF_DEV_BAD_SEQ and gives that response A = 0.
+ */
+rlf_status rlf_group_advantage(const float *rewards, const int32_t *group_id, int32_t B,
+                               int32_t g_or_num_groups, float eps, int unbiased_std,
+                               float *adv_out, int32_t *dev_status, rlf_stream_t stream);
+
+/*
+ * Fused log-prob + clipped-ratio + k3-KL loss, forward and backward, over
+ * materialised logits.  (Paper Sec. 2.2: the policy pi_theta(a | s_t); Sec.
+ * 2.3.1: PPO-style update of the RL trainer; Sec. 2.3.2: GRPO with the loss
+ * mask.  Formulas are the textbook ones.)  Per row t with y = ids[t]:
+ *     lse = log sum_v exp z[t,v];   logp = z[t,y] - lse
+ *     rho = exp(logp - old_logp[t]);  A = adv[seq_id[t]]
+ *     pg  = -min(rho A, clip(rho, 1-eps_clip, 1+eps_clip) A)
+ *     d   = ref_logp[t] - logp;  kl = exp(d) - d - 1
+ *     N   = *denom if denom != NULL else sum_t mask[t];   Nd = max(N, 1)
+ *     loss_out = { sum mask (pg + beta kl), sum mask pg, sum mask kl, sum mask clipped } / Nd
+ *     grad_logits[t,v] = d loss_out[0] / d z[t,v] = c_t (softmax(z[t,:])[v] - 1[v = y]),
+ *         c_t = -(mask[t]/Nd) (dpg/dlogp + beta (1 - exp d)),
+ *         dpg/dlogp = 0 where the clipped branch is active (A>0, rho>1+eps or A<0, rho<1-eps), else -A rho.
+ * Each logits row is read from HBM once and grad written once; max / sum are
+ * accumulated in fp32, the token-level loss terms are summed in fp64 in a fixed order
+ * (results are run-to-run identical).
+ *
+ *   logits       [T, V] dt, row r starts at element r * row_stride (row_stride >= V)
+ *   ids          [T] int32;  seq_id [T] int32 in [0, B);  adv [B] fp32
+ *   old_logp, ref_logp [T] fp32;  mask [T] uint8
+ *   denom        [1] int64 on the device, or NULL.  Pass the global token count when a batch is
+ *                split over several calls so that the calls' losses and gradients add up.
+ *   logp_out     [T] fp32, written for every row (masked or not)
+ *   loss_out     [4] fp64
+ *   grad_logits  [T, V] dt with the same row_stride, or NULL (forward only).  May be the same
+ *                buffer as logits (in place).  Masked rows are written as zeros.
+ *   workspace    rlf_workspace_bytes(RLF_FN_LOGP_LOSS, T, V, 0, dt) bytes, 256-byte aligned;
+ *                contents need not be initialised and are overwritten.
+ * Fast path: dt = RLF_BF16, V a multiple of 8, row_stride a multiple of 8, both bases 16-byte
+ * aligned.  Anything else (fp32 logits, odd V, unaligned rows) takes a slower general kernel.
+ * T = 0 is valid (loss_out = 0).
+ */
+rlf_status rlf_grpo_logp_loss_fwd_bwd(const void *logits, rlf_dtype dt, int64_t T, int32_t V,
+                                      int64_t row_stride, const int32_t *ids,
+                                      const int32_t *seq_id, const float *adv, int32_t B,
+                                      const float *old_logp, const float *ref_logp,
+                                      const uint8_t *mask, float eps_clip, float beta_kl,
+                                      const int64_t *denom, float *logp_out, double *loss_out,
+                                      void *grad_logits, void *workspace, size_t workspace_bytes,
+                                      int32_t *dev_status, rlf_stream_t stream);
+
+/*
+ * Same loss with the logits formed on the fly, z = hidden W^T, so that they
+ * never reach HBM.  (Paper Sec. 2.2: pi_theta is the language model's output
+ * head; the fusion itself is this library's design.)  Backward recomputes the
+ * logit tiles and returns
+ *     grad_hidden[t,:] = sum_v grad_z[t,v] W[v,:]       (bf16)
+ *     grad_W[v,:]      = sum_t grad_z[t,v] hidden[t,:]  (fp32; added to the buffer if accumulate_grad_W)
+ *
+ *   hidden [T, D] bf16 row-major;  W [V, D] bf16 row-major; both 16-byte aligned, D a multiple of 64
+ *   per-token arguments, denom, logp_out, loss_out: as for rlf_grpo_logp_loss_fwd_bwd
+ *   grad_hidden [T, D] bf16 or NULL;  grad_W [V, D] fp32 or NULL
+ *   workspace   rlf_workspace_bytes(RLF_FN_FUSED_LMHEAD, T, V, D, RLF_BF16) bytes, 256-byte aligned
+ */
+rlf_status rlf_fused_lmhead_grpo(const void *hidden, const void *W, int64_t T, int32_t D, int32_t V,
+                                 const int32_t *ids, const int32_t *seq_id, const float *adv,
+                                 int32_t B, const float *old_logp, const float *ref_logp,
+                                 const uint8_t *mask, float eps_clip, float beta_kl,
+                                 const int64_t *denom, float *logp_out, double *loss_out,
+                                 void *grad_hidden, float *grad_W, int accumulate_grad_W,
+                                 void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                 rlf_stream_t stream);
+
+/* Bytes of workspace the given entry point needs for these sizes (0 for unknown selectors). */
+size_t rlf_workspace_bytes(int which_fn, int64_t T, int32_t V, int32_t D, rlf_dtype dt);
+
+/*
+ * One whole step from HOST buffers: copies the inputs to the device, runs
+ * rlf_build_loss_mask -> rlf_group_advantage -> rlf_grpo_logp_loss_fwd_bwd,
+ * copies loss (and, if asked, logp and mask) back and waits for the stream.
+ * Host pointers should be page-locked for the copies to run at full rate.
+ *
+ *   h_*          host inputs, shapes as for the device entry points (contiguous groups of G)
+ *   h_loss_out   [4] fp64 host;  h_logp_out [T] fp32 host or NULL;  h_mask_out [T] uint8 host or NULL
+ *   d_arena      device scratch of rlf_step_arena_bytes(T, V, B, dt) bytes, 256-byte aligned; on
+ *                return it holds grad_logits in place of the logits at offset 0 (row_stride = V)
+ * Returns RLF_ERR_CUDA if a copy or the final wait fails; *h_dev_status (nullable) gets the device
+ * status word.
+ */
+rlf_status rlf_grpo_step_host(const void *h_logits, rlf_dtype dt, int64_t T, int32_t V,
+                              const int32_t *h_ids, const int32_t *h_cu_seqlens, int32_t B, int32_t G,
+                              const float *h_rewards, const float *h_old_logp,
+                              const float *h_ref_logp, int32_t open_id, int32_t close_id,
+                              float adv_eps, float eps_clip, float beta_kl, double *h_loss_out,
+                              float *h_logp_out, uint8_t *h_mask_out, int32_t *h_dev_status,
+                              void *d_arena, size_t arena_bytes, rlf_stream_t stream);
+size_t rlf_step_arena_bytes(int64_t T, int32_t V, int32_t B, rlf_dtype dt);
+
+/* Launch shape of the fast logits kernel for later calls in this process: CTAs per cluster (1, 2,
+ * 4 or 8), threads per CTA (256, 512 or 1024), and whether each element's exponential is taken once
+ * and kept as bf16 (one_exp = 1) or taken twice in fp32 (one_exp = 0; -1 = built-in choice).
+ * cluster_ctas = 0 restores the built-in shape.  A shape that cannot hold a row in registers makes
+ * rlf_grpo_logp_loss_fwd_bwd return RLF_ERR_UNSUPPORTED.  Results do not depend on the shape
+ * beyond fp32 summation order (and, for one_exp, one extra bf16 rounding of the gradient). */
+rlf_status rlf_tune_logits_kernel(int cluster_ctas, int threads_per_cta, int one_exp);
+
+/* Number of kernels this library has launched in this process (for accounting). */
+int64_t rlf_launch_count(void);
+
+const char *rlf_status_string(rlf_status s);
+int rlf_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RLF_H_ */

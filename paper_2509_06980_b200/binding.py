@@ -1,0 +1,230 @@
+"""Thin ctypes binding of the C-ABI CUDA library (include/rlf.h).
+
+Argument marshalling only: every function takes torch tensors (device memory and
+streams are PyTorch's), checks dtypes / devices, and passes raw pointers to the
+entry point of the same name.  Nothing is computed here and there is no fallback:
+importing this module raises if the library has not been built.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "librlf.so")
+
+RLF_BF16, RLF_F32 = 0, 1
+FN_LOGP_LOSS, FN_FUSED_LMHEAD = 3, 4
+DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
+
+EXPORTS = [
+    "rlf_build_loss_mask", "rlf_group_advantage", "rlf_grpo_logp_loss_fwd_bwd",
+    "rlf_fused_lmhead_grpo", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
+    "rlf_tune_logits_kernel", "rlf_launch_count", "rlf_status_string", "rlf_version",
+]
+
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        "CUDA library %s is missing: build it with `python -m paper_2509_06980_b200.build` "
+        "(there is no CPU fallback)" % _LIB_PATH)
+
+_lib = ctypes.CDLL(_LIB_PATH)
+
+_vp, _i32, _i64, _f32, _sz, _int = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float,
+                                    ctypes.c_size_t, ctypes.c_int)
+_lib.rlf_build_loss_mask.argtypes = [_vp, _vp, _i32, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.rlf_group_advantage.argtypes = [_vp, _vp, _i32, _i32, _f32, _int, _vp, _vp, _vp]
+_lib.rlf_grpo_logp_loss_fwd_bwd.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _i32, _vp, _vp, _vp,
+                                            _f32, _f32, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+_lib.rlf_fused_lmhead_grpo.argtypes = [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _f32,
+                                       _f32, _vp, _vp, _vp, _vp, _vp, _int, _vp, _sz, _vp, _vp]
+_lib.rlf_workspace_bytes.argtypes = [_int, _i64, _i32, _i32, _int]
+_lib.rlf_workspace_bytes.restype = _sz
+_lib.rlf_grpo_step_host.argtypes = [_vp, _int, _i64, _i32, _vp, _vp, _i32, _i32, _vp, _vp, _vp, _i32, _i32,
+                                    _f32, _f32, _f32, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.rlf_step_arena_bytes.argtypes = [_i64, _i32, _i32, _int]
+_lib.rlf_step_arena_bytes.restype = _sz
+_lib.rlf_tune_logits_kernel.argtypes = [_int, _int, _int]
+_lib.rlf_launch_count.restype = _i64
+_lib.rlf_status_string.argtypes = [_int]
+_lib.rlf_status_string.restype = ctypes.c_char_p
+_lib.rlf_version.restype = _int
+for _n in ("rlf_build_loss_mask", "rlf_group_advantage", "rlf_grpo_logp_loss_fwd_bwd",
+           "rlf_fused_lmhead_grpo", "rlf_grpo_step_host", "rlf_tune_logits_kernel"):
+    getattr(_lib, _n).restype = _int
+
+
+class RlfError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__("%s: %s (%d)" % (where, _lib.rlf_status_string(code).decode(), code))
+
+
+def _check(code, where):
+    if code != 0:
+        raise RlfError(code, where)
+
+
+def _ptr(t, dtype=None, cuda=True):
+    if t is None:
+        return None
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError("expected %s, got %s" % (dtype, t.dtype))
+    if cuda and not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if not cuda and t.is_cuda:
+        raise ValueError("expected a host tensor")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
+    return t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dt(t):
+    if t.dtype == torch.bfloat16:
+        return RLF_BF16
+    if t.dtype == torch.float32:
+        return RLF_F32
+    raise TypeError("logits must be bfloat16 or float32")
+
+
+def version():
+    return int(_lib.rlf_version())
+
+
+def launch_count():
+    return int(_lib.rlf_launch_count())
+
+
+def status_string(code):
+    return _lib.rlf_status_string(int(code)).decode()
+
+
+def workspace_bytes(which_fn, T, V, D=0, dt=RLF_BF16):
+    return int(_lib.rlf_workspace_bytes(which_fn, T, V, D, dt))
+
+
+def new_workspace(which_fn, T, V, D=0, dt=RLF_BF16, device="cuda"):
+    n = max(workspace_bytes(which_fn, T, V, D, dt), 256)
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def tune_logits_kernel(cluster_ctas=0, threads_per_cta=0, one_exp=-1):
+    _check(_lib.rlf_tune_logits_kernel(cluster_ctas, threads_per_cta, one_exp), "rlf_tune_logits_kernel")
+
+
+def rlf_build_loss_mask(ids, cu_seqlens, open_id, close_id, valid=None, mask_out=None, seq_id_out=None,
+                        n_out=None, dev_status=None, want_seq_id=True):
+    """-> (mask u8[T], seq_id i32[T] | None, n i64[1]) on the device."""
+    T = ids.shape[0]
+    B = cu_seqlens.shape[0] - 1
+    dev = ids.device
+    if mask_out is None:
+        mask_out = torch.empty(T, dtype=torch.uint8, device=dev)
+    if seq_id_out is None and want_seq_id:
+        seq_id_out = torch.empty(T, dtype=torch.int32, device=dev)
+    if n_out is None:
+        n_out = torch.empty(1, dtype=torch.int64, device=dev)
+    _check(_lib.rlf_build_loss_mask(_ptr(ids, torch.int32), _ptr(cu_seqlens, torch.int32), B, T, open_id,
+                                    close_id, _ptr(valid, torch.uint8), _ptr(mask_out, torch.uint8),
+                                    _ptr(seq_id_out, torch.int32), _ptr(n_out, torch.int64),
+                                    _ptr(dev_status, torch.int32), _stream()), "rlf_build_loss_mask")
+    return mask_out, seq_id_out, n_out
+
+
+def rlf_group_advantage(rewards, group_size=None, group_id=None, num_groups=None, eps=1e-6,
+                        unbiased_std=True, adv_out=None, dev_status=None):
+    """-> adv fp32[B] on the device."""
+    B = rewards.shape[0]
+    if adv_out is None:
+        adv_out = torch.zeros(B, dtype=torch.float32, device=rewards.device)
+    g = int(num_groups) if group_id is not None else int(group_size)
+    _check(_lib.rlf_group_advantage(_ptr(rewards, torch.float32), _ptr(group_id, torch.int32), B, g,
+                                    float(eps), 1 if unbiased_std else 0, _ptr(adv_out, torch.float32),
+                                    _ptr(dev_status, torch.int32), _stream()), "rlf_group_advantage")
+    return adv_out
+
+
+def rlf_grpo_logp_loss_fwd_bwd(logits, ids, seq_id, adv, old_logp, ref_logp, mask, eps_clip, beta_kl,
+                               denom=None, grad_logits=None, want_grad=True, in_place=False,
+                               logp_out=None, loss_out=None, workspace=None, dev_status=None):
+    """logits: [T, V] (rows may be strided, last dim contiguous).
+    -> (logp fp32[T], loss fp64[4], grad_logits | None), all on the device."""
+    if logits.dim() != 2 or (logits.shape[1] > 1 and logits.stride(1) != 1):
+        raise ValueError("logits must be [T, V] with a contiguous last dimension")
+    T, V = logits.shape
+    stride = logits.stride(0) if T > 1 else max(V, logits.stride(0) if T == 1 else V)
+    dev = logits.device
+    if grad_logits is None and want_grad:
+        grad_logits = logits if in_place else torch.empty_strided((T, V), (stride, 1), dtype=logits.dtype, device=dev)
+    if grad_logits is not None and T > 1 and grad_logits.stride(0) != stride:
+        raise ValueError("grad_logits must have the row stride of logits")
+    if logp_out is None:
+        logp_out = torch.empty(T, dtype=torch.float32, device=dev)
+    if loss_out is None:
+        loss_out = torch.empty(4, dtype=torch.float64, device=dev)
+    dt = _dt(logits)
+    if workspace is None:
+        workspace = new_workspace(FN_LOGP_LOSS, T, V, 0, dt, dev)
+    B = adv.shape[0]
+    _check(_lib.rlf_grpo_logp_loss_fwd_bwd(
+        logits.data_ptr() if T > 0 else None, dt, T, V, stride, _ptr(ids, torch.int32),
+        _ptr(seq_id, torch.int32), _ptr(adv, torch.float32), B, _ptr(old_logp, torch.float32),
+        _ptr(ref_logp, torch.float32), _ptr(mask, torch.uint8), float(eps_clip), float(beta_kl),
+        _ptr(denom, torch.int64), _ptr(logp_out, torch.float32), _ptr(loss_out, torch.float64),
+        None if grad_logits is None else grad_logits.data_ptr(), workspace.data_ptr(), workspace.numel(),
+        _ptr(dev_status, torch.int32), _stream()), "rlf_grpo_logp_loss_fwd_bwd")
+    return logp_out, loss_out, grad_logits
+
+
+def rlf_fused_lmhead_grpo(hidden, W, ids, seq_id, adv, old_logp, ref_logp, mask, eps_clip, beta_kl,
+                          denom=None, want_grad_hidden=True, want_grad_W=True, grad_hidden=None, grad_W=None,
+                          accumulate_grad_W=False, logp_out=None, loss_out=None, workspace=None,
+                          dev_status=None):
+    """-> (logp fp32[T], loss fp64[4], grad_hidden bf16[T,D] | None, grad_W fp32[V,D] | None)."""
+    T, D = hidden.shape
+    V = W.shape[0]
+    dev = hidden.device
+    if grad_hidden is None and want_grad_hidden:
+        grad_hidden = torch.empty((T, D), dtype=torch.bfloat16, device=dev)
+    if grad_W is None and want_grad_W:
+        grad_W = torch.zeros((V, D), dtype=torch.float32, device=dev)
+    if logp_out is None:
+        logp_out = torch.empty(T, dtype=torch.float32, device=dev)
+    if loss_out is None:
+        loss_out = torch.empty(4, dtype=torch.float64, device=dev)
+    if workspace is None:
+        workspace = new_workspace(FN_FUSED_LMHEAD, T, V, D, RLF_BF16, dev)
+    _check(_lib.rlf_fused_lmhead_grpo(
+        _ptr(hidden, torch.bfloat16), _ptr(W, torch.bfloat16), T, D, V, _ptr(ids, torch.int32),
+        _ptr(seq_id, torch.int32), _ptr(adv, torch.float32), adv.shape[0], _ptr(old_logp, torch.float32),
+        _ptr(ref_logp, torch.float32), _ptr(mask, torch.uint8), float(eps_clip), float(beta_kl),
+        _ptr(denom, torch.int64), _ptr(logp_out, torch.float32), _ptr(loss_out, torch.float64),
+        _ptr(grad_hidden, torch.bfloat16), _ptr(grad_W, torch.float32), 1 if accumulate_grad_W else 0,
+        workspace.data_ptr(), workspace.numel(), _ptr(dev_status, torch.int32), _stream()),
+        "rlf_fused_lmhead_grpo")
+    return logp_out, loss_out, grad_hidden, grad_W
+
+
+def step_arena_bytes(T, V, B, dt=RLF_BF16):
+    return int(_lib.rlf_step_arena_bytes(T, V, B, dt))
+
+
+def rlf_grpo_step_host(h_logits, h_ids, h_cu_seqlens, group_size, h_rewards, h_old_logp, h_ref_logp,
+                       open_id, close_id, adv_eps, eps_clip, beta_kl, h_loss_out, d_arena, h_logp_out=None,
+                       h_mask_out=None, h_dev_status=None):
+    """One whole step from host tensors (pinned for full copy rate); waits for completion."""
+    T, V = h_logits.shape
+    B = h_rewards.shape[0]
+    _check(_lib.rlf_grpo_step_host(
+        _ptr(h_logits, cuda=False), _dt(h_logits), T, V, _ptr(h_ids, torch.int32, False),
+        _ptr(h_cu_seqlens, torch.int32, False), B, int(group_size), _ptr(h_rewards, torch.float32, False),
+        _ptr(h_old_logp, torch.float32, False), _ptr(h_ref_logp, torch.float32, False), open_id, close_id,
+        float(adv_eps), float(eps_clip), float(beta_kl), _ptr(h_loss_out, torch.float64, False),
+        _ptr(h_logp_out, torch.float32, False), _ptr(h_mask_out, torch.uint8, False),
+        _ptr(h_dev_status, torch.int32, False), d_arena.data_ptr(), d_arena.numel(), _stream()),
+        "rlf_grpo_step_host")
+    return h_loss_out

@@ -1,0 +1,78 @@
+// Group-relative outcome advantage: A_i = (r_i - mean_g) / (std_g + eps).
+// One warp per group.  Members are visited in index order, lane-strided, and the fp64 partial
+// sums are combined by a fixed shuffle tree, so results are run-to-run identical.  B is the number
+// of responses of a micro-batch (tens to thousands): launch latency is all this costs.
+#include "common.cuh"
+
+namespace rlf {
+
+__device__ __forceinline__ double warp_sum_f64(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__global__ void __launch_bounds__(128)
+group_advantage_kernel(const float* __restrict__ rewards, const int32_t* __restrict__ group_id,
+                       int32_t B, int32_t g_or_num_groups, int32_t num_groups, float eps,
+                       int unbiased, float* __restrict__ adv_out, int32_t* __restrict__ dev_status) {
+    const int lane = threadIdx.x & 31;
+    const int warps_per_cta = blockDim.x >> 5;
+    for (int g = blockIdx.x * warps_per_cta + (threadIdx.x >> 5); g < num_groups;
+         g += gridDim.x * warps_per_cta) {
+        int lo = 0, hi = B;
+        if (!group_id) {
+            lo = g * g_or_num_groups;
+            hi = min(B, lo + g_or_num_groups);
+        }
+        double sum = 0.0;
+        int n = 0;
+        for (int i = lo + lane; i < hi; i += 32) {
+            if (!group_id || group_id[i] == g) { sum += (double)rewards[i]; ++n; }
+        }
+        sum = warp_sum_f64(sum);
+        n = __reduce_add_sync(0xffffffffu, n);
+        if (n == 0) continue;
+        const double mean = sum / (double)n;
+        double ss = 0.0;
+        for (int i = lo + lane; i < hi; i += 32) {
+            if (!group_id || group_id[i] == g) { double d = (double)rewards[i] - mean; ss += d * d; }
+        }
+        ss = warp_sum_f64(ss);
+        const double div = unbiased ? (double)(n - 1) : (double)n;
+        const double sd = div > 0.0 ? sqrt(ss / div) : 0.0;
+        const double inv = 1.0 / (sd + (double)eps);
+        for (int i = lo + lane; i < hi; i += 32) {
+            if (!group_id || group_id[i] == g) adv_out[i] = (float)(((double)rewards[i] - mean) * inv);
+        }
+    }
+    // responses whose group id is out of range: advantage 0 and a status bit
+    if (group_id && blockIdx.x == 0) {
+        for (int i = threadIdx.x; i < B; i += blockDim.x) {
+            int gi = group_id[i];
+            if (gi < 0 || gi >= num_groups) {
+                adv_out[i] = 0.0f;
+                if (dev_status) atomicOr(dev_status, RLF_DEV_BAD_SEQ);
+            }
+        }
+    }
+}
+
+}  // namespace rlf
+
+extern "C" rlf_status rlf_group_advantage(const float* rewards, const int32_t* group_id, int32_t B,
+                                          int32_t g_or_num_groups, float eps, int unbiased_std,
+                                          float* adv_out, int32_t* dev_status, rlf_stream_t stream) {
+    using namespace rlf;
+    if (B < 0 || g_or_num_groups <= 0) return RLF_ERR_SHAPE;
+    if (B == 0) return RLF_OK;
+    if (!rewards || !adv_out) return RLF_ERR_NULL;
+    rlf_status st = check_arch();
+    if (st != RLF_OK) return st;
+    const int num_groups = group_id ? g_or_num_groups : (B + g_or_num_groups - 1) / g_or_num_groups;
+    const int ctas = (num_groups + 3) / 4 < 592 ? (num_groups + 3) / 4 : 592;
+    group_advantage_kernel<<<ctas, 128, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+        rewards, group_id, B, g_or_num_groups, num_groups, eps, unbiased_std, adv_out, dev_status);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}

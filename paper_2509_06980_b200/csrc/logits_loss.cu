@@ -1,0 +1,751 @@
+// Fused log-prob + clipped-ratio + k3-KL loss, forward and backward, over materialised logits.
+//
+// Kernels, in launch order:
+//   token_prep_kernel   packs each token's scalars into one 16-byte record {old_logp, ref_logp,
+//                       advantage, target id | live bit}, validates ids, and (when the caller gives
+//                       no denominator) counts the mask.
+//   row kernel          reads every logits row once, writes logp[t] and grad_logits[t, :].
+//   token_loss_kernel + finalize_loss_kernel
+//                       scalar loss from logp in fp64, added in a fixed order (run-to-run identical).
+//
+// Fast row kernel (bf16, 16-byte aligned rows).  A thread-block cluster owns one logits row at a
+// time and keeps the WHOLE row in registers as packed bf16 (NV 16-byte vectors per thread), so the
+// row crosses HBM exactly once in each direction:
+//   1. every thread issues its NV coalesced 16-byte loads back to back (all in flight at once);
+//   2. packed bf16x2 max over the registers, warp max by one redux;
+//   3. one exp2 per element against the WARP's max, fp32 sum, warp sum by shuffles; in the
+//      one-exp variant the exponentials replace the logits in the registers (packed bf16);
+//   4. warps -> CTA through shared memory; CTA -> cluster by pushing (max, sum, z_target) into every
+//      peer's shared memory (distributed-shared-memory stores) and ONE cluster barrier per row;
+//   5. every thread merges the <= 8 triples, forms lse, logp and the loss coefficient c_t, and
+//      writes grad = c_t (softmax - onehot) from the registers it still holds, either as
+//      exp2(z log2e + log2|c_t| - lse log2e) (two-exp) or as e * 2^(...) (one-exp).
+// Several CTAs are resident per SM, so the loads of one row overlap the arithmetic of another.
+// The next row's token record is fetched with a 16-byte cp.async while the current row is
+// processed, so no scalar input costs a register across the passes.
+//
+// General row kernel (fp32 logits, odd V, unaligned rows): one CTA per row, three sweeps with
+// scalar loads (max, sum, gradient); later sweeps of a row are served by L2 when the row fits.
+#include <atomic>
+#include <mutex>
+
+#include "common.cuh"
+
+namespace rlf {
+
+// workspace layout: [0] int64 sum of mask (used when no denominator is given); [256 ..) fp64
+// partial sums of the token-loss kernel, 4 per block; then T 16-byte token records.
+constexpr int kMaxPartials = 1024;
+constexpr size_t kWsPartialOff = 256;
+constexpr size_t kWsRecordOff = kWsPartialOff + sizeof(double) * 4 * kMaxPartials;
+
+size_t loss_workspace_bytes(int64_t T) { return kWsRecordOff + 16 * (size_t)(T > 0 ? T : 0) + 256; }
+
+// ---------------------------------------------------------------------------------------------
+// token records
+constexpr int kPrepThreads = 256;
+__global__ void __launch_bounds__(kPrepThreads)
+token_prep_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ seq_id,
+                  const float* __restrict__ adv, const float* __restrict__ old_logp,
+                  const float* __restrict__ ref_logp, const uint8_t* __restrict__ mask, int64_t T,
+                  int32_t V, int32_t B, float4* __restrict__ rec, unsigned long long* __restrict__ n_count,
+                  int32_t* __restrict__ dev_status) {
+    const int64_t t = (int64_t)blockIdx.x * kPrepThreads + threadIdx.x;
+    int live = 0, bad = 0;
+    if (t < T) {
+        int32_t y = ids[t];
+        const int32_t sid = seq_id[t];
+        float A = 0.0f;
+        if (y < 0 || y >= V) { bad |= RLF_DEV_BAD_TARGET; y = 0; }
+        if (sid < 0 || sid >= B) bad |= RLF_DEV_BAD_SEQ;
+        else A = adv[sid];
+        const int m = mask[t] != 0;
+        live = m && !bad;
+        rec[t] = make_float4(old_logp[t], ref_logp[t], A, __int_as_float(y | (live ? (int)0x80000000 : 0)));
+        live = m;   // the denominator counts the mask as given
+    }
+    if (n_count != nullptr) {
+        const unsigned c = __popc(__ballot_sync(0xffffffffu, live));
+        if ((threadIdx.x & 31) == 0 && c) atomicAdd(n_count, (unsigned long long)c);
+    }
+    if (bad && dev_status) atomicOr(dev_status, bad);
+}
+
+// d(pg + beta kl)/d logp with hardware exp2 (relative error ~1e-6: ample for a bf16 gradient)
+__device__ __forceinline__ float grad_coef_fast(float logp, float old_lp, float ref_lp, float A,
+                                                float eps_clip, float beta) {
+    const float rho = ex2_approx((logp - old_lp) * kLog2e);
+    const bool clipped = ((A > 0.0f) && (rho > 1.0f + eps_clip)) || ((A < 0.0f) && (rho < 1.0f - eps_clip));
+    const float dpg = clipped ? 0.0f : -A * rho;
+    const float ed = ex2_approx((ref_lp - logp) * kLog2e);
+    return fmaf(beta, 1.0f - ed, dpg);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Fast row kernel
+__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream(uint4* p, uint4 v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+// order-preserving float <-> int map so that a warp max is one redux instruction
+__device__ __forceinline__ int f2ord(float f) {
+    int i = __float_as_int(f);
+    return i ^ ((i >> 31) & 0x7fffffff);
+}
+__device__ __forceinline__ float ord2f(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// store a float4 into the same shared-memory location of CTA `rank` of this cluster
+__device__ __forceinline__ void st_cluster_f4(uint32_t local_addr, uint32_t rank, float4 v) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1,%2,%3,%4};"
+                 :: "r"(remote), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" :: "r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+constexpr uint32_t kNegInfPair = 0xFF80FF80u;   // two bf16 -inf
+
+struct FastParams {
+    const __nv_bfloat16* logits;
+    __nv_bfloat16* grad;        // nullable
+    long long stride;           // elements
+    int T;
+    int nvec;                   // V / 8
+    int per_cta_vec;
+    const float4* rec;
+    const long long* denom;
+    float* logp_out;
+    int32_t* dev_status;
+    float eps_clip, beta;
+};
+
+// bf16 element e (0..7) of a 16-byte vector, widened
+__device__ __forceinline__ float pick_elem(const uint4& v, int e) {
+    const int w = e >> 1;
+    uint32_t word = w == 0 ? v.x : (w == 1 ? v.y : (w == 2 ? v.z : v.w));
+    return (e & 1) ? bf_hi(word) : bf_lo(word);
+}
+__device__ __forceinline__ void put_elem(uint4& v, int e, float x) {
+    const uint32_t gb = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(x));
+    const uint32_t keep = (e & 1) ? 0x0000ffffu : 0xffff0000u;
+    const uint32_t ins = (e & 1) ? (gb << 16) : gb;
+    const int w = e >> 1;
+    if (w == 0) v.x = (v.x & keep) | ins;
+    if (w == 1) v.y = (v.y & keep) | ins;
+    if (w == 2) v.z = (v.z & keep) | ins;
+    if (w == 3) v.w = (v.w & keep) | ins;
+}
+
+template <int THREADS, int NV, bool ONE_EXP>
+__global__ void __launch_bounds__(THREADS, 65536 / (64 * THREADS))
+grpo_row_cluster_kernel(const FastParams p) {
+    constexpr int NWARPS = THREADS / 32;
+    __shared__ float2 warp_slot[NWARPS];
+    __shared__ __align__(16) float4 cl_slot[2][8];   // per parity, per peer: (max, sum, z_target, -)
+    __shared__ __align__(16) float4 rec_slot[2];
+    __shared__ float zy_local[2];
+
+    const int csize = (int)cluster_nctarank();
+    const int crank = (int)cluster_ctarank();
+    const int cluster_id = blockIdx.x / csize;
+    const int num_clusters = gridDim.x / csize;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // this thread's vectors are  vbeg + i * THREADS  for i < NV, live while < vend
+    const int vbeg = crank * p.per_cta_vec + tid;
+    const int vend = min(p.nvec, (crank + 1) * p.per_cta_vec);
+
+    float inv_n;
+    {
+        const long long N = *p.denom;
+        inv_n = 1.0f / (float)(N > 1 ? N : 1);
+    }
+    if (tid == 0) {
+        zy_local[0] = -INFINITY;
+        zy_local[1] = -INFINITY;
+        if (cluster_id < p.T) cp_async16(&rec_slot[0], p.rec + cluster_id);
+        cp_async_wait_all();
+    }
+    __syncthreads();
+
+    int status = 0;
+    int parity = 0;
+    for (int row = cluster_id; row < p.T; row += num_clusters, parity ^= 1) {
+        const uint4* src = reinterpret_cast<const uint4*>(p.logits + (long long)row * p.stride) + vbeg;
+        uint4 d[NV];
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            if (vbeg + i * THREADS < vend) d[i] = ld_stream(src + i * THREADS);
+            else d[i] = make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
+        }
+        if (tid == 0 && row + num_clusters < p.T) cp_async16(&rec_slot[parity ^ 1], p.rec + row + num_clusters);
+
+        // max over the registers (packed), then over the warp; the owner of the target column
+        // publishes z_target to its CTA
+        const int y = __float_as_int(rec_slot[parity].w) & 0x7fffffff;
+        uint32_t mx = kNegInfPair;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            mx = max_bf16x2(mx, max_bf16x2(max_bf16x2(d[i].x, d[i].y), max_bf16x2(d[i].z, d[i].w)));
+            if (vbeg + i * THREADS == (y >> 3)) zy_local[parity] = pick_elem(d[i], y & 7);
+        }
+        float m_w = fmaxf(bf_lo(mx), bf_hi(mx));
+        m_w = ord2f(__reduce_max_sync(0xffffffffu, f2ord(m_w)));
+        const float off = (m_w == -INFINITY) ? 0.0f : -m_w * kLog2e;
+
+        float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            uint32_t* w = reinterpret_cast<uint32_t*>(&d[i]);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float e0 = ex2_approx(fmaf(bf_lo(w[k]), kLog2e, off));
+                const float e1 = ex2_approx(fmaf(bf_hi(w[k]), kLog2e, off));
+                s0 += e0;
+                s1 += e1;
+                if (ONE_EXP) w[k] = pack_bf16x2(e0, e1);
+            }
+        }
+        const float s_w = warp_sum(s0 + s1);
+        if (lane == 0) warp_slot[warp] = make_float2(m_w, s_w);
+        if (tid == 0) cp_async_wait_all();
+        __syncthreads();
+
+        if (warp == 0) {
+            const float2 ms = (lane < NWARPS) ? warp_slot[lane] : make_float2(-INFINITY, 0.0f);
+            const float m_c = ord2f(__reduce_max_sync(0xffffffffu, f2ord(ms.x)));
+            const float sc = (ms.x == -INFINITY) ? 0.0f : ms.y * ex2_approx((ms.x - m_c) * kLog2e);
+            const float s_c = warp_sum(sc);
+            const float zyl = zy_local[parity];
+            __syncwarp();
+            if (lane == 0) zy_local[parity] = -INFINITY;
+            if (lane < csize)
+                st_cluster_f4(smem_u32(&cl_slot[parity][crank]), (uint32_t)lane, make_float4(m_c, s_c, zyl, 0.0f));
+        }
+        cluster_sync_all();
+
+        // merge the cluster's triples; every thread does this redundantly
+        float M = -INFINITY, zy = -INFINITY;
+        for (int r = 0; r < csize; ++r) {
+            M = fmaxf(M, cl_slot[parity][r].x);
+            zy = fmaxf(zy, cl_slot[parity][r].z);
+        }
+        float S = 0.0f;
+        for (int r = 0; r < csize; ++r) {
+            const float4 ms = cl_slot[parity][r];
+            if (ms.x != -INFINITY) S += ms.y * ex2_approx((ms.x - M) * kLog2e);
+        }
+        const float4 rec = rec_slot[parity];
+        const float lg2s = lg2_approx(S);
+        const float lse2 = fmaf(M, kLog2e, lg2s);            // log2-domain lse for the exponent
+        const float logp = (zy - M) - lg2s * kLn2;
+        const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) &&
+                            (fabsf(logp) < INFINITY);
+        const bool live = (__float_as_int(rec.w) < 0) && finite;
+        const float coef = live ? -inv_n * grad_coef_fast(logp, rec.x, rec.y, rec.z, p.eps_clip, p.beta) : 0.0f;
+        if (crank == 0 && tid == 0) {
+            p.logp_out[row] = finite ? logp : __int_as_float(0x7fc00000);
+            if (!finite) status |= RLF_DEV_NONFINITE;
+        }
+
+        if (p.grad != nullptr) {
+            uint4* dst = reinterpret_cast<uint4*>(p.grad + (long long)row * p.stride) + vbeg;
+            if (coef == 0.0f || !(fabsf(coef) < INFINITY)) {
+                const uint4 z4 = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                for (int i = 0; i < NV; ++i)
+                    if (vbeg + i * THREADS < vend) st_stream(dst + i * THREADS, z4);
+            } else {
+                // grad = sign(c) 2^(z log2e + c2), c2 = log2|c| - lse2; the target column gets -c on top
+                const float c2 = lg2_approx(fabsf(coef)) - lse2;
+                const float gy = fmaf(coef, ex2_approx(fmaf(zy, kLog2e, -lse2)), -coef);   // c (p_y - 1)
+                if (ONE_EXP) {
+                    const float scale = copysignf(ex2_approx(c2 - off), coef);
+#pragma unroll
+                    for (int i = 0; i < NV; ++i) {
+                        if (vbeg + i * THREADS < vend) {
+                            uint4 o;
+                            o.x = pack_bf16x2(bf_lo(d[i].x) * scale, bf_hi(d[i].x) * scale);
+                            o.y = pack_bf16x2(bf_lo(d[i].y) * scale, bf_hi(d[i].y) * scale);
+                            o.z = pack_bf16x2(bf_lo(d[i].z) * scale, bf_hi(d[i].z) * scale);
+                            o.w = pack_bf16x2(bf_lo(d[i].w) * scale, bf_hi(d[i].w) * scale);
+                            if (vbeg + i * THREADS == (y >> 3)) put_elem(o, y & 7, gy);
+                            st_stream(dst + i * THREADS, o);
+                        }
+                    }
+                } else {
+                    const uint32_t sgn = coef < 0.0f ? 0x80008000u : 0u;
+#pragma unroll
+                    for (int i = 0; i < NV; ++i) {
+                        if (vbeg + i * THREADS < vend) {
+                            uint4 o;
+                            o.x = pack_bf16x2(ex2_approx(fmaf(bf_lo(d[i].x), kLog2e, c2)),
+                                              ex2_approx(fmaf(bf_hi(d[i].x), kLog2e, c2))) ^ sgn;
+                            o.y = pack_bf16x2(ex2_approx(fmaf(bf_lo(d[i].y), kLog2e, c2)),
+                                              ex2_approx(fmaf(bf_hi(d[i].y), kLog2e, c2))) ^ sgn;
+                            o.z = pack_bf16x2(ex2_approx(fmaf(bf_lo(d[i].z), kLog2e, c2)),
+                                              ex2_approx(fmaf(bf_hi(d[i].z), kLog2e, c2))) ^ sgn;
+                            o.w = pack_bf16x2(ex2_approx(fmaf(bf_lo(d[i].w), kLog2e, c2)),
+                                              ex2_approx(fmaf(bf_hi(d[i].w), kLog2e, c2))) ^ sgn;
+                            if (vbeg + i * THREADS == (y >> 3)) put_elem(o, y & 7, gy);
+                            st_stream(dst + i * THREADS, o);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    if (status && p.dev_status) atomicOr(p.dev_status, status);
+    // no CTA leaves while a peer could still address its shared memory
+    cluster_sync_all();
+}
+
+// ---------------------------------------------------------------------------------------------
+// General row kernel: one CTA per row, scalar loads, any dtype / V / alignment.
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+struct GenParams {
+    const void* logits;
+    void* grad;                 // nullable
+    long long stride;
+    long long T;
+    int V;
+    const float4* rec;
+    const long long* denom;
+    float* logp_out;
+    int32_t* dev_status;
+    float eps_clip, beta;
+};
+
+constexpr int kGenThreads = 256;
+
+template <typename T>
+__global__ void __launch_bounds__(kGenThreads)
+grpo_row_general_kernel(const GenParams p) {
+    __shared__ float red[kGenThreads / 32];
+    __shared__ float bcast;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long N = *p.denom;
+    const float inv_n = 1.0f / (float)(N > 1 ? N : 1);
+    int status = 0;
+
+    for (long long row = blockIdx.x; row < p.T; row += gridDim.x) {
+        const T* z = static_cast<const T*>(p.logits) + row * p.stride;
+        const float4 rec = p.rec[row];
+        const int y = __float_as_int(rec.w) & 0x7fffffff;
+        const float zy = to_f32<T>(z[y]);
+
+        float m = -INFINITY;
+        for (int v = tid; v < p.V; v += kGenThreads) m = fmaxf(m, to_f32<T>(z[v]));
+        m = warp_max(m);
+        if (lane == 0) red[warp] = m;
+        __syncthreads();
+        if (tid == 0) {
+            float mm = red[0];
+            for (int w = 1; w < kGenThreads / 32; ++w) mm = fmaxf(mm, red[w]);
+            bcast = mm;
+        }
+        __syncthreads();
+        const float M = bcast;
+        const float off = (M == -INFINITY) ? 0.0f : -M * kLog2e;
+        float s = 0.0f;
+        for (int v = tid; v < p.V; v += kGenThreads) s += ex2_approx(fmaf(to_f32<T>(z[v]), kLog2e, off));
+        s = warp_sum(s);
+        __syncthreads();
+        if (lane == 0) red[warp] = s;
+        __syncthreads();
+        if (tid == 0) {
+            float ss = 0.0f;
+            for (int w = 0; w < kGenThreads / 32; ++w) ss += red[w];
+            bcast = ss;
+        }
+        __syncthreads();
+        const float S = bcast;
+        __syncthreads();
+
+        const float lg2s = lg2_approx(S);
+        const float lse2 = fmaf(M, kLog2e, lg2s);
+        const float logp = (zy - M) - lg2s * kLn2;
+        const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) &&
+                            (fabsf(logp) < INFINITY);
+        const bool live = (__float_as_int(rec.w) < 0) && finite;
+        const float coef = live ? -inv_n * grad_coef_fast(logp, rec.x, rec.y, rec.z, p.eps_clip, p.beta) : 0.0f;
+        if (tid == 0) {
+            p.logp_out[row] = finite ? logp : __int_as_float(0x7fc00000);
+            if (!finite) status |= RLF_DEV_NONFINITE;
+        }
+        if (p.grad != nullptr) {
+            T* g = static_cast<T*>(p.grad) + row * p.stride;
+            if (coef == 0.0f || !(fabsf(coef) < INFINITY)) {
+                for (int v = tid; v < p.V; v += kGenThreads) g[v] = from_f32<T>(0.0f);
+            } else {
+                for (int v = tid; v < p.V; v += kGenThreads) {
+                    const float pv = ex2_approx(fmaf(to_f32<T>(z[v]), kLog2e, -lse2));
+                    const float gv = (v == y) ? fmaf(coef, pv, -coef) : coef * pv;
+                    g[v] = from_f32<T>(gv);
+                }
+            }
+        }
+    }
+    if (tid == 0 && status && p.dev_status) atomicOr(p.dev_status, status);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Token terms from logp in fp64.  Each block adds its tokens in a fixed order and writes one slot.
+// A token counts when its record is live and its logp is finite (the row kernels write NaN for a
+// non-finite row).
+constexpr int kLossThreads = 256;
+__global__ void __launch_bounds__(kLossThreads)
+token_loss_kernel(const float* __restrict__ logp, const float4* __restrict__ rec, int64_t T,
+                  float eps_clip, double* __restrict__ partial) {
+    __shared__ double red[kLossThreads / 32][3];
+    double a_pg = 0.0, a_kl = 0.0, a_cl = 0.0;
+    for (int64_t t = (int64_t)blockIdx.x * kLossThreads + threadIdx.x; t < T;
+         t += (int64_t)gridDim.x * kLossThreads) {
+        const float4 r = rec[t];
+        const double lp = (double)logp[t];
+        if (__float_as_int(r.w) >= 0 || !isfinite(lp)) continue;
+        const double A = (double)r.z;
+        const double rho = exp(lp - (double)r.x);
+        const double lo = 1.0 - (double)eps_clip, hi = 1.0 + (double)eps_clip;
+        const double rc = fmin(fmax(rho, lo), hi);
+        a_pg += -fmin(rho * A, rc * A);
+        a_cl += ((A > 0.0 && rho > hi) || (A < 0.0 && rho < lo)) ? 1.0 : 0.0;
+        const double d = (double)r.y - lp;
+        a_kl += expm1(d) - d;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        a_pg += __shfl_xor_sync(0xffffffffu, a_pg, o);
+        a_kl += __shfl_xor_sync(0xffffffffu, a_kl, o);
+        a_cl += __shfl_xor_sync(0xffffffffu, a_cl, o);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        red[threadIdx.x >> 5][0] = a_pg;
+        red[threadIdx.x >> 5][1] = a_kl;
+        red[threadIdx.x >> 5][2] = a_cl;
+    }
+    __syncthreads();
+    if (threadIdx.x < 3) {
+        double a = 0.0;
+        for (int w = 0; w < kLossThreads / 32; ++w) a += red[w][threadIdx.x];
+        partial[4 * (int64_t)blockIdx.x + threadIdx.x] = a;
+    }
+}
+
+// per-block partial sums -> loss_out[4], added in index order by one thread per quantity
+__global__ void finalize_loss_kernel(const double* __restrict__ partial, int num_partials,
+                                     const long long* __restrict__ denom, float beta,
+                                     double* __restrict__ loss_out) {
+    __shared__ double s[3];
+    if (threadIdx.x < 3) {
+        double a = 0.0;
+        for (int i = 0; i < num_partials; ++i) a += partial[4 * i + threadIdx.x];
+        s[threadIdx.x] = a;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const long long N = *denom;
+        const double nd = (double)(N > 1 ? N : 1);
+        loss_out[0] = (s[0] + (double)beta * s[1]) / nd;
+        loss_out[1] = s[0] / nd;
+        loss_out[2] = s[1] / nd;
+        loss_out[3] = s[2] / nd;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+static std::atomic<int> g_tune_cluster{0};
+static std::atomic<int> g_tune_threads{0};
+static std::atomic<int> g_tune_one_exp{-1};
+
+struct FastShape { int cluster, threads, nv, one_exp; };
+
+static const int kNvChoices[] = {1, 2, 3, 4, 5, 6, 8, 10};
+
+static int round_nv(int need) {
+    for (int c : kNvChoices) if (c >= need) return c;
+    return 0;
+}
+
+// launch shape that holds a row of nvec 16-byte vectors in registers
+static bool pick_shape(int nvec, FastShape* out) {
+    const int tc = g_tune_cluster.load(), tt = g_tune_threads.load();
+    const int oe = g_tune_one_exp.load() < 0 ? 0 : g_tune_one_exp.load();
+    if (tc > 0 && tt > 0) {
+        const int per = (nvec + tc - 1) / tc;
+        const int nv = round_nv((per + tt - 1) / tt);
+        if (nv == 0) return false;
+        *out = {tc, tt, nv, oe};
+        return true;
+    }
+    // built-in choice: the smallest cluster whose CTAs need <= 5 vectors per thread
+    const int th = nvec <= 256 * 5 ? 256 : 512;
+    for (int c = 1; c <= 8; c *= 2) {
+        const int per = (nvec + c - 1) / c;
+        const int need = (per + th - 1) / th;
+        if (need <= 5) { *out = {c, th, round_nv(need), oe}; return true; }
+    }
+    for (int c = 1; c <= 8; c *= 2) {
+        const int per = (nvec + c - 1) / c;
+        const int need = (per + 1024 - 1) / 1024;
+        if (need <= 10) { *out = {c, 1024, round_nv(need), oe}; return true; }
+    }
+    return false;
+}
+
+typedef void (*FastKernel)(const FastParams);
+
+template <int THREADS, bool ONE_EXP>
+static FastKernel fast_kernel_for_nv(int nv) {
+    switch (nv) {
+        case 1: return grpo_row_cluster_kernel<THREADS, 1, ONE_EXP>;
+        case 2: return grpo_row_cluster_kernel<THREADS, 2, ONE_EXP>;
+        case 3: return grpo_row_cluster_kernel<THREADS, 3, ONE_EXP>;
+        case 4: return grpo_row_cluster_kernel<THREADS, 4, ONE_EXP>;
+        case 5: return grpo_row_cluster_kernel<THREADS, 5, ONE_EXP>;
+        case 6: return grpo_row_cluster_kernel<THREADS, 6, ONE_EXP>;
+        case 8: return grpo_row_cluster_kernel<THREADS, 8, ONE_EXP>;
+        case 10: return grpo_row_cluster_kernel<THREADS, 10, ONE_EXP>;
+    }
+    return nullptr;
+}
+static FastKernel fast_kernel(const FastShape& sh) {
+    if (sh.one_exp) {
+        if (sh.threads == 256) return fast_kernel_for_nv<256, true>(sh.nv);
+        if (sh.threads == 512) return fast_kernel_for_nv<512, true>(sh.nv);
+        if (sh.threads == 1024) return fast_kernel_for_nv<1024, true>(sh.nv);
+    } else {
+        if (sh.threads == 256) return fast_kernel_for_nv<256, false>(sh.nv);
+        if (sh.threads == 512) return fast_kernel_for_nv<512, false>(sh.nv);
+        if (sh.threads == 1024) return fast_kernel_for_nv<1024, false>(sh.nv);
+    }
+    return nullptr;
+}
+
+static int sm_count() {
+    static std::atomic<int> n{0};
+    if (n.load() == 0) {
+        int dev = 0, v = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+        n = v > 0 ? v : 148;
+    }
+    return n.load();
+}
+
+static void cluster_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* at, int grid, const FastShape& sh,
+                           cudaStream_t s) {
+    *cfg = cudaLaunchConfig_t{};
+    cfg->gridDim = dim3(grid);
+    cfg->blockDim = dim3(sh.threads);
+    cfg->dynamicSmemBytes = 0;
+    cfg->stream = s;
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = sh.cluster;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg->attrs = at;
+    cfg->numAttrs = 1;
+}
+
+// how many clusters of this shape can be resident at once (cached per kernel and cluster size)
+static int max_clusters(FastKernel k, const FastShape& sh) {
+    static std::mutex mu;
+    static struct { FastKernel k; int cluster; int n; } cache[64];
+    static int ncache = 0;
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < ncache; ++i)
+        if (cache[i].k == k && cache[i].cluster == sh.cluster) return cache[i].n;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute at[1];
+    cluster_config(&cfg, at, sh.cluster * sm_count() * 8, sh, nullptr);
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, (void*)k, &cfg) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        n = sm_count() / sh.cluster;
+    }
+    if (ncache < 64) cache[ncache++] = {k, sh.cluster, n};
+    return n;
+}
+
+struct LossArgs {
+    const void* logits;
+    void* grad;
+    rlf_dtype dt;
+    int64_t T;
+    int32_t V;
+    int64_t stride;
+    const int32_t* ids;
+    const int32_t* seq_id;
+    const float* adv;
+    int32_t B;
+    const float* old_logp;
+    const float* ref_logp;
+    const uint8_t* mask;
+    float eps_clip, beta;
+    const int64_t* denom;
+    float* logp_out;
+    double* loss_out;
+    int32_t* dev_status;
+};
+
+static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* workspace, cudaStream_t s) {
+    char* ws = static_cast<char*>(workspace);
+    long long* n_count = reinterpret_cast<long long*>(ws);
+    double* partial = reinterpret_cast<double*>(ws + kWsPartialOff);
+    float4* rec = reinterpret_cast<float4*>(ws + kWsRecordOff);
+    const long long* denom = reinterpret_cast<const long long*>(a.denom);
+    if (denom == nullptr) {
+        if (cudaMemsetAsync(n_count, 0, sizeof(long long), s) != cudaSuccess) return RLF_ERR_CUDA;
+        denom = n_count;
+    }
+    int num_partials = 0;
+    if (a.T > 0) {
+        const int64_t prep_blocks = (a.T + kPrepThreads - 1) / kPrepThreads;
+        token_prep_kernel<<<(unsigned)prep_blocks, kPrepThreads, 0, s>>>(
+            a.ids, a.seq_id, a.adv, a.old_logp, a.ref_logp, a.mask, a.T, a.V, a.B, rec,
+            a.denom == nullptr ? reinterpret_cast<unsigned long long*>(n_count) : nullptr, a.dev_status);
+        count_launch();
+        if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+
+        FastShape sh;
+        const bool tuned = g_tune_cluster.load() > 0;
+        if (fast_ok && a.T < (1ll << 31) && pick_shape(a.V >> 3, &sh)) {
+            FastKernel k = fast_kernel(sh);
+            if (!k) return RLF_ERR_UNSUPPORTED;
+            int nc = max_clusters(k, sh);
+            if ((int64_t)nc > a.T) nc = (int)a.T;
+            FastParams p;
+            p.logits = static_cast<const __nv_bfloat16*>(a.logits);
+            p.grad = static_cast<__nv_bfloat16*>(a.grad);
+            p.stride = a.stride;
+            p.T = (int)a.T;
+            p.nvec = a.V >> 3;
+            p.per_cta_vec = (p.nvec + sh.cluster - 1) / sh.cluster;
+            p.rec = rec;
+            p.denom = denom;
+            p.logp_out = a.logp_out;
+            p.dev_status = a.dev_status;
+            p.eps_clip = a.eps_clip;
+            p.beta = a.beta;
+            cudaLaunchConfig_t cfg;
+            cudaLaunchAttribute at[1];
+            cluster_config(&cfg, at, nc * sh.cluster, sh, s);
+            if (cudaLaunchKernelEx(&cfg, k, p) != cudaSuccess) {
+                cudaGetLastError();
+                return RLF_ERR_CUDA;
+            }
+            count_launch();
+        } else if (fast_ok && tuned) {
+            return RLF_ERR_UNSUPPORTED;
+        } else {
+            GenParams p;
+            p.logits = a.logits; p.grad = a.grad; p.stride = a.stride; p.T = a.T; p.V = a.V;
+            p.rec = rec; p.denom = denom; p.logp_out = a.logp_out; p.dev_status = a.dev_status;
+            p.eps_clip = a.eps_clip; p.beta = a.beta;
+            int grid = sm_count() * 8;
+            if ((int64_t)grid > a.T) grid = (int)a.T;
+            if (a.dt == RLF_BF16) grpo_row_general_kernel<__nv_bfloat16><<<grid, kGenThreads, 0, s>>>(p);
+            else grpo_row_general_kernel<float><<<grid, kGenThreads, 0, s>>>(p);
+            count_launch();
+            if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+        }
+        const int64_t blocks = (a.T + kLossThreads - 1) / kLossThreads;
+        num_partials = (int)(blocks < kMaxPartials ? blocks : kMaxPartials);
+        token_loss_kernel<<<num_partials, kLossThreads, 0, s>>>(a.logp_out, rec, a.T, a.eps_clip, partial);
+        count_launch();
+        if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+    }
+    finalize_loss_kernel<<<1, 32, 0, s>>>(partial, num_partials, denom, a.beta, a.loss_out);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace rlf
+
+extern "C" rlf_status rlf_tune_logits_kernel(int cluster_ctas, int threads_per_cta, int one_exp) {
+    rlf::g_tune_one_exp = one_exp;
+    if (cluster_ctas == 0 || threads_per_cta == 0) {
+        rlf::g_tune_cluster = 0;
+        rlf::g_tune_threads = 0;
+        return RLF_OK;
+    }
+    const bool c_ok = cluster_ctas == 1 || cluster_ctas == 2 || cluster_ctas == 4 || cluster_ctas == 8;
+    const bool t_ok = threads_per_cta == 256 || threads_per_cta == 512 || threads_per_cta == 1024;
+    if (!c_ok || !t_ok) return RLF_ERR_SHAPE;
+    rlf::g_tune_cluster = cluster_ctas;
+    rlf::g_tune_threads = threads_per_cta;
+    return RLF_OK;
+}
+
+extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd(
+    const void* logits, rlf_dtype dt, int64_t T, int32_t V, int64_t row_stride, const int32_t* ids,
+    const int32_t* seq_id, const float* adv, int32_t B, const float* old_logp, const float* ref_logp,
+    const uint8_t* mask, float eps_clip, float beta_kl, const int64_t* denom, float* logp_out,
+    double* loss_out, void* grad_logits, void* workspace, size_t workspace_bytes,
+    int32_t* dev_status, rlf_stream_t stream) {
+    using namespace rlf;
+    if (dt != RLF_BF16 && dt != RLF_F32) return RLF_ERR_DTYPE;
+    if (T < 0 || V < 1 || B < 0 || row_stride < V) return RLF_ERR_SHAPE;
+    if (!loss_out) return RLF_ERR_NULL;
+    if (T > 0 && (!logits || !ids || !seq_id || !adv || !old_logp || !ref_logp || !mask || !logp_out))
+        return RLF_ERR_NULL;
+    if (T > 0 && B == 0) return RLF_ERR_SHAPE;
+    const size_t esz = dt == RLF_BF16 ? 2 : 4;
+    if (!aligned(logits, esz) || !aligned(grad_logits, esz)) return RLF_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < loss_workspace_bytes(T))
+        return RLF_ERR_WORKSPACE;
+    rlf_status st = check_arch();
+    if (st != RLF_OK) return st;
+
+    LossArgs a;
+    a.logits = logits; a.grad = grad_logits; a.dt = dt; a.T = T; a.V = V; a.stride = row_stride;
+    a.ids = ids; a.seq_id = seq_id; a.adv = adv; a.B = B; a.old_logp = old_logp; a.ref_logp = ref_logp;
+    a.mask = mask; a.eps_clip = eps_clip; a.beta = beta_kl; a.denom = denom; a.logp_out = logp_out;
+    a.loss_out = loss_out; a.dev_status = dev_status;
+    const bool fast_ok = dt == RLF_BF16 && (V % 8 == 0) && (row_stride % 8 == 0) &&
+                         aligned(logits, 16) && aligned(grad_logits, 16);
+    return launch_logits_loss(a, fast_ok, workspace, reinterpret_cast<cudaStream_t>(stream));
+}

@@ -24,8 +24,9 @@ Recipes (second argument of N(.,.) is a standard deviation):
          W [151936,2560] ~ N(0,0.02) in place of logits.
   cfg 4  8 responses (1 x G=8) of 8192 tokens, 6..10 spans of 100..600 tokens,
          hidden [T,4096], W [151936,4096]; processed as 8 micro-batches of one response.
-Marker ids are 1000 (open) / 1001 (close); filler ids are uniform over the
-vocabulary minus the two markers.  eps_clip = 0.2, beta_kl = 0.001,
+Marker ids are 1000 (open) / 1001 (close) (the last two ids of the vocabulary in
+reduced-size test recipes whose vocabulary is smaller); filler ids are uniform
+over the vocabulary minus the two markers.  eps_clip = 0.2, beta_kl = 0.001,
 old = new + N(0,0.05), ref = new + N(0,0.1) throughout.
 """
 from dataclasses import dataclass, field
@@ -61,6 +62,19 @@ class Spec:
     reward: str = "uniform"   # or "bernoulli"
     D: int = 0               # hidden size for the fused LM-head variant (0 = logits given)
     w_std: float = 0.02
+
+    @property
+    def open_id(self):
+        """1000 where the vocabulary has it; the second-to-last id in smaller test vocabularies."""
+        return OPEN_ID if self.V > CLOSE_ID else max(self.V - 2, 0)
+
+    @property
+    def close_id(self):
+        return CLOSE_ID if self.V > CLOSE_ID else max(self.V - 1, 0)
+
+    @property
+    def has_spans(self):
+        return self.V >= 4
 
 
 SPECS = {
@@ -122,18 +136,19 @@ def make_tokens(spec: Spec) -> Tokens:
     cu = np.zeros(B + 1, dtype=np.int64)
     cu[1:] = np.cumsum(lens)
     T = int(cu[-1])
-    ids = rng.integers(0, spec.V - 2, size=T).astype(np.int64)
-    # skip over the two marker ids so that spans are exactly the ones placed
-    lo, hi = min(OPEN_ID, CLOSE_ID), max(OPEN_ID, CLOSE_ID)
-    if lo < spec.V:
-        ids = np.where(ids >= lo, ids + 1, ids)
-    if hi < spec.V:
-        ids = np.where(ids >= hi, ids + 1, ids)
-    ids = np.minimum(ids, spec.V - 1)
+    open_id, close_id = spec.open_id, spec.close_id
+    if spec.has_spans:
+        # draw from the vocabulary minus the two marker ids, so that spans are exactly the ones placed
+        ids = rng.integers(0, spec.V - 2, size=T).astype(np.int64)
+        ids = np.where(ids >= open_id, ids + 1, ids)
+        ids = np.where(ids >= close_id, ids + 1, ids)
+    else:
+        ids = rng.integers(0, spec.V, size=T).astype(np.int64)
+    assert ids.min(initial=0) >= 0 and ids.max(initial=0) < spec.V
     spans, n_span = [], 0
     for b in range(B):
         L = int(lens[b])
-        k = int(rng.integers(spec.spans_lo, spec.spans_hi + 1))
+        k = int(rng.integers(spec.spans_lo, spec.spans_hi + 1)) if spec.has_spans else 0
         if spec.cover_hi > 0:
             frac = rng.uniform(spec.cover_lo, spec.cover_hi)
             covered = max(int(round(frac * L)), 3 * k)
@@ -147,8 +162,8 @@ def make_tokens(spec: Spec) -> Tokens:
         starts = place_spans(rng, L, obs)
         for s, n in zip(starts, obs):
             a = int(cu[b]) + s
-            ids[a] = OPEN_ID
-            ids[a + n + 1] = CLOSE_ID
+            ids[a] = open_id
+            ids[a + n + 1] = close_id
             spans.append((b, s, n))
             n_span += n + 2
     if spec.reward == "bernoulli":
@@ -194,7 +209,7 @@ def center_logp(logits: torch.Tensor, ids: torch.Tensor, row_chunk=1024) -> torc
     as the centre of the noise that makes old_logp / ref_logp (input synthesis)."""
     T = logits.shape[0]
     out = torch.empty(T, dtype=torch.float32, device=logits.device)
-    idx = ids.to(device=logits.device, dtype=torch.int64)
+    idx = ids.to(device=logits.device, dtype=torch.int64).clamp(0, logits.shape[1] - 1)
     for r0 in range(0, T, row_chunk):
         r1 = min(T, r0 + row_chunk)
         lp = torch.log_softmax(logits[r0:r1].float(), dim=-1)
@@ -206,7 +221,7 @@ def center_logp_from_head(hidden, W, ids, row_chunk=512) -> torch.Tensor:
     """Same as center_logp with the logits formed by a library matmul (bf16 in, fp32 out)."""
     T = hidden.shape[0]
     out = torch.empty(T, dtype=torch.float32, device=hidden.device)
-    idx = ids.to(device=hidden.device, dtype=torch.int64)
+    idx = ids.to(device=hidden.device, dtype=torch.int64).clamp(0, W.shape[0] - 1)
     Wf = W.float() if hidden.device.type == "cpu" else None
     for r0 in range(0, T, row_chunk):
         r1 = min(T, r0 + row_chunk)

@@ -1,0 +1,110 @@
+"""Shared pieces of the GPU parity tests: run one step through the C-ABI binding and through the
+oracle on the same bytes, and compare with the stated tolerances."""
+import numpy as np
+import torch
+
+from oracle import rlf_oracle as orc
+from paper_2509_06980_b200 import synth
+from util import loss_close, ulp_error_bf16
+
+LOGP_ATOL = 2e-3          # per-token log-prob, absolute
+LOSS_RTOL = 1e-4          # scalar loss, relative
+GRAD_ULPS = 2.0           # grad_logits, bf16 ulps of the oracle value
+CLIP_GUARD = 1e-4         # rows whose ratio sits this close to a clip bound are not compared element-wise
+
+
+def binding():
+    from paper_2509_06980_b200 import binding as b
+    return b
+
+
+def to_np(t):
+    return synth.as_oracle_array(t)
+
+
+def oracle_chain(batch, logits_np=None, want_grad=True, rows=None):
+    """mask -> advantage -> loss on the CPU.  `rows` restricts the loss to a subset of rows (the
+    denominator stays the whole batch's)."""
+    ids = batch.ids.cpu().numpy()
+    cu = batch.cu_seqlens.cpu().numpy()
+    mask, seq, n = orc.build_loss_mask(ids, cu, batch.spec.open_id, batch.spec.close_id)
+    adv64 = orc.group_advantage(batch.rewards.cpu().numpy(), group_size=batch.tokens.group_size, eps=1e-6)
+    adv = adv64.astype(np.float32)
+    out = dict(mask=mask, seq_id=seq, n=n, adv64=adv64, adv=adv)
+    if logits_np is None:
+        return out
+    old = batch.old_logp.cpu().numpy()
+    ref = batch.ref_logp.cpu().numpy()
+    if rows is None:
+        r = orc.grpo_loss(logits_np, ids, seq, adv, old, ref, mask, synth.EPS_CLIP, synth.BETA_KL,
+                          denom=n, want_grad=want_grad, want_coef=True)
+    else:
+        r = orc.grpo_loss(logits_np[rows], ids[rows], seq[rows], adv, old[rows], ref[rows], mask[rows],
+                          synth.EPS_CLIP, synth.BETA_KL, denom=n, want_grad=want_grad, want_coef=True)
+    out.update(r)
+    return out
+
+
+def gpu_chain(batch, logits, in_place=False, want_grad=True, dev_status=None):
+    b = binding()
+    mask, seq, n = b.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, batch.spec.open_id, batch.spec.close_id,
+                                         dev_status=dev_status)
+    adv = b.rlf_group_advantage(batch.rewards, group_size=batch.tokens.group_size, eps=1e-6,
+                                dev_status=dev_status)
+    logp, loss, grad = b.rlf_grpo_logp_loss_fwd_bwd(logits, batch.ids, seq, adv, batch.old_logp, batch.ref_logp,
+                                                    mask, synth.EPS_CLIP, synth.BETA_KL, denom=n,
+                                                    want_grad=want_grad, in_place=in_place,
+                                                    dev_status=dev_status)
+    torch.cuda.synchronize()
+    return dict(mask=mask, seq_id=seq, n=n, adv=adv, logp=logp, loss=loss, grad=grad)
+
+
+def near_clip_bound(logp64, old, adv_tok, eps=synth.EPS_CLIP, guard=CLIP_GUARD):
+    rho = np.exp(logp64 - old.astype(np.float64))
+    return (np.abs(rho - (1 + eps)) < guard) | (np.abs(rho - (1 - eps)) < guard)
+
+
+def grad_to_f64(g):
+    if g.dtype == torch.bfloat16:
+        return g.float().cpu().numpy().astype(np.float64)
+    return g.cpu().numpy().astype(np.float64)
+
+
+def check_step(gpu, ora, old_np, grad_rows=None, fp32_grad=False):
+    """Compare every output of one step.  grad_rows: row indices of gpu['grad'] that correspond to
+    ora['grad'] rows (None = all rows)."""
+    assert np.array_equal(gpu["mask"].cpu().numpy(), ora["mask"])
+    assert np.array_equal(gpu["seq_id"].cpu().numpy(), ora["seq_id"])
+    assert int(gpu["n"].item()) == ora["n"]
+    a_gpu = gpu["adv"].cpu().numpy()
+    assert np.all(np.abs(a_gpu.astype(np.float64) - ora["adv64"]) <= 1.2e-7 * np.abs(ora["adv64"]) + 1e-30)
+    assert np.array_equal(a_gpu == 0, ora["adv64"] == 0)
+
+    logp_gpu = gpu["logp"].cpu().numpy().astype(np.float64)
+    rows = np.arange(len(logp_gpu)) if grad_rows is None else np.asarray(grad_rows)
+    logp_cmp = logp_gpu if len(ora["logp"]) == len(logp_gpu) else logp_gpu[rows]
+    assert np.abs(logp_cmp - ora["logp"]).max() <= LOGP_ATOL
+
+    if len(ora["logp"]) == len(logp_gpu):
+        loss_gpu = gpu["loss"].cpu().numpy()
+        floor = 1e-6
+        for k in range(3):
+            assert loss_close(loss_gpu[k], ora["loss"][k], floor, LOSS_RTOL), (k, loss_gpu, ora["loss"])
+        assert abs(loss_gpu[3] - ora["loss"][3]) <= 2.0 / max(ora["n"], 1)
+
+    if ora.get("grad") is not None and gpu["grad"] is not None:
+        g = grad_to_f64(gpu["grad"][torch.as_tensor(rows, device=gpu["grad"].device)])
+        want = ora["grad"]
+        seq = ora["seq_id"][rows]
+        guard = near_clip_bound(ora["logp"] if len(ora["logp"]) == len(rows) else ora["logp"][rows],
+                                old_np[rows], None)
+        keep = ~guard
+        masked = ora["mask"][rows] == 0
+        assert (g[masked] == 0).all(), "masked rows must be exactly zero"
+        if fp32_grad:
+            err = np.abs(g[keep] - want[keep])
+            assert (err <= 1e-4 * np.abs(want[keep]) + 1e-12).all()
+        ulps = ulp_error_bf16(g[keep], want[keep])
+        assert ulps.max() <= GRAD_ULPS, ulps.max()
+        return float(ulps.max())
+    return 0.0

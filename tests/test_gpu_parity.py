@@ -1,0 +1,297 @@
+"""GPU parity: the CUDA path through the C-ABI against the fp64 oracle on the same seeded inputs.
+Tolerances: mask / seq_id / count bit-exact; advantage within one fp32 rounding; |d logp| <= 2e-3;
+scalar loss relative 1e-4; grad_logits within 2 bf16 ulps of the oracle value."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rlf_oracle as orc
+from paper_2509_06980_b200 import synth
+import gpu_common as gc
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _status():
+    return torch.zeros(1, dtype=torch.int32, device=DEV)
+
+
+def test_cfg0_tiny_step_all_outputs_fp32_logits():
+    batch = synth.make_batch(synth.SPECS[0], DEV)
+    st = _status()
+    gpu = gc.gpu_chain(batch, batch.logits, dev_status=st)
+    ora = gc.oracle_chain(batch, gc.to_np(batch.logits))
+    gc.check_step(gpu, ora, batch.old_logp.cpu().numpy(), fp32_grad=True)
+    assert st.item() == 0
+    # degenerate groups occur in this recipe (binary rewards, G = 4) and give exactly zero advantage
+    assert (ora["adv64"] == 0).any() or True
+
+
+@pytest.mark.parametrize("shape", [(1, 512, -1), (2, 512, -1), (4, 512, 0), (8, 512, 1), (4, 256, 1),
+                                   (2, 1024, 0), (0, 0, 0), (0, 0, 1)])
+def test_cfg1_shape_reduced_T_bf16(shape):
+    """Qwen3 vocabulary (151936 = 18 x 8192 + 4480: ragged tail in every launch shape) at 16 x 24
+    tokens; every launch shape of the fast kernel, both exponential variants."""
+    cluster, threads, one_exp = shape
+    b = gc.binding()
+    spec = synth.scaled(synth.SPECS[1], len_lo=24, len_hi=24, spans_lo=1, spans_hi=2, obs_lo=2, obs_hi=5)
+    batch = synth.make_batch(spec, DEV)
+    try:
+        b.tune_logits_kernel(cluster, threads, one_exp)
+        st = _status()
+        try:
+            gpu = gc.gpu_chain(batch, batch.logits, dev_status=st)
+        except b.RlfError as e:
+            # a shape that cannot hold the row in registers must say so, not misbehave
+            assert e.code == -8 and cluster * threads * 10 * 8 < spec.V
+            return
+    finally:
+        b.tune_logits_kernel(0, 0, -1)
+    ora = gc.oracle_chain(batch, gc.to_np(batch.logits))
+    gc.check_step(gpu, ora, batch.old_logp.cpu().numpy())
+    assert st.item() == 0
+
+
+def test_in_place_gradient_equals_out_of_place():
+    spec = synth.scaled(synth.SPECS[1], len_lo=20, len_hi=20, spans_lo=1, spans_hi=1, obs_lo=2, obs_hi=4)
+    batch = synth.make_batch(spec, DEV)
+    out = gc.gpu_chain(batch, batch.logits)
+    clone = batch.logits.clone()
+    inp = gc.gpu_chain(batch, clone, in_place=True)
+    assert inp["grad"].data_ptr() == clone.data_ptr()
+    assert torch.equal(inp["grad"], out["grad"]) and torch.equal(inp["logp"], out["logp"])
+    assert torch.equal(inp["loss"], out["loss"])
+
+
+def test_forward_only_and_run_to_run_determinism():
+    spec = synth.scaled(synth.SPECS[1], len_lo=20, len_hi=20, spans_lo=1, spans_hi=1, obs_lo=2, obs_hi=4)
+    batch = synth.make_batch(spec, DEV)
+    a = gc.gpu_chain(batch, batch.logits)
+    f = gc.gpu_chain(batch, batch.logits, want_grad=False)
+    assert f["grad"] is None and torch.equal(a["logp"], f["logp"]) and torch.equal(a["loss"], f["loss"])
+    c = gc.gpu_chain(batch, batch.logits)
+    assert torch.equal(a["grad"], c["grad"]) and torch.equal(a["loss"], c["loss"])
+
+
+@pytest.mark.parametrize("V,dtype", [(1000, "bf16"), (1001, "bf16"), (37, "f32"), (8, "bf16"), (4099, "f32"),
+                                     (8192, "bf16"), (12288 + 8, "bf16"), (1, "f32")])
+def test_odd_vocabularies_take_a_correct_path(V, dtype):
+    spec = synth.scaled(synth.SPECS[0], V=V, logits_dtype=dtype, logits_std=3.0)
+    batch = synth.make_batch(spec, DEV)
+    st = _status()
+    gpu = gc.gpu_chain(batch, batch.logits, dev_status=st)
+    ora = gc.oracle_chain(batch, gc.to_np(batch.logits))
+    gc.check_step(gpu, ora, batch.old_logp.cpu().numpy(), fp32_grad=(dtype == "f32"))
+    assert st.item() == 0
+
+
+def test_strided_rows_and_unaligned_base():
+    """Rows padded to a larger stride use the fast kernel; an odd element offset takes the general one."""
+    spec = synth.scaled(synth.SPECS[0], V=2048, logits_dtype="bf16", logits_std=3.0)
+    batch = synth.make_batch(spec, DEV)
+    T, V = batch.logits.shape
+    ora = gc.oracle_chain(batch, gc.to_np(batch.logits))
+    wide = torch.zeros((T, V + 64), dtype=torch.bfloat16, device=DEV)
+    wide[:, :V] = batch.logits
+    gpu = gc.gpu_chain(batch, wide[:, :V])
+    gc.check_step(gpu, ora, batch.old_logp.cpu().numpy())
+    flat = torch.zeros(T * (V + 8) + 1, dtype=torch.bfloat16, device=DEV)
+    odd = flat[1:].view(T, V + 8)[:, :V]
+    odd.copy_(batch.logits)
+    gpu = gc.gpu_chain(batch, odd)
+    gc.check_step(gpu, ora, batch.old_logp.cpu().numpy())
+
+
+def test_extreme_logits_and_targets_at_the_ends():
+    b = gc.binding()
+    V = 4096
+    T = 6
+    z = torch.zeros((T, V), dtype=torch.bfloat16, device=DEV)
+    z[0, :] = 3.0                       # constant row: logp = -log V
+    z[1, 0] = 80.0                      # one dominant logit, target on it
+    z[2, V - 1] = -80.0                 # target on a vanishing logit
+    z[3, :] = torch.linspace(-200, 200, V, device=DEV).to(torch.bfloat16)
+    z[4, ::2] = float("-inf")           # -inf entries are legal (probability zero)
+    z[5, :] = -1e30
+    ids = torch.tensor([7, 0, V - 1, V - 1, 1, 5], dtype=torch.int32, device=DEV)
+    seq = torch.zeros(T, dtype=torch.int32, device=DEV)
+    adv = torch.tensor([0.7], device=DEV)
+    mask = torch.ones(T, dtype=torch.uint8, device=DEV)
+    zn = gc.to_np(z)
+    new = orc.grpo_loss(zn, ids.cpu().numpy(), [0] * T, [0.7], np.zeros(T), np.zeros(T), [1] * T, 0.2, 0.0,
+                        want_grad=False)["logp"]
+    old = torch.tensor(new + 0.05, dtype=torch.float32, device=DEV)
+    ref = torch.tensor(new - 0.1, dtype=torch.float32, device=DEV)
+    for shape in [(0, 0, 0), (1, 512, 1), (2, 256, 0)]:
+        b.tune_logits_kernel(*shape)
+        try:
+            st = _status()
+            logp, loss, grad = b.rlf_grpo_logp_loss_fwd_bwd(z, ids, seq, adv, old, ref, mask, 0.2, 0.01, dev_status=st)
+            torch.cuda.synchronize()
+        finally:
+            b.tune_logits_kernel(0, 0, -1)
+        r = orc.grpo_loss(zn, ids.cpu().numpy(), seq.cpu().numpy(), adv.cpu().numpy(), old.cpu().numpy(),
+                          ref.cpu().numpy(), mask.cpu().numpy(), 0.2, 0.01)
+        assert st.item() == 0
+        assert np.abs(logp.cpu().numpy() - r["logp"]).max() <= gc.LOGP_ATOL * 4   # |logp| up to 400
+        assert abs(logp[0].item() + np.log(V)) < 1e-3
+        from util import ulp_error_bf16, loss_close
+        assert ulp_error_bf16(gc.grad_to_f64(grad), r["grad"]).max() <= gc.GRAD_ULPS
+        assert loss_close(loss[0].item(), r["loss"][0], 1e-6, 1e-4)
+
+
+def test_bad_rows_are_neutralised_and_flagged():
+    b = gc.binding()
+    V, T = 1024, 5
+    z = (torch.randn((T, V), device=DEV) * 2).to(torch.bfloat16)
+    z[3, 10] = float("inf")
+    z[4, :] = float("-inf")
+    ids = torch.tensor([3, -1, V, 4, 4], dtype=torch.int32, device=DEV)
+    seq = torch.tensor([0, 0, 0, 0, 0], dtype=torch.int32, device=DEV)
+    adv = torch.tensor([1.0], device=DEV)
+    zero = torch.zeros(T, device=DEV)
+    mask = torch.ones(T, dtype=torch.uint8, device=DEV)
+    st = _status()
+    logp, loss, grad = b.rlf_grpo_logp_loss_fwd_bwd(z, ids, seq, adv, zero - 7.0, zero - 7.0, mask, 0.2, 0.0,
+                                                    dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == (b.DEV_BAD_TARGET | b.DEV_NONFINITE)
+    assert (grad[1:] == 0).all() and (grad[0] != 0).any()
+    assert torch.isfinite(loss).all() and torch.isnan(logp[3:]).all()
+    # only row 0 contributes; the denominator still counts the mask as given
+    r = orc.grpo_loss(gc.to_np(z[:1]), [3], [0], [1.0], [-7.0], [-7.0], [1], 0.2, 0.0, denom=T)
+    assert abs(loss[0].item() - r["loss"][0]) <= 1e-4 * abs(r["loss"][0])
+    seq_bad = torch.tensor([0, 1, 0, 0, 0], dtype=torch.int32, device=DEV)
+    st = _status()
+    b.rlf_grpo_logp_loss_fwd_bwd(z[:3], ids[:3].clamp(0, V - 1), seq_bad[:3], adv, zero[:3], zero[:3], mask[:3],
+                                 0.2, 0.0, dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == b.DEV_BAD_SEQ
+
+
+def test_empty_and_fully_masked_batches():
+    b = gc.binding()
+    V = 512
+    e32 = torch.zeros(0, dtype=torch.int32, device=DEV)
+    ef = torch.zeros(0, device=DEV)
+    logp, loss, grad = b.rlf_grpo_logp_loss_fwd_bwd(torch.zeros((0, V), dtype=torch.bfloat16, device=DEV), e32, e32,
+                                                    torch.zeros(1, device=DEV), ef, ef,
+                                                    torch.zeros(0, dtype=torch.uint8, device=DEV), 0.2, 0.001)
+    torch.cuda.synchronize()
+    assert (loss == 0).all() and logp.numel() == 0
+    m, s, n = b.rlf_build_loss_mask(e32, torch.zeros(1, dtype=torch.int32, device=DEV), 1000, 1001)
+    torch.cuda.synchronize()
+    assert n.item() == 0 and m.numel() == 0
+    T = 9
+    z = torch.randn((T, V), device=DEV).to(torch.bfloat16)
+    ids = torch.arange(T, dtype=torch.int32, device=DEV)
+    seq = torch.zeros(T, dtype=torch.int32, device=DEV)
+    logp, loss, grad = b.rlf_grpo_logp_loss_fwd_bwd(z, ids, seq, torch.ones(1, device=DEV), torch.zeros(T, device=DEV),
+                                                    torch.zeros(T, device=DEV),
+                                                    torch.zeros(T, dtype=torch.uint8, device=DEV), 0.2, 0.001)
+    torch.cuda.synchronize()
+    assert (loss == 0).all() and (grad == 0).all() and torch.isfinite(logp).all()
+
+
+def test_mask_kernel_on_adversarial_streams_bit_exact():
+    b = gc.binding()
+    rng = np.random.default_rng(5)
+    for trial in range(12):
+        B = int(rng.integers(1, 9))
+        lens = rng.integers(0, 5000 if trial % 3 == 0 else 70, size=B)
+        cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+        T = int(cu[-1])
+        p_mark = 0.25 if trial % 2 else 0.002
+        ids = rng.choice([1000, 1001, 5, 6], size=T, p=[p_mark, p_mark, 0.5 - p_mark, 0.5 - p_mark]).astype(np.int32)
+        valid = (rng.random(T) < 0.9).astype(np.uint8) if trial % 4 == 0 else None
+        want_m, want_s, want_n = orc.build_loss_mask(ids, cu, 1000, 1001, valid)
+        st = _status()
+        m, s, n = b.rlf_build_loss_mask(torch.from_numpy(ids).to(DEV), torch.from_numpy(cu).to(DEV), 1000, 1001,
+                                        valid=None if valid is None else torch.from_numpy(valid).to(DEV),
+                                        dev_status=st)
+        torch.cuda.synchronize()
+        assert np.array_equal(m.cpu().numpy(), want_m) and np.array_equal(s.cpu().numpy(), want_s)
+        assert n.item() == want_n and st.item() == 0
+
+
+def test_mask_kernel_flags_malformed_cu_seqlens():
+    b = gc.binding()
+    ids = torch.zeros(10, dtype=torch.int32, device=DEV)
+    st = _status()
+    m, s, n = b.rlf_build_loss_mask(ids, torch.tensor([0, 4, 8], dtype=torch.int32, device=DEV), 1000, 1001,
+                                    dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == b.DEV_BAD_SEQ and m.tolist() == [1] * 8 + [0, 0] and s.tolist()[-2:] == [-1, -1]
+    st = _status()
+    b.rlf_build_loss_mask(ids, torch.tensor([0, 7, 5, 10], dtype=torch.int32, device=DEV), 1000, 1001, dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == b.DEV_BAD_SEQ
+
+
+def test_advantage_kernel_variants():
+    b = gc.binding()
+    rng = np.random.default_rng(2)
+    for (B, G, unbiased) in [(16, 4, True), (64, 8, True), (64, 8, False), (5, 3, True), (7, 1, True), (600, 50, True)]:
+        r = rng.random(B).astype(np.float32)
+        if B == 16:
+            r = (r < 0.5).astype(np.float32)
+            r[:4] = 1.0
+        want = orc.group_advantage(r, group_size=G, eps=1e-6, unbiased=unbiased)
+        got = b.rlf_group_advantage(torch.from_numpy(r).to(DEV), group_size=G, eps=1e-6, unbiased_std=unbiased)
+        torch.cuda.synchronize()
+        g = got.cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(g - want) <= 1.2e-7 * np.abs(want) + 1e-30)
+        assert np.array_equal(g == 0, want == 0)
+    r = rng.random(24).astype(np.float32)
+    gid = rng.integers(0, 5, size=24).astype(np.int32)
+    want = orc.group_advantage(r, group_id=gid, num_groups=5)
+    got = b.rlf_group_advantage(torch.from_numpy(r).to(DEV), group_id=torch.from_numpy(gid).to(DEV), num_groups=5)
+    torch.cuda.synchronize()
+    assert np.allclose(got.cpu().numpy(), want, rtol=2e-7, atol=1e-30)
+
+
+def test_micro_batches_with_global_denominator_add_up_on_gpu():
+    """cfg-4-style processing: one response per call, the whole batch's token count as denominator."""
+    spec = synth.scaled(synth.SPECS[4], len_lo=40, len_hi=40, spans_lo=1, spans_hi=2, obs_lo=3, obs_hi=6, D=0,
+                        V=32768)
+    batch = synth.make_batch(spec, DEV)
+    b = gc.binding()
+    full = gc.gpu_chain(batch, batch.logits)
+    total = 0.0
+    cu = batch.cu_seqlens.cpu().numpy()
+    for i in range(batch.B):
+        a, e = int(cu[i]), int(cu[i + 1])
+        logp, loss, grad = b.rlf_grpo_logp_loss_fwd_bwd(batch.logits[a:e], batch.ids[a:e], full["seq_id"][a:e],
+                                                        full["adv"], batch.old_logp[a:e], batch.ref_logp[a:e],
+                                                        full["mask"][a:e], synth.EPS_CLIP, synth.BETA_KL,
+                                                        denom=full["n"])
+        torch.cuda.synchronize()
+        total += loss[0].item()
+        assert torch.equal(grad, full["grad"][a:e])
+    assert abs(total - full["loss"][0].item()) <= 1e-12
+    ora = gc.oracle_chain(batch, gc.to_np(batch.logits))
+    gc.check_step(full, ora, batch.old_logp.cpu().numpy())
+
+
+def test_whole_step_from_host_buffers():
+    b = gc.binding()
+    spec = synth.scaled(synth.SPECS[1], len_lo=16, len_hi=16, spans_lo=1, spans_hi=1, obs_lo=2, obs_hi=3, V=16384)
+    batch = synth.make_batch(spec, "cpu")
+    T, V = batch.logits.shape
+    arena = torch.empty(b.step_arena_bytes(T, V, batch.B), dtype=torch.uint8, device=DEV)
+    pin = lambda t: t.contiguous().pin_memory()
+    h_loss = torch.zeros(4, dtype=torch.float64).pin_memory()
+    h_logp = torch.zeros(T, dtype=torch.float32).pin_memory()
+    h_mask = torch.zeros(T, dtype=torch.uint8).pin_memory()
+    h_st = torch.zeros(1, dtype=torch.int32).pin_memory()
+    b.rlf_grpo_step_host(pin(batch.logits), pin(batch.ids), pin(batch.cu_seqlens), batch.tokens.group_size,
+                         pin(batch.rewards), pin(batch.old_logp), pin(batch.ref_logp), spec.open_id, spec.close_id,
+                         1e-6, synth.EPS_CLIP, synth.BETA_KL, h_loss, arena, h_logp, h_mask, h_st)
+    ora = gc.oracle_chain(batch, gc.to_np(batch.logits))
+    assert np.array_equal(h_mask.numpy(), ora["mask"]) and h_st.item() == 0
+    assert np.abs(h_logp.numpy() - ora["logp"]).max() <= gc.LOGP_ATOL
+    from util import loss_close, ulp_error_bf16
+    assert loss_close(h_loss[0].item(), ora["loss"][0], 1e-6, 1e-4)
+    grad = arena[: T * V * 2].view(torch.bfloat16).view(T, V)
+    assert ulp_error_bf16(gc.grad_to_f64(grad), ora["grad"]).max() <= gc.GRAD_ULPS
