@@ -1,0 +1,381 @@
+#!/usr/bin/env python
+"""Benchmark of the GRPO policy-update loss path on B200.
+
+One step = one pass of the whole path over one synthetic micro-batch that is already resident in
+HBM:  rlf_build_loss_mask -> rlf_group_advantage -> rlf_grpo_logp_loss_fwd_bwd  (forward and
+backward over the full vocabulary).  The workload at one GPU is the Qwen3-4B-shaped micro-batch:
+16 responses x 2048 tokens, V = 151936 bf16 logits (9.96 GB in, 9.96 GB of grad_logits out).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line.  With N > 1 (under torchrun) every rank runs its own micro-batch (no data-path
+collective: tokens are independent given the per-batch token count), the time is the max over
+ranks, and the value is the tokens all ranks processed per second.
+`--impl reference` times the fp64 CPU oracle on the host cores instead (a deliberately slow
+definition-level program; rank 0 only).
+"""
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2509_06980_b200 import synth
+
+METRIC = "GRPO loss fwd+bwd tokens/s at V=151936 bf16"
+UNIT = "tokens/s"
+WORKLOAD = "cfg1_qwen3_4b_microbatch: 16 responses x 2048 tokens, V=151936 bf16 logits"
+
+# DRAM bytes of one row-kernel launch from the ncu capture summarised under profiles/, as bytes per
+# token; valid only for the kernel source it was taken from (else reported as null).
+NCU_TRAFFIC = {"logits_loss_cu_sha1": None, "dram_bytes_per_token": None}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def _kernel_sha1():
+    p = os.path.join(ROOT, "paper_2509_06980_b200", "csrc", "logits_loss.cu")
+    with open(p, "rb") as f:
+        return hashlib.sha1(f.read()).hexdigest()
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
+                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1]))
+                mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def shard_seed(base_seed, rank):
+    """Each rank draws its own micro-batch of the same recipe."""
+    return base_seed + 101 * rank
+
+
+def aggregate(tokens_per_rank, world, max_seconds):
+    """Whole-job throughput: the tokens all ranks processed over the slowest rank's time."""
+    return tokens_per_rank * world / max_seconds
+
+
+def max_over_ranks(seconds, world, device=None, backend_tensor=None):
+    """Slowest rank's time (an all-reduce MAX of one scalar; identity at world size 1)."""
+    if world <= 1:
+        return float(seconds)
+    import torch.distributed as dist
+    t = torch.tensor([seconds], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# ---------------------------------------------------------------------------------------------
+def oracle_step_sampler(batch, rows_per_call):
+    """Returns f(k) that runs the oracle chain on the k-th slice of `rows_per_call` rows (mask and
+    advantage for the whole batch, loss forward + backward on the slice) and returns rows done."""
+    from oracle import rlf_oracle as orc
+    ids = batch.ids.cpu().numpy()
+    cu = batch.cu_seqlens.cpu().numpy()
+    rewards = batch.rewards.cpu().numpy()
+    old = batch.old_logp.cpu().numpy()
+    ref = batch.ref_logp.cpu().numpy()
+    T = batch.T
+
+    def run(k):
+        r0 = (k * rows_per_call) % T
+        r1 = min(T, r0 + rows_per_call)
+        z = synth.as_oracle_array(batch.logits[r0:r1])
+        mask, seq, n = orc.build_loss_mask(ids, cu, batch.spec.open_id, batch.spec.close_id)
+        adv = orc.group_advantage(rewards, group_size=batch.tokens.group_size, eps=1e-6).astype(np.float32)
+        orc.grpo_loss(z, ids[r0:r1], seq[r0:r1], adv, old[r0:r1], ref[r0:r1], mask[r0:r1], synth.EPS_CLIP,
+                      synth.BETA_KL, denom=n, want_grad=True)
+        return r1 - r0
+    return run, orc.num_threads()
+
+
+def time_oracle(batch, budget_s, rows_per_call=256):
+    run, cores = oracle_step_sampler(batch, rows_per_call)
+    run(0)                                      # page in, build
+    done, k, t0 = 0, 0, time.perf_counter()
+    while True:
+        done += run(k)
+        k += 1
+        el = time.perf_counter() - t0
+        if el >= budget_s or k >= 4096:
+            break
+    return dict(value=done / el, unit=UNIT, cores=cores, kind="oracle",
+                sample="%d rows of the same micro-batch (full vocabulary, forward + fp64 gradient), %d calls of %d rows, %.1f s"
+                       % (done, k, rows_per_call, el))
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    spec = synth.SPECS[1]
+    rows = 256
+    # the oracle reads a row slice per step; draw only what the steps touch
+    need = rows * (args.steps + args.warmup)
+    per = max(need // 16 + 1, 64)
+    small = synth.scaled(spec, len_lo=per, len_hi=per, spans_lo=1, spans_hi=2, obs_lo=10, obs_hi=20)
+    batch = synth.make_batch(small, "cpu")
+    run, cores = oracle_step_sampler(batch, rows)
+    for k in range(args.warmup):
+        run(k)
+    t0 = time.perf_counter()
+    done = 0
+    for k in range(args.steps):
+        done += run(args.warmup + k)
+    el = time.perf_counter() - t0
+    val = done / el
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * el / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD,
+                   "step": "fp64 CPU oracle on %d rows per step (bounded sample of the workload)" % rows},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": "%d rows per step x %d steps, full vocabulary, forward + fp64 gradient"
+                                   % (rows, args.steps)},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+def run_cuda(args):
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2509_06980_b200 import binding as rlf
+
+    spec = synth.scaled(synth.SPECS[1], seed=shard_seed(synth.SPECS[1].seed, rank))
+    if args.tokens_per_response:
+        spec = synth.scaled(spec, len_lo=args.tokens_per_response, len_hi=args.tokens_per_response)
+    batch = synth.make_batch(spec, dev)
+    T, V, B = batch.T, spec.V, batch.B
+    G = batch.tokens.group_size
+
+    # CPU baseline first (rank 0, one GPU only): the oracle on a bounded sample of this workload
+    cpu_baseline = None
+    if rank == 0 and world == 1 and args.cpu_seconds > 0:
+        cpu_baseline = time_oracle(batch, args.cpu_seconds)
+
+    grad = torch.empty_like(batch.logits)
+    mask = torch.empty(T, dtype=torch.uint8, device=dev)
+    seq_id = torch.empty(T, dtype=torch.int32, device=dev)
+    n_tok = torch.empty(1, dtype=torch.int64, device=dev)
+    adv = torch.empty(B, dtype=torch.float32, device=dev)
+    logp = torch.empty(T, dtype=torch.float32, device=dev)
+    loss = torch.empty(4, dtype=torch.float64, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = rlf.new_workspace(rlf.FN_LOGP_LOSS, T, V, 0, rlf.RLF_BF16, dev)
+
+    def step(ev=None):
+        rlf.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, spec.open_id, spec.close_id, mask_out=mask,
+                                seq_id_out=seq_id, n_out=n_tok, dev_status=status)
+        rlf.rlf_group_advantage(batch.rewards, group_size=G, eps=1e-6, adv_out=adv, dev_status=status)
+        if ev is not None:
+            ev[0].record()
+        rlf.rlf_grpo_logp_loss_fwd_bwd(batch.logits, batch.ids, seq_id, adv, batch.old_logp, batch.ref_logp, mask,
+                                       synth.EPS_CLIP, synth.BETA_KL, denom=n_tok, grad_logits=grad,
+                                       logp_out=logp, loss_out=loss, workspace=ws, dev_status=status)
+        if ev is not None:
+            ev[1].record()
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = rlf.launch_count()
+    barrier()
+    e0.record()
+    for k in range(args.steps):
+        step(kev[k])
+    e1.record()
+    barrier()
+    launches = rlf.launch_count() - launches0
+    ms_total = e0.elapsed_time(e1)
+    kernel_ms = [a.elapsed_time(b) for a, b in kev]
+    time.sleep(0.25)
+    clocks = sampler.stop()
+    if status.item() != 0:
+        raise SystemExit("device status %d after the timed region" % status.item())
+
+    ms_total_max = max_over_ranks(ms_total, world, dev)
+    value = aggregate(T * args.steps, world, ms_total_max / 1e3)
+
+    # end to end through the host-buffer entry point: inputs start in pinned host memory, the loss
+    # (and per-token log-probs) come back to the host, every step
+    e2e = None
+    if not args.no_e2e:
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        h_logits = torch.empty((T, V), dtype=torch.bfloat16).pin_memory()
+        h_logits.copy_(batch.logits)
+        pin = lambda t: t.cpu().contiguous().pin_memory()
+        h_ids, h_cu, h_rw = pin(batch.ids), pin(batch.cu_seqlens), pin(batch.rewards)
+        h_old, h_ref = pin(batch.old_logp), pin(batch.ref_logp)
+        h_loss = torch.zeros(4, dtype=torch.float64).pin_memory()
+        h_logp = torch.zeros(T, dtype=torch.float32).pin_memory()
+        h_st = torch.zeros(1, dtype=torch.int32).pin_memory()
+        del grad
+        arena = torch.empty(rlf.step_arena_bytes(T, V, B), dtype=torch.uint8, device=dev)
+
+        def host_step():
+            rlf.rlf_grpo_step_host(h_logits, h_ids, h_cu, G, h_rw, h_old, h_ref, spec.open_id, spec.close_id, 1e-6,
+                                   synth.EPS_CLIP, synth.BETA_KL, h_loss, arena, h_logp_out=h_logp, h_dev_status=h_st)
+        host_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            host_step()              # waits for its stream before returning
+        barrier()
+        el = max_over_ranks(time.perf_counter() - t0, world, dev)
+        h2d = T * V * 2 + T * 4 * 3 + (B + 1) * 4 + B * 4
+        d2h = 4 * 8 + T * 4 + 4
+        e2e = {"value": aggregate(T * e2e_steps, world, el), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+               "loss": float(h_loss[0].item())}
+
+    if rank != 0:
+        return
+    peak, peak_kind = _peaks()
+    k_ms = statistics.mean(kernel_ms)
+    alg_bytes = T * V * 4                      # bf16 logits read once + bf16 grad written once
+    achieved = alg_bytes / (k_ms * 1e-3) / 1e9
+    traffic = None
+    if NCU_TRAFFIC["dram_bytes_per_token"] and NCU_TRAFFIC["logits_loss_cu_sha1"] == _kernel_sha1():
+        traffic = NCU_TRAFFIC["dram_bytes_per_token"] * T
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": ms_total_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD if not args.tokens_per_response
+                   else "cfg1 recipe at %d tokens per response" % args.tokens_per_response,
+                   "T": T, "V": V, "B": B, "G": G, "eps_clip": synth.EPS_CLIP, "beta_kl": synth.BETA_KL,
+                   "arithmetic": "bf16 in/out, fp32 accumulate, fp64 loss sum",
+                   "l2": "inputs (%.1f GB per step) exceed L2; no flush needed" % (T * V * 2 / 1e9),
+                   "grad": "out of place",
+                   "parallelism": "independent micro-batch per GPU" if world > 1 else "single GPU"},
+        "logits_gbs": achieved,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": "of " + peak_kind, "frac_of_nominal_8tbs": achieved / 8000.0, "traffic": traffic,
+                     "kernel": "grpo_row_cluster_kernel (timed as the rlf_grpo_logp_loss_fwd_bwd call: "
+                               "row kernel + 3 sub-10us kernels)",
+                     "kernel_ms": k_ms, "kernel_ms_min": min(kernel_ms), "algorithmic_bytes": alg_bytes},
+        "gpu_launches": int(launches),
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"]},
+        "loss": float(loss[0].item()),
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if cpu_baseline is not None:
+        line["cpu_baseline"] = cpu_baseline
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="time budget of the CPU-oracle baseline leg")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--tokens-per-response", type=int, default=0,
+                    help="smaller micro-batch of the same recipe (profiling captures); 0 = the full 2048")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+        if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+            import torch.distributed as dist
+            if dist.is_initialized():
+                dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -20,6 +20,8 @@
 //   5. every thread merges the <= 8 triples, forms lse, logp and the loss coefficient c_t, and
 //      writes grad = c_t (softmax - onehot) from the registers it still holds, either as
 //      exp2(z log2e + log2|c_t| - lse log2e) (two-exp) or as e * 2^(...) (one-exp).
+// Exponents are formed by one FFMA per element; rows whose maximum is huge in magnitude switch to
+// a subtract-first form so that the result stays accurate for any finite logits.
 // Several CTAs are resident per SM, so the loads of one row overlap the arithmetic of another.
 // The next row's token record is fetched with a 16-byte cp.async while the current row is
 // processed, so no scalar input costs a register across the passes.
@@ -171,6 +173,44 @@ __device__ __forceinline__ void put_elem(uint4& v, int e, float x) {
     if (w == 3) v.w = (v.w & keep) | ins;
 }
 
+// exponent of one element.  Fast form: one FFMA, z log2e + off with off = -m log2e rounded to fp32,
+// accurate while |m| is moderate (the rounding of off is an absolute error of |m| 2^-24 log2e in
+// the exponent).  Robust form for rows with a huge maximum: (z - m) log2e + add, subtraction first.
+constexpr float kRobustAbove = 2048.0f;
+template <bool ROBUST>
+__device__ __forceinline__ float expo(float z, float m, float off) {
+    return ROBUST ? fmaf(z - m, kLog2e, off) : fmaf(z, kLog2e, off);
+}
+
+// sum of 2^expo over this thread's registers; ONE_EXP keeps the exponentials in place as bf16
+template <int NV, bool ONE_EXP, bool ROBUST>
+__device__ __forceinline__ float exp_sum_pass(uint4 (&d)[NV], float m, float off) {
+    float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+        uint32_t* w = reinterpret_cast<uint32_t*>(&d[i]);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float e0 = ex2_approx(expo<ROBUST>(bf_lo(w[k]), m, off));
+            const float e1 = ex2_approx(expo<ROBUST>(bf_hi(w[k]), m, off));
+            s0 += e0;
+            s1 += e1;
+            if (ONE_EXP) w[k] = pack_bf16x2(e0, e1);
+        }
+    }
+    return s0 + s1;
+}
+
+template <bool ROBUST>
+__device__ __forceinline__ uint4 grad_vec_two_exp(const uint4& v, float m, float off, uint32_t sgn) {
+    uint4 o;
+    o.x = pack_bf16x2(ex2_approx(expo<ROBUST>(bf_lo(v.x), m, off)), ex2_approx(expo<ROBUST>(bf_hi(v.x), m, off))) ^ sgn;
+    o.y = pack_bf16x2(ex2_approx(expo<ROBUST>(bf_lo(v.y), m, off)), ex2_approx(expo<ROBUST>(bf_hi(v.y), m, off))) ^ sgn;
+    o.z = pack_bf16x2(ex2_approx(expo<ROBUST>(bf_lo(v.z), m, off)), ex2_approx(expo<ROBUST>(bf_hi(v.z), m, off))) ^ sgn;
+    o.w = pack_bf16x2(ex2_approx(expo<ROBUST>(bf_lo(v.w), m, off)), ex2_approx(expo<ROBUST>(bf_hi(v.w), m, off))) ^ sgn;
+    return o;
+}
+
 template <int THREADS, int NV, bool ONE_EXP>
 __global__ void __launch_bounds__(THREADS, 65536 / (64 * THREADS))
 grpo_row_cluster_kernel(const FastParams p) {
@@ -226,22 +266,12 @@ grpo_row_cluster_kernel(const FastParams p) {
         }
         float m_w = fmaxf(bf_lo(mx), bf_hi(mx));
         m_w = ord2f(__reduce_max_sync(0xffffffffu, f2ord(m_w)));
-        const float off = (m_w == -INFINITY) ? 0.0f : -m_w * kLog2e;
-
-        float s0 = 0.0f, s1 = 0.0f;
-#pragma unroll
-        for (int i = 0; i < NV; ++i) {
-            uint32_t* w = reinterpret_cast<uint32_t*>(&d[i]);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float e0 = ex2_approx(fmaf(bf_lo(w[k]), kLog2e, off));
-                const float e1 = ex2_approx(fmaf(bf_hi(w[k]), kLog2e, off));
-                s0 += e0;
-                s1 += e1;
-                if (ONE_EXP) w[k] = pack_bf16x2(e0, e1);
-            }
-        }
-        const float s_w = warp_sum(s0 + s1);
+        // exponent base of this warp: 2^((z - m_w) log2e); all lanes agree on the form
+        const float m_ws = (m_w == -INFINITY) ? 0.0f : m_w;
+        const bool robust_w = fabsf(m_ws) > kRobustAbove;
+        const float s_t = robust_w ? exp_sum_pass<NV, ONE_EXP, true>(d, m_ws, 0.0f)
+                                   : exp_sum_pass<NV, ONE_EXP, false>(d, 0.0f, -m_ws * kLog2e);
+        const float s_w = warp_sum(s_t);
         if (lane == 0) warp_slot[warp] = make_float2(m_w, s_w);
         if (tid == 0) cp_async_wait_all();
         __syncthreads();
@@ -272,7 +302,6 @@ grpo_row_cluster_kernel(const FastParams p) {
         }
         const float4 rec = rec_slot[parity];
         const float lg2s = lg2_approx(S);
-        const float lse2 = fmaf(M, kLog2e, lg2s);            // log2-domain lse for the exponent
         const float logp = (zy - M) - lg2s * kLn2;
         const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) &&
                             (fabsf(logp) < INFINITY);
@@ -291,11 +320,12 @@ grpo_row_cluster_kernel(const FastParams p) {
                 for (int i = 0; i < NV; ++i)
                     if (vbeg + i * THREADS < vend) st_stream(dst + i * THREADS, z4);
             } else {
-                // grad = sign(c) 2^(z log2e + c2), c2 = log2|c| - lse2; the target column gets -c on top
-                const float c2 = lg2_approx(fabsf(coef)) - lse2;
-                const float gy = fmaf(coef, ex2_approx(fmaf(zy, kLog2e, -lse2)), -coef);   // c (p_y - 1)
+                // grad = sign(c) 2^((z - M) log2e + lc), lc = log2|c| - log2 S; the target column gets -c on top
+                const float lc = lg2_approx(fabsf(coef)) - lg2s;
+                const float gy = fmaf(coef, ex2_approx(fmaf(zy - M, kLog2e, -lg2s)), -coef);   // c (p_y - 1)
                 if (ONE_EXP) {
-                    const float scale = copysignf(ex2_approx(c2 - off), coef);
+                    // the registers hold 2^((z - m_w) log2e): rescale from the warp's base to the row's
+                    const float scale = copysignf(ex2_approx(fmaf(m_ws - M, kLog2e, lc)), coef);
 #pragma unroll
                     for (int i = 0; i < NV; ++i) {
                         if (vbeg + i * THREADS < vend) {
@@ -310,18 +340,13 @@ grpo_row_cluster_kernel(const FastParams p) {
                     }
                 } else {
                     const uint32_t sgn = coef < 0.0f ? 0x80008000u : 0u;
+                    const bool robust_r = fabsf(M) > kRobustAbove;
+                    const float c2 = lc - M * kLog2e;
 #pragma unroll
                     for (int i = 0; i < NV; ++i) {
                         if (vbeg + i * THREADS < vend) {
-                            uint4 o;
-                            o.x = pack_bf16x2(ex2_approx(fmaf(bf_lo(d[i].x), kLog2e, c2)),
-                                              ex2_approx(fmaf(bf_hi(d[i].x), kLog2e, c2))) ^ sgn;
-                            o.y = pack_bf16x2(ex2_approx(fmaf(bf_lo(d[i].y), kLog2e, c2)),
-                                              ex2_approx(fmaf(bf_hi(d[i].y), kLog2e, c2))) ^ sgn;
-                            o.z = pack_bf16x2(ex2_approx(fmaf(bf_lo(d[i].z), kLog2e, c2)),
-                                              ex2_approx(fmaf(bf_hi(d[i].z), kLog2e, c2))) ^ sgn;
-                            o.w = pack_bf16x2(ex2_approx(fmaf(bf_lo(d[i].w), kLog2e, c2)),
-                                              ex2_approx(fmaf(bf_hi(d[i].w), kLog2e, c2))) ^ sgn;
+                            uint4 o = robust_r ? grad_vec_two_exp<true>(d[i], M, lc, sgn)
+                                               : grad_vec_two_exp<false>(d[i], 0.0f, c2, sgn);
                             if (vbeg + i * THREADS == (y >> 3)) put_elem(o, y & 7, gy);
                             st_stream(dst + i * THREADS, o);
                         }
@@ -387,9 +412,9 @@ grpo_row_general_kernel(const GenParams p) {
         }
         __syncthreads();
         const float M = bcast;
-        const float off = (M == -INFINITY) ? 0.0f : -M * kLog2e;
+        const float Ms = (M == -INFINITY) ? 0.0f : M;
         float s = 0.0f;
-        for (int v = tid; v < p.V; v += kGenThreads) s += ex2_approx(fmaf(to_f32<T>(z[v]), kLog2e, off));
+        for (int v = tid; v < p.V; v += kGenThreads) s += ex2_approx((to_f32<T>(z[v]) - Ms) * kLog2e);
         s = warp_sum(s);
         __syncthreads();
         if (lane == 0) red[warp] = s;
@@ -404,7 +429,6 @@ grpo_row_general_kernel(const GenParams p) {
         __syncthreads();
 
         const float lg2s = lg2_approx(S);
-        const float lse2 = fmaf(M, kLog2e, lg2s);
         const float logp = (zy - M) - lg2s * kLn2;
         const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) &&
                             (fabsf(logp) < INFINITY);
@@ -420,7 +444,7 @@ grpo_row_general_kernel(const GenParams p) {
                 for (int v = tid; v < p.V; v += kGenThreads) g[v] = from_f32<T>(0.0f);
             } else {
                 for (int v = tid; v < p.V; v += kGenThreads) {
-                    const float pv = ex2_approx(fmaf(to_f32<T>(z[v]), kLog2e, -lse2));
+                    const float pv = ex2_approx(fmaf(to_f32<T>(z[v]) - M, kLog2e, -lg2s));
                     const float gv = (v == y) ? fmaf(coef, pv, -coef) : coef * pv;
                     g[v] = from_f32<T>(gv);
                 }

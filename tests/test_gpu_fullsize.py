@@ -1,0 +1,90 @@
+"""Full-size parity in the launch configuration the benchmark times: the Qwen3-4B-shaped micro-batch
+(32768 x 151936 bf16, out of place).  The scalar loss and every row's log-prob are compared with
+the oracle run over all rows; grad_logits is compared element by element on sampled rows (rows are
+independent given the batch's token count), plus properties that hold at any size on all rows."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2509_06980_b200 import synth
+import gpu_common as gc
+from util import loss_close, ulp_error_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def test_cfg1_full_size_against_oracle():
+    dev = "cuda"
+    batch = synth.make_batch(synth.SPECS[1], dev)
+    T, V = batch.logits.shape
+    assert (T, V) == (32768, 151936)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    gpu = gc.gpu_chain(batch, batch.logits, dev_status=st)
+    assert st.item() == 0
+
+    # all rows: log-prob and scalar loss (oracle forward over the whole batch)
+    z_np = gc.to_np(batch.logits)
+    ora = gc.oracle_chain(batch, z_np, want_grad=False)
+    assert np.array_equal(gpu["mask"].cpu().numpy(), ora["mask"]) and gpu["n"].item() == ora["n"]
+    assert np.abs(gpu["logp"].cpu().numpy() - ora["logp"]).max() <= gc.LOGP_ATOL
+    lg = gpu["loss"].cpu().numpy()
+    for k in range(3):
+        assert loss_close(lg[k], ora["loss"][k], 1e-6, gc.LOSS_RTOL), (k, lg, ora["loss"])
+
+    # sampled rows: gradient element by element
+    rng = np.random.default_rng(0)
+    rows = np.unique(np.concatenate([[0, 1, T - 1], rng.integers(0, T, size=93)]))
+    sub = gc.oracle_chain(batch, z_np, want_grad=True, rows=rows)
+    g = gc.grad_to_f64(gpu["grad"][torch.as_tensor(rows, device=dev)])
+    guard = gc.near_clip_bound(sub["logp"], batch.old_logp.cpu().numpy()[rows], None)
+    ulps = ulp_error_bf16(g[~guard], sub["grad"][~guard])
+    assert ulps.max() <= gc.GRAD_ULPS
+    assert (g[ora["mask"][rows] == 0] == 0).all()
+
+    # all rows: masked rows are zero; live rows sum to ~0 (bf16 rounding noise only)
+    grad = gpu["grad"]
+    m = gpu["mask"].bool()
+    coef_scale = np.abs(ora["coef"]).max()
+    for r0 in range(0, T, 4096):
+        blk = grad[r0:r0 + 4096]
+        mb = m[r0:r0 + 4096]
+        assert not blk[~mb].any()
+        assert blk[mb].float().sum(dim=1).abs().max().item() <= 0.05 * coef_scale
+
+
+def test_cfg2_ragged_sampled_rows():
+    """Ragged varlen packing (64 responses, lengths 256..4096): tokens and masks at full size, logits
+    for a sampled subset of rows (parity needs only independent rows and the batch's token count)."""
+    dev = "cuda"
+    spec = synth.SPECS[2]
+    tok = synth.make_tokens(spec)
+    T = len(tok.ids)
+    b = gc.binding()
+    ids = torch.from_numpy(tok.ids).to(dev)
+    cu = torch.from_numpy(tok.cu_seqlens).to(dev)
+    mask, seq, n = b.rlf_build_loss_mask(ids, cu, spec.open_id, spec.close_id)
+    adv = b.rlf_group_advantage(torch.from_numpy(tok.rewards).to(dev), group_size=spec.group_size)
+    torch.cuda.synchronize()
+    from oracle import rlf_oracle as orc
+    m_o, s_o, n_o = orc.build_loss_mask(tok.ids, tok.cu_seqlens, spec.open_id, spec.close_id)
+    assert np.array_equal(mask.cpu().numpy(), m_o) and np.array_equal(seq.cpu().numpy(), s_o) and n.item() == n_o
+    assert n_o == T - tok.n_span_tokens
+
+    rng = np.random.default_rng(1)
+    rows = np.sort(rng.choice(T, size=600, replace=False))
+    sub = synth.scaled(spec, seed=77)
+    logits = synth.make_logits(sub, len(rows), dev)
+    rows_t = torch.as_tensor(rows, device=dev)
+    ids_s, seq_s, mask_s = ids[rows_t].contiguous(), seq[rows_t].contiguous(), mask[rows_t].contiguous()
+    center = synth.center_logp(logits, ids_s)
+    old, ref = synth.perturbed_logps(sub, center)
+    logp, loss, grad = b.rlf_grpo_logp_loss_fwd_bwd(logits, ids_s, seq_s, adv, old, ref, mask_s, synth.EPS_CLIP,
+                                                    synth.BETA_KL, denom=n, in_place=False)
+    torch.cuda.synchronize()
+    a_o = orc.group_advantage(tok.rewards, group_size=spec.group_size, eps=1e-6).astype(np.float32)
+    r = orc.grpo_loss(gc.to_np(logits), tok.ids[rows], s_o[rows], a_o, old.cpu().numpy(), ref.cpu().numpy(),
+                      m_o[rows], synth.EPS_CLIP, synth.BETA_KL, denom=n_o)
+    assert np.abs(logp.cpu().numpy() - r["logp"]).max() <= gc.LOGP_ATOL
+    assert loss_close(loss[0].item(), r["loss"][0], 1e-9, gc.LOSS_RTOL)
+    guard = gc.near_clip_bound(r["logp"], old.cpu().numpy(), None)
+    assert ulp_error_bf16(gc.grad_to_f64(grad)[~guard], r["grad"][~guard]).max() <= gc.GRAD_ULPS
