@@ -167,8 +167,11 @@ static void token_terms(double logp, double old_lp, double ref_lp, double A, dou
     *dkl = 1.0 - exp(d);
 }
 
-/* log-softmax statistics of one row: max, log-sum-exp. */
-static double row_lse(const void *logits, int dtype, int64_t off, int32_t V)
+/* log-softmax statistics of one row: m = max_v z, and log s with s = sum_v exp(z - m), so that
+ * lse = m + log s.  The two parts are returned separately and every use below subtracts m from a
+ * logit FIRST, (z - m) - log s: the same quantity as z - lse, but it keeps full precision when
+ * |m| is so large that m + log s would absorb log s. */
+static void row_stats(const void *logits, int dtype, int64_t off, int32_t V, double *m_out, double *logs_out)
 {
     double m = -INFINITY;
     for (int32_t v = 0; v < V; ++v) {
@@ -178,7 +181,8 @@ static double row_lse(const void *logits, int dtype, int64_t off, int32_t V)
     double s = 0.0;
     for (int32_t v = 0; v < V; ++v)
         s += exp(widen(logits, dtype, off + v) - m);
-    return m + log(s);
+    *m_out = m;
+    *logs_out = log(s);
 }
 
 /*
@@ -219,8 +223,9 @@ int orc_grpo_loss(const void *logits, int dtype, int64_t T, int32_t V, int64_t r
             bad = 1;
             continue;
         }
-        double lse = row_lse(logits, dtype, off, V);
-        double logp = widen(logits, dtype, off + y) - lse;
+        double m, logs;
+        row_stats(logits, dtype, off, V, &m, &logs);
+        double logp = (widen(logits, dtype, off + y) - m) - logs;
         logp_out[t] = logp;
         double A = (double)adv[seq_id[t]];
         double pg, kl, dpg, dkl;
@@ -235,7 +240,7 @@ int orc_grpo_loss(const void *logits, int dtype, int64_t T, int32_t V, int64_t r
         if (coef_out) coef_out[t] = -g;
         if (grad) {
             for (int32_t v = 0; v < V; ++v) {
-                double p = exp(widen(logits, dtype, off + v) - lse);
+                double p = exp((widen(logits, dtype, off + v) - m) - logs);
                 grad[t * (int64_t)V + v] = g * ((v == y ? 1.0 : 0.0) - p);
             }
         }
