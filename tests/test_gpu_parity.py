@@ -132,12 +132,12 @@ def test_extreme_logits_and_targets_at_the_ends():
         finally:
             b.tune_logits_kernel(0, 0, -1)
         r = orc.grpo_loss(zn, ids.cpu().numpy(), seq.cpu().numpy(), adv.cpu().numpy(), old.cpu().numpy(),
-                          ref.cpu().numpy(), mask.cpu().numpy(), 0.2, 0.01)
+                          ref.cpu().numpy(), mask.cpu().numpy(), 0.2, 0.01, want_coef=True)
         assert st.item() == 0
         assert np.abs(logp.cpu().numpy() - r["logp"]).max() <= gc.LOGP_ATOL * 4   # |logp| up to 400
         assert abs(logp[0].item() + np.log(V)) < 1e-3
         from util import ulp_error_bf16, loss_close
-        assert ulp_error_bf16(gc.grad_to_f64(grad), r["grad"]).max() <= gc.GRAD_ULPS
+        assert gc.grad_ulps(gc.grad_to_f64(grad), r["grad"], ids.cpu().numpy(), r["coef"]).max() <= gc.GRAD_ULPS
         assert loss_close(loss[0].item(), r["loss"][0], 1e-6, 1e-4)
 
 
