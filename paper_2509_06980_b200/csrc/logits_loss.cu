@@ -11,7 +11,10 @@
 // Fast row kernel (bf16, 16-byte aligned rows).  A thread-block cluster owns one logits row at a
 // time and keeps the WHOLE row in registers as packed bf16 (NV 16-byte vectors per thread), so the
 // row crosses HBM exactly once in each direction:
-//   1. every thread issues its NV coalesced 16-byte loads back to back (all in flight at once);
+//   1. every thread copies its NV coalesced 16-byte vectors of the NEXT row into its own slots of
+//      a shared-memory staging buffer with cp.async (no registers held, no barrier needed: a
+//      thread only reads back what it copied itself), then pulls the CURRENT row from the other
+//      buffer into registers, so HBM reads of row r+1 run under all the arithmetic of row r;
 //   2. packed bf16x2 max over the registers, warp max by one redux;
 //   3. one exp2 per element against the WARP's max, fp32 sum, warp sum by shuffles; in the
 //      one-exp variant the exponentials replace the logits in the registers (packed bf16);
@@ -22,9 +25,8 @@
 //      exp2(z log2e + log2|c_t| - lse log2e) (two-exp) or as e * 2^(...) (one-exp).
 // Exponents are formed by one FFMA per element; rows whose maximum is huge in magnitude switch to
 // a subtract-first form so that the result stays accurate for any finite logits.
-// Several CTAs are resident per SM, so the loads of one row overlap the arithmetic of another.
-// The next row's token record is fetched with a 16-byte cp.async while the current row is
-// processed, so no scalar input costs a register across the passes.
+// Token records ride the same cp.async groups two rows ahead, so no scalar input costs a register
+// across the passes.
 //
 // General row kernel (fp32 logits, odd V, unaligned rows): one CTA per row, three sweeps with
 // scalar loads (max, sum, gradient); later sweeps of a row are served by L2 when the row fits.
@@ -138,6 +140,11 @@ __device__ __forceinline__ void st_cluster_f4(uint32_t local_addr, uint32_t rank
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" :: "r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
 }
+__device__ __forceinline__ void cp_async16_cg(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_group1() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
 constexpr uint32_t kNegInfPair = 0xFF80FF80u;   // two bf16 -inf
@@ -211,13 +218,26 @@ __device__ __forceinline__ uint4 grad_vec_two_exp(const uint4& v, float m, float
     return o;
 }
 
+// Resident CTAs per SM: bounded by registers (64 per thread) and by the two staging buffers.
+constexpr int kSmemBudget = 220 * 1024;
+constexpr int stage_bytes(int threads, int nv) { return 2 * nv * threads * 16; }
+constexpr int ctas_per_sm(int threads, int nv) {
+    const int by_regs = 65536 / (64 * threads);
+    const int by_smem = kSmemBudget / (stage_bytes(threads, nv) + 1024);
+    const int m = by_regs < by_smem ? by_regs : by_smem;
+    return m < 1 ? 1 : m;
+}
+
 template <int THREADS, int NV, bool ONE_EXP>
-__global__ void __launch_bounds__(THREADS, 65536 / (64 * THREADS))
+__global__ void __launch_bounds__(THREADS, ctas_per_sm(THREADS, NV))
 grpo_row_cluster_kernel(const FastParams p) {
     constexpr int NWARPS = THREADS / 32;
+    // staging: [2 buffers][NV][THREADS] 16-byte slots; each thread only ever touches its own slots,
+    // so a thread's cp.async.wait_group is all the synchronisation the logits data needs
+    extern __shared__ __align__(16) uint4 stage[];
     __shared__ float2 warp_slot[NWARPS];
     __shared__ __align__(16) float4 cl_slot[2][8];   // per parity, per peer: (max, sum, z_target, -)
-    __shared__ __align__(16) float4 rec_slot[2];
+    __shared__ __align__(16) float4 rec_slot[4];     // token records, ring over rows
     __shared__ float zy_local[2];
 
     const int csize = (int)cluster_nctarank();
@@ -235,29 +255,53 @@ grpo_row_cluster_kernel(const FastParams p) {
         const long long N = *p.denom;
         inv_n = 1.0f / (float)(N > 1 ? N : 1);
     }
+
+    // queue this thread's part of a row into staging buffer `buf` (one cp.async group per row;
+    // thread 0's group also carries the token record of the row after it)
+    auto prefetch = [&](int row, int buf, int it) {
+        if (row < p.T) {
+            const uint4* src = reinterpret_cast<const uint4*>(p.logits + (long long)row * p.stride) + vbeg;
+            uint4* dst = stage + (size_t)buf * NV * THREADS + tid;
+#pragma unroll
+            for (int i = 0; i < NV; ++i)
+                if (vbeg + i * THREADS < vend) cp_async16_cg(dst + i * THREADS, src + i * THREADS);
+        }
+        if (tid == 0 && row + num_clusters < p.T)
+            cp_async16(&rec_slot[(it + 1) & 3], p.rec + row + num_clusters);
+        cp_async_commit();
+    };
+
     if (tid == 0) {
         zy_local[0] = -INFINITY;
         zy_local[1] = -INFINITY;
         if (cluster_id < p.T) cp_async16(&rec_slot[0], p.rec + cluster_id);
-        cp_async_wait_all();
     }
-    __syncthreads();
+    prefetch(cluster_id, 0, 0);          // row 0 of this cluster (+ record of row 1)
+    cp_async_wait_all();
+    // every CTA of the cluster is running (and its shared memory initialised) before any peer
+    // may address it
+    cluster_sync_all();
 
     int status = 0;
-    int parity = 0;
-    for (int row = cluster_id; row < p.T; row += num_clusters, parity ^= 1) {
-        const uint4* src = reinterpret_cast<const uint4*>(p.logits + (long long)row * p.stride) + vbeg;
+    int it = 0;
+    for (int row = cluster_id; row < p.T; row += num_clusters, ++it) {
+        const int parity = it & 1;
+        // next row of this cluster goes to the other buffer while this one is processed
+        prefetch(row + num_clusters, parity ^ 1, it + 1);
+        cp_async_wait_group1();          // everything but the group just queued has landed
         uint4 d[NV];
+        {
+            const uint4* own = stage + (size_t)parity * NV * THREADS + tid;
 #pragma unroll
-        for (int i = 0; i < NV; ++i) {
-            if (vbeg + i * THREADS < vend) d[i] = ld_stream(src + i * THREADS);
-            else d[i] = make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
+            for (int i = 0; i < NV; ++i) {
+                if (vbeg + i * THREADS < vend) d[i] = own[i * THREADS];
+                else d[i] = make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
+            }
         }
-        if (tid == 0 && row + num_clusters < p.T) cp_async16(&rec_slot[parity ^ 1], p.rec + row + num_clusters);
 
         // max over the registers (packed), then over the warp; the owner of the target column
         // publishes z_target to its CTA
-        const int y = __float_as_int(rec_slot[parity].w) & 0x7fffffff;
+        const int y = __float_as_int(rec_slot[it & 3].w) & 0x7fffffff;
         uint32_t mx = kNegInfPair;
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
@@ -273,7 +317,6 @@ grpo_row_cluster_kernel(const FastParams p) {
                                    : exp_sum_pass<NV, ONE_EXP, false>(d, 0.0f, -m_ws * kLog2e);
         const float s_w = warp_sum(s_t);
         if (lane == 0) warp_slot[warp] = make_float2(m_w, s_w);
-        if (tid == 0) cp_async_wait_all();
         __syncthreads();
 
         if (warp == 0) {
@@ -300,7 +343,7 @@ grpo_row_cluster_kernel(const FastParams p) {
             const float4 ms = cl_slot[parity][r];
             if (ms.x != -INFINITY) S += ms.y * ex2_approx((ms.x - M) * kLog2e);
         }
-        const float4 rec = rec_slot[parity];
+        const float4 rec = rec_slot[it & 3];
         const float lg2s = lg2_approx(S);
         const float logp = (zy - M) - lg2s * kLn2;
         const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) &&
@@ -604,7 +647,7 @@ static void cluster_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* at, int
     *cfg = cudaLaunchConfig_t{};
     cfg->gridDim = dim3(grid);
     cfg->blockDim = dim3(sh.threads);
-    cfg->dynamicSmemBytes = 0;
+    cfg->dynamicSmemBytes = (size_t)stage_bytes(sh.threads, sh.nv);
     cfg->stream = s;
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = sh.cluster;
@@ -614,23 +657,31 @@ static void cluster_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* at, int
     cfg->numAttrs = 1;
 }
 
-// how many clusters of this shape can be resident at once (cached per kernel and cluster size)
+// how many clusters of this shape can be resident at once; also opts the kernel in to its staging
+// buffers.  Cached per device, kernel and cluster size.
 static int max_clusters(FastKernel k, const FastShape& sh) {
     static std::mutex mu;
-    static struct { FastKernel k; int cluster; int n; } cache[64];
+    static struct { int dev; FastKernel k; int cluster; int n; } cache[128];
     static int ncache = 0;
+    int dev = 0;
+    cudaGetDevice(&dev);
     std::lock_guard<std::mutex> lock(mu);
     for (int i = 0; i < ncache; ++i)
-        if (cache[i].k == k && cache[i].cluster == sh.cluster) return cache[i].n;
+        if (cache[i].dev == dev && cache[i].k == k && cache[i].cluster == sh.cluster) return cache[i].n;
+    if (cudaFuncSetAttribute((const void*)k, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             stage_bytes(sh.threads, sh.nv)) != cudaSuccess) {
+        cudaGetLastError();
+        return -1;
+    }
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute at[1];
     cluster_config(&cfg, at, sh.cluster * sm_count() * 8, sh, nullptr);
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, (void*)k, &cfg) != cudaSuccess || n <= 0) {
         cudaGetLastError();
-        n = sm_count() / sh.cluster;
+        return -1;
     }
-    if (ncache < 64) cache[ncache++] = {k, sh.cluster, n};
+    if (ncache < 128) cache[ncache++] = {dev, k, sh.cluster, n};
     return n;
 }
 
@@ -680,6 +731,7 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
             FastKernel k = fast_kernel(sh);
             if (!k) return RLF_ERR_UNSUPPORTED;
             int nc = max_clusters(k, sh);
+            if (nc <= 0) return RLF_ERR_UNSUPPORTED;      // this shape does not fit on the device
             if ((int64_t)nc > a.T) nc = (int)a.T;
             FastParams p;
             p.logits = static_cast<const __nv_bfloat16*>(a.logits);
