@@ -11,18 +11,19 @@
 // Fast row kernel (bf16, 16-byte aligned rows).  A thread-block cluster owns one logits row at a
 // time and keeps the WHOLE row in registers as packed bf16 (NV 16-byte vectors per thread), so the
 // row crosses HBM exactly once in each direction:
-//   1. every thread copies its NV coalesced 16-byte vectors of the NEXT row into its own slots of
-//      a shared-memory staging buffer with cp.async (no registers held, no barrier needed: a
-//      thread only reads back what it copied itself), then pulls the CURRENT row from the other
-//      buffer into registers, so HBM reads of row r+1 run under all the arithmetic of row r;
-//   2. packed bf16x2 max over the registers, warp max by one redux;
-//   3. one exp2 per element against the WARP's max, fp32 sum, warp sum by shuffles; in the
+//   1. cp.async brings each thread's NV coalesced 16-byte vectors into its own slots of a
+//      shared-memory staging buffer (no registers held, no barrier: a thread only reads back what
+//      it copied itself); the thread pulls them into registers, takes the packed bf16x2 max, and
+//      immediately re-queues the same slots with the cluster's NEXT row, so HBM reads of row r+1
+//      run under the rest of row r;
+//   2. one exp2 per element against the WARP's max, fp32 sum, warp sum by shuffles; in the
 //      one-exp variant the exponentials replace the logits in the registers (packed bf16);
-//   4. warps -> CTA through shared memory; CTA -> cluster by pushing (max, sum, z_target) into every
-//      peer's shared memory (distributed-shared-memory stores) and ONE cluster barrier per row;
-//   5. every thread merges the <= 8 triples, forms lse, logp and the loss coefficient c_t, and
-//      writes grad = c_t (softmax - onehot) from the registers it still holds, either as
-//      exp2(z log2e + log2|c_t| - lse log2e) (two-exp) or as e * 2^(...) (one-exp).
+//   3. every warp stores its (max, sum) into every CTA of the cluster (distributed-shared-memory
+//      stores), the owner of the target column likewise sends z_target, and ONE cluster barrier
+//      per row follows; there is no other barrier in the loop;
+//   4. every warp merges all pairs of the row (lanes in parallel), forms lse, logp and the loss
+//      coefficient c_t, and writes grad = c_t (softmax - onehot) from the registers it still
+//      holds, either as exp2(z log2e + log2|c_t| - lse log2e) (two-exp) or as e * 2^(...) (one-exp).
 // Exponents are formed by one FFMA per element; rows whose maximum is huge in magnitude switch to
 // a subtract-first form so that the result stays accurate for any finite logits.
 // Token records ride the same cp.async groups two rows ahead, so no scalar input costs a register
@@ -218,33 +219,45 @@ __device__ __forceinline__ uint4 grad_vec_two_exp(const uint4& v, float m, float
     return o;
 }
 
-// Resident CTAs per SM: bounded by registers (64 per thread) and by the two staging buffers.
+// Resident CTAs per SM: bounded by registers (64 per thread) and by the staging buffer.
 constexpr int kSmemBudget = 220 * 1024;
-constexpr int stage_bytes(int threads, int nv) { return 2 * nv * threads * 16; }
+constexpr int stage_bytes(int threads, int nv) { return nv * threads * 16; }
 constexpr int ctas_per_sm(int threads, int nv) {
     const int by_regs = 65536 / (64 * threads);
-    const int by_smem = kSmemBudget / (stage_bytes(threads, nv) + 1024);
+    const int by_smem = kSmemBudget / (stage_bytes(threads, nv) + 4096);
     const int m = by_regs < by_smem ? by_regs : by_smem;
     return m < 1 ? 1 : m;
+}
+
+__device__ __forceinline__ void st_cluster_f2(uint32_t local_addr, uint32_t rank, float a, float b) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" :: "r"(remote), "f"(a), "f"(b) : "memory");
+}
+__device__ __forceinline__ void st_cluster_f1(uint32_t local_addr, uint32_t rank, float a) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" :: "r"(remote), "f"(a) : "memory");
 }
 
 template <int THREADS, int NV, bool ONE_EXP>
 __global__ void __launch_bounds__(THREADS, ctas_per_sm(THREADS, NV))
 grpo_row_cluster_kernel(const FastParams p) {
     constexpr int NWARPS = THREADS / 32;
-    // staging: [2 buffers][NV][THREADS] 16-byte slots; each thread only ever touches its own slots,
-    // so a thread's cp.async.wait_group is all the synchronisation the logits data needs
+    constexpr int MAXE = 8 * NWARPS;          // (max, sum) pairs per row: one per warp of the cluster
+    // staging: [NV][THREADS] 16-byte slots; a thread only ever touches its own slots, so its own
+    // cp.async wait is all the synchronisation the logits data needs
     extern __shared__ __align__(16) uint4 stage[];
-    __shared__ float2 warp_slot[NWARPS];
-    __shared__ __align__(16) float4 cl_slot[2][8];   // per parity, per peer: (max, sum, z_target, -)
-    __shared__ __align__(16) float4 rec_slot[4];     // token records, ring over rows
-    __shared__ float zy_local[2];
+    __shared__ __align__(8) float2 pair_slot[2][MAXE];   // per row parity: every warp's (max, sum)
+    __shared__ __align__(16) float4 rec_slot[4];         // token records, ring over rows
+    __shared__ float zy_slot[2];                         // per row parity: the target logit
 
     const int csize = (int)cluster_nctarank();
     const int crank = (int)cluster_ctarank();
     const int cluster_id = blockIdx.x / csize;
     const int num_clusters = gridDim.x / csize;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int npairs = csize * NWARPS;
 
     // this thread's vectors are  vbeg + i * THREADS  for i < NV, live while < vend
     const int vbeg = crank * p.per_cta_vec + tid;
@@ -256,58 +269,55 @@ grpo_row_cluster_kernel(const FastParams p) {
         inv_n = 1.0f / (float)(N > 1 ? N : 1);
     }
 
-    // queue this thread's part of a row into staging buffer `buf` (one cp.async group per row;
-    // thread 0's group also carries the token record of the row after it)
-    auto prefetch = [&](int row, int buf, int it) {
+    // queue this thread's part of a row into the staging buffer (one cp.async group per row;
+    // thread 0's group also carries the token record of the row after it, into ring slot `rslot`)
+    auto prefetch = [&](int row, int rslot) {
         if (row < p.T) {
             const uint4* src = reinterpret_cast<const uint4*>(p.logits + (long long)row * p.stride) + vbeg;
-            uint4* dst = stage + (size_t)buf * NV * THREADS + tid;
+            uint4* dst = stage + tid;
 #pragma unroll
             for (int i = 0; i < NV; ++i)
                 if (vbeg + i * THREADS < vend) cp_async16_cg(dst + i * THREADS, src + i * THREADS);
         }
         if (tid == 0 && row + num_clusters < p.T)
-            cp_async16(&rec_slot[(it + 1) & 3], p.rec + row + num_clusters);
+            cp_async16(&rec_slot[rslot & 3], p.rec + row + num_clusters);
         cp_async_commit();
     };
 
-    if (tid == 0) {
-        zy_local[0] = -INFINITY;
-        zy_local[1] = -INFINITY;
-        if (cluster_id < p.T) cp_async16(&rec_slot[0], p.rec + cluster_id);
-    }
-    prefetch(cluster_id, 0, 0);          // row 0 of this cluster (+ record of row 1)
-    cp_async_wait_all();
-    // every CTA of the cluster is running (and its shared memory initialised) before any peer
-    // may address it
+    if (tid == 0 && cluster_id < p.T) cp_async16(&rec_slot[0], p.rec + cluster_id);
+    prefetch(cluster_id, 1);             // first row of this cluster (+ record of its second row)
+    cp_async_wait_all();                 // the first two records must be visible CTA-wide below
+    // every CTA of the cluster is running before any peer may address its shared memory
     cluster_sync_all();
 
     int status = 0;
     int it = 0;
     for (int row = cluster_id; row < p.T; row += num_clusters, ++it) {
         const int parity = it & 1;
-        // next row of this cluster goes to the other buffer while this one is processed
-        prefetch(row + num_clusters, parity ^ 1, it + 1);
-        cp_async_wait_group1();          // everything but the group just queued has landed
+        cp_async_wait_all();             // this thread's part of the row has landed
         uint4 d[NV];
-        {
-            const uint4* own = stage + (size_t)parity * NV * THREADS + tid;
 #pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                if (vbeg + i * THREADS < vend) d[i] = own[i * THREADS];
-                else d[i] = make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
-            }
+        for (int i = 0; i < NV; ++i) {
+            if (vbeg + i * THREADS < vend) d[i] = stage[i * THREADS + tid];
+            else d[i] = make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
         }
 
         // max over the registers (packed), then over the warp; the owner of the target column
-        // publishes z_target to its CTA
+        // sends z_target to every CTA of the cluster
         const int y = __float_as_int(rec_slot[it & 3].w) & 0x7fffffff;
         uint32_t mx = kNegInfPair;
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
             mx = max_bf16x2(mx, max_bf16x2(max_bf16x2(d[i].x, d[i].y), max_bf16x2(d[i].z, d[i].w)));
-            if (vbeg + i * THREADS == (y >> 3)) zy_local[parity] = pick_elem(d[i], y & 7);
+            if (vbeg + i * THREADS == (y >> 3) && vbeg + i * THREADS < vend) {
+                const float zt = pick_elem(d[i], y & 7);
+                for (int r = 0; r < csize; ++r) st_cluster_f1(smem_u32(&zy_slot[parity]), (uint32_t)r, zt);
+            }
         }
+        // the staging slots have been consumed (the max needed every register): refill them with
+        // the cluster's next row while this one is processed
+        prefetch(row + num_clusters, it + 2);
+
         float m_w = fmaxf(bf_lo(mx), bf_hi(mx));
         m_w = ord2f(__reduce_max_sync(0xffffffffu, f2ord(m_w)));
         // exponent base of this warp: 2^((z - m_w) log2e); all lanes agree on the form
@@ -316,33 +326,27 @@ grpo_row_cluster_kernel(const FastParams p) {
         const float s_t = robust_w ? exp_sum_pass<NV, ONE_EXP, true>(d, m_ws, 0.0f)
                                    : exp_sum_pass<NV, ONE_EXP, false>(d, 0.0f, -m_ws * kLog2e);
         const float s_w = warp_sum(s_t);
-        if (lane == 0) warp_slot[warp] = make_float2(m_w, s_w);
-        __syncthreads();
-
-        if (warp == 0) {
-            const float2 ms = (lane < NWARPS) ? warp_slot[lane] : make_float2(-INFINITY, 0.0f);
-            const float m_c = ord2f(__reduce_max_sync(0xffffffffu, f2ord(ms.x)));
-            const float sc = (ms.x == -INFINITY) ? 0.0f : ms.y * ex2_approx((ms.x - m_c) * kLog2e);
-            const float s_c = warp_sum(sc);
-            const float zyl = zy_local[parity];
-            __syncwarp();
-            if (lane == 0) zy_local[parity] = -INFINITY;
-            if (lane < csize)
-                st_cluster_f4(smem_u32(&cl_slot[parity][crank]), (uint32_t)lane, make_float4(m_c, s_c, zyl, 0.0f));
-        }
+        // every warp hands its (max, sum) to every CTA of the cluster; one barrier per row
+        if (lane < csize)
+            st_cluster_f2(smem_u32(&pair_slot[parity][crank * NWARPS + warp]), (uint32_t)lane, m_w, s_w);
         cluster_sync_all();
 
-        // merge the cluster's triples; every thread does this redundantly
-        float M = -INFINITY, zy = -INFINITY;
-        for (int r = 0; r < csize; ++r) {
-            M = fmaxf(M, cl_slot[parity][r].x);
-            zy = fmaxf(zy, cl_slot[parity][r].z);
+        // merge all pairs of the row, lanes in parallel, identically in every warp
+        float M = -INFINITY;
+        float2 e[MAXE / 32 > 0 ? MAXE / 32 : 1];
+#pragma unroll
+        for (int j = 0; j < (MAXE + 31) / 32; ++j) {
+            const int k = lane + 32 * j;
+            e[j] = (k < npairs) ? pair_slot[parity][k] : make_float2(-INFINITY, 0.0f);
+            M = fmaxf(M, e[j].x);
         }
+        M = ord2f(__reduce_max_sync(0xffffffffu, f2ord(M)));
         float S = 0.0f;
-        for (int r = 0; r < csize; ++r) {
-            const float4 ms = cl_slot[parity][r];
-            if (ms.x != -INFINITY) S += ms.y * ex2_approx((ms.x - M) * kLog2e);
-        }
+#pragma unroll
+        for (int j = 0; j < (MAXE + 31) / 32; ++j)
+            if (e[j].x != -INFINITY) S += e[j].y * ex2_approx((e[j].x - M) * kLog2e);
+        S = warp_sum(S);
+        const float zy = zy_slot[parity];
         const float4 rec = rec_slot[it & 3];
         const float lg2s = lg2_approx(S);
         const float logp = (zy - M) - lg2s * kLn2;
@@ -579,7 +583,7 @@ static int round_nv(int need) {
 // launch shape that holds a row of nvec 16-byte vectors in registers
 static bool pick_shape(int nvec, FastShape* out) {
     const int tc = g_tune_cluster.load(), tt = g_tune_threads.load();
-    const int oe = g_tune_one_exp.load() < 0 ? 0 : g_tune_one_exp.load();
+    const int oe = g_tune_one_exp.load() < 0 ? 1 : g_tune_one_exp.load();
     if (tc > 0 && tt > 0) {
         const int per = (nvec + tc - 1) / tc;
         const int nv = round_nv((per + tt - 1) / tt);
@@ -587,17 +591,17 @@ static bool pick_shape(int nvec, FastShape* out) {
         *out = {tc, tt, nv, oe};
         return true;
     }
-    // built-in choice: the smallest cluster whose CTAs need <= 5 vectors per thread
-    const int th = nvec <= 256 * 5 ? 256 : 512;
-    for (int c = 1; c <= 8; c *= 2) {
-        const int per = (nvec + c - 1) / c;
-        const int need = (per + th - 1) / th;
-        if (need <= 5) { *out = {c, th, round_nv(need), oe}; return true; }
-    }
-    for (int c = 1; c <= 8; c *= 2) {
-        const int per = (nvec + c - 1) / c;
-        const int need = (per + 1024 - 1) / 1024;
-        if (need <= 10) { *out = {c, 1024, round_nv(need), oe}; return true; }
+    // built-in choice: 256-thread CTAs holding up to 10 vectors per thread (four CTAs per SM), in
+    // the smallest cluster that covers the row; wider CTAs only for rows beyond 8 x 256 x 10 vectors
+    for (int th = 256; th <= 1024; th *= 2) {
+        for (int c = 1; c <= 8; c *= 2) {
+            const int per = (nvec + c - 1) / c;
+            const int need = (per + th - 1) / th;
+            if (need <= 10 && stage_bytes(th, round_nv(need)) <= kSmemBudget) {
+                *out = {c, th, round_nv(need), oe};
+                return true;
+            }
+        }
     }
     return false;
 }
@@ -658,7 +662,7 @@ static void cluster_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* at, int
 }
 
 // how many clusters of this shape can be resident at once; also opts the kernel in to its staging
-// buffers.  Cached per device, kernel and cluster size.
+// buffer.  Cached per device, kernel and cluster size.
 static int max_clusters(FastKernel k, const FastShape& sh) {
     static std::mutex mu;
     static struct { int dev; FastKernel k; int cluster; int n; } cache[128];
