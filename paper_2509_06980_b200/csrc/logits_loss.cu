@@ -18,9 +18,11 @@
 //      run under the rest of row r;
 //   2. one exp2 per element against the WARP's max, fp32 sum, warp sum by shuffles; in the
 //      one-exp variant the exponentials replace the logits in the registers (packed bf16);
-//   3. every warp stores its (max, sum) into every CTA of the cluster (distributed-shared-memory
-//      stores), the owner of the target column likewise sends z_target, and ONE cluster barrier
-//      per row follows; there is no other barrier in the loop;
+//   3. every warp stores its (max, sum) into every CTA of the cluster and the owner of the target
+//      column likewise sends z_target, as asynchronous distributed-shared-memory stores that credit
+//      an mbarrier in the receiving CTA; each warp then waits (bounded) on its own CTA's mbarrier
+//      for the row's byte count.  There is no thread barrier and no memory fence in the loop, so
+//      a row's exchange never waits for the previous row's gradient stores to drain;
 //   4. every warp merges all pairs of the row (lanes in parallel), forms lse, logp and the loss
 //      coefficient c_t, and writes grad = c_t (softmax - onehot) from the registers it still
 //      holds, either as exp2(z log2e + log2|c_t| - lse log2e) (two-exp) or as e * 2^(...) (one-exp).
@@ -229,15 +231,41 @@ constexpr int ctas_per_sm(int threads, int nv) {
     return m < 1 ? 1 : m;
 }
 
-__device__ __forceinline__ void st_cluster_f2(uint32_t local_addr, uint32_t rank, float a, float b) {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    asm volatile("st.shared::cluster.v2.f32 [%0], {%1,%2};" :: "r"(remote), "f"(a), "f"(b) : "memory");
+// Asynchronous stores into the shared memory of CTA `rank` of this cluster: the data is written to
+// the peer's copy of `local_addr` and its byte count is credited to the peer's copy of the mbarrier
+// at `local_mbar`, which is how the peer learns that it has arrived (no fence, no thread barrier).
+__device__ __forceinline__ void st_async_f2(uint32_t local_addr, uint32_t local_mbar, uint32_t rank, float a, float b) {
+    uint32_t raddr, rbar;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(local_addr), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(local_mbar), "r"(rank));
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
+                 :: "r"(raddr), "f"(a), "f"(b), "r"(rbar) : "memory");
 }
-__device__ __forceinline__ void st_cluster_f1(uint32_t local_addr, uint32_t rank, float a) {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
-    asm volatile("st.shared::cluster.f32 [%0], %1;" :: "r"(remote), "f"(a) : "memory");
+__device__ __forceinline__ void st_async_f1(uint32_t local_addr, uint32_t local_mbar, uint32_t rank, float a) {
+    uint32_t raddr, rbar;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(local_addr), "r"(rank));
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(local_mbar), "r"(rank));
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];"
+                 :: "r"(raddr), "f"(a), "r"(rbar) : "memory");
+}
+__device__ __forceinline__ void mbar_init(uint32_t mbar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(mbar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t mbar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(mbar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t mbar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait for one phase of an mbarrier: false when it gives up (about a second).
+constexpr int kWaitPolls = 1 << 22;
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t mbar, uint32_t parity) {
+    for (int i = 0; i < kWaitPolls; ++i)
+        if (mbar_try_wait(mbar, parity)) return true;
+    return false;
 }
 
 template <int THREADS, int NV, bool ONE_EXP>
@@ -251,6 +279,7 @@ grpo_row_cluster_kernel(const FastParams p) {
     __shared__ __align__(8) float2 pair_slot[2][MAXE];   // per row parity: every warp's (max, sum)
     __shared__ __align__(16) float4 rec_slot[4];         // token records, ring over rows
     __shared__ float zy_slot[2];                         // per row parity: the target logit
+    __shared__ __align__(8) unsigned long long row_bar[2];   // per row parity: "all pairs and z_target are here"
 
     const int csize = (int)cluster_nctarank();
     const int crank = (int)cluster_ctarank();
@@ -262,6 +291,8 @@ grpo_row_cluster_kernel(const FastParams p) {
     // this thread's vectors are  vbeg + i * THREADS  for i < NV, live while < vend
     const int vbeg = crank * p.per_cta_vec + tid;
     const int vend = min(p.nvec, (crank + 1) * p.per_cta_vec);
+    // number of live vectors of this thread (they are the first nvalid of the NV), same for every row
+    const int nvalid = vend > vbeg ? min(NV, (vend - vbeg + THREADS - 1) / THREADS) : 0;
 
     float inv_n;
     {
@@ -277,14 +308,21 @@ grpo_row_cluster_kernel(const FastParams p) {
             uint4* dst = stage + tid;
 #pragma unroll
             for (int i = 0; i < NV; ++i)
-                if (vbeg + i * THREADS < vend) cp_async16_cg(dst + i * THREADS, src + i * THREADS);
+                if (i < nvalid) cp_async16_cg(dst + i * THREADS, src + i * THREADS);
         }
         if (tid == 0 && row + num_clusters < p.T)
             cp_async16(&rec_slot[rslot & 3], p.rec + row + num_clusters);
         cp_async_commit();
     };
 
-    if (tid == 0 && cluster_id < p.T) cp_async16(&rec_slot[0], p.rec + cluster_id);
+    // per row every CTA receives one (max, sum) pair from every warp of the cluster and z_target
+    const uint32_t row_bytes = (uint32_t)npairs * 8u + 4u;
+    if (tid == 0) {
+        mbar_init(smem_u32(&row_bar[0]), 1);
+        mbar_init(smem_u32(&row_bar[1]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (cluster_id < p.T) cp_async16(&rec_slot[0], p.rec + cluster_id);
+    }
     prefetch(cluster_id, 1);             // first row of this cluster (+ record of its second row)
     cp_async_wait_all();                 // the first two records must be visible CTA-wide below
     // every CTA of the cluster is running before any peer may address its shared memory
@@ -292,27 +330,33 @@ grpo_row_cluster_kernel(const FastParams p) {
 
     int status = 0;
     int it = 0;
+    bool gave_up = false;                // a wait ran out: stop waiting, finish the loop, report
     for (int row = cluster_id; row < p.T; row += num_clusters, ++it) {
         const int parity = it & 1;
+        const uint32_t bar = smem_u32(&row_bar[parity]);
+        if (tid == 0) mbar_arrive_expect_tx(bar, row_bytes);
         cp_async_wait_all();             // this thread's part of the row has landed
         uint4 d[NV];
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
-            if (vbeg + i * THREADS < vend) d[i] = stage[i * THREADS + tid];
+            if (i < nvalid) d[i] = stage[i * THREADS + tid];
             else d[i] = make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
         }
 
         // max over the registers (packed), then over the warp; the owner of the target column
         // sends z_target to every CTA of the cluster
         const int y = __float_as_int(rec_slot[it & 3].w) & 0x7fffffff;
+        const int yrel = (y >> 3) - vbeg;             // owner iff a multiple of THREADS below nvalid * THREADS
+        const bool owner = yrel >= 0 && (yrel & (THREADS - 1)) == 0 && (yrel / THREADS) < nvalid;
         uint32_t mx = kNegInfPair;
 #pragma unroll
-        for (int i = 0; i < NV; ++i) {
+        for (int i = 0; i < NV; ++i)
             mx = max_bf16x2(mx, max_bf16x2(max_bf16x2(d[i].x, d[i].y), max_bf16x2(d[i].z, d[i].w)));
-            if (vbeg + i * THREADS == (y >> 3) && vbeg + i * THREADS < vend) {
-                const float zt = pick_elem(d[i], y & 7);
-                for (int r = 0; r < csize; ++r) st_cluster_f1(smem_u32(&zy_slot[parity]), (uint32_t)r, zt);
-            }
+        if (owner) {
+            // the target logit still sits in this thread's staging slot
+            const __nv_bfloat16* sv = reinterpret_cast<const __nv_bfloat16*>(&stage[yrel + tid]);
+            const float zt = __bfloat162float(sv[y & 7]);
+            for (int r = 0; r < csize; ++r) st_async_f1(smem_u32(&zy_slot[parity]), bar, (uint32_t)r, zt);
         }
         // the staging slots have been consumed (the max needed every register): refill them with
         // the cluster's next row while this one is processed
@@ -326,10 +370,14 @@ grpo_row_cluster_kernel(const FastParams p) {
         const float s_t = robust_w ? exp_sum_pass<NV, ONE_EXP, true>(d, m_ws, 0.0f)
                                    : exp_sum_pass<NV, ONE_EXP, false>(d, 0.0f, -m_ws * kLog2e);
         const float s_w = warp_sum(s_t);
-        // every warp hands its (max, sum) to every CTA of the cluster; one barrier per row
+        // every warp hands its (max, sum) to every CTA of the cluster, then waits until its own CTA
+        // has received the whole row's worth (the only synchronisation in the loop)
         if (lane < csize)
-            st_cluster_f2(smem_u32(&pair_slot[parity][crank * NWARPS + warp]), (uint32_t)lane, m_w, s_w);
-        cluster_sync_all();
+            st_async_f2(smem_u32(&pair_slot[parity][crank * NWARPS + warp]), bar, (uint32_t)lane, m_w, s_w);
+        if (!gave_up && !mbar_wait_bounded(bar, (uint32_t)(it >> 1) & 1u)) {
+            gave_up = true;
+            status |= RLF_DEV_TIMEOUT;
+        }
 
         // merge all pairs of the row, lanes in parallel, identically in every warp
         float M = -INFINITY;
@@ -365,7 +413,7 @@ grpo_row_cluster_kernel(const FastParams p) {
                 const uint4 z4 = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
                 for (int i = 0; i < NV; ++i)
-                    if (vbeg + i * THREADS < vend) st_stream(dst + i * THREADS, z4);
+                    if (i < nvalid) st_stream(dst + i * THREADS, z4);
             } else {
                 // grad = sign(c) 2^((z - M) log2e + lc), lc = log2|c| - log2 S; the target column gets -c on top
                 const float lc = lg2_approx(fabsf(coef)) - lg2s;
@@ -375,13 +423,12 @@ grpo_row_cluster_kernel(const FastParams p) {
                     const float scale = copysignf(ex2_approx(fmaf(m_ws - M, kLog2e, lc)), coef);
 #pragma unroll
                     for (int i = 0; i < NV; ++i) {
-                        if (vbeg + i * THREADS < vend) {
+                        if (i < nvalid) {
                             uint4 o;
                             o.x = pack_bf16x2(bf_lo(d[i].x) * scale, bf_hi(d[i].x) * scale);
                             o.y = pack_bf16x2(bf_lo(d[i].y) * scale, bf_hi(d[i].y) * scale);
                             o.z = pack_bf16x2(bf_lo(d[i].z) * scale, bf_hi(d[i].z) * scale);
                             o.w = pack_bf16x2(bf_lo(d[i].w) * scale, bf_hi(d[i].w) * scale);
-                            if (vbeg + i * THREADS == (y >> 3)) put_elem(o, y & 7, gy);
                             st_stream(dst + i * THREADS, o);
                         }
                     }
@@ -391,14 +438,15 @@ grpo_row_cluster_kernel(const FastParams p) {
                     const float c2 = lc - M * kLog2e;
 #pragma unroll
                     for (int i = 0; i < NV; ++i) {
-                        if (vbeg + i * THREADS < vend) {
+                        if (i < nvalid) {
                             uint4 o = robust_r ? grad_vec_two_exp<true>(d[i], M, lc, sgn)
                                                : grad_vec_two_exp<false>(d[i], 0.0f, c2, sgn);
-                            if (vbeg + i * THREADS == (y >> 3)) put_elem(o, y & 7, gy);
                             st_stream(dst + i * THREADS, o);
                         }
                     }
                 }
+                // the owner overwrites the target column of the vector it has just stored
+                if (owner) p.grad[(long long)row * p.stride + y] = __float2bfloat16_rn(gy);
             }
         }
     }
