@@ -44,7 +44,8 @@ typedef enum {
     RLF_ERR_WORKSPACE = -5, /* workspace NULL, misaligned or smaller than rlf_workspace_bytes() */
     RLF_ERR_ARCH = -6,      /* current device is not sm_100 */
     RLF_ERR_CUDA = -7,      /* a CUDA runtime call failed (launch, memset, copy) */
-    RLF_ERR_UNSUPPORTED = -8 /* valid request outside what this build implements */
+    RLF_ERR_UNSUPPORTED = -8, /* valid request outside what this build implements */
+    RLF_ERR_TOO_LARGE = -9   /* more tokens than the built-in scratch of a *_static entry point holds */
 } rlf_status;
 
 typedef enum { RLF_BF16 = 0, RLF_F32 = 1 } rlf_dtype;
@@ -145,6 +146,40 @@ rlf_status rlf_grpo_logp_loss_fwd_bwd(const void *logits, rlf_dtype dt, int64_t 
                                       const int64_t *denom, float *logp_out, double *loss_out,
                                       void *grad_logits, void *workspace, size_t workspace_bytes,
                                       int32_t *dev_status, rlf_stream_t stream);
+
+/*
+ * rlf_grpo_logp_loss_fwd_bwd without a workspace argument, for callers that cannot allocate.
+ * (The paper has no counterpart: this is a packaging variant of the entry point above.)
+ *
+ * Who needs it: code that sits where device allocation is not an option -- a training-loop thread
+ * that must not trigger the device-wide synchronisation cudaMalloc / cudaFree imply, a process
+ * whose framework has already claimed all device memory for its own pool, or a plug-in that has
+ * no handle on the host framework's allocator.  Such a caller still owns every input and output
+ * buffer; only the kernels' scratch (token records and partial sums) moves into the library.
+ *
+ * The scratch is a fixed array in the library's device image, RLF_STATIC_MAX_TOKENS tokens large
+ * (about 1.1 MB; every GPU that loads the library holds it until the process exits).  This call
+ * allocates nothing, on the device or through any library: T > RLF_STATIC_MAX_TOKENS returns
+ * RLF_ERR_TOO_LARGE before anything is queued.  All other arguments, results and errors are
+ * those of rlf_grpo_logp_loss_fwd_bwd, and the same kernels run.
+ *
+ * The first call on each device looks the array's device address up (one runtime query, made with
+ * that device current, its result checked and remembered); make that first call outside any stream
+ * capture.  Every call on a device uses the same array: it keeps the previous call's contents,
+ * which is harmless (each call rewrites what it reads and zeroes its token counter itself), but
+ * two calls whose kernels overlap on the GPU -- different streams without an ordering between
+ * them -- race on it.  Serialise such calls or give the second one its own workspace through
+ * rlf_grpo_logp_loss_fwd_bwd.
+ */
+#define RLF_STATIC_MAX_TOKENS 65536
+rlf_status rlf_grpo_logp_loss_fwd_bwd_static(const void *logits, rlf_dtype dt, int64_t T, int32_t V,
+                                             int64_t row_stride, const int32_t *ids,
+                                             const int32_t *seq_id, const float *adv, int32_t B,
+                                             const float *old_logp, const float *ref_logp,
+                                             const uint8_t *mask, float eps_clip, float beta_kl,
+                                             const int64_t *denom, float *logp_out,
+                                             double *loss_out, void *grad_logits,
+                                             int32_t *dev_status, rlf_stream_t stream);
 
 /*
  * Same loss with the logits formed on the fly, z = hidden W^T, so that they

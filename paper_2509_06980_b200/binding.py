@@ -19,7 +19,7 @@ DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
 
 EXPORTS = [
     "rlf_build_loss_mask", "rlf_group_advantage", "rlf_grpo_logp_loss_fwd_bwd",
-    "rlf_fused_lmhead_grpo", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
+    "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_fused_lmhead_grpo", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
     "rlf_tune_logits_kernel", "rlf_launch_count", "rlf_status_string", "rlf_version",
 ]
 
@@ -36,6 +36,9 @@ _lib.rlf_build_loss_mask.argtypes = [_vp, _vp, _i32, _i64, _i32, _i32, _vp, _vp,
 _lib.rlf_group_advantage.argtypes = [_vp, _vp, _i32, _i32, _f32, _int, _vp, _vp, _vp]
 _lib.rlf_grpo_logp_loss_fwd_bwd.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _i32, _vp, _vp, _vp,
                                             _f32, _f32, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+_lib.rlf_grpo_logp_loss_fwd_bwd_static.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _i32, _vp, _vp, _vp,
+                                                   _f32, _f32, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.rlf_grpo_logp_loss_fwd_bwd_static.restype = _int
 _lib.rlf_fused_lmhead_grpo.argtypes = [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _f32,
                                        _f32, _vp, _vp, _vp, _vp, _vp, _int, _vp, _sz, _vp, _vp]
 _lib.rlf_workspace_bytes.argtypes = [_int, _i64, _i32, _i32, _int]
@@ -177,6 +180,27 @@ def rlf_grpo_logp_loss_fwd_bwd(logits, ids, seq_id, adv, old_logp, ref_logp, mas
         _ptr(denom, torch.int64), _ptr(logp_out, torch.float32), _ptr(loss_out, torch.float64),
         None if grad_logits is None else grad_logits.data_ptr(), workspace.data_ptr(), workspace.numel(),
         _ptr(dev_status, torch.int32), _stream()), "rlf_grpo_logp_loss_fwd_bwd")
+    return logp_out, loss_out, grad_logits
+
+
+STATIC_MAX_TOKENS = 65536
+
+
+def rlf_grpo_logp_loss_fwd_bwd_static(logits, ids, seq_id, adv, old_logp, ref_logp, mask, eps_clip, beta_kl,
+                                      denom, logp_out, loss_out, grad_logits=None, dev_status=None):
+    """The loss entry point for callers that cannot allocate: no workspace argument (the scratch is a
+    fixed array inside the library, at most STATIC_MAX_TOKENS tokens) and, unlike the wrapper above,
+    this wrapper creates no tensor either: every output buffer is passed in.  Calls on one device
+    share the scratch, so do not let two of them overlap on the GPU."""
+    T, V = logits.shape
+    stride = logits.stride(0) if T > 1 else V
+    _check(_lib.rlf_grpo_logp_loss_fwd_bwd_static(
+        logits.data_ptr() if T > 0 else None, _dt(logits), T, V, stride, _ptr(ids, torch.int32),
+        _ptr(seq_id, torch.int32), _ptr(adv, torch.float32), adv.shape[0], _ptr(old_logp, torch.float32),
+        _ptr(ref_logp, torch.float32), _ptr(mask, torch.uint8), float(eps_clip), float(beta_kl),
+        _ptr(denom, torch.int64), _ptr(logp_out, torch.float32), _ptr(loss_out, torch.float64),
+        None if grad_logits is None else grad_logits.data_ptr(), _ptr(dev_status, torch.int32), _stream()),
+        "rlf_grpo_logp_loss_fwd_bwd_static")
     return logp_out, loss_out, grad_logits
 
 

@@ -877,3 +877,49 @@ extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd(
                          aligned(logits, 16) && aligned(grad_logits, 16);
     return launch_logits_loss(a, fast_ok, workspace, reinterpret_cast<cudaStream_t>(stream));
 }
+
+// ---------------------------------------------------------------------------------------------
+// Variant for callers that cannot allocate: the scratch lives in the library's device image.
+namespace rlf {
+
+constexpr size_t kStaticScratchBytes = kWsRecordOff + 16 * (size_t)RLF_STATIC_MAX_TOKENS + 256;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of the scratch array on the current device.  In host code the array's name only
+// stands for the symbol; the address a kernel can use comes from the runtime, per device.
+static rlf_status static_scratch_ptr(void** out) {
+    static std::mutex mu;
+    static void* ptr_of_device[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return RLF_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return RLF_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(mu);
+    if (ptr_of_device[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) {
+            cudaGetLastError();
+            return RLF_ERR_CUDA;
+        }
+        ptr_of_device[dev] = ptr;
+    }
+    *out = ptr_of_device[dev];
+    return RLF_OK;
+}
+
+}  // namespace rlf
+
+extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd_static(
+    const void* logits, rlf_dtype dt, int64_t T, int32_t V, int64_t row_stride, const int32_t* ids,
+    const int32_t* seq_id, const float* adv, int32_t B, const float* old_logp, const float* ref_logp,
+    const uint8_t* mask, float eps_clip, float beta_kl, const int64_t* denom, float* logp_out,
+    double* loss_out, void* grad_logits, int32_t* dev_status, rlf_stream_t stream) {
+    if (T > RLF_STATIC_MAX_TOKENS) return RLF_ERR_TOO_LARGE;
+    rlf_status st = rlf::check_arch();
+    if (st != RLF_OK) return st;
+    void* scratch = nullptr;
+    st = rlf::static_scratch_ptr(&scratch);
+    if (st != RLF_OK) return st;
+    return rlf_grpo_logp_loss_fwd_bwd(logits, dt, T, V, row_stride, ids, seq_id, adv, B, old_logp, ref_logp,
+                                      mask, eps_clip, beta_kl, denom, logp_out, loss_out, grad_logits,
+                                      scratch, rlf::kStaticScratchBytes, dev_status, stream);
+}
