@@ -15,6 +15,14 @@ void count_launch(int n = 1);
 // RLF_OK iff the current device is compute capability 10.x
 rlf_status check_arch();
 
+// token-record and scalar-loss stages (logits_loss.cu), also used by the fused LM-head path
+rlf_status launch_token_prep(const int32_t* ids, const int32_t* seq_id, const float* adv, const float* old_logp,
+                             const float* ref_logp, const uint8_t* mask, int64_t T, int32_t V, int32_t B,
+                             void* rec, long long* n_count_or_null, int32_t* dev_status, cudaStream_t s);
+rlf_status launch_token_loss(const float* logp, const void* rec, int64_t T, float eps_clip, float beta,
+                             double* partial, const long long* denom, double* loss_out, cudaStream_t s);
+size_t token_loss_partial_bytes();
+
 inline rlf_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? RLF_OK : RLF_ERR_CUDA; }
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }

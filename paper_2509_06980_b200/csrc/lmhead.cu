@@ -1,14 +1,713 @@
-// Fused LM-head variant (placeholder until the tcgen05 kernels land).
+// Fused LM-head variant: the logits z = hidden W^T are formed tile by tile on the tensor cores
+// (tcgen05.mma, operands staged in shared memory by TMA, accumulators in tensor memory) and consumed
+// by the softmax / loss epilogue straight from tensor memory, so they never reach HBM.
+//
+// One warp-specialised kernel template serves four contractions (all bf16 x bf16 -> fp32):
+//   LSE   z tile = H W^T, epilogue keeps a running (max, sum exp) per token      -> log-sum-exp
+//   DZ    z tile recomputed, epilogue turns it into dZ = c_t (softmax - onehot)  -> bf16 scratch
+//   GH    grad_hidden = dZ W      (A = dZ K-major, B = W vocabulary-major rows: N-major operand)
+//   GW    grad_W     += dZ^T H    (both operands token-major rows: M-/N-major operands)
+// CTA = 192 threads: warp 0 issues TMA loads into a 4-stage ring (48 KB per stage), warp 1 issues
+// the MMAs (one thread) into a double-buffered 128 x 256 fp32 accumulator (all 512 TMEM columns),
+// warps 2..5 drain the accumulator with tcgen05.ld (one token row per thread) while the next tile
+// is being multiplied.  Every mbarrier wait is bounded; a wait that runs out raises a CTA-wide
+// abort flag, all roles leave their loops, tensor memory is released and RLF_DEV_TIMEOUT is set.
+//
+// Backward is by token chunks: DZ writes a [chunk, V] bf16 scratch, GH and GW read it.  The
+// logits themselves are never stored; the dZ scratch is (stated in the entry point's contract).
+#include <cuda.h>
+
+#include <mutex>
+
 #include "common.cuh"
 
 namespace rlf {
-size_t lmhead_workspace_bytes(int64_t, int32_t, int32_t) { return 0; }
+namespace lm {
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int kStages = 4;
+constexpr int kABytes = BM * BK * 2;
+constexpr int kBBytes = BN * BK * 2;
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+constexpr int kSlabBytes = 64 * BK * 2;      // one 64-wide slab of an MN-major operand: 64 k-rows of 128 B
+
+enum Mode { kLse = 0, kDz = 1, kGradHidden = 2, kGradW = 3 };
+
+struct GemmParams {
+    int mode;
+    int M, N;                 // extent of the output tile grid in rows / columns (valid elements)
+    int m_tiles, n_tiles, k_slabs;
+    int nsplit, n_tiles_per_split;
+    float2* part;             // kLse: [M][nsplit] (max, sum exp)
+    const float* lse;         // kDz: per row of this launch
+    const float* coef;
+    const int32_t* ids;
+    __nv_bfloat16* dz;        // kDz out, row stride dz_stride
+    long long dz_stride;
+    __nv_bfloat16* out_bf16;  // kGradHidden out [M][out_stride]
+    float* out_f32;           // kGradW out [M][out_stride]
+    long long out_stride;
+    int accumulate;
+    int32_t* dev_status;
+};
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+constexpr int kWaitPolls = 1 << 22;
+// bounded wait; on failure (or if another role already gave up) returns false
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (int i = 0; i < kWaitPolls; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 1023) == 1023 && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 :: "r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                   "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                   "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory operand descriptor, 128-byte swizzle, descriptor version 1.
+//   K-major tile  (rows of 64 bf16 = 128 B, 8-row groups 1024 B apart): LBO 1, SBO 1024 B.
+//   MN-major tile (64-wide slabs, each 64 k-rows of 128 B): LBO = slab pitch 8192 B, SBO 1024 B.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major) {
+    const uint64_t lbo = mn_major ? (uint64_t)(kSlabBytes >> 4) : 1ull;
+    return (uint64_t)((addr & 0x3FFFF) >> 4) | (lbo << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+           (2ull << 61);
+}
+// Instruction descriptor: D fp32, A and B bf16, M = 128, N = 256, majorness per operand.
+__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+           ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+struct SmemCtl {
+    unsigned long long full[kStages];
+    unsigned long long empty[kStages];
+    unsigned long long tmem_full[2];
+    unsigned long long tmem_empty[2];
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+
+// ---- the kernel -----------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const GemmParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    // operand stages must sit on 1024-byte boundaries (swizzle atom)
+    const uint32_t raw = smem_addr(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;
+    SmemCtl* ctl = reinterpret_cast<SmemCtl*>(smem_raw + (tiles - raw) + kStages * kStageBytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool a_mn = p.mode == kGradW;
+    const bool b_mn = p.mode == kGradHidden || p.mode == kGradW;
+    const bool sweep = p.mode == kLse || p.mode == kDz;     // a unit sweeps several vocabulary tiles
+    const int units = sweep ? p.m_tiles * p.nsplit : p.m_tiles * p.n_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_addr(&ctl->full[s]), 1);
+            mbar_init(smem_addr(&ctl->empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_addr(&ctl->tmem_full[b]), 1);
+            mbar_init(smem_addr(&ctl->tmem_empty[b]), 4);
+        }
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     :: "r"(smem_addr(&ctl->tmem_base)), "r"((uint32_t)kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    // unit -> (m tile, first n tile, one-past-last n tile)
+    auto unit_range = [&](int u, int& m, int& n0, int& n1) {
+        if (sweep) {
+            m = u % p.m_tiles;
+            const int sp = u / p.m_tiles;
+            n0 = sp * p.n_tiles_per_split;
+            n1 = min(p.n_tiles, n0 + p.n_tiles_per_split);
+        } else {
+            m = u % p.m_tiles;
+            n0 = u / p.m_tiles;
+            n1 = n0 + 1;
+        }
+    };
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+                int m, n0, n1;
+                unit_range(u, m, n0, n1);
+                for (int n = n0; n < n1 && ok; ++n) {
+                    for (int kb = 0; kb < p.k_slabs; ++kb) {
+                        if (!mbar_wait(smem_addr(&ctl->empty[stage]), phase ^ 1u, &ctl->abort_flag)) { ok = false; break; }
+                        const uint32_t bar = smem_addr(&ctl->full[stage]);
+                        const uint32_t sa = tiles + stage * kStageBytes;
+                        const uint32_t sb = sa + kABytes;
+                        mbar_expect_tx(bar, kStageBytes);
+                        if (!a_mn) {
+                            tma_load_2d(sa, &map_a, bar, kb * BK, m * BM);
+                        } else {
+                            for (int j = 0; j < BM / 64; ++j)
+                                tma_load_2d(sa + j * kSlabBytes, &map_a, bar, m * BM + j * 64, kb * BK);
+                        }
+                        if (!b_mn) {
+                            tma_load_2d(sb, &map_b, bar, kb * BK, n * BN);
+                        } else {
+                            for (int j = 0; j < BN / 64; ++j)
+                                tma_load_2d(sb + j * kSlabBytes, &map_b, bar, n * BN + j * 64, kb * BK);
+                        }
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(a_mn, b_mn);
+            const uint32_t a_kstep = a_mn ? (16 * 128) >> 4 : 32 >> 4;   // 16 k per instruction, in 16-byte units
+            const uint32_t b_kstep = b_mn ? (16 * 128) >> 4 : 32 >> 4;
+            int stage = 0;
+            uint32_t phase = 0;
+            int buf = 0;
+            uint32_t tphase[2] = {0, 0};
+            bool ok = true;
+            for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+                int m, n0, n1;
+                unit_range(u, m, n0, n1);
+                for (int n = n0; n < n1 && ok; ++n) {
+                    if (!mbar_wait(smem_addr(&ctl->tmem_empty[buf]), tphase[buf] ^ 1u, &ctl->abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + (uint32_t)buf * BN;
+                    for (int kb = 0; kb < p.k_slabs; ++kb) {
+                        if (!mbar_wait(smem_addr(&ctl->full[stage]), phase, &ctl->abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t sa = tiles + stage * kStageBytes;
+                        const uint64_t adesc = smem_desc(sa, a_mn);
+                        const uint64_t bdesc = smem_desc(sa + kABytes, b_mn);
+#pragma unroll
+                        for (int k = 0; k < BK / 16; ++k)
+                            tc_mma(d_tmem, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc,
+                                   (kb | k) ? 1u : 0u);
+                        tc_commit(smem_addr(&ctl->empty[stage]));      // frees the stage when these MMAs retire
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!ok) break;
+                    tc_commit(smem_addr(&ctl->tmem_full[buf]));        // accumulator complete
+                    tphase[buf] ^= 1u;
+                    buf ^= 1;
+                }
+            }
+        }
+    } else {
+        // ---------------- epilogue: warps 2..5, one accumulator row per thread ----------------
+        const int quarter = warp & 3;                    // TMEM lane quarter this warp may read
+        const int row_in_tile = quarter * 32 + lane;
+        int buf = 0;
+        uint32_t tphase[2] = {0, 0};
+        bool ok = true;
+        for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+            int m, n0, n1;
+            unit_range(u, m, n0, n1);
+            const int row = m * BM + row_in_tile;
+            const bool row_ok = row < p.M;
+            float run_m = -INFINITY, run_s = 0.0f;       // kLse
+            float c2 = 0.0f, coef = 0.0f;                // kDz
+            uint32_t sgn = 0;
+            int y = -1;
+            if (p.mode == kDz && row_ok) {
+                coef = p.coef[row];
+                y = p.ids[row];
+                if (coef != 0.0f) {
+                    c2 = lg2_approx(fabsf(coef)) - p.lse[row] * kLog2e;
+                    sgn = coef < 0.0f ? 0x80008000u : 0u;
+                }
+            }
+            for (int n = n0; n < n1 && ok; ++n) {
+                if (!mbar_wait(smem_addr(&ctl->tmem_full[buf]), tphase[buf], &ctl->abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * BN;
+                const int col0 = n * BN;
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    const int cb = col0 + c * 32;
+                    if (cb >= p.N) break;                // whole chunk beyond the valid columns (warp-uniform)
+                    uint32_t v[32];
+                    tc_ld32(t_row + (uint32_t)(c * 32), v);
+                    const int nvalid = min(32, p.N - cb);
+                    if (p.mode == kLse) {
+                        float cm = -INFINITY;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (i < nvalid) cm = fmaxf(cm, __uint_as_float(v[i]));
+                        if (cm > run_m) {
+                            run_s *= ex2_approx((run_m - cm) * kLog2e);   // exp2(-inf) = 0 on the first chunk
+                            run_m = cm;
+                        }
+                        const float off = -run_m * kLog2e;
+                        float s0 = 0.0f, s1 = 0.0f;
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2) {
+                            if (i < nvalid) s0 += ex2_approx(fmaf(__uint_as_float(v[i]), kLog2e, off));
+                            if (i + 1 < nvalid) s1 += ex2_approx(fmaf(__uint_as_float(v[i + 1]), kLog2e, off));
+                        }
+                        run_s += s0 + s1;
+                    } else if (p.mode == kDz) {
+                        if (row_ok) {
+                            uint32_t o[16];
+                            if (coef == 0.0f) {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) o[i] = 0u;
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) {
+                                    float g0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), kLog2e, c2));
+                                    float g1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), kLog2e, c2));
+                                    uint32_t pk;
+                                    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(g1), "f"(g0));
+                                    o[i] = pk ^ sgn;
+                                }
+                                if (y >= cb && y < cb + 32) {
+                                    // target column: c (p_y - 1), rounded once
+                                    const int e = y - cb;
+                                    float zy = 0.0f;
+#pragma unroll
+                                    for (int i = 0; i < 32; ++i)
+                                        if (i == e) zy = __uint_as_float(v[i]);
+                                    const float py = ex2_approx(fmaf(zy, kLog2e, -p.lse[row] * kLog2e));
+                                    const uint32_t gb = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(fmaf(coef, py, -coef)));
+#pragma unroll
+                                    for (int i = 0; i < 16; ++i)
+                                        if (i == (e >> 1))
+                                            o[i] = (e & 1) ? ((o[i] & 0x0000ffffu) | (gb << 16)) : ((o[i] & 0xffff0000u) | gb);
+                                }
+                            }
+                            __nv_bfloat16* dst = p.dz + (long long)row * p.dz_stride + cb;
+                            if (nvalid == 32) {
+                                uint4* d4 = reinterpret_cast<uint4*>(dst);
+                                d4[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                                d4[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                                d4[2] = make_uint4(o[8], o[9], o[10], o[11]);
+                                d4[3] = make_uint4(o[12], o[13], o[14], o[15]);
+                            } else {
+                                for (int i = 0; i < nvalid; ++i)
+                                    dst[i] = __ushort_as_bfloat16((unsigned short)((i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xffffu)));
+                            }
+                        }
+                    } else if (p.mode == kGradHidden) {
+                        if (row_ok) {
+                            __nv_bfloat16* dst = p.out_bf16 + (long long)row * p.out_stride + cb;
+                            if (nvalid == 32) {
+                                uint32_t o[16];
+#pragma unroll
+                                for (int i = 0; i < 16; ++i)
+                                    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[i])
+                                        : "f"(__uint_as_float(v[2 * i + 1])), "f"(__uint_as_float(v[2 * i])));
+                                uint4* d4 = reinterpret_cast<uint4*>(dst);
+                                d4[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                                d4[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                                d4[2] = make_uint4(o[8], o[9], o[10], o[11]);
+                                d4[3] = make_uint4(o[12], o[13], o[14], o[15]);
+                            } else {
+                                for (int i = 0; i < nvalid; ++i) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                            }
+                        }
+                    } else {   // kGradW
+                        if (row_ok) {
+                            float* dst = p.out_f32 + (long long)row * p.out_stride + cb;
+                            if (nvalid == 32) {
+                                float4* d4 = reinterpret_cast<float4*>(dst);
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    float4 a = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                                           __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+                                    if (p.accumulate) {
+                                        const float4 old = d4[i];
+                                        a.x += old.x; a.y += old.y; a.z += old.z; a.w += old.w;
+                                    }
+                                    d4[i] = a;
+                                }
+                            } else {
+                                for (int i = 0; i < nvalid; ++i)
+                                    dst[i] = __uint_as_float(v[i]) + (p.accumulate ? dst[i] : 0.0f);
+                            }
+                        }
+                    }
+                }
+                // hand the accumulator buffer back to the MMA warp
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_addr(&ctl->tmem_empty[buf]));
+                tphase[buf] ^= 1u;
+                buf ^= 1;
+            }
+            if (p.mode == kLse && row_ok && ok) {
+                const int sp = u / p.m_tiles;
+                p.part[(long long)row * p.nsplit + sp] = make_float2(run_m, run_s);
+            }
+        }
+    }
+
+    // ---------------- teardown ----------------
+    tc_fence_before();
+    __syncthreads();
+    if (ctl->abort_flag) {
+        // copies or MMAs may still be in flight: give them time before the memory is released
+        if (threadIdx.x == 0 && p.dev_status) atomicOr(p.dev_status, RLF_DEV_TIMEOUT);
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    }
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+    }
+}
+
+// ---- small kernels around it ----------------------------------------------------------------
+// z_target[t] = <hidden[t, :], W[ids[t], :]> in fp32: one warp per token
+__global__ void __launch_bounds__(256)
+target_logit_kernel(const __nv_bfloat16* __restrict__ hidden, const __nv_bfloat16* __restrict__ W,
+                    const float4* __restrict__ rec, int64_t T, int32_t D, float* __restrict__ zy) {
+    const int64_t t = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (t >= T) return;
+    const int lane = threadIdx.x & 31;
+    const int y = __float_as_int(rec[t].w) & 0x7fffffff;
+    const uint4* h = reinterpret_cast<const uint4*>(hidden + t * (int64_t)D);
+    const uint4* w = reinterpret_cast<const uint4*>(W + (int64_t)y * D);
+    float acc = 0.0f;
+    for (int i = lane; i < D / 8; i += 32) {
+        const uint4 a = h[i], b = w[i];
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            acc = fmaf(__uint_as_float(aw[k] << 16), __uint_as_float(bw[k] << 16), acc);
+            acc = fmaf(__uint_as_float(aw[k] & 0xffff0000u), __uint_as_float(bw[k] & 0xffff0000u), acc);
+        }
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) zy[t] = acc;
+}
+
+// merge the per-split (max, sum exp) pairs of every token into lse, logp and the gradient coefficient
+__global__ void __launch_bounds__(256)
+combine_kernel(const float2* __restrict__ part, int nsplit, const float* __restrict__ zy,
+               const float4* __restrict__ rec, int64_t T, const long long* __restrict__ denom, float eps_clip,
+               float beta, float* __restrict__ logp_out, float* __restrict__ lse_out, float* __restrict__ coef_out,
+               int32_t* __restrict__ dev_status) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    float M = -INFINITY;
+    for (int j = 0; j < nsplit; ++j) M = fmaxf(M, part[t * nsplit + j].x);
+    float S = 0.0f;
+    for (int j = 0; j < nsplit; ++j) {
+        const float2 ms = part[t * nsplit + j];
+        if (ms.x != -INFINITY) S += ms.y * expf(ms.x - M);
+    }
+    const float lse = M + logf(S);
+    const float logp = (zy[t] - M) - logf(S);
+    const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) && (fabsf(logp) < INFINITY);
+    const float4 r = rec[t];
+    const bool live = (__float_as_int(r.w) < 0) && finite;
+    float coef = 0.0f;
+    if (live) {
+        const long long N = *denom;
+        const float inv_n = 1.0f / (float)(N > 1 ? N : 1);
+        const float A = r.z;
+        const float rho = expf(logp - r.x);
+        const bool clipped = ((A > 0.0f) && (rho > 1.0f + eps_clip)) || ((A < 0.0f) && (rho < 1.0f - eps_clip));
+        const float dpg = clipped ? 0.0f : -A * rho;
+        coef = -inv_n * fmaf(beta, -expm1f(r.y - logp), dpg);
+    }
+    logp_out[t] = finite ? logp : __int_as_float(0x7fc00000);
+    lse_out[t] = finite ? lse : 0.0f;
+    coef_out[t] = coef;
+    if (!finite && dev_status) atomicOr(dev_status, RLF_DEV_NONFINITE);
+}
+
+// ---- host side ------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static std::mutex mu;
+    static EncodeTiledFn fn = nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 row-major matrix [rows][cols] (cols contiguous); box = box_cols x box_rows, 128-byte swizzle
+static bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t row_stride_elems,
+                     uint32_t box_cols, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {row_stride_elems * 2};
+    const cuuint32_t box[2] = {box_cols, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int sm_count_lm() {
+    int dev = 0, v = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+    return v > 0 ? v : 148;
+}
+
+static rlf_status launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, cudaStream_t s) {
+    static std::mutex mu;
+    static bool opted[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (dev >= 0 && dev < 64 && !opted[dev]) {
+            if (cudaFuncSetAttribute((const void*)umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kSmemBytes) != cudaSuccess) {
+                cudaGetLastError();
+                return RLF_ERR_CUDA;
+            }
+            opted[dev] = true;
+        }
+    }
+    const bool sweep = p.mode == kLse || p.mode == kDz;
+    const int units = sweep ? p.m_tiles * p.nsplit : p.m_tiles * p.n_tiles;
+    if (units <= 0) return RLF_OK;
+    int grid = sm_count_lm();
+    if (grid > units) grid = units;
+    umma_gemm_kernel<<<grid, kThreads, kSmemBytes, s>>>(ma, mb, p);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+constexpr int kChunkTokens = 8192;          // rows of dZ held in scratch at a time
+constexpr int kSplit = 4;                   // vocabulary splits of the forward sweep
+
+struct LmWs {
+    size_t n_count, partial, rec, zy, lse, coef, part, dz, total;
+};
+static size_t up1k(size_t x) { return (x + 1023) & ~(size_t)1023; }
+static LmWs lm_workspace(int64_t T, int32_t V) {
+    LmWs w;
+    size_t o = 0;
+    const size_t Tn = (size_t)(T > 0 ? T : 0);
+    w.n_count = o; o += 1024;
+    w.partial = o; o += up1k(token_loss_partial_bytes());
+    w.rec = o;     o += up1k(16 * Tn);
+    w.zy = o;      o += up1k(4 * Tn);
+    w.lse = o;     o += up1k(4 * Tn);
+    w.coef = o;    o += up1k(4 * Tn);
+    w.part = o;    o += up1k(8 * Tn * kSplit);
+    w.dz = o;
+    const size_t chunk = Tn < (size_t)kChunkTokens ? Tn : (size_t)kChunkTokens;
+    o += up1k(chunk * (size_t)V * 2);
+    w.total = o + 1024;
+    return w;
+}
+
+}  // namespace lm
+
+size_t lmhead_workspace_bytes(int64_t T, int32_t V, int32_t D) {
+    (void)D;
+    if (V < 1) return 0;
+    return lm::lm_workspace(T, V).total;
+}
+
 }  // namespace rlf
 
-extern "C" rlf_status rlf_fused_lmhead_grpo(const void*, const void*, int64_t, int32_t, int32_t,
-                                            const int32_t*, const int32_t*, const float*, int32_t,
-                                            const float*, const float*, const uint8_t*, float, float,
-                                            const int64_t*, float*, double*, void*, float*, int,
-                                            void*, size_t, int32_t*, rlf_stream_t) {
-    return RLF_ERR_UNSUPPORTED;
+extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, int64_t T, int32_t D, int32_t V,
+                                            const int32_t* ids, const int32_t* seq_id, const float* adv, int32_t B,
+                                            const float* old_logp, const float* ref_logp, const uint8_t* mask,
+                                            float eps_clip, float beta_kl, const int64_t* denom, float* logp_out,
+                                            double* loss_out, void* grad_hidden, float* grad_W,
+                                            int accumulate_grad_W, void* workspace, size_t workspace_bytes,
+                                            int32_t* dev_status, rlf_stream_t stream) {
+    using namespace rlf;
+    using namespace rlf::lm;
+    if (T < 0 || V < 1 || D < 1 || B < 0) return RLF_ERR_SHAPE;
+    if (D % 64 != 0 || V % 8 != 0) return RLF_ERR_SHAPE;
+    if (T >= (1ll << 30)) return RLF_ERR_UNSUPPORTED;
+    if (!loss_out) return RLF_ERR_NULL;
+    if (T > 0 && (!hidden || !W || !ids || !seq_id || !adv || !old_logp || !ref_logp || !mask || !logp_out))
+        return RLF_ERR_NULL;
+    if (T > 0 && B == 0) return RLF_ERR_SHAPE;
+    if (!aligned(hidden, 16) || !aligned(W, 16) || !aligned(grad_hidden, 16) || !aligned(grad_W, 16))
+        return RLF_ERR_ALIGN;
+    const LmWs w = lm_workspace(T, V);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < w.total) return RLF_ERR_WORKSPACE;
+    rlf_status st = check_arch();
+    if (st != RLF_OK) return st;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+
+    // 1 KB alignment of the scratch pieces that TMA reads
+    char* ws = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(workspace) + 1023) & ~(uintptr_t)1023);
+    long long* n_count = reinterpret_cast<long long*>(ws + w.n_count);
+    double* partial = reinterpret_cast<double*>(ws + w.partial);
+    float4* rec = reinterpret_cast<float4*>(ws + w.rec);
+    float* zy = reinterpret_cast<float*>(ws + w.zy);
+    float* lse = reinterpret_cast<float*>(ws + w.lse);
+    float* coef = reinterpret_cast<float*>(ws + w.coef);
+    float2* part = reinterpret_cast<float2*>(ws + w.part);
+    __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(ws + w.dz);
+    const __nv_bfloat16* H = static_cast<const __nv_bfloat16*>(hidden);
+    const __nv_bfloat16* Wm = static_cast<const __nv_bfloat16*>(W);
+
+    const long long* dn = reinterpret_cast<const long long*>(denom);
+    if (dn == nullptr) {
+        if (cudaMemsetAsync(n_count, 0, sizeof(long long), s) != cudaSuccess) return RLF_ERR_CUDA;
+        dn = n_count;
+    }
+    if (T == 0) return launch_token_loss(logp_out, rec, 0, eps_clip, beta_kl, partial, dn, loss_out, s);
+
+    st = launch_token_prep(ids, seq_id, adv, old_logp, ref_logp, mask, T, V, B, rec, denom == nullptr ? n_count : nullptr,
+                           dev_status, s);
+    if (st != RLF_OK) return st;
+    target_logit_kernel<<<(unsigned)((T + 7) / 8), 256, 0, s>>>(H, Wm, rec, T, D, zy);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+
+    // forward sweep: running (max, sum exp) per token and vocabulary split
+    CUtensorMap mapH, mapW;
+    if (!make_map(&mapH, H, (uint64_t)T, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
+    if (!make_map(&mapW, Wm, (uint64_t)V, (uint64_t)D, (uint64_t)D, BK, BN)) return RLF_ERR_CUDA;
+    GemmParams g = {};
+    g.mode = kLse;
+    g.M = (int)T;
+    g.N = V;
+    g.m_tiles = (int)((T + BM - 1) / BM);
+    g.n_tiles = (V + BN - 1) / BN;
+    g.k_slabs = D / BK;
+    g.nsplit = kSplit;
+    g.n_tiles_per_split = (g.n_tiles + kSplit - 1) / kSplit;
+    g.part = part;
+    g.dev_status = dev_status;
+    st = launch_gemm(mapH, mapW, g, s);
+    if (st != RLF_OK) return st;
+    combine_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(part, kSplit, zy, rec, T, dn, eps_clip, beta_kl, logp_out,
+                                                                lse, coef, dev_status);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+    st = launch_token_loss(logp_out, rec, T, eps_clip, beta_kl, partial, dn, loss_out, s);
+    if (st != RLF_OK) return st;
+    if (!grad_hidden && !grad_W) return RLF_OK;
+
+    // backward by token chunks: dZ chunk -> grad_hidden rows of the chunk, grad_W += chunk's part
+    for (int64_t t0 = 0; t0 < T; t0 += kChunkTokens) {
+        const int64_t tc = (T - t0) < kChunkTokens ? (T - t0) : kChunkTokens;
+        CUtensorMap mapHc;
+        if (!make_map(&mapHc, H + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
+        GemmParams z = g;
+        z.mode = kDz;
+        z.M = (int)tc;
+        z.m_tiles = (int)((tc + BM - 1) / BM);
+        z.lse = lse + t0;
+        z.coef = coef + t0;
+        z.ids = ids + t0;
+        z.dz = dz;
+        z.dz_stride = V;
+        st = launch_gemm(mapHc, mapW, z, s);
+        if (st != RLF_OK) return st;
+        if (grad_hidden) {
+            // grad_hidden[chunk] = dZ[chunk, V] W[V, D]
+            CUtensorMap mapDzK, mapWn;
+            if (!make_map(&mapDzK, dz, (uint64_t)tc, (uint64_t)V, (uint64_t)V, BK, BM)) return RLF_ERR_CUDA;
+            if (!make_map(&mapWn, Wm, (uint64_t)V, (uint64_t)D, (uint64_t)D, 64, BK)) return RLF_ERR_CUDA;
+            GemmParams h = {};
+            h.mode = kGradHidden;
+            h.M = (int)tc;
+            h.N = D;
+            h.m_tiles = (int)((tc + BM - 1) / BM);
+            h.n_tiles = (D + BN - 1) / BN;
+            h.k_slabs = (V + BK - 1) / BK;
+            h.out_bf16 = static_cast<__nv_bfloat16*>(grad_hidden) + t0 * D;
+            h.out_stride = D;
+            h.dev_status = dev_status;
+            st = launch_gemm(mapDzK, mapWn, h, s);
+            if (st != RLF_OK) return st;
+        }
+        if (grad_W) {
+            // grad_W[V, D] (+)= dZ[chunk, V]^T hidden[chunk, D]
+            CUtensorMap mapDzM, mapHn;
+            if (!make_map(&mapDzM, dz, (uint64_t)tc, (uint64_t)V, (uint64_t)V, 64, BK)) return RLF_ERR_CUDA;
+            if (!make_map(&mapHn, H + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, 64, BK)) return RLF_ERR_CUDA;
+            GemmParams q = {};
+            q.mode = kGradW;
+            q.M = V;
+            q.N = D;
+            q.m_tiles = (V + BM - 1) / BM;
+            q.n_tiles = (D + BN - 1) / BN;
+            q.k_slabs = (int)((tc + BK - 1) / BK);
+            q.out_f32 = grad_W;
+            q.out_stride = D;
+            q.accumulate = (accumulate_grad_W || t0 > 0) ? 1 : 0;
+            q.dev_status = dev_status;
+            st = launch_gemm(mapDzM, mapHn, q, s);
+            if (st != RLF_OK) return st;
+        }
+    }
+    return RLF_OK;
 }

@@ -879,6 +879,42 @@ extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd(
 }
 
 // ---------------------------------------------------------------------------------------------
+// Token-record and scalar-loss stages, shared with the fused LM-head path.
+namespace rlf {
+
+rlf_status launch_token_prep(const int32_t* ids, const int32_t* seq_id, const float* adv, const float* old_logp,
+                             const float* ref_logp, const uint8_t* mask, int64_t T, int32_t V, int32_t B,
+                             void* rec, long long* n_count_or_null, int32_t* dev_status, cudaStream_t s) {
+    if (T <= 0) return RLF_OK;
+    const int64_t blocks = (T + kPrepThreads - 1) / kPrepThreads;
+    token_prep_kernel<<<(unsigned)blocks, kPrepThreads, 0, s>>>(
+        ids, seq_id, adv, old_logp, ref_logp, mask, T, V, B, static_cast<float4*>(rec),
+        reinterpret_cast<unsigned long long*>(n_count_or_null), dev_status);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+rlf_status launch_token_loss(const float* logp, const void* rec, int64_t T, float eps_clip, float beta,
+                             double* partial, const long long* denom, double* loss_out, cudaStream_t s) {
+    int num_partials = 0;
+    if (T > 0) {
+        const int64_t blocks = (T + kLossThreads - 1) / kLossThreads;
+        num_partials = (int)(blocks < kMaxPartials ? blocks : kMaxPartials);
+        token_loss_kernel<<<num_partials, kLossThreads, 0, s>>>(logp, static_cast<const float4*>(rec), T, eps_clip,
+                                                               partial);
+        count_launch();
+        if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+    }
+    finalize_loss_kernel<<<1, 32, 0, s>>>(partial, num_partials, denom, beta, loss_out);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+size_t token_loss_partial_bytes() { return sizeof(double) * 4 * kMaxPartials; }
+
+}  // namespace rlf
+
+// ---------------------------------------------------------------------------------------------
 // Variant for callers that cannot allocate: the scratch lives in the library's device image.
 namespace rlf {
 

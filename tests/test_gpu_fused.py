@@ -1,0 +1,83 @@
+"""GPU parity of the fused LM-head variant (logits formed on the tensor cores, never stored) against
+the fp64 oracle.  Tolerances: |d logp| <= 2e-3, loss relative 1e-4; grad_hidden (bf16) and grad_W
+(fp32) are sums over V resp. T of bf16-rounded dZ terms, so they are compared per tensor:
+max |g - g*| <= 2^-7 max |g*| and cosine similarity >= 0.9999 per row, plus the invariants that hold
+at any size (masked rows of grad_hidden are zero, the columns of grad_W sum to zero over V)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rlf_oracle as orc
+from paper_2509_06980_b200 import synth
+import gpu_common as gc
+from util import loss_close
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _run(spec, want_grads=True, accumulate=False):
+    b = gc.binding()
+    batch = synth.make_batch(spec, DEV)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    mask, seq, n = b.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, spec.open_id, spec.close_id, dev_status=st)
+    adv = b.rlf_group_advantage(batch.rewards, group_size=batch.tokens.group_size, dev_status=st)
+    gw0 = None
+    if accumulate:
+        gw0 = torch.randn((spec.V, spec.D), device=DEV)
+    logp, loss, gh, gw = b.rlf_fused_lmhead_grpo(batch.hidden, batch.W, batch.ids, seq, adv, batch.old_logp,
+                                                 batch.ref_logp, mask, synth.EPS_CLIP, synth.BETA_KL, denom=n,
+                                                 want_grad_hidden=want_grads, want_grad_W=want_grads,
+                                                 grad_W=None if gw0 is None else gw0.clone(),
+                                                 accumulate_grad_W=accumulate, dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0, st.item()
+    ora = gc.oracle_chain(batch)
+    r = orc.fused_lmhead_grpo(synth.bf16_bits(batch.hidden), synth.bf16_bits(batch.W), batch.ids.cpu().numpy(),
+                              ora["seq_id"], ora["adv"], batch.old_logp.cpu().numpy(), batch.ref_logp.cpu().numpy(),
+                              ora["mask"], synth.EPS_CLIP, synth.BETA_KL, denom=ora["n"],
+                              want_grad_hidden=want_grads, want_grad_W=want_grads)
+    assert np.array_equal(mask.cpu().numpy(), ora["mask"])
+    assert np.abs(logp.cpu().numpy() - r["logp"]).max() <= gc.LOGP_ATOL
+    lg = loss.cpu().numpy()
+    for k in range(3):
+        assert loss_close(lg[k], r["loss"][k], 1e-6, gc.LOSS_RTOL), (k, lg, r["loss"])
+    return batch, ora, r, gh, gw, gw0
+
+
+def _close_tensor(got, want, name):
+    got = got.astype(np.float64)
+    scale = np.abs(want).max()
+    assert np.abs(got - want).max() <= 2.0 ** -7 * scale, (name, np.abs(got - want).max(), scale)
+    num = (got * want).sum(axis=1)
+    den = np.sqrt((got * got).sum(axis=1) * (want * want).sum(axis=1))
+    nz = den > 1e-30 * max(scale, 1e-300) ** 2
+    assert (num[nz] / den[nz]).min() >= 0.9999, name
+
+
+SMALL = dict(len_lo=20, len_hi=20, spans_lo=1, spans_hi=2, obs_lo=2, obs_hi=4)
+
+
+@pytest.mark.parametrize("V,D", [(2048, 128), (1032, 64), (4096 + 264, 192)])
+def test_fused_forward_small(V, D):
+    """Forward only: several vocabulary tiles with a ragged last tile, one and several k-slabs,
+    a token tile that is not full (T = 320 = 2.5 tiles)."""
+    spec = synth.scaled(synth.SPECS[3], V=V, D=D, w_std=0.3, **SMALL)
+    _run(spec, want_grads=False)
+
+
+@pytest.mark.parametrize("V,D", [(2048, 128), (1032, 64), (4096 + 264, 320)])
+def test_fused_backward_small(V, D):
+    spec = synth.scaled(synth.SPECS[3], V=V, D=D, w_std=0.3, **SMALL)
+    batch, ora, r, gh, gw, _ = _run(spec)
+    _close_tensor(gh.float().cpu().numpy(), r["grad_hidden"], "grad_hidden")
+    _close_tensor(gw.cpu().numpy(), r["grad_W"], "grad_W")
+    assert not gh[torch.from_numpy(ora["mask"] == 0).to(DEV)].any()
+    colsum = gw.double().sum(dim=0).abs().max().item()
+    assert colsum <= 1e-3 * np.abs(r["grad_W"]).sum(axis=0).max() + 2.0 ** -7 * np.abs(r["grad_W"]).max()
+
+
+def test_fused_grad_W_accumulates():
+    spec = synth.scaled(synth.SPECS[3], V=2048, D=128, w_std=0.3, **SMALL)
+    batch, ora, r, gh, gw, gw0 = _run(spec, accumulate=True)
+    _close_tensor((gw - gw0).cpu().numpy(), r["grad_W"], "grad_W accumulate")
