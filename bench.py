@@ -49,6 +49,70 @@ def _peaks():
     return 6650.0, "fallback"
 
 
+def _tensor_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            j = json.load(f)
+        return float(j["bf16_tflops"]), float(j["bf16_tflops_sustained"]), "measured"
+    return 1590.0, 1400.0, "fallback"
+
+
+def time_fused_lmhead(rlf, dev, steps):
+    """The fused LM-head variant on the Qwen3-4B head (T = 32768, D = 2560, V = 151936): forward
+    (log-probs and loss, logits never stored) and forward + backward (grad_hidden, grad_W)."""
+    spec = synth.SPECS[3]
+    tok = synth.make_tokens(spec)
+    T = len(tok.ids)
+    ids = torch.from_numpy(tok.ids).to(dev)
+    cu = torch.from_numpy(tok.cu_seqlens).to(dev)
+    H, W = synth.make_hidden_and_head(spec, T, dev)
+    mask, seq, n = rlf.rlf_build_loss_mask(ids, cu, spec.open_id, spec.close_id)
+    adv = rlf.rlf_group_advantage(torch.from_numpy(tok.rewards).to(dev), group_size=spec.group_size)
+    center = synth.center_logp_from_head(H, W, ids)
+    old, ref = synth.perturbed_logps(spec, center)
+    del center
+    ws = rlf.new_workspace(rlf.FN_FUSED_LMHEAD, T, spec.V, spec.D, rlf.RLF_BF16, dev)
+    gh = torch.empty((T, spec.D), dtype=torch.bfloat16, device=dev)
+    gw = torch.empty((spec.V, spec.D), dtype=torch.float32, device=dev)
+    logp = torch.empty(T, dtype=torch.float32, device=dev)
+    loss = torch.empty(4, dtype=torch.float64, device=dev)
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def run(bwd):
+        rlf.rlf_fused_lmhead_grpo(H, W, ids, seq, adv, old, ref, mask, synth.EPS_CLIP, synth.BETA_KL, denom=n,
+                                  want_grad_hidden=bwd, want_grad_W=bwd, grad_hidden=gh if bwd else None,
+                                  grad_W=gw if bwd else None, logp_out=logp, loss_out=loss, workspace=ws,
+                                  dev_status=st)
+    out = {"workload": "cfg3_fused_lmhead_4b: hidden [32768, 2560] x W [151936, 2560] bf16", "T": T, "D": spec.D,
+           "V": spec.V}
+    burst, sustained, kind = _tensor_peaks()
+    for name, bwd, gemms, executed in (("fwd", False, 1, 1), ("fwd_bwd", True, 3, 4)):
+        for _ in range(2):
+            run(bwd)
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(steps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            run(bwd)
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        ms = statistics.mean(ts)
+        useful = 2.0 * T * spec.V * spec.D * gemms / ms / 1e9
+        out[name] = {"ms": ms, "tokens_per_s": T / ms * 1e3, "useful_tflops": useful,
+                     "executed_tflops": 2.0 * T * spec.V * spec.D * executed / ms / 1e9,
+                     "roofline": {"bound": "tensor", "achieved": useful, "peak": burst, "unit": "TFLOP/s",
+                                  "frac": useful / burst, "peak_kind": "of " + kind + " (burst)",
+                                  "frac_of_sustained": useful / sustained, "frac_of_nominal_2250": useful / 2250.0,
+                                  "traffic": None}}
+    if st.item() != 0:
+        out["device_status"] = int(st.item())
+    out["loss"] = float(loss[0].item())
+    return out
+
+
 def _kernel_sha1():
     p = os.path.join(ROOT, "paper_2509_06980_b200", "csrc", "logits_loss.cu")
     with open(p, "rb") as f:
@@ -317,6 +381,10 @@ def run_cuda(args):
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                "loss": float(h_loss[0].item())}
 
+    fused = None
+    if rank == 0 and world == 1 and not args.skip_fused:
+        fused = time_fused_lmhead(rlf, dev, max(2, min(args.steps, 5)))
+
     if rank != 0:
         return
     peak, peak_kind = _peaks()
@@ -352,6 +420,8 @@ def run_cuda(args):
         line["e2e"] = e2e
     if cpu_baseline is not None:
         line["cpu_baseline"] = cpu_baseline
+    if fused is not None:
+        line["fused_lmhead"] = fused
     print(json.dumps(line))
 
 
@@ -364,6 +434,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="time budget of the CPU-oracle baseline leg")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--skip-fused", action="store_true", help="do not time the fused LM-head variant")
     ap.add_argument("--tokens-per-response", type=int, default=0,
                     help="smaller micro-batch of the same recipe (profiling captures); 0 = the full 2048")
     args = ap.parse_args()

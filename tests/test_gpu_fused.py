@@ -81,3 +81,60 @@ def test_fused_grad_W_accumulates():
     spec = synth.scaled(synth.SPECS[3], V=2048, D=128, w_std=0.3, **SMALL)
     batch, ora, r, gh, gw, gw0 = _run(spec, accumulate=True)
     _close_tensor((gw - gw0).cpu().numpy(), r["grad_W"], "grad_W accumulate")
+
+
+def test_fused_full_vocabulary_and_hidden_reduced_T():
+    """Qwen3-4B head (V = 151936 = 593 x 256 + 128, D = 2560 = 40 k-slabs) at 16 x 8 tokens: every
+    vocabulary / hidden tile of the full-size launch, with all outputs compared in full."""
+    spec = synth.scaled(synth.SPECS[3], len_lo=8, len_hi=8, spans_lo=1, spans_hi=1, obs_lo=1, obs_hi=2)
+    batch, ora, r, gh, gw, _ = _run(spec)
+    _close_tensor(gh.float().cpu().numpy(), r["grad_hidden"], "grad_hidden")
+    _close_tensor(gw.cpu().numpy(), r["grad_W"], "grad_W")
+
+
+def test_cfg3_full_size_sampled_rows_and_invariants():
+    """The launch configuration the benchmark times (T = 32768, D = 2560, V = 151936): log-probs and
+    grad_hidden rows of sampled tokens against the oracle (a token's row depends only on that token
+    and the batch's token count); the scalar loss against the token terms evaluated in fp64 from the
+    returned log-probs; grad_W through the invariant that its columns sum to zero over the vocabulary."""
+    b = gc.binding()
+    spec = synth.SPECS[3]
+    batch = synth.make_batch(spec, DEV)
+    T = batch.T
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    mask, seq, n = b.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, spec.open_id, spec.close_id, dev_status=st)
+    adv = b.rlf_group_advantage(batch.rewards, group_size=batch.tokens.group_size, dev_status=st)
+    logp, loss, gh, gw = b.rlf_fused_lmhead_grpo(batch.hidden, batch.W, batch.ids, seq, adv, batch.old_logp,
+                                                 batch.ref_logp, mask, synth.EPS_CLIP, synth.BETA_KL, denom=n,
+                                                 dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    ora = gc.oracle_chain(batch)
+    assert np.array_equal(mask.cpu().numpy(), ora["mask"]) and n.item() == ora["n"]
+
+    rng = np.random.default_rng(3)
+    live = np.flatnonzero(ora["mask"])
+    rows = np.unique(np.concatenate([[0, T - 1], rng.choice(live, size=30, replace=False),
+                                     rng.integers(0, T, size=8)]))
+    rt = torch.as_tensor(rows, device=DEV)
+    r = orc.fused_lmhead_grpo(synth.bf16_bits(batch.hidden[rt]), synth.bf16_bits(batch.W),
+                              batch.ids.cpu().numpy()[rows], ora["seq_id"][rows], ora["adv"],
+                              batch.old_logp.cpu().numpy()[rows], batch.ref_logp.cpu().numpy()[rows],
+                              ora["mask"][rows], synth.EPS_CLIP, synth.BETA_KL, denom=ora["n"],
+                              want_grad_hidden=True, want_grad_W=False)
+    assert np.abs(logp[rt].cpu().numpy() - r["logp"]).max() <= gc.LOGP_ATOL
+    _close_tensor(gh[rt].float().cpu().numpy(), r["grad_hidden"], "grad_hidden rows")
+    assert not gh[~mask.bool()].any()
+
+    # scalar loss = masked token mean of the token terms at the returned log-probs
+    lp = logp.double().cpu()
+    A = torch.from_numpy(ora["adv"].astype(np.float64))[torch.from_numpy(ora["seq_id"]).long()]
+    rho = torch.exp(lp - batch.old_logp.double().cpu())
+    pg = -torch.minimum(rho * A, torch.clamp(rho, 1 - synth.EPS_CLIP, 1 + synth.EPS_CLIP) * A)
+    d = batch.ref_logp.double().cpu() - lp
+    m = torch.from_numpy(ora["mask"].astype(np.float64))
+    want = float((m * (pg + synth.BETA_KL * (torch.exp(d) - d - 1))).sum() / ora["n"])
+    assert loss_close(loss[0].item(), want, 1e-6, gc.LOSS_RTOL)
+
+    col = gw.double().sum(dim=0).abs().max().item()
+    assert col <= 1e-3 * gw.double().abs().sum(dim=0).max().item()
