@@ -236,6 +236,11 @@ size_t rlf_step_arena_bytes(int64_t T, int32_t V, int32_t B, rlf_dtype dt);
  * beyond fp32 summation order (and, for one_exp, one extra bf16 rounding of the gradient). */
 rlf_status rlf_tune_logits_kernel(int cluster_ctas, int threads_per_cta, int one_exp);
 
+/* Form of the fused LM-head contractions for later calls in this process: 1 = pairs of CTAs share a
+ * 256 x 256 tile (tcgen05 cta_group::2; the built-in choice), 0 = one CTA per 128 x 256 tile.
+ * Results are identical up to fp32 summation order. */
+rlf_status rlf_tune_lmhead(int pair_ctas);
+
 /* Number of kernels this library has launched in this process (for accounting). */
 int64_t rlf_launch_count(void);
 

@@ -20,7 +20,7 @@ DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
 EXPORTS = [
     "rlf_build_loss_mask", "rlf_group_advantage", "rlf_grpo_logp_loss_fwd_bwd",
     "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_fused_lmhead_grpo", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
-    "rlf_tune_logits_kernel", "rlf_launch_count", "rlf_status_string", "rlf_version",
+    "rlf_tune_logits_kernel", "rlf_tune_lmhead", "rlf_launch_count", "rlf_status_string", "rlf_version",
 ]
 
 if not os.path.exists(_LIB_PATH):
@@ -117,6 +117,12 @@ def new_workspace(which_fn, T, V, D=0, dt=RLF_BF16, device="cuda"):
 
 def tune_logits_kernel(cluster_ctas=0, threads_per_cta=0, one_exp=-1):
     _check(_lib.rlf_tune_logits_kernel(cluster_ctas, threads_per_cta, one_exp), "rlf_tune_logits_kernel")
+
+
+def tune_lmhead(pair_ctas=1):
+    _lib.rlf_tune_lmhead.argtypes = [_int]
+    _lib.rlf_tune_lmhead.restype = _int
+    _check(_lib.rlf_tune_lmhead(int(pair_ctas)), "rlf_tune_lmhead")
 
 
 def rlf_build_loss_mask(ids, cu_seqlens, open_id, close_id, valid=None, mask_out=None, seq_id_out=None,

@@ -17,6 +17,7 @@
 // logits themselves are never stored; the dZ scratch is (stated in the entry point's contract).
 #include <cuda.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "common.cuh"
@@ -25,13 +26,22 @@ namespace rlf {
 namespace lm {
 
 constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int kStages = 4;
+// Single-CTA form: each CTA multiplies a 128 x 256 tile (A 16 KB + B 32 KB per stage, 4 stages).
+// Pair form (cta_group::2): two CTAs of a cluster multiply a 256 x 256 tile; each stages its own 128
+// rows of A and HALF of B (16 KB + 16 KB per stage, 6 stages), the leader CTA issues the MMAs, and
+// each CTA's tensor memory receives its own 128 rows of the accumulator.  Per flop the pair form
+// moves two thirds of the shared-memory bytes of the single form.
 constexpr int kABytes = BM * BK * 2;
-constexpr int kBBytes = BN * BK * 2;
-constexpr int kStageBytes = kABytes + kBBytes;
+template <bool PAIR> struct Cfg {
+    static constexpr int kStages = PAIR ? 6 : 4;
+    static constexpr int kBRows = PAIR ? BN / 2 : BN;
+    static constexpr int kBBytes = kBRows * BK * 2;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+};
+constexpr int kMaxStages = 6;
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
 constexpr int kSlabBytes = 64 * BK * 2;      // one 64-wide slab of an MN-major operand: 64 k-rows of 128 B
 
 enum Mode { kLse = 0, kDz = 1, kGradHidden = 2, kGradW = 3 };
@@ -95,6 +105,39 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
 }
+// cta_group::2 forms: the MMA spans both CTAs of the pair; its commit arrives on the same barrier
+// offset in both CTAs; TMA loads of either CTA credit a barrier in the leader CTA.
+__device__ __forceinline__ void tc_mma2(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tc_commit2(uint32_t bar) {
+    const unsigned short both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 :: "r"(bar), "h"(both) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t leader_bar, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 :: "r"(dst), "l"(map), "r"(leader_bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" :: "r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ uint32_t pair_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void pair_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // 32 consecutive fp32 columns of this thread's TMEM lane
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -117,14 +160,14 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major) {
            (2ull << 61);
 }
 // Instruction descriptor: D fp32, A and B bf16, M = 128, N = 256, majorness per operand.
-__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn) {
+__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn, int m) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-           ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+           ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 struct SmemCtl {
-    unsigned long long full[kStages];
-    unsigned long long empty[kStages];
+    unsigned long long full[kMaxStages];
+    unsigned long long empty[kMaxStages];
     unsigned long long tmem_full[2];
     unsigned long long tmem_empty[2];
     uint32_t tmem_base;
@@ -132,94 +175,114 @@ struct SmemCtl {
 };
 
 // ---- the kernel -----------------------------------------------------------------------------
+template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const GemmParams p) {
+    using C = Cfg<PAIR>;
     extern __shared__ unsigned char smem_raw[];
     // operand stages must sit on 1024-byte boundaries (swizzle atom)
     const uint32_t raw = smem_addr(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
-    SmemCtl* ctl = reinterpret_cast<SmemCtl*>(smem_raw + (tiles - raw) + kStages * kStageBytes);
+    SmemCtl* ctl = reinterpret_cast<SmemCtl*>(smem_raw + (tiles - raw) + C::kStages * C::kStageBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool a_mn = p.mode == kGradW;
     const bool b_mn = p.mode == kGradHidden || p.mode == kGradW;
     const bool sweep = p.mode == kLse || p.mode == kDz;     // a unit sweeps several vocabulary tiles
-    const int units = sweep ? p.m_tiles * p.nsplit : p.m_tiles * p.n_tiles;
+    // in pair form the scheduling unit covers two token tiles: this CTA takes tile 2 * mp + rank
+    const int rank = PAIR ? (int)pair_rank() : 0;
+    const int m_units = PAIR ? (p.m_tiles + 1) / 2 : p.m_tiles;
+    const int units = sweep ? m_units * p.nsplit : m_units * p.n_tiles;
+    const int worker = PAIR ? blockIdx.x >> 1 : blockIdx.x;
+    const int workers = PAIR ? gridDim.x >> 1 : gridDim.x;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < C::kStages; ++s) {
             mbar_init(smem_addr(&ctl->full[s]), 1);
             mbar_init(smem_addr(&ctl->empty[s]), 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_addr(&ctl->tmem_full[b]), 1);
-            mbar_init(smem_addr(&ctl->tmem_empty[b]), 4);
+            mbar_init(smem_addr(&ctl->tmem_empty[b]), PAIR ? 8 : 4);
         }
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     :: "r"(smem_addr(&ctl->tmem_base)), "r"((uint32_t)kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         :: "r"(smem_addr(&ctl->tmem_base)), "r"((uint32_t)kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         :: "r"(smem_addr(&ctl->tmem_base)), "r"((uint32_t)kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) pair_sync();        // both CTAs' barriers exist before either signals the other
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
-    // unit -> (m tile, first n tile, one-past-last n tile)
+    // unit -> (m unit, first n tile, one-past-last n tile)
     auto unit_range = [&](int u, int& m, int& n0, int& n1) {
         if (sweep) {
-            m = u % p.m_tiles;
-            const int sp = u / p.m_tiles;
+            m = u % m_units;
+            const int sp = u / m_units;
             n0 = sp * p.n_tiles_per_split;
             n1 = min(p.n_tiles, n0 + p.n_tiles_per_split);
         } else {
-            m = u % p.m_tiles;
-            n0 = u / p.m_tiles;
+            m = u % m_units;
+            n0 = u / m_units;
             n1 = n0 + 1;
         }
     };
 
     if (warp == 0) {
-        // ---------------- TMA producer ----------------
+        // ---------------- TMA producer (one per CTA) ----------------
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+            for (int u = worker; u < units && ok; u += workers) {
                 int m, n0, n1;
                 unit_range(u, m, n0, n1);
+                const int my_m = PAIR ? 2 * m + rank : m;
                 for (int n = n0; n < n1 && ok; ++n) {
+                    const int b_row0 = n * BN + rank * C::kBRows;      // this CTA's rows of the B tile
                     for (int kb = 0; kb < p.k_slabs; ++kb) {
                         if (!mbar_wait(smem_addr(&ctl->empty[stage]), phase ^ 1u, &ctl->abort_flag)) { ok = false; break; }
-                        const uint32_t bar = smem_addr(&ctl->full[stage]);
-                        const uint32_t sa = tiles + stage * kStageBytes;
+                        const uint32_t own_bar = smem_addr(&ctl->full[stage]);
+                        const uint32_t bar = PAIR ? map_to_cta(own_bar, 0) : own_bar;   // the leader's barrier
+                        const uint32_t sa = tiles + stage * C::kStageBytes;
                         const uint32_t sb = sa + kABytes;
-                        mbar_expect_tx(bar, kStageBytes);
+                        if (!PAIR) mbar_expect_tx(own_bar, C::kStageBytes);
+                        else if (rank == 0) mbar_expect_tx(own_bar, 2 * C::kStageBytes);
+                        auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
+                            if (PAIR) tma_load_2d_pair(dst, map, bar, x, y);
+                            else tma_load_2d(dst, map, bar, x, y);
+                        };
                         if (!a_mn) {
-                            tma_load_2d(sa, &map_a, bar, kb * BK, m * BM);
+                            load(sa, &map_a, kb * BK, my_m * BM);
                         } else {
-                            for (int j = 0; j < BM / 64; ++j)
-                                tma_load_2d(sa + j * kSlabBytes, &map_a, bar, m * BM + j * 64, kb * BK);
+                            for (int j = 0; j < BM / 64; ++j) load(sa + j * kSlabBytes, &map_a, my_m * BM + j * 64, kb * BK);
                         }
                         if (!b_mn) {
-                            tma_load_2d(sb, &map_b, bar, kb * BK, n * BN);
+                            load(sb, &map_b, kb * BK, b_row0);
                         } else {
-                            for (int j = 0; j < BN / 64; ++j)
-                                tma_load_2d(sb + j * kSlabBytes, &map_b, bar, n * BN + j * 64, kb * BK);
+                            for (int j = 0; j < C::kBRows / 64; ++j) load(sb + j * kSlabBytes, &map_b, b_row0 + j * 64, kb * BK);
                         }
-                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                        if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                     }
                 }
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            const uint32_t idesc = instr_desc(a_mn, b_mn);
+        // ---------------- MMA issuer (in pair form: the leader CTA only) ----------------
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = instr_desc(a_mn, b_mn, PAIR ? 2 * BM : BM);
             const uint32_t a_kstep = a_mn ? (16 * 128) >> 4 : 32 >> 4;   // 16 k per instruction, in 16-byte units
             const uint32_t b_kstep = b_mn ? (16 * 128) >> 4 : 32 >> 4;
             int stage = 0;
@@ -227,7 +290,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             int buf = 0;
             uint32_t tphase[2] = {0, 0};
             bool ok = true;
-            for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+            for (int u = worker; u < units && ok; u += workers) {
                 int m, n0, n1;
                 unit_range(u, m, n0, n1);
                 for (int n = n0; n < n1 && ok; ++n) {
@@ -237,18 +300,25 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     for (int kb = 0; kb < p.k_slabs; ++kb) {
                         if (!mbar_wait(smem_addr(&ctl->full[stage]), phase, &ctl->abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        const uint32_t sa = tiles + stage * kStageBytes;
+                        const uint32_t sa = tiles + stage * C::kStageBytes;
                         const uint64_t adesc = smem_desc(sa, a_mn);
                         const uint64_t bdesc = smem_desc(sa + kABytes, b_mn);
 #pragma unroll
-                        for (int k = 0; k < BK / 16; ++k)
-                            tc_mma(d_tmem, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc,
-                                   (kb | k) ? 1u : 0u);
-                        tc_commit(smem_addr(&ctl->empty[stage]));      // frees the stage when these MMAs retire
-                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                        for (int k = 0; k < BK / 16; ++k) {
+                            if (PAIR) tc_mma2(d_tmem, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc,
+                                              (kb | k) ? 1u : 0u);
+                            else tc_mma(d_tmem, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc,
+                                        (kb | k) ? 1u : 0u);
+                        }
+                        // frees the stage (in both CTAs) when these MMAs retire
+                        if (PAIR) tc_commit2(smem_addr(&ctl->empty[stage]));
+                        else tc_commit(smem_addr(&ctl->empty[stage]));
+                        if (++stage == C::kStages) { stage = 0; phase ^= 1u; }
                     }
                     if (!ok) break;
-                    tc_commit(smem_addr(&ctl->tmem_full[buf]));        // accumulator complete
+                    // accumulator complete (in both CTAs)
+                    if (PAIR) tc_commit2(smem_addr(&ctl->tmem_full[buf]));
+                    else tc_commit(smem_addr(&ctl->tmem_full[buf]));
                     tphase[buf] ^= 1u;
                     buf ^= 1;
                 }
@@ -261,10 +331,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         int buf = 0;
         uint32_t tphase[2] = {0, 0};
         bool ok = true;
-        for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+        for (int u = worker; u < units && ok; u += workers) {
             int m, n0, n1;
             unit_range(u, m, n0, n1);
-            const int row = m * BM + row_in_tile;
+            const int row = (PAIR ? 2 * m + rank : m) * BM + row_in_tile;
             const bool row_ok = row < p.M;
             float run_m = -INFINITY, run_s = 0.0f;       // kLse
             float c2 = 0.0f, coef = 0.0f;                // kDz
@@ -392,12 +462,15 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 // hand the accumulator buffer back to the MMA warp
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_addr(&ctl->tmem_empty[buf]));
+                if (lane == 0) {
+                    if (PAIR) mbar_arrive_cluster(map_to_cta(smem_addr(&ctl->tmem_empty[buf]), 0));
+                    else mbar_arrive(smem_addr(&ctl->tmem_empty[buf]));
+                }
                 tphase[buf] ^= 1u;
                 buf ^= 1;
             }
             if (p.mode == kLse && row_ok && ok) {
-                const int sp = u / p.m_tiles;
+                const int sp = u / m_units;
                 p.part[(long long)row * p.nsplit + sp] = make_float2(run_m, run_s);
             }
         }
@@ -411,9 +484,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         if (threadIdx.x == 0 && p.dev_status) atomicOr(p.dev_status, RLF_DEV_TIMEOUT);
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
     }
+    if (PAIR) pair_sync();        // the peer may still be signalling this CTA's barriers until here
     if (warp == 0) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+        if (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
     }
 }
 
@@ -518,7 +595,10 @@ static int sm_count_lm() {
     return v > 0 ? v : 148;
 }
 
-static rlf_status launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, cudaStream_t s) {
+static std::atomic<int> g_pair{1};       // 1: cta_group::2 pair form, 0: single-CTA form
+
+template <bool PAIR>
+static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, cudaStream_t s) {
     static std::mutex mu;
     static bool opted[64] = {};
     int dev = 0;
@@ -526,8 +606,8 @@ static rlf_status launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, cons
     {
         std::lock_guard<std::mutex> lock(mu);
         if (dev >= 0 && dev < 64 && !opted[dev]) {
-            if (cudaFuncSetAttribute((const void*)umma_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     kSmemBytes) != cudaSuccess) {
+            if (cudaFuncSetAttribute((const void*)umma_gemm_kernel<PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     Cfg<PAIR>::kSmemBytes) != cudaSuccess) {
                 cudaGetLastError();
                 return RLF_ERR_CUDA;
             }
@@ -535,16 +615,39 @@ static rlf_status launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, cons
         }
     }
     const bool sweep = p.mode == kLse || p.mode == kDz;
-    const int units = sweep ? p.m_tiles * p.nsplit : p.m_tiles * p.n_tiles;
+    const int m_units = PAIR ? (p.m_tiles + 1) / 2 : p.m_tiles;
+    const int units = sweep ? m_units * p.nsplit : m_units * p.n_tiles;
     if (units <= 0) return RLF_OK;
-    int grid = sm_count_lm();
-    if (grid > units) grid = units;
-    umma_gemm_kernel<<<grid, kThreads, kSmemBytes, s>>>(ma, mb, p);
+    int workers = PAIR ? sm_count_lm() / 2 : sm_count_lm();
+    if (workers > units) workers = units;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(PAIR ? 2 * workers : workers);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = Cfg<PAIR>::kSmemBytes;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = PAIR ? 2 : 1;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, umma_gemm_kernel<PAIR>, ma, mb, p) != cudaSuccess) {
+        cudaGetLastError();
+        return RLF_ERR_CUDA;
+    }
     count_launch();
-    return cuda_ok(cudaGetLastError());
+    return RLF_OK;
 }
 
-constexpr int kChunkTokens = 8192;          // rows of dZ held in scratch at a time
+static rlf_status launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, bool pair,
+                              cudaStream_t s) {
+    return pair ? launch_gemm_t<true>(ma, mb, p, s) : launch_gemm_t<false>(ma, mb, p, s);
+}
+
+// rows of dZ held in scratch at a time: 74 token tiles, so that the dZ sweep (74 x 4 units) and the
+// grad_hidden contraction (74 x D/256 tiles) fill whole waves of 148 SMs
+constexpr int kChunkTokens = 74 * BM;
 constexpr int kSplit = 4;                   // vocabulary splits of the forward sweep
 
 struct LmWs {
@@ -631,9 +734,11 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
     if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
 
     // forward sweep: running (max, sum exp) per token and vocabulary split
+    const bool pair = g_pair.load() != 0;
+    const uint32_t b_rows = pair ? BN / 2 : BN;       // rows of a K-major B tile that one CTA stages
     CUtensorMap mapH, mapW;
     if (!make_map(&mapH, H, (uint64_t)T, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
-    if (!make_map(&mapW, Wm, (uint64_t)V, (uint64_t)D, (uint64_t)D, BK, BN)) return RLF_ERR_CUDA;
+    if (!make_map(&mapW, Wm, (uint64_t)V, (uint64_t)D, (uint64_t)D, BK, b_rows)) return RLF_ERR_CUDA;
     GemmParams g = {};
     g.mode = kLse;
     g.M = (int)T;
@@ -645,7 +750,7 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
     g.n_tiles_per_split = (g.n_tiles + kSplit - 1) / kSplit;
     g.part = part;
     g.dev_status = dev_status;
-    st = launch_gemm(mapH, mapW, g, s);
+    st = launch_gemm(mapH, mapW, g, pair, s);
     if (st != RLF_OK) return st;
     combine_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(part, kSplit, zy, rec, T, dn, eps_clip, beta_kl, logp_out,
                                                                 lse, coef, dev_status);
@@ -669,7 +774,7 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
         z.ids = ids + t0;
         z.dz = dz;
         z.dz_stride = V;
-        st = launch_gemm(mapHc, mapW, z, s);
+        st = launch_gemm(mapHc, mapW, z, pair, s);
         if (st != RLF_OK) return st;
         if (grad_hidden) {
             // grad_hidden[chunk] = dZ[chunk, V] W[V, D]
@@ -686,7 +791,7 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
             h.out_bf16 = static_cast<__nv_bfloat16*>(grad_hidden) + t0 * D;
             h.out_stride = D;
             h.dev_status = dev_status;
-            st = launch_gemm(mapDzK, mapWn, h, s);
+            st = launch_gemm(mapDzK, mapWn, h, pair, s);
             if (st != RLF_OK) return st;
         }
         if (grad_W) {
@@ -705,9 +810,15 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
             q.out_stride = D;
             q.accumulate = (accumulate_grad_W || t0 > 0) ? 1 : 0;
             q.dev_status = dev_status;
-            st = launch_gemm(mapDzM, mapHn, q, s);
+            st = launch_gemm(mapDzM, mapHn, q, pair, s);
             if (st != RLF_OK) return st;
         }
     }
+    return RLF_OK;
+}
+
+extern "C" rlf_status rlf_tune_lmhead(int pair_ctas) {
+    if (pair_ctas != 0 && pair_ctas != 1) return RLF_ERR_SHAPE;
+    rlf::lm::g_pair = pair_ctas;
     return RLF_OK;
 }

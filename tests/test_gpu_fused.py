@@ -16,6 +16,15 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
+@pytest.fixture(params=[1, 0], ids=["pair", "single"])
+def form(request):
+    """Both forms of the contraction kernel: CTA pairs on 256 x 256 tiles, and one CTA per 128 x 256."""
+    b = gc.binding()
+    b.tune_lmhead(request.param)
+    yield request.param
+    b.tune_lmhead(1)
+
+
 def _run(spec, want_grads=True, accumulate=False):
     b = gc.binding()
     batch = synth.make_batch(spec, DEV)
@@ -59,7 +68,7 @@ SMALL = dict(len_lo=20, len_hi=20, spans_lo=1, spans_hi=2, obs_lo=2, obs_hi=4)
 
 
 @pytest.mark.parametrize("V,D", [(2048, 128), (1032, 64), (4096 + 264, 192)])
-def test_fused_forward_small(V, D):
+def test_fused_forward_small(V, D, form):
     """Forward only: several vocabulary tiles with a ragged last tile, one and several k-slabs,
     a token tile that is not full (T = 320 = 2.5 tiles)."""
     spec = synth.scaled(synth.SPECS[3], V=V, D=D, w_std=0.3, **SMALL)
@@ -67,7 +76,7 @@ def test_fused_forward_small(V, D):
 
 
 @pytest.mark.parametrize("V,D", [(2048, 128), (1032, 64), (4096 + 264, 320)])
-def test_fused_backward_small(V, D):
+def test_fused_backward_small(V, D, form):
     spec = synth.scaled(synth.SPECS[3], V=V, D=D, w_std=0.3, **SMALL)
     batch, ora, r, gh, gw, _ = _run(spec)
     _close_tensor(gh.float().cpu().numpy(), r["grad_hidden"], "grad_hidden")
@@ -77,7 +86,7 @@ def test_fused_backward_small(V, D):
     assert colsum <= 1e-3 * np.abs(r["grad_W"]).sum(axis=0).max() + 2.0 ** -7 * np.abs(r["grad_W"]).max()
 
 
-def test_fused_grad_W_accumulates():
+def test_fused_grad_W_accumulates(form):
     spec = synth.scaled(synth.SPECS[3], V=2048, D=128, w_std=0.3, **SMALL)
     batch, ora, r, gh, gw, gw0 = _run(spec, accumulate=True)
     _close_tensor((gw - gw0).cpu().numpy(), r["grad_W"], "grad_W accumulate")
