@@ -234,8 +234,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             n0 = sp * p.n_tiles_per_split;
             n1 = min(p.n_tiles, n0 + p.n_tiles_per_split);
         } else {
-            m = u % m_units;
-            n0 = u / m_units;
+            // column tiles fastest: the CTAs running at the same time share their A slabs (the dZ
+            // rows or columns) in L2 instead of each streaming the whole scratch from HBM
+            n0 = u % p.n_tiles;
+            m = u / p.n_tiles;
             n1 = n0 + 1;
         }
     };
