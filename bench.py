@@ -58,10 +58,12 @@ def _tensor_peaks():
     return 1590.0, 1400.0, "fallback"
 
 
-def time_fused_lmhead(rlf, dev, steps):
+def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0):
     """The fused LM-head variant on the Qwen3-4B head (T = 32768, D = 2560, V = 151936): forward
     (log-probs and loss, logits never stored) and forward + backward (grad_hidden, grad_W)."""
     spec = synth.SPECS[3]
+    if tokens_per_response:
+        spec = synth.scaled(spec, len_lo=tokens_per_response, len_hi=tokens_per_response)
     tok = synth.make_tokens(spec)
     T = len(tok.ids)
     ids = torch.from_numpy(tok.ids).to(dev)
@@ -84,11 +86,11 @@ def time_fused_lmhead(rlf, dev, steps):
                                   want_grad_hidden=bwd, want_grad_W=bwd, grad_hidden=gh if bwd else None,
                                   grad_W=gw if bwd else None, logp_out=logp, loss_out=loss, workspace=ws,
                                   dev_status=st)
-    out = {"workload": "cfg3_fused_lmhead_4b: hidden [32768, 2560] x W [151936, 2560] bf16", "T": T, "D": spec.D,
+    out = {"workload": "cfg3_fused_lmhead_4b: hidden [%d, 2560] x W [151936, 2560] bf16" % T, "T": T, "D": spec.D,
            "V": spec.V}
     burst, sustained, kind = _tensor_peaks()
     for name, bwd, gemms, executed in (("fwd", False, 1, 1), ("fwd_bwd", True, 3, 4)):
-        for _ in range(2):
+        for _ in range(1 if tokens_per_response else 2):
             run(bwd)
         torch.cuda.synchronize()
         ts = []
@@ -271,10 +273,22 @@ def run_reference(args):
 
 
 # ---------------------------------------------------------------------------------------------
+def run_fused_only(args):
+    """Only the fused LM-head variant, optionally at a reduced token count (profiling captures)."""
+    from paper_2509_06980_b200 import binding as rlf
+    torch.cuda.set_device(0)
+    out = time_fused_lmhead(rlf, torch.device("cuda", 0), max(1, args.steps), args.tokens_per_response)
+    print(json.dumps({"fused_lmhead": out, "gpu_launches": rlf.launch_count()}))
+
+
 def run_cuda(args):
     rank, world, local = dist_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    if args.fused_only:
+        if rank == 0:
+            run_fused_only(args)
+        return
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1:
@@ -435,6 +449,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--skip-fused", action="store_true", help="do not time the fused LM-head variant")
+    ap.add_argument("--fused-only", action="store_true", help="time only the fused LM-head variant (rank 0)")
     ap.add_argument("--tokens-per-response", type=int, default=0,
                     help="smaller micro-batch of the same recipe (profiling captures); 0 = the full 2048")
     args = ap.parse_args()
