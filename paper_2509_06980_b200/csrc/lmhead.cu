@@ -7,8 +7,8 @@
 //   DZ    z tile recomputed, epilogue turns it into dZ = c_t (softmax - onehot)  -> bf16 scratch
 //   GH    grad_hidden = dZ W      (A = dZ K-major, B = W vocabulary-major rows: N-major operand)
 //   GW    grad_W     += dZ^T H    (both operands token-major rows: M-/N-major operands)
-// CTA = 192 threads: warp 0 issues TMA loads into a 4-stage ring (48 KB per stage), warp 1 issues
-// the MMAs (one thread) into a double-buffered 128 x 256 fp32 accumulator (all 512 TMEM columns),
+// CTA = 192 threads: warp 0 issues TMA loads into a multi-stage ring, warp 1 issues the MMAs (one
+// thread) into a double-buffered 128 x 256 fp32 accumulator (all 512 TMEM columns),
 // warps 2..5 drain the accumulator with tcgen05.ld (one token row per thread) while the next tile
 // is being multiplied.  Every mbarrier wait is bounded; a wait that runs out raises a CTA-wide
 // abort flag, all roles leave their loops, tensor memory is released and RLF_DEV_TIMEOUT is set.
