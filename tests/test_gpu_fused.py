@@ -147,3 +147,40 @@ def test_cfg3_full_size_sampled_rows_and_invariants():
 
     col = gw.double().sum(dim=0).abs().max().item()
     assert col <= 1e-3 * gw.double().abs().sum(dim=0).max().item()
+
+
+def test_cfg4_head_shape_reduced_T():
+    """Qwen3-8B head (D = 4096 = 64 k-slabs, V = 151936) at 8 x 8 tokens, all outputs in full."""
+    spec = synth.scaled(synth.SPECS[4], len_lo=8, len_hi=8, spans_lo=1, spans_hi=1, obs_lo=1, obs_hi=2)
+    batch, ora, r, gh, gw, _ = _run(spec)
+    _close_tensor(gh.float().cpu().numpy(), r["grad_hidden"], "grad_hidden")
+    _close_tensor(gw.cpu().numpy(), r["grad_W"], "grad_W")
+
+
+def test_fused_micro_batches_with_global_denominator_accumulate():
+    """cfg-4-style processing: one response per call, the batch's token count as denominator, grad_W
+    accumulated across calls; the sum must equal the single-call result."""
+    b = gc.binding()
+    spec = synth.scaled(synth.SPECS[4], len_lo=40, len_hi=40, spans_lo=1, spans_hi=2, obs_lo=3, obs_hi=6, V=4096 + 264,
+                        D=256, w_std=0.3)
+    batch = synth.make_batch(spec, DEV)
+    mask, seq, n = b.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, spec.open_id, spec.close_id)
+    adv = b.rlf_group_advantage(batch.rewards, group_size=batch.tokens.group_size)
+    full = b.rlf_fused_lmhead_grpo(batch.hidden, batch.W, batch.ids, seq, adv, batch.old_logp, batch.ref_logp, mask,
+                                   synth.EPS_CLIP, synth.BETA_KL, denom=n)
+    torch.cuda.synchronize()
+    gw = torch.zeros_like(full[3])
+    total = 0.0
+    cu = batch.cu_seqlens.cpu().numpy()
+    for i in range(batch.B):
+        a, e = int(cu[i]), int(cu[i + 1])
+        logp, loss, gh, _ = b.rlf_fused_lmhead_grpo(batch.hidden[a:e], batch.W, batch.ids[a:e], seq[a:e], adv,
+                                                    batch.old_logp[a:e], batch.ref_logp[a:e], mask[a:e], synth.EPS_CLIP,
+                                                    synth.BETA_KL, denom=n, grad_W=gw, accumulate_grad_W=True)
+        torch.cuda.synchronize()
+        total += loss[0].item()
+        assert torch.equal(logp, full[0][a:e])
+        assert (gh.float() - full[2][a:e].float()).abs().max().item() <= 2.0 ** -7 * full[2].float().abs().max().item()
+    assert abs(total - full[1][0].item()) <= 1e-9 + 1e-6 * abs(full[1][0].item())
+    scale = full[3].abs().max().item()
+    assert (gw - full[3]).abs().max().item() <= 2.0 ** -7 * scale
