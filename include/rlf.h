@@ -148,6 +148,22 @@ rlf_status rlf_grpo_logp_loss_fwd_bwd(const void *logits, rlf_dtype dt, int64_t 
                                       int32_t *dev_status, rlf_stream_t stream);
 
 /*
+ * Forward-only log-prob of given target tokens, and the entropy of each row's distribution: the pass
+ * that produces old_logp / ref_logp for the update above (the behaviour and reference policies of
+ * the PPO-style update, paper Sec. 2.3.1; the policy pi_theta(a | s_t) of Sec. 2.2).  Per row t:
+ *     logp[t]    = z[t, ids[t]] - log sum_v exp z[t, v]
+ *     entropy[t] = - sum_v p_v log p_v,  p = softmax(z[t, :])      (terms with p_v = 0 contribute 0)
+ * Each logits row is read from HBM once (2 V bytes per token at bf16); nothing else of size T x V
+ * is touched.  Same fast-path conditions, general fallback, workspace size
+ * (rlf_workspace_bytes(RLF_FN_LOGP_LOSS, ...)) and device status bits as rlf_grpo_logp_loss_fwd_bwd;
+ * a row with a target outside [0, V) or a non-finite log-sum-exp gets NaN.
+ *   logits [T, V] dt with row_stride;  ids [T] int32;  logp_out [T] fp32;  entropy_out [T] fp32 or NULL
+ */
+rlf_status rlf_logp_entropy_fwd(const void *logits, rlf_dtype dt, int64_t T, int32_t V, int64_t row_stride,
+                                const int32_t *ids, float *logp_out, float *entropy_out, void *workspace,
+                                size_t workspace_bytes, int32_t *dev_status, rlf_stream_t stream);
+
+/*
  * rlf_grpo_logp_loss_fwd_bwd without a workspace argument, for callers that cannot allocate.
  * (The paper has no counterpart: this is a packaging variant of the entry point above.)
  *

@@ -321,6 +321,42 @@ int orc_fused_lmhead_grpo(const uint16_t *hidden, const uint16_t *W, int64_t T, 
     return rc;
 }
 
+/*
+ * Forward-only log-prob and entropy of each row's softmax (the behaviour / reference policy pass that
+ * produces old_logp and ref_logp for the PPO-style update of Sec. 2.3.1; the policy of Sec. 2.2):
+ *     logp_t = z[t, y_t] - lse_t
+ *     H_t    = - sum_v p_v log p_v,   p_v = exp(z_v - lse_t),   a term with p_v = 0 counts 0
+ * entropy_out may be NULL.
+ */
+int orc_logp_entropy(const void *logits, int dtype, int64_t T, int32_t V, int64_t row_stride,
+                     const int32_t *ids, double *logp_out, double *entropy_out)
+{
+    int bad = 0;
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int64_t t = 0; t < T; ++t) {
+        int64_t off = t * row_stride;
+        int32_t y = ids[t];
+        if (y < 0 || y >= V) {
+#pragma omp atomic write
+            bad = 1;
+            continue;
+        }
+        double m, logs;
+        row_stats(logits, dtype, off, V, &m, &logs);
+        logp_out[t] = (widen(logits, dtype, off + y) - m) - logs;
+        if (entropy_out) {
+            double h = 0.0;
+            for (int32_t v = 0; v < V; ++v) {
+                double lp = (widen(logits, dtype, off + v) - m) - logs;   /* log p_v */
+                double pv = exp(lp);
+                if (pv > 0.0) h -= pv * lp;
+            }
+            entropy_out[t] = h;
+        }
+    }
+    return bad ? -2 : 0;
+}
+
 /* Rule reward, Eq. 1: R = sum_i w_i r_i over n rule scores, for each of B responses.
  * scores is [B, n] row-major. */
 int orc_rule_reward(const float *scores, const float *weights, int32_t B, int32_t n, double *R)

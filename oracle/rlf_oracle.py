@@ -125,6 +125,20 @@ def grpo_loss(logits, ids, seq_id, adv, old_logp, ref_logp, mask, eps_clip, beta
     return dict(logp=logp, loss=loss, grad=grad, coef=coef)
 
 
+def logp_entropy(logits, ids, want_entropy=True):
+    """-> (logp f64[T], entropy f64[T] | None) of each row's softmax at the given targets."""
+    assert logits.ndim == 2 and (logits.shape[1] <= 1 or logits.strides[1] == logits.itemsize)
+    T, V = logits.shape
+    stride = logits.strides[0] // logits.itemsize if T > 1 else V
+    ids = _c(ids, np.int32)
+    logp = np.zeros(T, np.float64)
+    ent = np.zeros(T, np.float64) if want_entropy else None
+    rc = lib().orc_logp_entropy(_p(logits), ctypes.c_int(_dtype_code(logits)), ctypes.c_int64(T), ctypes.c_int32(V),
+                                ctypes.c_int64(stride), _p(ids), _p(logp), _p(ent))
+    _check(rc, "logp_entropy")
+    return logp, ent
+
+
 def fused_lmhead_grpo(hidden, W, ids, seq_id, adv, old_logp, ref_logp, mask, eps_clip, beta_kl,
                       denom=None, want_grad_hidden=True, want_grad_W=True, want_z=False):
     """hidden [T,D], W [V,D]: uint16 arrays holding bf16 bit patterns.

@@ -19,7 +19,7 @@ DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
 
 EXPORTS = [
     "rlf_build_loss_mask", "rlf_group_advantage", "rlf_grpo_logp_loss_fwd_bwd",
-    "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_fused_lmhead_grpo", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
+    "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
     "rlf_tune_logits_kernel", "rlf_tune_lmhead", "rlf_launch_count", "rlf_status_string", "rlf_version",
 ]
 
@@ -187,6 +187,28 @@ def rlf_grpo_logp_loss_fwd_bwd(logits, ids, seq_id, adv, old_logp, ref_logp, mas
         None if grad_logits is None else grad_logits.data_ptr(), workspace.data_ptr(), workspace.numel(),
         _ptr(dev_status, torch.int32), _stream()), "rlf_grpo_logp_loss_fwd_bwd")
     return logp_out, loss_out, grad_logits
+
+
+def rlf_logp_entropy_fwd(logits, ids, want_entropy=True, logp_out=None, entropy_out=None, workspace=None,
+                         dev_status=None):
+    """Forward only: -> (logp fp32[T], entropy fp32[T] | None) of the rows of `logits` at targets `ids`."""
+    T, V = logits.shape
+    stride = logits.stride(0) if T > 1 else V
+    dev = logits.device
+    if logp_out is None:
+        logp_out = torch.empty(T, dtype=torch.float32, device=dev)
+    if entropy_out is None and want_entropy:
+        entropy_out = torch.empty(T, dtype=torch.float32, device=dev)
+    dt = _dt(logits)
+    if workspace is None:
+        workspace = new_workspace(FN_LOGP_LOSS, T, V, 0, dt, dev)
+    _lib.rlf_logp_entropy_fwd.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+    _lib.rlf_logp_entropy_fwd.restype = _int
+    _check(_lib.rlf_logp_entropy_fwd(logits.data_ptr() if T > 0 else None, dt, T, V, stride, _ptr(ids, torch.int32),
+                                     _ptr(logp_out, torch.float32), _ptr(entropy_out, torch.float32),
+                                     workspace.data_ptr(), workspace.numel(), _ptr(dev_status, torch.int32),
+                                     _stream()), "rlf_logp_entropy_fwd")
+    return logp_out, entropy_out
 
 
 STATIC_MAX_TOKENS = 65536

@@ -162,6 +162,7 @@ struct FastParams {
     const float4* rec;
     const long long* denom;
     float* logp_out;
+    float* entropy_out;         // entropy variant only, nullable
     int32_t* dev_status;
     float eps_clip, beta;
 };
@@ -209,6 +210,29 @@ __device__ __forceinline__ float exp_sum_pass(uint4 (&d)[NV], float m, float off
         }
     }
     return s0 + s1;
+}
+
+// forward-only variant with entropy: besides s = sum 2^x it accumulates u = sum 2^x * x, where
+// x = (z - m) log2e is the element's exponent (clamped below so that a vanishing term contributes
+// 0 * finite instead of 0 * inf); the entropy is ln S - ln2 * U / S once merged over the row
+template <int NV, bool ROBUST>
+__device__ __forceinline__ float2 exp_sum_ent_pass(const uint4 (&d)[NV], float m, float off) {
+    float s0 = 0.0f, s1 = 0.0f, u0 = 0.0f, u1 = 0.0f;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+        const uint32_t w[4] = {d[i].x, d[i].y, d[i].z, d[i].w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float x0 = fmaxf(expo<ROBUST>(bf_lo(w[k]), m, off), -1e30f);
+            const float x1 = fmaxf(expo<ROBUST>(bf_hi(w[k]), m, off), -1e30f);
+            const float e0 = ex2_approx(x0), e1 = ex2_approx(x1);
+            s0 += e0;
+            s1 += e1;
+            u0 = fmaf(e0, x0, u0);
+            u1 = fmaf(e1, x1, u1);
+        }
+    }
+    return make_float2(s0 + s1, u0 + u1);
 }
 
 template <bool ROBUST>
@@ -268,7 +292,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t mbar, uint32_t parity
     return false;
 }
 
-template <int THREADS, int NV, bool ONE_EXP>
+template <int THREADS, int NV, bool ONE_EXP, bool ENT = false>
 __global__ void __launch_bounds__(THREADS, ctas_per_sm(THREADS, NV))
 grpo_row_cluster_kernel(const FastParams p) {
     constexpr int NWARPS = THREADS / 32;
@@ -279,6 +303,7 @@ grpo_row_cluster_kernel(const FastParams p) {
     __shared__ __align__(8) float2 pair_slot[2][MAXE];   // per row parity: every warp's (max, sum)
     __shared__ __align__(16) float4 rec_slot[4];         // token records, ring over rows
     __shared__ float zy_slot[2];                         // per row parity: the target logit
+    __shared__ float ent_slot[2][ENT ? MAXE : 1];        // entropy variant: every warp's sum 2^x * x
     __shared__ __align__(8) unsigned long long row_bar[2];   // per row parity: "all pairs and z_target are here"
 
     const int csize = (int)cluster_nctarank();
@@ -316,7 +341,7 @@ grpo_row_cluster_kernel(const FastParams p) {
     };
 
     // per row every CTA receives one (max, sum) pair from every warp of the cluster and z_target
-    const uint32_t row_bytes = (uint32_t)npairs * 8u + 4u;
+    const uint32_t row_bytes = (uint32_t)npairs * (ENT ? 12u : 8u) + 4u;
     if (tid == 0) {
         mbar_init(smem_u32(&row_bar[0]), 1);
         mbar_init(smem_u32(&row_bar[1]), 1);
@@ -367,13 +392,23 @@ grpo_row_cluster_kernel(const FastParams p) {
         // exponent base of this warp: 2^((z - m_w) log2e); all lanes agree on the form
         const float m_ws = (m_w == -INFINITY) ? 0.0f : m_w;
         const bool robust_w = fabsf(m_ws) > kRobustAbove;
-        const float s_t = robust_w ? exp_sum_pass<NV, ONE_EXP, true>(d, m_ws, 0.0f)
-                                   : exp_sum_pass<NV, ONE_EXP, false>(d, 0.0f, -m_ws * kLog2e);
+        float s_t, u_w = 0.0f;
+        if (ENT) {
+            const float2 su = robust_w ? exp_sum_ent_pass<NV, true>(d, m_ws, 0.0f)
+                                       : exp_sum_ent_pass<NV, false>(d, 0.0f, -m_ws * kLog2e);
+            s_t = su.x;
+            u_w = warp_sum(su.y);
+        } else {
+            s_t = robust_w ? exp_sum_pass<NV, ONE_EXP, true>(d, m_ws, 0.0f)
+                           : exp_sum_pass<NV, ONE_EXP, false>(d, 0.0f, -m_ws * kLog2e);
+        }
         const float s_w = warp_sum(s_t);
         // every warp hands its (max, sum) to every CTA of the cluster, then waits until its own CTA
         // has received the whole row's worth (the only synchronisation in the loop)
-        if (lane < csize)
+        if (lane < csize) {
             st_async_f2(smem_u32(&pair_slot[parity][crank * NWARPS + warp]), bar, (uint32_t)lane, m_w, s_w);
+            if (ENT) st_async_f1(smem_u32(&ent_slot[parity][crank * NWARPS + warp]), bar, (uint32_t)lane, u_w);
+        }
         if (!gave_up && !mbar_wait_bounded(bar, (uint32_t)(it >> 1) & 1u)) {
             gave_up = true;
             status |= RLF_DEV_TIMEOUT;
@@ -389,11 +424,23 @@ grpo_row_cluster_kernel(const FastParams p) {
             M = fmaxf(M, e[j].x);
         }
         M = ord2f(__reduce_max_sync(0xffffffffu, f2ord(M)));
-        float S = 0.0f;
+        float S = 0.0f, U = 0.0f;
 #pragma unroll
-        for (int j = 0; j < (MAXE + 31) / 32; ++j)
-            if (e[j].x != -INFINITY) S += e[j].y * ex2_approx((e[j].x - M) * kLog2e);
+        for (int j = 0; j < (MAXE + 31) / 32; ++j) {
+            if (e[j].x != -INFINITY) {
+                const float dx = (e[j].x - M) * kLog2e;          // this warp's base relative to the row's
+                const float f = ex2_approx(dx);
+                S += e[j].y * f;
+                if (ENT) {
+                    const int k = lane + 32 * j;
+                    // exponents relative to the row maximum are x + dx; a warp whose weight f
+                    // vanishes contributes nothing (its dx may be -huge)
+                    if (f > 0.0f) U += f * fmaf(e[j].y, dx, ent_slot[parity][k < npairs ? k : 0]);
+                }
+            }
+        }
         S = warp_sum(S);
+        if (ENT) U = warp_sum(U);
         const float zy = zy_slot[parity];
         const float4 rec = rec_slot[it & 3];
         const float lg2s = lg2_approx(S);
@@ -403,11 +450,15 @@ grpo_row_cluster_kernel(const FastParams p) {
         const bool live = (__float_as_int(rec.w) < 0) && finite;
         const float coef = live ? -inv_n * grad_coef_fast(logp, rec.x, rec.y, rec.z, p.eps_clip, p.beta) : 0.0f;
         if (crank == 0 && tid == 0) {
-            p.logp_out[row] = finite ? logp : __int_as_float(0x7fc00000);
+            // forward-only variant: a row whose target id was out of range has no log-prob
+            const bool has_logp = finite && (!ENT || __float_as_int(rec.w) < 0);
+            p.logp_out[row] = has_logp ? logp : __int_as_float(0x7fc00000);
             if (!finite) status |= RLF_DEV_NONFINITE;
+            // H = ln S - ln2 * U / S  (= lse - E[z])
+            if (ENT && p.entropy_out) p.entropy_out[row] = finite ? (lg2s - U / S) * kLn2 : __int_as_float(0x7fc00000);
         }
 
-        if (p.grad != nullptr) {
+        if (!ENT && p.grad != nullptr) {
             uint4* dst = reinterpret_cast<uint4*>(p.grad + (long long)row * p.stride) + vbeg;
             if (coef == 0.0f || !(fabsf(coef) < INFINITY)) {
                 const uint4 z4 = make_uint4(0u, 0u, 0u, 0u);
@@ -473,6 +524,8 @@ struct GenParams {
     const float4* rec;
     const long long* denom;
     float* logp_out;
+    float* entropy_out;         // nullable: also return the row's entropy (forward-only use)
+    int fwd_only;               // forward-only entry point: a row with a bad target id gets NaN
     int32_t* dev_status;
     float eps_clip, beta;
 };
@@ -483,7 +536,8 @@ template <typename T>
 __global__ void __launch_bounds__(kGenThreads)
 grpo_row_general_kernel(const GenParams p) {
     __shared__ float red[kGenThreads / 32];
-    __shared__ float bcast;
+    __shared__ float red_u[kGenThreads / 32];
+    __shared__ float bcast, bcast_u;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long N = *p.denom;
     const float inv_n = 1.0f / (float)(N > 1 ? N : 1);
@@ -508,19 +562,27 @@ grpo_row_general_kernel(const GenParams p) {
         __syncthreads();
         const float M = bcast;
         const float Ms = (M == -INFINITY) ? 0.0f : M;
-        float s = 0.0f;
-        for (int v = tid; v < p.V; v += kGenThreads) s += ex2_approx((to_f32<T>(z[v]) - Ms) * kLog2e);
+        float s = 0.0f, u = 0.0f;
+        for (int v = tid; v < p.V; v += kGenThreads) {
+            const float x = fmaxf((to_f32<T>(z[v]) - Ms) * kLog2e, -1e30f);
+            const float e = ex2_approx(x);
+            s += e;
+            u = fmaf(e, x, u);                 // for the entropy: sum 2^x * x
+        }
         s = warp_sum(s);
+        u = warp_sum(u);
         __syncthreads();
-        if (lane == 0) red[warp] = s;
+        if (lane == 0) { red[warp] = s; red_u[warp] = u; }
         __syncthreads();
         if (tid == 0) {
-            float ss = 0.0f;
-            for (int w = 0; w < kGenThreads / 32; ++w) ss += red[w];
+            float ss = 0.0f, uu = 0.0f;
+            for (int w = 0; w < kGenThreads / 32; ++w) { ss += red[w]; uu += red_u[w]; }
             bcast = ss;
+            bcast_u = uu;
         }
         __syncthreads();
         const float S = bcast;
+        const float U = bcast_u;
         __syncthreads();
 
         const float lg2s = lg2_approx(S);
@@ -530,8 +592,10 @@ grpo_row_general_kernel(const GenParams p) {
         const bool live = (__float_as_int(rec.w) < 0) && finite;
         const float coef = live ? -inv_n * grad_coef_fast(logp, rec.x, rec.y, rec.z, p.eps_clip, p.beta) : 0.0f;
         if (tid == 0) {
-            p.logp_out[row] = finite ? logp : __int_as_float(0x7fc00000);
+            const bool has_logp = finite && (!p.fwd_only || __float_as_int(rec.w) < 0);
+            p.logp_out[row] = has_logp ? logp : __int_as_float(0x7fc00000);
             if (!finite) status |= RLF_DEV_NONFINITE;
+            if (p.entropy_out) p.entropy_out[row] = finite ? (lg2s - U / S) * kLn2 : __int_as_float(0x7fc00000);
         }
         if (p.grad != nullptr) {
             T* g = static_cast<T*>(p.grad) + row * p.stride;
@@ -798,6 +862,7 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
             p.dev_status = a.dev_status;
             p.eps_clip = a.eps_clip;
             p.beta = a.beta;
+            p.entropy_out = nullptr;
             cudaLaunchConfig_t cfg;
             cudaLaunchAttribute at[1];
             cluster_config(&cfg, at, nc * sh.cluster, sh, s);
@@ -812,7 +877,7 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
             GenParams p;
             p.logits = a.logits; p.grad = a.grad; p.stride = a.stride; p.T = a.T; p.V = a.V;
             p.rec = rec; p.denom = denom; p.logp_out = a.logp_out; p.dev_status = a.dev_status;
-            p.eps_clip = a.eps_clip; p.beta = a.beta;
+            p.eps_clip = a.eps_clip; p.beta = a.beta; p.entropy_out = nullptr; p.fwd_only = 0;
             int grid = sm_count() * 8;
             if ((int64_t)grid > a.T) grid = (int)a.T;
             if (a.dt == RLF_BF16) grpo_row_general_kernel<__nv_bfloat16><<<grid, kGenThreads, 0, s>>>(p);
@@ -876,6 +941,111 @@ extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd(
     const bool fast_ok = dt == RLF_BF16 && (V % 8 == 0) && (row_stride % 8 == 0) &&
                          aligned(logits, 16) && aligned(grad_logits, 16);
     return launch_logits_loss(a, fast_ok, workspace, reinterpret_cast<cudaStream_t>(stream));
+}
+
+// ---------------------------------------------------------------------------------------------
+// Forward-only log-prob (+ entropy) of given target ids: the pass that produces old_logp / ref_logp.
+namespace rlf {
+
+__global__ void __launch_bounds__(256)
+ids_to_record_kernel(const int32_t* __restrict__ ids, int64_t T, int32_t V, float4* __restrict__ rec,
+                     long long* __restrict__ one, int32_t* __restrict__ dev_status) {
+    const int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (t == 0) *one = 1;                       // the row kernels read a denominator; unused here
+    if (t >= T) return;
+    int32_t y = ids[t];
+    const bool bad = y < 0 || y >= V;
+    if (bad) {
+        y = 0;
+        if (dev_status) atomicOr(dev_status, RLF_DEV_BAD_TARGET);
+    }
+    rec[t] = make_float4(0.0f, 0.0f, 0.0f, __int_as_float(bad ? y : (y | (int)0x80000000)));
+}
+
+template <int THREADS>
+static FastKernel entropy_kernel_for_nv(int nv) {
+    switch (nv) {
+        case 1: return grpo_row_cluster_kernel<THREADS, 1, false, true>;
+        case 2: return grpo_row_cluster_kernel<THREADS, 2, false, true>;
+        case 3: return grpo_row_cluster_kernel<THREADS, 3, false, true>;
+        case 4: return grpo_row_cluster_kernel<THREADS, 4, false, true>;
+        case 5: return grpo_row_cluster_kernel<THREADS, 5, false, true>;
+        case 6: return grpo_row_cluster_kernel<THREADS, 6, false, true>;
+        case 8: return grpo_row_cluster_kernel<THREADS, 8, false, true>;
+        case 10: return grpo_row_cluster_kernel<THREADS, 10, false, true>;
+    }
+    return nullptr;
+}
+
+}  // namespace rlf
+
+extern "C" rlf_status rlf_logp_entropy_fwd(const void* logits, rlf_dtype dt, int64_t T, int32_t V,
+                                           int64_t row_stride, const int32_t* ids, float* logp_out,
+                                           float* entropy_out, void* workspace, size_t workspace_bytes,
+                                           int32_t* dev_status, rlf_stream_t stream) {
+    using namespace rlf;
+    if (dt != RLF_BF16 && dt != RLF_F32) return RLF_ERR_DTYPE;
+    if (T < 0 || V < 1 || row_stride < V) return RLF_ERR_SHAPE;
+    if (T == 0) return RLF_OK;
+    if (!logits || !ids || !logp_out) return RLF_ERR_NULL;
+    const size_t esz = dt == RLF_BF16 ? 2 : 4;
+    if (!aligned(logits, esz)) return RLF_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < loss_workspace_bytes(T)) return RLF_ERR_WORKSPACE;
+    rlf_status st = check_arch();
+    if (st != RLF_OK) return st;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    long long* one = reinterpret_cast<long long*>(ws);
+    float4* rec = reinterpret_cast<float4*>(ws + kWsRecordOff);
+    ids_to_record_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(ids, T, V, rec, one, dev_status);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+
+    const bool fast_ok = dt == RLF_BF16 && (V % 8 == 0) && (row_stride % 8 == 0) && aligned(logits, 16) &&
+                         T < (1ll << 30);
+    FastShape sh;
+    if (fast_ok && pick_shape(V >> 3, &sh)) {
+        FastKernel k = sh.threads == 256 ? entropy_kernel_for_nv<256>(sh.nv)
+                     : sh.threads == 512 ? entropy_kernel_for_nv<512>(sh.nv)
+                                         : entropy_kernel_for_nv<1024>(sh.nv);
+        if (!k) return RLF_ERR_UNSUPPORTED;
+        int nc = max_clusters(k, sh);
+        if (nc <= 0) return RLF_ERR_UNSUPPORTED;
+        if ((int64_t)nc > T) nc = (int)T;
+        FastParams p;
+        p.logits = static_cast<const __nv_bfloat16*>(logits);
+        p.grad = nullptr;
+        p.stride = row_stride;
+        p.T = (int)T;
+        p.nvec = V >> 3;
+        p.per_cta_vec = (p.nvec + sh.cluster - 1) / sh.cluster;
+        p.rec = rec;
+        p.denom = one;
+        p.logp_out = logp_out;
+        p.entropy_out = entropy_out;
+        p.dev_status = dev_status;
+        p.eps_clip = 0.0f;
+        p.beta = 0.0f;
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute at[1];
+        cluster_config(&cfg, at, nc * sh.cluster, sh, s);
+        if (cudaLaunchKernelEx(&cfg, k, p) != cudaSuccess) {
+            cudaGetLastError();
+            return RLF_ERR_CUDA;
+        }
+        count_launch();
+        return RLF_OK;
+    }
+    GenParams g;
+    g.logits = logits; g.grad = nullptr; g.stride = row_stride; g.T = T; g.V = V; g.rec = rec; g.denom = one;
+    g.logp_out = logp_out; g.entropy_out = entropy_out; g.dev_status = dev_status; g.eps_clip = 0.0f; g.beta = 0.0f;
+    g.fwd_only = 1;
+    int grid = sm_count() * 8;
+    if ((int64_t)grid > T) grid = (int)T;
+    if (dt == RLF_BF16) grpo_row_general_kernel<__nv_bfloat16><<<grid, kGenThreads, 0, s>>>(g);
+    else grpo_row_general_kernel<float><<<grid, kGenThreads, 0, s>>>(g);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
 }
 
 // ---------------------------------------------------------------------------------------------
