@@ -399,6 +399,28 @@ def run_cuda(args):
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                "loss": float(h_loss[0].item())}
 
+    # forward-only log-prob + entropy over the same logits (the old / reference policy pass): read-only
+    fwd_only = None
+    if rank == 0 and world == 1:
+        ent = torch.empty(T, dtype=torch.float32, device=dev)
+        for _ in range(2):
+            rlf.rlf_logp_entropy_fwd(batch.logits, batch.ids, logp_out=logp, entropy_out=ent, workspace=ws)
+        torch.cuda.synchronize()
+        fe = []
+        for _ in range(max(3, min(args.steps, 10))):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            rlf.rlf_logp_entropy_fwd(batch.logits, batch.ids, logp_out=logp, entropy_out=ent, workspace=ws)
+            b.record()
+            torch.cuda.synchronize()
+            fe.append(a.elapsed_time(b))
+        fms = statistics.mean(fe)
+        hbm_peak, hbm_kind = _peaks()
+        fwd_only = {"entry": "rlf_logp_entropy_fwd", "ms": fms, "tokens_per_s": T / fms * 1e3,
+                    "roofline": {"bound": "hbm", "achieved": T * V * 2 / fms / 1e6, "peak": hbm_peak, "unit": "GB/s",
+                                 "frac": T * V * 2 / fms / 1e6 / hbm_peak, "peak_kind": "of " + hbm_kind,
+                                 "traffic": None, "algorithmic_bytes": T * V * 2}}
+
     fused = None
     if rank == 0 and world == 1 and not args.skip_fused:
         fused = time_fused_lmhead(rlf, dev, max(2, min(args.steps, 5)))
@@ -438,6 +460,8 @@ def run_cuda(args):
         line["e2e"] = e2e
     if cpu_baseline is not None:
         line["cpu_baseline"] = cpu_baseline
+    if fwd_only is not None:
+        line["logp_entropy_fwd"] = fwd_only
     if fused is not None:
         line["fused_lmhead"] = fused
     print(json.dumps(line))
