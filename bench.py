@@ -421,6 +421,35 @@ def run_cuda(args):
                                  "frac": T * V * 2 / fms / 1e6 / hbm_peak, "peak_kind": "of " + hbm_kind,
                                  "traffic": None, "algorithmic_bytes": T * V * 2}}
 
+    # skip-masked variant on the same batch: rows without loss weight are neither read nor computed
+    skip_masked = None
+    if rank == 0 and world == 1:
+        g2 = torch.empty_like(batch.logits)
+        skip_masked = {"entry": "rlf_grpo_logp_loss_fwd_bwd_skip_masked", "live_fraction": float(mask.float().mean().item())}
+        for zero in (True, False):
+            def run_skip():
+                rlf.rlf_grpo_logp_loss_fwd_bwd_skip_masked(batch.logits, batch.ids, seq_id, adv, batch.old_logp,
+                                                           batch.ref_logp, mask, synth.EPS_CLIP, synth.BETA_KL,
+                                                           denom=n_tok, grad_logits=g2, zero_masked_grad=zero,
+                                                           logp_out=logp, loss_out=loss, workspace=ws)
+            for _ in range(2):
+                run_skip()
+            torch.cuda.synchronize()
+            ts = []
+            for _ in range(max(3, min(args.steps, 10))):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                run_skip()
+                b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            sms = statistics.mean(ts)
+            n_live = int(mask.sum().item())
+            moved = n_live * V * 4 + ((T - n_live) * V * 2 if zero else 0)
+            skip_masked["zero_fill" if zero else "no_fill"] = {"ms": sms, "tokens_per_s": T / sms * 1e3,
+                                                               "algorithmic_bytes": moved, "gbs": moved / sms / 1e6}
+        del g2
+
     fused = None
     if rank == 0 and world == 1 and not args.skip_fused:
         fused = time_fused_lmhead(rlf, dev, max(2, min(args.steps, 5)))
@@ -462,6 +491,8 @@ def run_cuda(args):
         line["cpu_baseline"] = cpu_baseline
     if fwd_only is not None:
         line["logp_entropy_fwd"] = fwd_only
+    if skip_masked is not None:
+        line["skip_masked"] = skip_masked
     if fused is not None:
         line["fused_lmhead"] = fused
     print(json.dumps(line))

@@ -148,6 +148,30 @@ rlf_status rlf_grpo_logp_loss_fwd_bwd(const void *logits, rlf_dtype dt, int64_t 
                                       int32_t *dev_status, rlf_stream_t stream);
 
 /*
+ * rlf_grpo_logp_loss_fwd_bwd that neither reads nor computes rows without loss weight.  (Paper
+ * Sec. 2.2 / Sec. 2.3.2: observation tokens take no part in the loss; in multi-turn tool-use batches
+ * they are a large share of all tokens, so their logits rows need not be touched at all.)
+ * Rows with mask 0 (and rows neutralised for a bad target / sequence id) are skipped:
+ *   - logp_out[t] of a skipped row is NaN;
+ *   - its grad_logits row is written as zeros if zero_masked_grad != 0, and left untouched
+ *     otherwise (for callers that zero the buffer themselves or never read those rows);
+ *   - loss_out and the live rows' logp / grad are exactly those of rlf_grpo_logp_loss_fwd_bwd.
+ * Arguments otherwise as for rlf_grpo_logp_loss_fwd_bwd; same workspace size.  HBM traffic is
+ * 4 V bytes per live token plus 2 V per skipped token that is zero-filled.  Logits that do not
+ * qualify for the fast path are processed in full by the general kernel (same results).
+ */
+rlf_status rlf_grpo_logp_loss_fwd_bwd_skip_masked(const void *logits, rlf_dtype dt, int64_t T, int32_t V,
+                                                  int64_t row_stride, const int32_t *ids,
+                                                  const int32_t *seq_id, const float *adv, int32_t B,
+                                                  const float *old_logp, const float *ref_logp,
+                                                  const uint8_t *mask, float eps_clip, float beta_kl,
+                                                  const int64_t *denom, float *logp_out,
+                                                  double *loss_out, void *grad_logits,
+                                                  int zero_masked_grad, void *workspace,
+                                                  size_t workspace_bytes, int32_t *dev_status,
+                                                  rlf_stream_t stream);
+
+/*
  * Forward-only log-prob of given target tokens, and the entropy of each row's distribution: the pass
  * that produces old_logp / ref_logp for the update above (the behaviour and reference policies of
  * the PPO-style update, paper Sec. 2.3.1; the policy pi_theta(a | s_t) of Sec. 2.2).  Per row t:

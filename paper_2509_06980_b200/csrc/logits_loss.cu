@@ -46,7 +46,12 @@ constexpr int kMaxPartials = 1024;
 constexpr size_t kWsPartialOff = 256;
 constexpr size_t kWsRecordOff = kWsPartialOff + sizeof(double) * 4 * kMaxPartials;
 
-size_t loss_workspace_bytes(int64_t T) { return kWsRecordOff + 16 * (size_t)(T > 0 ? T : 0) + 256; }
+// the skip-masked variant adds, after the records: compacted records (16 B per token), the list of
+// live rows (4 B per token); its live-row counter sits at byte 128 of the workspace
+static size_t ws_tokens(int64_t T) { return (size_t)(T > 0 ? T : 0); }
+static size_t ws_compact_rec_off(int64_t T) { return kWsRecordOff + 16 * ws_tokens(T) + 256; }
+static size_t ws_row_list_off(int64_t T) { return ws_compact_rec_off(T) + 16 * ws_tokens(T) + 256; }
+size_t loss_workspace_bytes(int64_t T) { return ws_row_list_off(T) + 4 * ws_tokens(T) + 256; }
 
 // ---------------------------------------------------------------------------------------------
 // token records
@@ -146,6 +151,9 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
 __device__ __forceinline__ void cp_async16_cg(void* smem_dst, const void* gmem_src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
 }
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" :: "r"(smem_u32(smem_dst)), "l"(gmem_src) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_group1() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
@@ -163,6 +171,8 @@ struct FastParams {
     const long long* denom;
     float* logp_out;
     float* entropy_out;         // entropy variant only, nullable
+    const int* row_list;        // skip-masked variant: rows to process, rec[] is indexed like this list
+    const int* n_rows;          // skip-masked variant: device count of listed rows
     int32_t* dev_status;
     float eps_clip, beta;
 };
@@ -292,7 +302,9 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t mbar, uint32_t parity
     return false;
 }
 
-template <int THREADS, int NV, bool ONE_EXP, bool ENT = false>
+// SKIP: the rows to process come from a compacted list (rows whose loss weight is zero are
+// neither read nor computed); token records are then indexed like the list.
+template <int THREADS, int NV, bool ONE_EXP, bool ENT = false, bool SKIP = false>
 __global__ void __launch_bounds__(THREADS, ctas_per_sm(THREADS, NV))
 grpo_row_cluster_kernel(const FastParams p) {
     constexpr int NWARPS = THREADS / 32;
@@ -301,7 +313,10 @@ grpo_row_cluster_kernel(const FastParams p) {
     // cp.async wait is all the synchronisation the logits data needs
     extern __shared__ __align__(16) uint4 stage[];
     __shared__ __align__(8) float2 pair_slot[2][MAXE];   // per row parity: every warp's (max, sum)
-    __shared__ __align__(16) float4 rec_slot[4];         // token records, ring over rows
+    constexpr int RM = SKIP ? 7 : 3;                     // ring mask of the per-row metadata
+    constexpr int AHEAD = SKIP ? 3 : 2;                  // how many rows ahead thread 0 fetches metadata
+    __shared__ __align__(16) float4 rec_slot[RM + 1];    // token records, ring over rows
+    __shared__ int row_slot[SKIP ? 8 : 1];               // skip variant: row index of each listed row
     __shared__ float zy_slot[2];                         // per row parity: the target logit
     __shared__ float ent_slot[2][ENT ? MAXE : 1];        // entropy variant: every warp's sum 2^x * x
     __shared__ __align__(8) unsigned long long row_bar[2];   // per row parity: "all pairs and z_target are here"
@@ -325,18 +340,27 @@ grpo_row_cluster_kernel(const FastParams p) {
         inv_n = 1.0f / (float)(N > 1 ? N : 1);
     }
 
-    // queue this thread's part of a row into the staging buffer (one cp.async group per row;
-    // thread 0's group also carries the token record of the row after it, into ring slot `rslot`)
-    auto prefetch = [&](int row, int rslot) {
-        if (row < p.T) {
+    const int nrows = SKIP ? *p.n_rows : p.T;
+    // thread 0 fetches the metadata of the row this cluster handles in iteration `j` (its token
+    // record; in the skip variant also its row index) into the rings
+    auto fetch_meta = [&](int j) {
+        const long long k = (long long)cluster_id + (long long)j * num_clusters;
+        if (tid == 0 && j >= 0 && k < nrows) {
+            cp_async16(&rec_slot[j & RM], p.rec + k);
+            if (SKIP) cp_async4(&row_slot[j & RM], p.row_list + k);
+        }
+    };
+    // queue this thread's part of a row into the staging buffer (one cp.async group per row; thread
+    // 0's group also carries metadata of a later row)
+    auto prefetch = [&](int row, bool have, int meta_j) {
+        if (have) {
             const uint4* src = reinterpret_cast<const uint4*>(p.logits + (long long)row * p.stride) + vbeg;
             uint4* dst = stage + tid;
 #pragma unroll
             for (int i = 0; i < NV; ++i)
                 if (i < nvalid) cp_async16_cg(dst + i * THREADS, src + i * THREADS);
         }
-        if (tid == 0 && row + num_clusters < p.T)
-            cp_async16(&rec_slot[rslot & 3], p.rec + row + num_clusters);
+        fetch_meta(meta_j);
         cp_async_commit();
     };
 
@@ -346,21 +370,33 @@ grpo_row_cluster_kernel(const FastParams p) {
         mbar_init(smem_u32(&row_bar[0]), 1);
         mbar_init(smem_u32(&row_bar[1]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        if (cluster_id < p.T) cp_async16(&rec_slot[0], p.rec + cluster_id);
     }
-    prefetch(cluster_id, 1);             // first row of this cluster (+ record of its second row)
-    cp_async_wait_all();                 // the first two records must be visible CTA-wide below
+    for (int j = 0; j < AHEAD; ++j) fetch_meta(j);
+    if (SKIP) {
+        // the first row's index is needed to start its copy
+        cp_async_wait_all();
+        __syncthreads();
+    }
+    {
+        const bool have0 = cluster_id < nrows;
+        const int row0 = SKIP ? (have0 ? row_slot[0] : 0) : cluster_id;
+        prefetch(row0, have0, -1);       // first row of this cluster (no further metadata yet)
+    }
+    cp_async_wait_all();                 // the first records must be visible CTA-wide below
     // every CTA of the cluster is running before any peer may address its shared memory
     cluster_sync_all();
 
     int status = 0;
     int it = 0;
     bool gave_up = false;                // a wait ran out: stop waiting, finish the loop, report
-    for (int row = cluster_id; row < p.T; row += num_clusters, ++it) {
+    for (int k = cluster_id; k < nrows; k += num_clusters, ++it) {
         const int parity = it & 1;
+        const int row = SKIP ? row_slot[it & RM] : k;
         const uint32_t bar = smem_u32(&row_bar[parity]);
+        cp_async_wait_all();             // this thread's part of the row (and thread 0's metadata) has landed
+        // an arrive releases what this thread did before it: the landed metadata becomes visible to
+        // every thread that later sees this barrier's phase complete
         if (tid == 0) mbar_arrive_expect_tx(bar, row_bytes);
-        cp_async_wait_all();             // this thread's part of the row has landed
         uint4 d[NV];
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
@@ -370,7 +406,7 @@ grpo_row_cluster_kernel(const FastParams p) {
 
         // max over the registers (packed), then over the warp; the owner of the target column
         // sends z_target to every CTA of the cluster
-        const int y = __float_as_int(rec_slot[it & 3].w) & 0x7fffffff;
+        const int y = __float_as_int(rec_slot[it & RM].w) & 0x7fffffff;
         const int yrel = (y >> 3) - vbeg;             // owner iff a multiple of THREADS below nvalid * THREADS
         const bool owner = yrel >= 0 && (yrel & (THREADS - 1)) == 0 && (yrel / THREADS) < nvalid;
         uint32_t mx = kNegInfPair;
@@ -385,7 +421,11 @@ grpo_row_cluster_kernel(const FastParams p) {
         }
         // the staging slots have been consumed (the max needed every register): refill them with
         // the cluster's next row while this one is processed
-        prefetch(row + num_clusters, it + 2);
+        {
+            const bool have_next = k + num_clusters < nrows;
+            const int next_row = SKIP ? (have_next ? row_slot[(it + 1) & RM] : 0) : k + num_clusters;
+            prefetch(next_row, have_next, it + AHEAD);
+        }
 
         float m_w = fmaxf(bf_lo(mx), bf_hi(mx));
         m_w = ord2f(__reduce_max_sync(0xffffffffu, f2ord(m_w)));
@@ -442,7 +482,7 @@ grpo_row_cluster_kernel(const FastParams p) {
         S = warp_sum(S);
         if (ENT) U = warp_sum(U);
         const float zy = zy_slot[parity];
-        const float4 rec = rec_slot[it & 3];
+        const float4 rec = rec_slot[it & RM];
         const float lg2s = lg2_approx(S);
         const float logp = (zy - M) - lg2s * kLn2;
         const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) &&
@@ -863,6 +903,8 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
             p.eps_clip = a.eps_clip;
             p.beta = a.beta;
             p.entropy_out = nullptr;
+            p.row_list = nullptr;
+            p.n_rows = nullptr;
             cudaLaunchConfig_t cfg;
             cudaLaunchAttribute at[1];
             cluster_config(&cfg, at, nc * sh.cluster, sh, s);
@@ -1023,6 +1065,8 @@ extern "C" rlf_status rlf_logp_entropy_fwd(const void* logits, rlf_dtype dt, int
         p.denom = one;
         p.logp_out = logp_out;
         p.entropy_out = entropy_out;
+        p.row_list = nullptr;
+        p.n_rows = nullptr;
         p.dev_status = dev_status;
         p.eps_clip = 0.0f;
         p.beta = 0.0f;
@@ -1046,6 +1090,160 @@ extern "C" rlf_status rlf_logp_entropy_fwd(const void* logits, rlf_dtype dt, int
     else grpo_row_general_kernel<float><<<grid, kGenThreads, 0, s>>>(g);
     count_launch();
     return cuda_ok(cudaGetLastError());
+}
+
+// ---------------------------------------------------------------------------------------------
+// Skip-masked variant: rows with zero loss weight are neither read nor computed.
+namespace rlf {
+
+// live rows (record's live bit) -> compacted list of row indices and of their records, in arbitrary
+// order (rows are independent, so the order does not affect any result)
+__global__ void __launch_bounds__(256)
+compact_live_kernel(const float4* __restrict__ rec, int64_t T, int* __restrict__ row_list,
+                    float4* __restrict__ rec_c, int* __restrict__ counter) {
+    const int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    bool live = false;
+    if (t < T) {
+        r = rec[t];
+        live = __float_as_int(r.w) < 0;
+    }
+    const unsigned m = __ballot_sync(0xffffffffu, live);
+    if (m == 0) return;
+    const int lane = threadIdx.x & 31;
+    int base = 0;
+    if (lane == 0) base = atomicAdd(counter, __popc(m));
+    base = __shfl_sync(0xffffffffu, base, 0);
+    if (live) {
+        const int k = base + __popc(m & ((1u << lane) - 1u));
+        row_list[k] = (int)t;
+        rec_c[k] = r;
+    }
+}
+
+// rows that are not live: log-prob NaN and (optionally) an all-zero gradient row
+template <typename T>
+__global__ void __launch_bounds__(256)
+fill_dead_rows_kernel(const float4* __restrict__ rec, int64_t Tn, int32_t V, long long stride, T* __restrict__ grad,
+                      int zero_grad, float* __restrict__ logp_out) {
+    for (int64_t row = blockIdx.x; row < Tn; row += gridDim.x) {
+        if (__float_as_int(rec[row].w) < 0) continue;
+        if (threadIdx.x == 0) logp_out[row] = __int_as_float(0x7fc00000);
+        if (grad == nullptr || !zero_grad) continue;
+        T* g = grad + row * stride;
+        const bool vec = (sizeof(T) * V) % 16 == 0 && (reinterpret_cast<uintptr_t>(g) % 16) == 0;
+        if (vec) {
+            uint4* g4 = reinterpret_cast<uint4*>(g);
+            const int n4 = (int)(sizeof(T) * V / 16);
+            for (int i = threadIdx.x; i < n4; i += 256) st_stream(g4 + i, make_uint4(0u, 0u, 0u, 0u));
+        } else {
+            for (int v = threadIdx.x; v < V; v += 256) g[v] = from_f32<T>(0.0f);
+        }
+    }
+}
+
+template <int THREADS>
+static FastKernel skip_kernel_for_nv(int nv) {
+    switch (nv) {
+        case 1: return grpo_row_cluster_kernel<THREADS, 1, true, false, true>;
+        case 2: return grpo_row_cluster_kernel<THREADS, 2, true, false, true>;
+        case 3: return grpo_row_cluster_kernel<THREADS, 3, true, false, true>;
+        case 4: return grpo_row_cluster_kernel<THREADS, 4, true, false, true>;
+        case 5: return grpo_row_cluster_kernel<THREADS, 5, true, false, true>;
+        case 6: return grpo_row_cluster_kernel<THREADS, 6, true, false, true>;
+        case 8: return grpo_row_cluster_kernel<THREADS, 8, true, false, true>;
+        case 10: return grpo_row_cluster_kernel<THREADS, 10, true, false, true>;
+    }
+    return nullptr;
+}
+
+}  // namespace rlf
+
+extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd_skip_masked(
+    const void* logits, rlf_dtype dt, int64_t T, int32_t V, int64_t row_stride, const int32_t* ids,
+    const int32_t* seq_id, const float* adv, int32_t B, const float* old_logp, const float* ref_logp,
+    const uint8_t* mask, float eps_clip, float beta_kl, const int64_t* denom, float* logp_out,
+    double* loss_out, void* grad_logits, int zero_masked_grad, void* workspace, size_t workspace_bytes,
+    int32_t* dev_status, rlf_stream_t stream) {
+    using namespace rlf;
+    if (dt != RLF_BF16 && dt != RLF_F32) return RLF_ERR_DTYPE;
+    if (T < 0 || V < 1 || B < 0 || row_stride < V) return RLF_ERR_SHAPE;
+    if (!loss_out) return RLF_ERR_NULL;
+    if (T > 0 && (!logits || !ids || !seq_id || !adv || !old_logp || !ref_logp || !mask || !logp_out))
+        return RLF_ERR_NULL;
+    if (T > 0 && B == 0) return RLF_ERR_SHAPE;
+    const size_t esz = dt == RLF_BF16 ? 2 : 4;
+    if (!aligned(logits, esz) || !aligned(grad_logits, esz)) return RLF_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < loss_workspace_bytes(T)) return RLF_ERR_WORKSPACE;
+    const bool fast_ok = dt == RLF_BF16 && (V % 8 == 0) && (row_stride % 8 == 0) && aligned(logits, 16) &&
+                         aligned(grad_logits, 16) && T < (1ll << 30);
+    FastShape sh;
+    if (T == 0 || !fast_ok || !pick_shape(V >> 3, &sh)) {
+        // nothing to gain on the general path: process every row, then mark the dead rows' log-probs
+        rlf_status st0 = rlf_grpo_logp_loss_fwd_bwd(logits, dt, T, V, row_stride, ids, seq_id, adv, B, old_logp, ref_logp,
+                                                    mask, eps_clip, beta_kl, denom, logp_out, loss_out, grad_logits,
+                                                    workspace, workspace_bytes, dev_status, stream);
+        if (st0 != RLF_OK || T == 0) return st0;
+        const float4* rec0 = reinterpret_cast<const float4*>(static_cast<char*>(workspace) + kWsRecordOff);
+        fill_dead_rows_kernel<float><<<sm_count() * 4, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+            rec0, T, V, row_stride, nullptr, 0, logp_out);
+        count_launch();
+        return cuda_ok(cudaGetLastError());
+    }
+    rlf_status st = check_arch();
+    if (st != RLF_OK) return st;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    long long* n_count = reinterpret_cast<long long*>(ws);
+    int* n_live = reinterpret_cast<int*>(ws + 128);
+    double* partial = reinterpret_cast<double*>(ws + kWsPartialOff);
+    float4* rec = reinterpret_cast<float4*>(ws + kWsRecordOff);
+    float4* rec_c = reinterpret_cast<float4*>(ws + ws_compact_rec_off(T));
+    int* row_list = reinterpret_cast<int*>(ws + ws_row_list_off(T));
+    if (cudaMemsetAsync(ws, 0, 256, s) != cudaSuccess) return RLF_ERR_CUDA;
+    const long long* dn = denom ? reinterpret_cast<const long long*>(denom) : n_count;
+    st = launch_token_prep(ids, seq_id, adv, old_logp, ref_logp, mask, T, V, B, rec, denom ? nullptr : n_count,
+                           dev_status, s);
+    if (st != RLF_OK) return st;
+    compact_live_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(rec, T, row_list, rec_c, n_live);
+    count_launch();
+    fill_dead_rows_kernel<__nv_bfloat16><<<sm_count() * 4, 256, 0, s>>>(
+        rec, T, V, row_stride, static_cast<__nv_bfloat16*>(grad_logits), zero_masked_grad, logp_out);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+
+    FastKernel k = sh.threads == 256 ? skip_kernel_for_nv<256>(sh.nv)
+                 : sh.threads == 512 ? skip_kernel_for_nv<512>(sh.nv)
+                                     : skip_kernel_for_nv<1024>(sh.nv);
+    if (!k) return RLF_ERR_UNSUPPORTED;
+    int nc = max_clusters(k, sh);
+    if (nc <= 0) return RLF_ERR_UNSUPPORTED;
+    if ((int64_t)nc > T) nc = (int)T;
+    FastParams p;
+    p.logits = static_cast<const __nv_bfloat16*>(logits);
+    p.grad = static_cast<__nv_bfloat16*>(grad_logits);
+    p.stride = row_stride;
+    p.T = (int)T;
+    p.nvec = V >> 3;
+    p.per_cta_vec = (p.nvec + sh.cluster - 1) / sh.cluster;
+    p.rec = rec_c;
+    p.denom = dn;
+    p.logp_out = logp_out;
+    p.entropy_out = nullptr;
+    p.row_list = row_list;
+    p.n_rows = n_live;
+    p.dev_status = dev_status;
+    p.eps_clip = eps_clip;
+    p.beta = beta_kl;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute at[1];
+    cluster_config(&cfg, at, nc * sh.cluster, sh, s);
+    if (cudaLaunchKernelEx(&cfg, k, p) != cudaSuccess) {
+        cudaGetLastError();
+        return RLF_ERR_CUDA;
+    }
+    count_launch();
+    return launch_token_loss(logp_out, rec, T, eps_clip, beta_kl, partial, dn, loss_out, s);
 }
 
 // ---------------------------------------------------------------------------------------------
