@@ -106,6 +106,14 @@ rlf_status rlf_group_advantage(const float *rewards, const int32_t *group_id, in
                                float *adv_out, int32_t *dev_status, rlf_stream_t stream);
 
 /*
+ * Rule reward.  (Paper Eq. 1: R_rule = sum_i w_i r_i over the n rule dimensions, e.g. call-format
+ * validity, task completion, efficiency.)  The result feeds rlf_group_advantage as `rewards`.
+ *   scores [B, n] fp32 row-major;  weights [n] fp32;  reward_out [B] fp32 (fp64 accumulation)
+ */
+rlf_status rlf_rule_reward(const float *scores, const float *weights, int32_t B, int32_t n,
+                           float *reward_out, rlf_stream_t stream);
+
+/*
  * Fused log-prob + clipped-ratio + k3-KL loss, forward and backward, over
  * materialised logits.  (Paper Sec. 2.2: the policy pi_theta(a | s_t); Sec.
  * 2.3.1: PPO-style update of the RL trainer; Sec. 2.3.2: GRPO with the loss

@@ -31,9 +31,11 @@ def build(force=False):
 
 
 def lib():
+    """The compiled oracle.  RLF_ORACLE_LIB names another build of it (used by the mutation tests,
+    which check that the pins notice a planted mistake)."""
     global _lib
     if _lib is None:
-        _lib = ctypes.CDLL(build())
+        _lib = ctypes.CDLL(os.environ.get("RLF_ORACLE_LIB") or build())
     return _lib
 
 

@@ -18,7 +18,7 @@ FN_LOGP_LOSS, FN_FUSED_LMHEAD = 3, 4
 DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
 
 EXPORTS = [
-    "rlf_build_loss_mask", "rlf_group_advantage", "rlf_grpo_logp_loss_fwd_bwd",
+    "rlf_build_loss_mask", "rlf_group_advantage", "rlf_rule_reward", "rlf_grpo_logp_loss_fwd_bwd",
     "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_grpo_logp_loss_fwd_bwd_skip_masked", "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
     "rlf_tune_logits_kernel", "rlf_tune_lmhead", "rlf_launch_count", "rlf_status_string", "rlf_version",
 ]
@@ -155,6 +155,18 @@ def rlf_group_advantage(rewards, group_size=None, group_id=None, num_groups=None
                                     float(eps), 1 if unbiased_std else 0, _ptr(adv_out, torch.float32),
                                     _ptr(dev_status, torch.int32), _stream()), "rlf_group_advantage")
     return adv_out
+
+
+def rlf_rule_reward(scores, weights, reward_out=None):
+    """Eq. 1: weighted sum of rule scores.  scores [B, n], weights [n] -> rewards fp32[B]."""
+    B, n = scores.shape
+    if reward_out is None:
+        reward_out = torch.empty(B, dtype=torch.float32, device=scores.device)
+    _lib.rlf_rule_reward.argtypes = [_vp, _vp, _i32, _i32, _vp, _vp]
+    _lib.rlf_rule_reward.restype = _int
+    _check(_lib.rlf_rule_reward(_ptr(scores, torch.float32), _ptr(weights, torch.float32), B, n,
+                                _ptr(reward_out, torch.float32), _stream()), "rlf_rule_reward")
+    return reward_out
 
 
 def rlf_grpo_logp_loss_fwd_bwd(logits, ids, seq_id, adv, old_logp, ref_logp, mask, eps_clip, beta_kl,

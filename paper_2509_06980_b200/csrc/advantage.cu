@@ -76,3 +76,32 @@ extern "C" rlf_status rlf_group_advantage(const float* rewards, const int32_t* g
     count_launch();
     return cuda_ok(cudaGetLastError());
 }
+
+// ---------------------------------------------------------------------------------------------
+// Rule reward (paper Eq. 1): R_b = sum_i w_i r_{b,i}.  One thread per response, fp64 accumulation in
+// index order (n is a handful of rule dimensions).
+namespace rlf {
+__global__ void __launch_bounds__(128)
+rule_reward_kernel(const float* __restrict__ scores, const float* __restrict__ weights, int32_t B, int32_t n,
+                   float* __restrict__ reward_out) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    double acc = 0.0;
+    for (int i = 0; i < n; ++i) acc += (double)weights[i] * (double)scores[(long long)b * n + i];
+    reward_out[b] = (float)acc;
+}
+}  // namespace rlf
+
+extern "C" rlf_status rlf_rule_reward(const float* scores, const float* weights, int32_t B, int32_t n,
+                                      float* reward_out, rlf_stream_t stream) {
+    using namespace rlf;
+    if (B < 0 || n < 0) return RLF_ERR_SHAPE;
+    if (B == 0) return RLF_OK;
+    if (!reward_out || (n > 0 && (!scores || !weights))) return RLF_ERR_NULL;
+    rlf_status st = check_arch();
+    if (st != RLF_OK) return st;
+    rule_reward_kernel<<<(B + 127) / 128, 128, 0, reinterpret_cast<cudaStream_t>(stream)>>>(scores, weights, B, n,
+                                                                                          reward_out);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}

@@ -297,3 +297,18 @@ def test_whole_step_from_host_buffers():
     assert loss_close(h_loss[0].item(), ora["loss"][0], 1e-6, 1e-4)
     grad = arena[: T * V * 2].view(torch.bfloat16).view(T, V)
     assert ulp_error_bf16(gc.grad_to_f64(grad), ora["grad"]).max() <= gc.GRAD_ULPS
+
+
+def test_rule_reward_eq1_feeds_the_advantage():
+    b = gc.binding()
+    rng = np.random.default_rng(8)
+    B, n = 24, 3
+    scores = rng.random((B, n)).astype(np.float32)
+    w = np.array([0.2, 1.0, -0.05], np.float32)
+    want = orc.rule_reward(scores, w)
+    got = b.rlf_rule_reward(torch.from_numpy(scores).to(DEV), torch.from_numpy(w).to(DEV))
+    adv = b.rlf_group_advantage(got, group_size=8)
+    torch.cuda.synchronize()
+    assert np.abs(got.cpu().numpy() - want).max() <= 1e-7 * np.abs(want).max()
+    want_adv = orc.group_advantage(got.cpu().numpy(), group_size=8)
+    assert np.allclose(adv.cpu().numpy(), want_adv, rtol=2e-7, atol=1e-30)
