@@ -237,10 +237,18 @@ rlf_status rlf_grpo_logp_loss_fwd_bwd_static(const void *logits, rlf_dtype dt, i
  *     grad_hidden[t,:] = sum_v grad_z[t,v] W[v,:]       (bf16)
  *     grad_W[v,:]      = sum_t grad_z[t,v] hidden[t,:]  (fp32; added to the buffer if accumulate_grad_W)
  *
- *   hidden [T, D] bf16 row-major;  W [V, D] bf16 row-major; both 16-byte aligned, D a multiple of 64
+ *   hidden [T, D] bf16 row-major;  W [V, D] bf16 row-major; both 16-byte aligned, D a multiple of
+ *               64 and V a multiple of 8 (else RLF_ERR_SHAPE)
  *   per-token arguments, denom, logp_out, loss_out: as for rlf_grpo_logp_loss_fwd_bwd
- *   grad_hidden [T, D] bf16 or NULL;  grad_W [V, D] fp32 or NULL
- *   workspace   rlf_workspace_bytes(RLF_FN_FUSED_LMHEAD, T, V, D, RLF_BF16) bytes, 256-byte aligned
+ *   grad_hidden [T, D] bf16 or NULL;  grad_W [V, D] fp32 or NULL (both NULL: forward only)
+ *   workspace   rlf_workspace_bytes(RLF_FN_FUSED_LMHEAD, T, V, D, RLF_BF16) bytes, 256-byte aligned.
+ *               It holds per-token records and partial sums and, for the backward, one chunk of
+ *               dZ = grad_z as bf16, [min(T, 9472), V] (2.9 GB at V = 151936): the logits are never
+ *               stored, this chunk of their gradient is, between the kernel that forms it and the
+ *               two contractions that consume it.
+ * Tensor-core contractions are bf16 x bf16 with fp32 accumulation in tensor memory; grad_z is
+ * rounded to bf16 before the two gradient contractions.  Waits inside the kernels are bounded: if
+ * one runs out, RLF_DEV_TIMEOUT is set in *dev_status and the outputs are not valid.
  */
 rlf_status rlf_fused_lmhead_grpo(const void *hidden, const void *W, int64_t T, int32_t D, int32_t V,
                                  const int32_t *ids, const int32_t *seq_id, const float *adv,
