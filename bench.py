@@ -58,10 +58,10 @@ def _tensor_peaks():
     return 1590.0, 1400.0, "fallback"
 
 
-def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0):
+def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3):
     """The fused LM-head variant on the Qwen3-4B head (T = 32768, D = 2560, V = 151936): forward
     (log-probs and loss, logits never stored) and forward + backward (grad_hidden, grad_W)."""
-    spec = synth.SPECS[3]
+    spec = synth.SPECS[cfg]
     if tokens_per_response:
         spec = synth.scaled(spec, len_lo=tokens_per_response, len_hi=tokens_per_response)
     tok = synth.make_tokens(spec)
@@ -86,7 +86,7 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0):
                                   want_grad_hidden=bwd, want_grad_W=bwd, grad_hidden=gh if bwd else None,
                                   grad_W=gw if bwd else None, logp_out=logp, loss_out=loss, workspace=ws,
                                   dev_status=st)
-    out = {"workload": "cfg3_fused_lmhead_4b: hidden [%d, 2560] x W [151936, 2560] bf16" % T, "T": T, "D": spec.D,
+    out = {"workload": "%s: hidden [%d, %d] x W [151936, %d] bf16" % (spec.name, T, spec.D, spec.D), "T": T, "D": spec.D,
            "V": spec.V}
     burst, sustained, kind = _tensor_peaks()
     for name, bwd, gemms, executed in (("fwd", False, 1, 1), ("fwd_bwd", True, 3, 4)):
@@ -285,13 +285,84 @@ def run_fused_only(args):
     print(json.dumps({"fused_lmhead": out, "gpu_launches": rlf.launch_count()}))
 
 
+def run_other_configs(args):
+    """The configurations that are parity cases rather than the headline: cfg 2 (ragged packing, ~133k
+    tokens, logits processed in place) and cfg 4 (8 micro-batches of 8192 tokens with a global
+    denominator; logits path and fused LM-head path).  Prints one JSON line."""
+    from paper_2509_06980_b200 import binding as rlf
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    steps = max(2, min(args.steps, 5))
+    out = {}
+
+    def timed(fn, n):
+        fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(n):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return statistics.mean(ts)
+
+    # cfg 2: in place over the whole packed batch (the gradient overwrites the logits, so every timed
+    # call sees the previous call's output as its logits: same bytes moved, values irrelevant to time)
+    spec = synth.SPECS[2]
+    batch = synth.make_batch(spec, dev)
+    T, V = batch.T, spec.V
+    mask, seq, n = rlf.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, spec.open_id, spec.close_id)
+    adv = rlf.rlf_group_advantage(batch.rewards, group_size=spec.group_size)
+    ws = rlf.new_workspace(rlf.FN_LOGP_LOSS, T, V)
+    logp = torch.empty(T, dtype=torch.float32, device=dev)
+    loss = torch.empty(4, dtype=torch.float64, device=dev)
+    ms = timed(lambda: rlf.rlf_grpo_logp_loss_fwd_bwd(batch.logits, batch.ids, seq, adv, batch.old_logp, batch.ref_logp,
+                                                      mask, synth.EPS_CLIP, synth.BETA_KL, denom=n, in_place=True,
+                                                      logp_out=logp, loss_out=loss, workspace=ws), steps)
+    out["cfg2_ragged_in_place"] = {"T": T, "responses": batch.B, "ms": ms, "tokens_per_s": T / ms * 1e3,
+                                   "logits_gbs": T * V * 4 / ms / 1e6, "logits_gb": T * V * 2 / 1e9}
+    del batch, ws
+    torch.cuda.empty_cache()
+
+    # cfg 4, logits path: 8 micro-batches of one 8192-token response, global denominator
+    spec = synth.SPECS[4]
+    tok = synth.make_tokens(spec)
+    T = len(tok.ids)
+    ids = torch.from_numpy(tok.ids).to(dev)
+    cu = torch.from_numpy(tok.cu_seqlens).to(dev)
+    mask, seq, n = rlf.rlf_build_loss_mask(ids, cu, spec.open_id, spec.close_id)
+    adv = rlf.rlf_group_advantage(torch.from_numpy(tok.rewards).to(dev), group_size=spec.group_size)
+    mb = 8192
+    logits = synth.make_logits(synth.scaled(spec, D=0), mb, dev)      # one micro-batch worth, reused
+    grad = torch.empty_like(logits)
+    old = torch.full((T,), -14.0, device=dev)
+    ws = rlf.new_workspace(rlf.FN_LOGP_LOSS, mb, V)
+    logp = torch.empty(mb, dtype=torch.float32, device=dev)
+
+    def logits_path():
+        for i in range(T // mb):
+            sl = slice(i * mb, (i + 1) * mb)
+            rlf.rlf_grpo_logp_loss_fwd_bwd(logits, ids[sl], seq[sl], adv, old[sl], old[sl], mask[sl], synth.EPS_CLIP,
+                                           synth.BETA_KL, denom=n, grad_logits=grad, logp_out=logp, loss_out=loss,
+                                           workspace=ws)
+    ms = timed(logits_path, steps)
+    out["cfg4_logits_path_8_microbatches"] = {"T": T, "ms": ms, "tokens_per_s": T / ms * 1e3,
+                                              "logits_gbs": T * V * 4 / ms / 1e6}
+    del logits, grad, ws
+    torch.cuda.empty_cache()
+    out["cfg4_fused_lmhead"] = time_fused_lmhead(rlf, dev, 2, 0, cfg=4)
+    print(json.dumps({"other_configs": out, "gpu_launches": rlf.launch_count()}))
+
+
 def run_cuda(args):
     rank, world, local = dist_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
-    if args.fused_only:
+    if args.fused_only or args.other_configs:
         if rank == 0:
-            run_fused_only(args)
+            run_other_configs(args) if args.other_configs else run_fused_only(args)
         return
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
@@ -509,6 +580,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--skip-fused", action="store_true", help="do not time the fused LM-head variant")
     ap.add_argument("--fused-only", action="store_true", help="time only the fused LM-head variant (rank 0)")
+    ap.add_argument("--other-configs", action="store_true",
+                    help="time cfg 2 (ragged, in place) and cfg 4 (micro-batched; both paths) instead (rank 0)")
     ap.add_argument("--tokens-per-response", type=int, default=0,
                     help="smaller micro-batch of the same recipe (profiling captures); 0 = the full 2048")
     args = ap.parse_args()
