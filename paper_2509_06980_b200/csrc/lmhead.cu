@@ -650,7 +650,25 @@ static rlf_status launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, cons
 // rows of dZ held in scratch at a time: 74 token tiles, so that the dZ sweep (74 x 4 units) and the
 // grad_hidden contraction (74 x D/256 tiles) fill whole waves of 148 SMs
 constexpr int kChunkTokens = 74 * BM;
-constexpr int kSplit = 4;                   // vocabulary splits of the forward sweep
+constexpr int kMaxSplit = 64;               // most vocabulary splits a sweep may use (sizes the partials)
+
+// Number of vocabulary splits for a sweep over m_units row units and n_tiles column tiles on
+// `workers` CTAs (or CTA pairs): the smallest count >= 4 whose m_units * splits work units fill
+// whole waves best, each split keeping at least 8 column tiles.
+static int pick_split(int m_units, int n_tiles, int workers) {
+    int best = 1;
+    double best_eff = 0.0;
+    for (int sp = 1; sp <= kMaxSplit; ++sp) {
+        const int per = (n_tiles + sp - 1) / sp;
+        if (sp > 1 && per < 8) break;
+        const int used = (n_tiles + per - 1) / per;            // splits that actually hold tiles
+        const long long units = (long long)m_units * used;
+        const long long waves = (units + workers - 1) / workers;
+        const double eff = (double)units / (double)(waves * workers) * ((double)n_tiles / (double)(per * used));
+        if (eff > best_eff + 0.02) { best_eff = eff; best = sp; }
+    }
+    return best;
+}
 
 struct LmWs {
     size_t n_count, partial, rec, zy, lse, coef, part, dz, total;
@@ -666,7 +684,7 @@ static LmWs lm_workspace(int64_t T, int32_t V) {
     w.zy = o;      o += up1k(4 * Tn);
     w.lse = o;     o += up1k(4 * Tn);
     w.coef = o;    o += up1k(4 * Tn);
-    w.part = o;    o += up1k(8 * Tn * kSplit);
+    w.part = o;    o += up1k(8 * Tn * kMaxSplit);
     w.dz = o;
     const size_t chunk = Tn < (size_t)kChunkTokens ? Tn : (size_t)kChunkTokens;
     o += up1k(chunk * (size_t)V * 2);
@@ -748,13 +766,14 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
     g.m_tiles = (int)((T + BM - 1) / BM);
     g.n_tiles = (V + BN - 1) / BN;
     g.k_slabs = D / BK;
-    g.nsplit = kSplit;
-    g.n_tiles_per_split = (g.n_tiles + kSplit - 1) / kSplit;
+    const int workers = pair ? sm_count_lm() / 2 : sm_count_lm();
+    g.nsplit = pick_split(pair ? (g.m_tiles + 1) / 2 : g.m_tiles, g.n_tiles, workers);
+    g.n_tiles_per_split = (g.n_tiles + g.nsplit - 1) / g.nsplit;
     g.part = part;
     g.dev_status = dev_status;
     st = launch_gemm(mapH, mapW, g, pair, s);
     if (st != RLF_OK) return st;
-    combine_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(part, kSplit, zy, rec, T, dn, eps_clip, beta_kl, logp_out,
+    combine_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(part, g.nsplit, zy, rec, T, dn, eps_clip, beta_kl, logp_out,
                                                                 lse, coef, dev_status);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
@@ -771,6 +790,8 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
         z.mode = kDz;
         z.M = (int)tc;
         z.m_tiles = (int)((tc + BM - 1) / BM);
+        z.nsplit = pick_split(pair ? (z.m_tiles + 1) / 2 : z.m_tiles, z.n_tiles, workers);
+        z.n_tiles_per_split = (z.n_tiles + z.nsplit - 1) / z.nsplit;
         z.lse = lse + t0;
         z.coef = coef + t0;
         z.ids = ids + t0;
