@@ -152,11 +152,10 @@ int orc_group_advantage(const float *rewards, const int32_t *group_id, int32_t B
  *               (A>0 and rho>1+e, or A<0 and rho<1-e), else -A*rho
  *   dkl/dlogp = 1 - exp(d)
  */
-static void token_terms(double logp, double old_lp, double ref_lp, double A, double eps_clip,
-                        double *pg, double *kl, double *dpg, double *dkl, int *clipped)
+static void token_terms_lohi(double logp, double old_lp, double ref_lp, double A, double lo, double hi,
+                             double *pg, double *kl, double *dpg, double *dkl, int *clipped)
 {
     double rho = exp(logp - old_lp);
-    double lo = 1.0 - eps_clip, hi = 1.0 + eps_clip;
     double rc = rho < lo ? lo : (rho > hi ? hi : rho);
     double s1 = rho * A, s2 = rc * A;
     *pg = -(s1 < s2 ? s1 : s2);
@@ -165,6 +164,12 @@ static void token_terms(double logp, double old_lp, double ref_lp, double A, dou
     double d = ref_lp - logp;
     *kl = exp(d) - d - 1.0;
     *dkl = 1.0 - exp(d);
+}
+
+static void token_terms(double logp, double old_lp, double ref_lp, double A, double eps_clip,
+                        double *pg, double *kl, double *dpg, double *dkl, int *clipped)
+{
+    token_terms_lohi(logp, old_lp, ref_lp, A, 1.0 - eps_clip, 1.0 + eps_clip, pg, kl, dpg, dkl, clipped);
 }
 
 /* log-softmax statistics of one row: m = max_v z, and log s with s = sum_v exp(z - m), so that
@@ -260,6 +265,90 @@ int orc_grpo_loss(const void *logits, int dtype, int64_t T, int32_t V, int64_t r
     loss_out[3] = s_cl / nd;
     free(pg_t); free(kl_t); free(cl_t);
     return 0;
+}
+
+/*
+ * Objective variants of orc_grpo_loss (the paper names GRPO / a PPO-style update in Sec. 2.3 and
+ * prints no objective; these are the common alternatives to the symmetric-clip token mean):
+ *   - asymmetric clip range: clip(rho, 1 - eps_low, 1 + eps_high);
+ *   - aggregation 0: masked token mean, weight w_t = mask_t / max(N, 1), N = denom or sum of mask;
+ *     aggregation 1: mean over sequences of each sequence's masked token mean,
+ *         w_t = mask_t / (n_b * max(S, 1)),  n_b = sum of mask in the sequence b of token t,
+ *         S = denom if denom >= 0 else the number of sequences with n_b > 0.
+ *   loss_out[k] = sum_t w_t x_t for x in {pg + beta kl, pg, kl, clipped};
+ *   grad[t,v] = w_t (dpg_t + beta dkl_t) (1[v = y_t] - p[t,v]).
+ * num_seqs = number of sequences (seq_id values lie in [0, num_seqs)).
+ */
+int orc_grpo_loss_obj(const void *logits, int dtype, int64_t T, int32_t V, int64_t row_stride,
+                      const int32_t *ids, const int32_t *seq_id, const float *adv, int32_t num_seqs,
+                      const float *old_logp, const float *ref_logp, const uint8_t *mask,
+                      double eps_low, double eps_high, double beta_kl, int aggregation, int64_t denom,
+                      double *logp_out, double *loss_out, double *grad, double *coef_out)
+{
+    double *w = (double *)calloc((size_t)(T > 0 ? T : 1), sizeof(double));
+    int64_t *nb = (int64_t *)calloc((size_t)(num_seqs > 0 ? num_seqs : 1), sizeof(int64_t));
+    if (!w || !nb) return -7;
+    for (int64_t t = 0; t < T; ++t) {
+        if (seq_id[t] < 0 || seq_id[t] >= num_seqs) { free(w); free(nb); return -2; }
+        if (mask[t]) nb[seq_id[t]] += 1;
+    }
+    if (aggregation == 0) {
+        int64_t n = 0;
+        for (int32_t b = 0; b < num_seqs; ++b) n += nb[b];
+        if (denom >= 0) n = denom;
+        double nd = n > 1 ? (double)n : 1.0;
+        for (int64_t t = 0; t < T; ++t) w[t] = mask[t] ? 1.0 / nd : 0.0;
+    } else {
+        int64_t S = 0;
+        for (int32_t b = 0; b < num_seqs; ++b) S += nb[b] > 0 ? 1 : 0;
+        if (denom >= 0) S = denom;
+        double sd = S > 1 ? (double)S : 1.0;
+        for (int64_t t = 0; t < T; ++t) w[t] = mask[t] ? 1.0 / ((double)nb[seq_id[t]] * sd) : 0.0;
+    }
+    double *terms = (double *)calloc((size_t)(T > 0 ? T : 1) * 3, sizeof(double));
+    if (!terms) { free(w); free(nb); return -7; }
+    int bad = 0;
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int64_t t = 0; t < T; ++t) {
+        int64_t off = t * row_stride;
+        int32_t y = ids[t];
+        if (y < 0 || y >= V) {
+#pragma omp atomic write
+            bad = 1;
+            continue;
+        }
+        double m, logs;
+        row_stats(logits, dtype, off, V, &m, &logs);
+        double logp = (widen(logits, dtype, off + y) - m) - logs;
+        logp_out[t] = logp;
+        double pg, kl, dpg, dkl;
+        int clipped;
+        token_terms_lohi(logp, (double)old_logp[t], (double)ref_logp[t], (double)adv[seq_id[t]],
+                         1.0 - eps_low, 1.0 + eps_high, &pg, &kl, &dpg, &dkl, &clipped);
+        terms[3 * t] = pg;
+        terms[3 * t + 1] = kl;
+        terms[3 * t + 2] = (double)clipped;
+        double g = w[t] * (dpg + beta_kl * dkl);
+        if (coef_out) coef_out[t] = -g;
+        if (grad) {
+            for (int32_t v = 0; v < V; ++v) {
+                double p = exp((widen(logits, dtype, off + v) - m) - logs);
+                grad[t * (int64_t)V + v] = g * ((v == y ? 1.0 : 0.0) - p);
+            }
+        }
+    }
+    double s_pg = 0.0, s_kl = 0.0, s_cl = 0.0;
+    for (int64_t t = 0; t < T; ++t) {
+        s_pg += w[t] * terms[3 * t];
+        s_kl += w[t] * terms[3 * t + 1];
+        s_cl += w[t] * terms[3 * t + 2];
+    }
+    loss_out[0] = s_pg + beta_kl * s_kl;
+    loss_out[1] = s_pg;
+    loss_out[2] = s_kl;
+    loss_out[3] = s_cl;
+    free(w); free(nb); free(terms);
+    return bad ? -2 : 0;
 }
 
 /*

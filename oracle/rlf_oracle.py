@@ -127,6 +127,33 @@ def grpo_loss(logits, ids, seq_id, adv, old_logp, ref_logp, mask, eps_clip, beta
     return dict(logp=logp, loss=loss, grad=grad, coef=coef)
 
 
+def grpo_loss_obj(logits, ids, seq_id, adv, old_logp, ref_logp, mask, eps_low, eps_high, beta_kl, aggregation=0,
+                  denom=None, want_grad=True, want_coef=False):
+    """Objective variants: asymmetric clip range and token-mean (0) / sequence-mean (1) aggregation.
+    -> dict(logp, loss f64[4], grad | None, coef | None)."""
+    assert logits.ndim == 2 and (logits.shape[1] <= 1 or logits.strides[1] == logits.itemsize)
+    T, V = logits.shape
+    stride = logits.strides[0] // logits.itemsize if T > 1 else V
+    ids = _c(ids, np.int32)
+    seq_id = _c(seq_id, np.int32)
+    adv = _c(adv, np.float32)
+    old_logp = _c(old_logp, np.float32)
+    ref_logp = _c(ref_logp, np.float32)
+    mask = _c(mask, np.uint8)
+    logp = np.zeros(T, np.float64)
+    loss = np.zeros(4, np.float64)
+    grad = np.zeros((T, V), np.float64) if want_grad else None
+    coef = np.zeros(T, np.float64) if want_coef else None
+    rc = lib().orc_grpo_loss_obj(_p(logits), ctypes.c_int(_dtype_code(logits)), ctypes.c_int64(T), ctypes.c_int32(V),
+                                 ctypes.c_int64(stride), _p(ids), _p(seq_id), _p(adv), ctypes.c_int32(adv.shape[0]),
+                                 _p(old_logp), _p(ref_logp), _p(mask), ctypes.c_double(eps_low),
+                                 ctypes.c_double(eps_high), ctypes.c_double(beta_kl), ctypes.c_int(aggregation),
+                                 ctypes.c_int64(-1 if denom is None else int(denom)), _p(logp), _p(loss), _p(grad),
+                                 _p(coef))
+    _check(rc, "grpo_loss_obj")
+    return dict(logp=logp, loss=loss, grad=grad, coef=coef)
+
+
 def logp_entropy(logits, ids, want_entropy=True):
     """-> (logp f64[T], entropy f64[T] | None) of each row's softmax at the given targets."""
     assert logits.ndim == 2 and (logits.shape[1] <= 1 or logits.strides[1] == logits.itemsize)

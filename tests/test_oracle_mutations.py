@@ -27,6 +27,8 @@ MUTATIONS = [
     ("denominator_ignores_override", "if (denom >= 0) n = denom;", "", "test_oracle_loss.py"),
     ("head_transposed", "widen(W, ORC_BF16, v * (int64_t)D + k);\n            z[t", "widen(W, ORC_BF16, (v * (int64_t)D + k) % ((int64_t)V * D - 1));\n            z[t", "test_oracle_fused.py"),
     ("grad_W_uses_wrong_operand", "acc += gz[t * (int64_t)V + v] * widen(hidden, ORC_BF16, t * (int64_t)D + k);", "acc += gz[t * (int64_t)V + v] * widen(hidden, ORC_BF16, t * (int64_t)D + (D - 1 - k));", "test_oracle_fused.py"),
+    ("asymmetric_clip_uses_low_for_both", "1.0 - eps_low, 1.0 + eps_high, &pg", "1.0 - eps_low, 1.0 + eps_low, &pg", "test_oracle_objective.py"),
+    ("sequence_mean_weighs_by_batch_count", "w[t] = mask[t] ? 1.0 / ((double)nb[seq_id[t]] * sd) : 0.0;", "w[t] = mask[t] ? 1.0 / ((double)T * sd) : 0.0;", "test_oracle_objective.py"),
     ("entropy_sign", "if (pv > 0.0) h -= pv * lp;", "if (pv > 0.0) h += pv * lp;", "test_oracle_entropy.py"),
 ]
 
