@@ -156,6 +156,29 @@ rlf_status rlf_grpo_logp_loss_fwd_bwd(const void *logits, rlf_dtype dt, int64_t 
                                       int32_t *dev_status, rlf_stream_t stream);
 
 /*
+ * rlf_grpo_logp_loss_fwd_bwd with the objective's common variants.  (The paper names GRPO and a
+ * PPO-style update, Sec. 2.3, without printing the objective; these are the usual alternatives.)
+ *   clip range     clip(rho, 1 - eps_clip_low, 1 + eps_clip_high)
+ *   aggregation 0  masked token mean over the call (N = *denom or the sum of mask), as above
+ *   aggregation 1  mean over responses of each response's masked token mean: token t of response b
+ *                  has weight mask[t] / (n_b S), n_b = live tokens of b, S = *denom if denom != NULL
+ *                  (number of responses of the whole batch when it is split over calls), else the
+ *                  number of responses with n_b > 0 in this call.  Needs B <= T + 1.
+ * loss_out[k] = sum of weight x {pg + beta kl, pg, kl, clipped}; grad_logits scales accordingly.
+ * All other arguments, the workspace size and the error behaviour are those of
+ * rlf_grpo_logp_loss_fwd_bwd, which equals this call with eps_clip_low = eps_clip_high, aggregation 0.
+ */
+rlf_status rlf_grpo_logp_loss_fwd_bwd_obj(const void *logits, rlf_dtype dt, int64_t T, int32_t V,
+                                          int64_t row_stride, const int32_t *ids, const int32_t *seq_id,
+                                          const float *adv, int32_t B, const float *old_logp,
+                                          const float *ref_logp, const uint8_t *mask,
+                                          float eps_clip_low, float eps_clip_high, float beta_kl,
+                                          int aggregation, const int64_t *denom, float *logp_out,
+                                          double *loss_out, void *grad_logits, void *workspace,
+                                          size_t workspace_bytes, int32_t *dev_status,
+                                          rlf_stream_t stream);
+
+/*
  * rlf_grpo_logp_loss_fwd_bwd that neither reads nor computes rows without loss weight.  (Paper
  * Sec. 2.2 / Sec. 2.3.2: observation tokens take no part in the loss; in multi-turn tool-use batches
  * they are a large share of all tokens, so their logits rows need not be touched at all.)

@@ -19,7 +19,7 @@ DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
 
 EXPORTS = [
     "rlf_build_loss_mask", "rlf_group_advantage", "rlf_rule_reward", "rlf_grpo_logp_loss_fwd_bwd",
-    "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_grpo_logp_loss_fwd_bwd_skip_masked", "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
+    "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_grpo_logp_loss_fwd_bwd_skip_masked", "rlf_grpo_logp_loss_fwd_bwd_obj", "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
     "rlf_tune_logits_kernel", "rlf_tune_lmhead", "rlf_launch_count", "rlf_status_string", "rlf_version",
 ]
 
@@ -198,6 +198,35 @@ def rlf_grpo_logp_loss_fwd_bwd(logits, ids, seq_id, adv, old_logp, ref_logp, mas
         _ptr(denom, torch.int64), _ptr(logp_out, torch.float32), _ptr(loss_out, torch.float64),
         None if grad_logits is None else grad_logits.data_ptr(), workspace.data_ptr(), workspace.numel(),
         _ptr(dev_status, torch.int32), _stream()), "rlf_grpo_logp_loss_fwd_bwd")
+    return logp_out, loss_out, grad_logits
+
+
+def rlf_grpo_logp_loss_fwd_bwd_obj(logits, ids, seq_id, adv, old_logp, ref_logp, mask, eps_clip_low, eps_clip_high,
+                                   beta_kl, aggregation=0, denom=None, grad_logits=None, want_grad=True,
+                                   in_place=False, logp_out=None, loss_out=None, workspace=None, dev_status=None):
+    """Objective variants: asymmetric clip range; aggregation 0 = token mean, 1 = sequence mean."""
+    T, V = logits.shape
+    stride = logits.stride(0) if T > 1 else V
+    dev = logits.device
+    if grad_logits is None and want_grad:
+        grad_logits = logits if in_place else torch.empty_strided((T, V), (stride, 1), dtype=logits.dtype, device=dev)
+    if logp_out is None:
+        logp_out = torch.empty(T, dtype=torch.float32, device=dev)
+    if loss_out is None:
+        loss_out = torch.empty(4, dtype=torch.float64, device=dev)
+    dt = _dt(logits)
+    if workspace is None:
+        workspace = new_workspace(FN_LOGP_LOSS, T, V, 0, dt, dev)
+    f = _lib.rlf_grpo_logp_loss_fwd_bwd_obj
+    f.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _f32, _f32, _f32, _int, _vp, _vp, _vp,
+                  _vp, _vp, _sz, _vp, _vp]
+    f.restype = _int
+    _check(f(logits.data_ptr() if T > 0 else None, dt, T, V, stride, _ptr(ids, torch.int32), _ptr(seq_id, torch.int32),
+             _ptr(adv, torch.float32), adv.shape[0], _ptr(old_logp, torch.float32), _ptr(ref_logp, torch.float32),
+             _ptr(mask, torch.uint8), float(eps_clip_low), float(eps_clip_high), float(beta_kl), int(aggregation),
+             _ptr(denom, torch.int64), _ptr(logp_out, torch.float32), _ptr(loss_out, torch.float64),
+             None if grad_logits is None else grad_logits.data_ptr(), workspace.data_ptr(), workspace.numel(),
+             _ptr(dev_status, torch.int32), _stream()), "rlf_grpo_logp_loss_fwd_bwd_obj")
     return logp_out, loss_out, grad_logits
 
 

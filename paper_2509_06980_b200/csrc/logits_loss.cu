@@ -51,7 +51,11 @@ constexpr size_t kWsRecordOff = kWsPartialOff + sizeof(double) * 4 * kMaxPartial
 static size_t ws_tokens(int64_t T) { return (size_t)(T > 0 ? T : 0); }
 static size_t ws_compact_rec_off(int64_t T) { return kWsRecordOff + 16 * ws_tokens(T) + 256; }
 static size_t ws_row_list_off(int64_t T) { return ws_compact_rec_off(T) + 16 * ws_tokens(T) + 256; }
-size_t loss_workspace_bytes(int64_t T) { return ws_row_list_off(T) + 4 * ws_tokens(T) + 256; }
+// then per-token weights (4 B per token) and per-sequence counters (4 B x (T + 1)) of the
+// sequence-mean aggregation
+static size_t ws_wtok_off(int64_t T) { return ws_row_list_off(T) + 4 * ws_tokens(T) + 256; }
+static size_t ws_seqcnt_off(int64_t T) { return ws_wtok_off(T) + 4 * ws_tokens(T) + 256; }
+size_t loss_workspace_bytes(int64_t T) { return ws_seqcnt_off(T) + 4 * (ws_tokens(T) + 1) + 256; }
 
 // ---------------------------------------------------------------------------------------------
 // token records
@@ -85,9 +89,9 @@ token_prep_kernel(const int32_t* __restrict__ ids, const int32_t* __restrict__ s
 
 // d(pg + beta kl)/d logp with hardware exp2 (relative error ~1e-6: ample for a bf16 gradient)
 __device__ __forceinline__ float grad_coef_fast(float logp, float old_lp, float ref_lp, float A,
-                                                float eps_clip, float beta) {
+                                                float eps_lo, float eps_hi, float beta) {
     const float rho = ex2_approx((logp - old_lp) * kLog2e);
-    const bool clipped = ((A > 0.0f) && (rho > 1.0f + eps_clip)) || ((A < 0.0f) && (rho < 1.0f - eps_clip));
+    const bool clipped = ((A > 0.0f) && (rho > 1.0f + eps_hi)) || ((A < 0.0f) && (rho < 1.0f - eps_lo));
     const float dpg = clipped ? 0.0f : -A * rho;
     const float ed = ex2_approx((ref_lp - logp) * kLog2e);
     return fmaf(beta, 1.0f - ed, dpg);
@@ -173,8 +177,9 @@ struct FastParams {
     float* entropy_out;         // entropy variant only, nullable
     const int* row_list;        // skip-masked variant: rows to process, rec[] is indexed like this list
     const int* n_rows;          // skip-masked variant: device count of listed rows
+    const float* wtok;          // per-token loss weights (sequence-mean aggregation) or NULL: 1 / N
     int32_t* dev_status;
-    float eps_clip, beta;
+    float eps_clip, eps_hi, beta;   // clip range [1 - eps_clip, 1 + eps_hi]
 };
 
 // bf16 element e (0..7) of a 16-byte vector, widened
@@ -317,6 +322,7 @@ grpo_row_cluster_kernel(const FastParams p) {
     constexpr int AHEAD = SKIP ? 3 : 2;                  // how many rows ahead thread 0 fetches metadata
     __shared__ __align__(16) float4 rec_slot[RM + 1];    // token records, ring over rows
     __shared__ int row_slot[SKIP ? 8 : 1];               // skip variant: row index of each listed row
+    __shared__ float w_slot[RM + 1];                     // per-token loss weight, when the caller gives them
     __shared__ float zy_slot[2];                         // per row parity: the target logit
     __shared__ float ent_slot[2][ENT ? MAXE : 1];        // entropy variant: every warp's sum 2^x * x
     __shared__ __align__(8) unsigned long long row_bar[2];   // per row parity: "all pairs and z_target are here"
@@ -348,6 +354,7 @@ grpo_row_cluster_kernel(const FastParams p) {
         if (tid == 0 && j >= 0 && k < nrows) {
             cp_async16(&rec_slot[j & RM], p.rec + k);
             if (SKIP) cp_async4(&row_slot[j & RM], p.row_list + k);
+            if (p.wtok) cp_async4(&w_slot[j & RM], p.wtok + k);
         }
     };
     // queue this thread's part of a row into the staging buffer (one cp.async group per row; thread
@@ -488,7 +495,8 @@ grpo_row_cluster_kernel(const FastParams p) {
         const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) &&
                             (fabsf(logp) < INFINITY);
         const bool live = (__float_as_int(rec.w) < 0) && finite;
-        const float coef = live ? -inv_n * grad_coef_fast(logp, rec.x, rec.y, rec.z, p.eps_clip, p.beta) : 0.0f;
+        const float w_row = p.wtok ? w_slot[it & RM] : inv_n;
+        const float coef = live ? -w_row * grad_coef_fast(logp, rec.x, rec.y, rec.z, p.eps_clip, p.eps_hi, p.beta) : 0.0f;
         if (crank == 0 && tid == 0) {
             // forward-only variant: a row whose target id was out of range has no log-prob
             const bool has_logp = finite && (!ENT || __float_as_int(rec.w) < 0);
@@ -566,8 +574,9 @@ struct GenParams {
     float* logp_out;
     float* entropy_out;         // nullable: also return the row's entropy (forward-only use)
     int fwd_only;               // forward-only entry point: a row with a bad target id gets NaN
+    const float* wtok;          // per-token loss weights or NULL: 1 / N
     int32_t* dev_status;
-    float eps_clip, beta;
+    float eps_clip, eps_hi, beta;
 };
 
 constexpr int kGenThreads = 256;
@@ -630,7 +639,8 @@ grpo_row_general_kernel(const GenParams p) {
         const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) &&
                             (fabsf(logp) < INFINITY);
         const bool live = (__float_as_int(rec.w) < 0) && finite;
-        const float coef = live ? -inv_n * grad_coef_fast(logp, rec.x, rec.y, rec.z, p.eps_clip, p.beta) : 0.0f;
+        const float w_row = p.wtok ? p.wtok[row] : inv_n;
+        const float coef = live ? -w_row * grad_coef_fast(logp, rec.x, rec.y, rec.z, p.eps_clip, p.eps_hi, p.beta) : 0.0f;
         if (tid == 0) {
             const bool has_logp = finite && (!p.fwd_only || __float_as_int(rec.w) < 0);
             p.logp_out[row] = has_logp ? logp : __int_as_float(0x7fc00000);
@@ -660,7 +670,7 @@ grpo_row_general_kernel(const GenParams p) {
 constexpr int kLossThreads = 256;
 __global__ void __launch_bounds__(kLossThreads)
 token_loss_kernel(const float* __restrict__ logp, const float4* __restrict__ rec, int64_t T,
-                  float eps_clip, double* __restrict__ partial) {
+                  float eps_clip, float eps_hi, const float* __restrict__ wtok, double* __restrict__ partial) {
     __shared__ double red[kLossThreads / 32][3];
     double a_pg = 0.0, a_kl = 0.0, a_cl = 0.0;
     for (int64_t t = (int64_t)blockIdx.x * kLossThreads + threadIdx.x; t < T;
@@ -670,12 +680,13 @@ token_loss_kernel(const float* __restrict__ logp, const float4* __restrict__ rec
         if (__float_as_int(r.w) >= 0 || !isfinite(lp)) continue;
         const double A = (double)r.z;
         const double rho = exp(lp - (double)r.x);
-        const double lo = 1.0 - (double)eps_clip, hi = 1.0 + (double)eps_clip;
+        const double lo = 1.0 - (double)eps_clip, hi = 1.0 + (double)eps_hi;
         const double rc = fmin(fmax(rho, lo), hi);
-        a_pg += -fmin(rho * A, rc * A);
-        a_cl += ((A > 0.0 && rho > hi) || (A < 0.0 && rho < lo)) ? 1.0 : 0.0;
+        const double w = wtok ? (double)wtok[t] : 1.0;      // token mean: divided by N at the end
+        a_pg += w * -fmin(rho * A, rc * A);
+        a_cl += ((A > 0.0 && rho > hi) || (A < 0.0 && rho < lo)) ? w : 0.0;
         const double d = (double)r.y - lp;
-        a_kl += expm1(d) - d;
+        a_kl += w * (expm1(d) - d);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -698,7 +709,7 @@ token_loss_kernel(const float* __restrict__ logp, const float4* __restrict__ rec
 
 // per-block partial sums -> loss_out[4], added in index order by one thread per quantity
 __global__ void finalize_loss_kernel(const double* __restrict__ partial, int num_partials,
-                                     const long long* __restrict__ denom, float beta,
+                                     const long long* __restrict__ denom, float beta, int weighted,
                                      double* __restrict__ loss_out) {
     __shared__ double s[3];
     if (threadIdx.x < 3) {
@@ -709,7 +720,7 @@ __global__ void finalize_loss_kernel(const double* __restrict__ partial, int num
     __syncthreads();
     if (threadIdx.x == 0) {
         const long long N = *denom;
-        const double nd = (double)(N > 1 ? N : 1);
+        const double nd = weighted ? 1.0 : (double)(N > 1 ? N : 1);   // weighted sums are already means
         loss_out[0] = (s[0] + (double)beta * s[1]) / nd;
         loss_out[1] = s[0] / nd;
         loss_out[2] = s[1] / nd;
@@ -856,11 +867,47 @@ struct LossArgs {
     const float* ref_logp;
     const uint8_t* mask;
     float eps_clip, beta;
+    float eps_hi;               // upper clip width (the lower one is eps_clip)
+    int aggregation;            // 0 token mean, 1 sequence mean (per-token weights built in the workspace)
     const int64_t* denom;
     float* logp_out;
     double* loss_out;
     int32_t* dev_status;
 };
+
+// sequence-mean aggregation: w_t = live_t / (n_b * S), n_b = live tokens of the token's sequence,
+// S = *denom if given else the number of sequences with n_b > 0
+__global__ void __launch_bounds__(256)
+seq_count_kernel(const float4* __restrict__ rec, const int32_t* __restrict__ seq_id, int64_t T, int* __restrict__ cnt) {
+    const int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (t < T && __float_as_int(rec[t].w) < 0) atomicAdd(&cnt[seq_id[t]], 1);
+}
+__global__ void __launch_bounds__(1024)
+seq_live_kernel(const int* __restrict__ cnt, int32_t B, const long long* __restrict__ denom, long long* __restrict__ s_out) {
+    __shared__ int red[32];
+    int c = 0;
+    for (int b = threadIdx.x; b < B; b += 1024) c += cnt[b] > 0 ? 1 : 0;
+    c = __reduce_add_sync(0xffffffffu, c);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int s = 0;
+        for (int w = 0; w < 32; ++w) s += red[w];
+        *s_out = denom ? *denom : (long long)s;
+    }
+}
+__global__ void __launch_bounds__(256)
+seq_weight_kernel(const float4* __restrict__ rec, const int32_t* __restrict__ seq_id, int64_t T,
+                  const int* __restrict__ cnt, const long long* __restrict__ s_in, float* __restrict__ wtok) {
+    const int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (t >= T) return;
+    float w = 0.0f;
+    if (__float_as_int(rec[t].w) < 0) {
+        const long long S = *s_in;
+        w = (float)(1.0 / ((double)cnt[seq_id[t]] * (double)(S > 1 ? S : 1)));
+    }
+    wtok[t] = w;
+}
 
 static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* workspace, cudaStream_t s) {
     char* ws = static_cast<char*>(workspace);
@@ -873,6 +920,7 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
         denom = n_count;
     }
     int num_partials = 0;
+    float* wtok = nullptr;
     if (a.T > 0) {
         const int64_t prep_blocks = (a.T + kPrepThreads - 1) / kPrepThreads;
         token_prep_kernel<<<(unsigned)prep_blocks, kPrepThreads, 0, s>>>(
@@ -880,6 +928,18 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
             a.denom == nullptr ? reinterpret_cast<unsigned long long*>(n_count) : nullptr, a.dev_status);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+        if (a.aggregation == 1) {
+            // per-token weights of the sequence mean; here `denom`, if given, counts sequences
+            int* cnt = reinterpret_cast<int*>(ws + ws_seqcnt_off(a.T));
+            long long* s_slot = reinterpret_cast<long long*>(ws + 64);
+            wtok = reinterpret_cast<float*>(ws + ws_wtok_off(a.T));
+            if (cudaMemsetAsync(cnt, 0, sizeof(int) * (size_t)a.B, s) != cudaSuccess) return RLF_ERR_CUDA;
+            seq_count_kernel<<<(unsigned)prep_blocks, 256, 0, s>>>(rec, a.seq_id, a.T, cnt);
+            seq_live_kernel<<<1, 1024, 0, s>>>(cnt, a.B, reinterpret_cast<const long long*>(a.denom), s_slot);
+            seq_weight_kernel<<<(unsigned)prep_blocks, 256, 0, s>>>(rec, a.seq_id, a.T, cnt, s_slot, wtok);
+            count_launch(3);
+            if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+        }
 
         FastShape sh;
         const bool tuned = g_tune_cluster.load() > 0;
@@ -901,7 +961,9 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
             p.logp_out = a.logp_out;
             p.dev_status = a.dev_status;
             p.eps_clip = a.eps_clip;
+            p.eps_hi = a.eps_hi;
             p.beta = a.beta;
+            p.wtok = wtok;
             p.entropy_out = nullptr;
             p.row_list = nullptr;
             p.n_rows = nullptr;
@@ -919,7 +981,8 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
             GenParams p;
             p.logits = a.logits; p.grad = a.grad; p.stride = a.stride; p.T = a.T; p.V = a.V;
             p.rec = rec; p.denom = denom; p.logp_out = a.logp_out; p.dev_status = a.dev_status;
-            p.eps_clip = a.eps_clip; p.beta = a.beta; p.entropy_out = nullptr; p.fwd_only = 0;
+            p.eps_clip = a.eps_clip; p.eps_hi = a.eps_hi; p.beta = a.beta; p.entropy_out = nullptr; p.fwd_only = 0;
+            p.wtok = wtok;
             int grid = sm_count() * 8;
             if ((int64_t)grid > a.T) grid = (int)a.T;
             if (a.dt == RLF_BF16) grpo_row_general_kernel<__nv_bfloat16><<<grid, kGenThreads, 0, s>>>(p);
@@ -929,11 +992,11 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
         }
         const int64_t blocks = (a.T + kLossThreads - 1) / kLossThreads;
         num_partials = (int)(blocks < kMaxPartials ? blocks : kMaxPartials);
-        token_loss_kernel<<<num_partials, kLossThreads, 0, s>>>(a.logp_out, rec, a.T, a.eps_clip, partial);
+        token_loss_kernel<<<num_partials, kLossThreads, 0, s>>>(a.logp_out, rec, a.T, a.eps_clip, a.eps_hi, wtok, partial);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
     }
-    finalize_loss_kernel<<<1, 32, 0, s>>>(partial, num_partials, denom, a.beta, a.loss_out);
+    finalize_loss_kernel<<<1, 32, 0, s>>>(partial, num_partials, denom, a.beta, wtok != nullptr, a.loss_out);
     count_launch();
     return cuda_ok(cudaGetLastError());
 }
@@ -980,6 +1043,39 @@ extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd(
     a.ids = ids; a.seq_id = seq_id; a.adv = adv; a.B = B; a.old_logp = old_logp; a.ref_logp = ref_logp;
     a.mask = mask; a.eps_clip = eps_clip; a.beta = beta_kl; a.denom = denom; a.logp_out = logp_out;
     a.loss_out = loss_out; a.dev_status = dev_status;
+    a.eps_hi = eps_clip; a.aggregation = 0;
+    const bool fast_ok = dt == RLF_BF16 && (V % 8 == 0) && (row_stride % 8 == 0) &&
+                         aligned(logits, 16) && aligned(grad_logits, 16);
+    return launch_logits_loss(a, fast_ok, workspace, reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd_obj(
+    const void* logits, rlf_dtype dt, int64_t T, int32_t V, int64_t row_stride, const int32_t* ids,
+    const int32_t* seq_id, const float* adv, int32_t B, const float* old_logp, const float* ref_logp,
+    const uint8_t* mask, float eps_clip_low, float eps_clip_high, float beta_kl, int aggregation,
+    const int64_t* denom, float* logp_out, double* loss_out, void* grad_logits, void* workspace,
+    size_t workspace_bytes, int32_t* dev_status, rlf_stream_t stream) {
+    using namespace rlf;
+    if (dt != RLF_BF16 && dt != RLF_F32) return RLF_ERR_DTYPE;
+    if (T < 0 || V < 1 || B < 0 || row_stride < V) return RLF_ERR_SHAPE;
+    if (aggregation != 0 && aggregation != 1) return RLF_ERR_SHAPE;
+    if (aggregation == 1 && (int64_t)B > T + 1) return RLF_ERR_SHAPE;
+    if (!loss_out) return RLF_ERR_NULL;
+    if (T > 0 && (!logits || !ids || !seq_id || !adv || !old_logp || !ref_logp || !mask || !logp_out))
+        return RLF_ERR_NULL;
+    if (T > 0 && B == 0) return RLF_ERR_SHAPE;
+    const size_t esz = dt == RLF_BF16 ? 2 : 4;
+    if (!aligned(logits, esz) || !aligned(grad_logits, esz)) return RLF_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < loss_workspace_bytes(T))
+        return RLF_ERR_WORKSPACE;
+    rlf_status st = check_arch();
+    if (st != RLF_OK) return st;
+    LossArgs a;
+    a.logits = logits; a.grad = grad_logits; a.dt = dt; a.T = T; a.V = V; a.stride = row_stride;
+    a.ids = ids; a.seq_id = seq_id; a.adv = adv; a.B = B; a.old_logp = old_logp; a.ref_logp = ref_logp;
+    a.mask = mask; a.eps_clip = eps_clip_low; a.beta = beta_kl; a.denom = denom; a.logp_out = logp_out;
+    a.loss_out = loss_out; a.dev_status = dev_status;
+    a.eps_hi = eps_clip_high; a.aggregation = aggregation;
     const bool fast_ok = dt == RLF_BF16 && (V % 8 == 0) && (row_stride % 8 == 0) &&
                          aligned(logits, 16) && aligned(grad_logits, 16);
     return launch_logits_loss(a, fast_ok, workspace, reinterpret_cast<cudaStream_t>(stream));
@@ -1069,6 +1165,8 @@ extern "C" rlf_status rlf_logp_entropy_fwd(const void* logits, rlf_dtype dt, int
         p.n_rows = nullptr;
         p.dev_status = dev_status;
         p.eps_clip = 0.0f;
+        p.eps_hi = 0.0f;
+        p.wtok = nullptr;
         p.beta = 0.0f;
         cudaLaunchConfig_t cfg;
         cudaLaunchAttribute at[1];
@@ -1083,6 +1181,7 @@ extern "C" rlf_status rlf_logp_entropy_fwd(const void* logits, rlf_dtype dt, int
     GenParams g;
     g.logits = logits; g.grad = nullptr; g.stride = row_stride; g.T = T; g.V = V; g.rec = rec; g.denom = one;
     g.logp_out = logp_out; g.entropy_out = entropy_out; g.dev_status = dev_status; g.eps_clip = 0.0f; g.beta = 0.0f;
+    g.eps_hi = 0.0f; g.wtok = nullptr;
     g.fwd_only = 1;
     int grid = sm_count() * 8;
     if ((int64_t)grid > T) grid = (int)T;
@@ -1234,6 +1333,8 @@ extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd_skip_masked(
     p.n_rows = n_live;
     p.dev_status = dev_status;
     p.eps_clip = eps_clip;
+    p.eps_hi = eps_clip;
+    p.wtok = nullptr;
     p.beta = beta_kl;
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute at[1];
@@ -1269,11 +1370,11 @@ rlf_status launch_token_loss(const float* logp, const void* rec, int64_t T, floa
         const int64_t blocks = (T + kLossThreads - 1) / kLossThreads;
         num_partials = (int)(blocks < kMaxPartials ? blocks : kMaxPartials);
         token_loss_kernel<<<num_partials, kLossThreads, 0, s>>>(logp, static_cast<const float4*>(rec), T, eps_clip,
-                                                               partial);
+                                                               eps_clip, nullptr, partial);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
     }
-    finalize_loss_kernel<<<1, 32, 0, s>>>(partial, num_partials, denom, beta, loss_out);
+    finalize_loss_kernel<<<1, 32, 0, s>>>(partial, num_partials, denom, beta, 0, loss_out);
     count_launch();
     return cuda_ok(cudaGetLastError());
 }
