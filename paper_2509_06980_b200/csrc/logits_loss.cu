@@ -309,7 +309,8 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t mbar, uint32_t parity
 
 // SKIP: the rows to process come from a compacted list (rows whose loss weight is zero are
 // neither read nor computed); token records are then indexed like the list.
-template <int THREADS, int NV, bool ONE_EXP, bool ENT = false, bool SKIP = false>
+// WT: per-token loss weights from the caller replace the common 1 / N.
+template <int THREADS, int NV, bool ONE_EXP, bool ENT = false, bool SKIP = false, bool WT = false>
 __global__ void __launch_bounds__(THREADS, ctas_per_sm(THREADS, NV))
 grpo_row_cluster_kernel(const FastParams p) {
     constexpr int NWARPS = THREADS / 32;
@@ -322,7 +323,7 @@ grpo_row_cluster_kernel(const FastParams p) {
     constexpr int AHEAD = SKIP ? 3 : 2;                  // how many rows ahead thread 0 fetches metadata
     __shared__ __align__(16) float4 rec_slot[RM + 1];    // token records, ring over rows
     __shared__ int row_slot[SKIP ? 8 : 1];               // skip variant: row index of each listed row
-    __shared__ float w_slot[RM + 1];                     // per-token loss weight, when the caller gives them
+    __shared__ float w_slot[WT ? RM + 1 : 1];            // per-token loss weight (WT variant)
     __shared__ float zy_slot[2];                         // per row parity: the target logit
     __shared__ float ent_slot[2][ENT ? MAXE : 1];        // entropy variant: every warp's sum 2^x * x
     __shared__ __align__(8) unsigned long long row_bar[2];   // per row parity: "all pairs and z_target are here"
@@ -354,7 +355,7 @@ grpo_row_cluster_kernel(const FastParams p) {
         if (tid == 0 && j >= 0 && k < nrows) {
             cp_async16(&rec_slot[j & RM], p.rec + k);
             if (SKIP) cp_async4(&row_slot[j & RM], p.row_list + k);
-            if (p.wtok) cp_async4(&w_slot[j & RM], p.wtok + k);
+            if (WT) cp_async4(&w_slot[j & RM], p.wtok + k);
         }
     };
     // queue this thread's part of a row into the staging buffer (one cp.async group per row; thread
@@ -495,7 +496,7 @@ grpo_row_cluster_kernel(const FastParams p) {
         const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) &&
                             (fabsf(logp) < INFINITY);
         const bool live = (__float_as_int(rec.w) < 0) && finite;
-        const float w_row = p.wtok ? w_slot[it & RM] : inv_n;
+        const float w_row = WT ? w_slot[it & RM] : inv_n;
         const float coef = live ? -w_row * grad_coef_fast(logp, rec.x, rec.y, rec.z, p.eps_clip, p.eps_hi, p.beta) : 0.0f;
         if (crank == 0 && tid == 0) {
             // forward-only variant: a row whose target id was out of range has no log-prob
@@ -785,6 +786,26 @@ static FastKernel fast_kernel_for_nv(int nv) {
     }
     return nullptr;
 }
+template <int THREADS>
+static FastKernel weighted_kernel_for_nv(int nv) {
+    switch (nv) {
+        case 1: return grpo_row_cluster_kernel<THREADS, 1, true, false, false, true>;
+        case 2: return grpo_row_cluster_kernel<THREADS, 2, true, false, false, true>;
+        case 3: return grpo_row_cluster_kernel<THREADS, 3, true, false, false, true>;
+        case 4: return grpo_row_cluster_kernel<THREADS, 4, true, false, false, true>;
+        case 5: return grpo_row_cluster_kernel<THREADS, 5, true, false, false, true>;
+        case 6: return grpo_row_cluster_kernel<THREADS, 6, true, false, false, true>;
+        case 8: return grpo_row_cluster_kernel<THREADS, 8, true, false, false, true>;
+        case 10: return grpo_row_cluster_kernel<THREADS, 10, true, false, false, true>;
+    }
+    return nullptr;
+}
+static FastKernel weighted_kernel(const FastShape& sh) {
+    if (sh.threads == 256) return weighted_kernel_for_nv<256>(sh.nv);
+    if (sh.threads == 512) return weighted_kernel_for_nv<512>(sh.nv);
+    if (sh.threads == 1024) return weighted_kernel_for_nv<1024>(sh.nv);
+    return nullptr;
+}
 static FastKernel fast_kernel(const FastShape& sh) {
     if (sh.one_exp) {
         if (sh.threads == 256) return fast_kernel_for_nv<256, true>(sh.nv);
@@ -944,7 +965,7 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
         FastShape sh;
         const bool tuned = g_tune_cluster.load() > 0;
         if (fast_ok && a.T < (1ll << 31) && pick_shape(a.V >> 3, &sh)) {
-            FastKernel k = fast_kernel(sh);
+            FastKernel k = wtok ? weighted_kernel(sh) : fast_kernel(sh);
             if (!k) return RLF_ERR_UNSUPPORTED;
             int nc = max_clusters(k, sh);
             if (nc <= 0) return RLF_ERR_UNSUPPORTED;      // this shape does not fit on the device
