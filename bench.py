@@ -38,7 +38,7 @@ WORKLOAD = "cfg1_qwen3_4b_microbatch: 16 responses x 2048 tokens, V=151936 bf16 
 
 # DRAM bytes of one row-kernel launch from the ncu capture summarised under profiles/, as bytes per
 # token; valid only for the row kernel's source text it was taken from (else reported as null).
-NCU_TRAFFIC = {"logits_loss_cu_sha1": "e87d0edb678454321ca2c0be075e0e050f25499f", "dram_bytes_per_token": 595845.0}
+NCU_TRAFFIC = {"logits_loss_cu_sha1": "beae1f6cbc292ea9da59db4c5f59b105793ed141", "dram_bytes_per_token": 596259.0}
 
 
 def _peaks():
