@@ -193,7 +193,7 @@ def aggregate(tokens_per_rank, world, max_seconds):
     return tokens_per_rank * world / max_seconds
 
 
-def max_over_ranks(seconds, world, device=None, backend_tensor=None):
+def max_over_ranks(seconds, world, device=None):
     """Slowest rank's time (an all-reduce MAX of one scalar; identity at world size 1)."""
     if world <= 1:
         return float(seconds)
