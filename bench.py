@@ -474,14 +474,15 @@ def run_cuda(args):
     fwd_only = None
     if rank == 0 and world == 1:
         ent = torch.empty(T, dtype=torch.float32, device=dev)
+        ws_ent = rlf.new_workspace(rlf.FN_LOGP_ENTROPY, T, V, 0, rlf.RLF_BF16, dev)
         for _ in range(2):
-            rlf.rlf_logp_entropy_fwd(batch.logits, batch.ids, logp_out=logp, entropy_out=ent, workspace=ws)
+            rlf.rlf_logp_entropy_fwd(batch.logits, batch.ids, logp_out=logp, entropy_out=ent, workspace=ws_ent)
         torch.cuda.synchronize()
         fe = []
         for _ in range(max(3, min(args.steps, 10))):
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
-            rlf.rlf_logp_entropy_fwd(batch.logits, batch.ids, logp_out=logp, entropy_out=ent, workspace=ws)
+            rlf.rlf_logp_entropy_fwd(batch.logits, batch.ids, logp_out=logp, entropy_out=ent, workspace=ws_ent)
             b.record()
             torch.cuda.synchronize()
             fe.append(a.elapsed_time(b))

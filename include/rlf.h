@@ -59,6 +59,7 @@ typedef enum { RLF_BF16 = 0, RLF_F32 = 1 } rlf_dtype;
 /* selectors for rlf_workspace_bytes */
 #define RLF_FN_LOGP_LOSS 3
 #define RLF_FN_FUSED_LMHEAD 4
+#define RLF_FN_LOGP_ENTROPY 5
 
 typedef struct CUstream_st *rlf_stream_t;
 
@@ -209,9 +210,11 @@ rlf_status rlf_grpo_logp_loss_fwd_bwd_skip_masked(const void *logits, rlf_dtype 
  *     logp[t]    = z[t, ids[t]] - log sum_v exp z[t, v]
  *     entropy[t] = - sum_v p_v log p_v,  p = softmax(z[t, :])      (terms with p_v = 0 contribute 0)
  * Each logits row is read from HBM once (2 V bytes per token at bf16); nothing else of size T x V
- * is touched.  Same fast-path conditions, general fallback, workspace size
- * (rlf_workspace_bytes(RLF_FN_LOGP_LOSS, ...)) and device status bits as rlf_grpo_logp_loss_fwd_bwd;
- * a row with a target outside [0, V) or a non-finite log-sum-exp gets NaN.
+ * is touched.  Same fast-path conditions, general fallback and device status bits as
+ * rlf_grpo_logp_loss_fwd_bwd; a row with a target outside [0, V) or a non-finite log-sum-exp gets
+ * NaN.  workspace: rlf_workspace_bytes(RLF_FN_LOGP_ENTROPY, T, V, 0, dt) bytes select the streaming
+ * form (rows cut into chunks whose partial statistics a second kernel merges); with only
+ * rlf_workspace_bytes(RLF_FN_LOGP_LOSS, ...) bytes the row-per-cluster form runs instead.
  *   logits [T, V] dt with row_stride;  ids [T] int32;  logp_out [T] fp32;  entropy_out [T] fp32 or NULL
  */
 rlf_status rlf_logp_entropy_fwd(const void *logits, rlf_dtype dt, int64_t T, int32_t V, int64_t row_stride,

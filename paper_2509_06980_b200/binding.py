@@ -14,7 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "librlf.so")
 
 RLF_BF16, RLF_F32 = 0, 1
-FN_LOGP_LOSS, FN_FUSED_LMHEAD = 3, 4
+FN_LOGP_LOSS, FN_FUSED_LMHEAD, FN_LOGP_ENTROPY = 3, 4, 5
 DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
 
 EXPORTS = [
@@ -273,7 +273,7 @@ def rlf_logp_entropy_fwd(logits, ids, want_entropy=True, logp_out=None, entropy_
         entropy_out = torch.empty(T, dtype=torch.float32, device=dev)
     dt = _dt(logits)
     if workspace is None:
-        workspace = new_workspace(FN_LOGP_LOSS, T, V, 0, dt, dev)
+        workspace = new_workspace(FN_LOGP_ENTROPY, T, V, 0, dt, dev)
     _lib.rlf_logp_entropy_fwd.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
     _lib.rlf_logp_entropy_fwd.restype = _int
     _check(_lib.rlf_logp_entropy_fwd(logits.data_ptr() if T > 0 else None, dt, T, V, stride, _ptr(ids, torch.int32),

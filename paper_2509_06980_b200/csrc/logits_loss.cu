@@ -1121,6 +1121,185 @@ ids_to_record_kernel(const int32_t* __restrict__ ids, int64_t T, int32_t V, floa
     rec[t] = make_float4(0.0f, 0.0f, 0.0f, __int_as_float(bad ? y : (y | (int)0x80000000)));
 }
 
+// Streaming form of the forward-only pass.  Log-sum-exp statistics are associative, so a row need not
+// be owned by anyone: a work unit is one CHUNK of one row (up to 256 x 10 vectors), every WARP turns
+// its share of a unit into a partial (max, sum 2^x, sum 2^x x) in global memory and a second kernel
+// merges the partials of a row and gathers the target logit.  No cluster, no exchange and no CTA
+// barrier: a thread only ever reads the staging slots it filled itself (cp.async, refilled with the
+// CTA's next unit as soon as they are in registers), so the warps of a CTA drift freely and the
+// exponential unit, the busiest pipe of this pass, is kept fed while other warps wait on loads.
+constexpr int kStreamThreads = 256;
+constexpr int kStreamWarps = kStreamThreads / 32;
+constexpr int kStreamNV = 10;
+constexpr int kStreamCtasPerSm = 4;
+
+// Packed fp32 pairs (one instruction, two lanes of arithmetic): with one instruction per element
+// for each of the multiply-adds around the exponential the pass is bound by instruction issue.
+__device__ __forceinline__ uint64_t f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f32x2_split(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+constexpr uint32_t kFloorPair = 0xFE96FE96u;   // two bf16 -9.97e37: keeps x finite, so that 2^x * x is 0, not NaN
+
+// (sum 2^x, sum 2^x x) with x = z log2e + off over this thread's registers; WANT_U = false drops the
+// second sum.  Only for moderate |max| (the caller takes the subtract-first form otherwise).
+template <int NV, bool WANT_U>
+__device__ __forceinline__ float2 stream_exp_pass(const uint4 (&d)[NV], float off) {
+    const uint64_t c2 = f32x2(kLog2e, kLog2e), off2 = f32x2(off, off);
+    uint64_t s2a = 0, s2b = 0, u2a = 0, u2b = 0;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+        const uint32_t w[4] = {d[i].x, d[i].y, d[i].z, d[i].w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t wc = WANT_U ? max_bf16x2(w[k], kFloorPair) : w[k];
+            const uint64_t x2 = fma_f32x2(f32x2(bf_lo(wc), bf_hi(wc)), c2, off2);
+            float x0, x1;
+            f32x2_split(x2, x0, x1);
+            const uint64_t e2 = f32x2(ex2_approx(x0), ex2_approx(x1));
+            if (k & 1) {
+                s2b = add_f32x2(s2b, e2);
+                if (WANT_U) u2b = fma_f32x2(e2, x2, u2b);
+            } else {
+                s2a = add_f32x2(s2a, e2);
+                if (WANT_U) u2a = fma_f32x2(e2, x2, u2a);
+            }
+        }
+    }
+    float a, b, c, e;
+    f32x2_split(add_f32x2(s2a, s2b), a, b);
+    f32x2_split(add_f32x2(u2a, u2b), c, e);
+    return make_float2(a + b, c + e);
+}
+
+struct StreamParams {
+    const __nv_bfloat16* logits;
+    long long stride;
+    long long units;            // T * chunks
+    int chunks;                 // chunks per row
+    int per_chunk_vec;          // vectors per chunk (the last chunk of a row may hold fewer)
+    int nvec;                   // V / 8
+    float4* partial;            // [units][kStreamWarps] (max, sum, usum, -)
+};
+
+template <bool WANT_U>
+__global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm)
+logp_entropy_stream_kernel(const StreamParams p) {
+    constexpr int NV = kStreamNV, THREADS = kStreamThreads;
+    extern __shared__ __align__(16) uint4 stage[];      // [NV][THREADS], slot (i, tid) private to thread tid
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    auto unit_geometry = [&](long long u, const uint4*& src, int& nvalid) {
+        const long long row = u / p.chunks;
+        const int chunk = (int)(u - row * p.chunks);
+        const int vbeg = chunk * p.per_chunk_vec + tid;
+        const int vend = min(p.nvec, (chunk + 1) * p.per_chunk_vec);
+        nvalid = vend > vbeg ? min(NV, (vend - vbeg + THREADS - 1) / THREADS) : 0;
+        src = reinterpret_cast<const uint4*>(p.logits + row * p.stride) + vbeg;
+    };
+    auto prefetch = [&](long long u) {
+        if (u < p.units) {
+            const uint4* src;
+            int nvalid;
+            unit_geometry(u, src, nvalid);
+#pragma unroll
+            for (int i = 0; i < NV; ++i)
+                if (i < nvalid) cp_async16_cg(stage + i * THREADS + tid, src + i * THREADS);
+        }
+        cp_async_commit();
+    };
+
+    prefetch(blockIdx.x);
+    for (long long u = blockIdx.x; u < p.units; u += gridDim.x) {
+        const uint4* src_unused;
+        int nvalid;
+        unit_geometry(u, src_unused, nvalid);
+        cp_async_wait_all();
+        uint4 d[NV];
+        if (nvalid == NV) {
+#pragma unroll
+            for (int i = 0; i < NV; ++i) d[i] = stage[i * THREADS + tid];
+        } else {
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                if (i < nvalid) d[i] = stage[i * THREADS + tid];
+                else d[i] = make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
+            }
+        }
+        prefetch(u + gridDim.x);          // the slots are in registers: refill them with the next unit
+        uint32_t mx = kNegInfPair;
+#pragma unroll
+        for (int i = 0; i < NV; ++i)
+            mx = max_bf16x2(mx, max_bf16x2(max_bf16x2(d[i].x, d[i].y), max_bf16x2(d[i].z, d[i].w)));
+        float m_w = fmaxf(bf_lo(mx), bf_hi(mx));
+        m_w = ord2f(__reduce_max_sync(0xffffffffu, f2ord(m_w)));
+        const float m_ws = (m_w == -INFINITY) ? 0.0f : m_w;
+        const float2 su = fabsf(m_ws) > kRobustAbove ? exp_sum_ent_pass<NV, true>(d, m_ws, 0.0f)
+                                                     : stream_exp_pass<NV, WANT_U>(d, -m_ws * kLog2e);
+        const float s_w = warp_sum(su.x), u_w = WANT_U ? warp_sum(su.y) : 0.0f;
+        if (lane == 0) p.partial[u * kStreamWarps + warp] = make_float4(m_w, s_w, u_w, 0.0f);
+    }
+    cp_async_wait_all();
+}
+
+// merge the warp partials of every row: one warp per row
+__global__ void __launch_bounds__(256)
+logp_entropy_merge_kernel(const float4* __restrict__ partial, int per_row, const __nv_bfloat16* __restrict__ logits,
+                          long long stride, const int32_t* __restrict__ ids, int64_t T, int32_t V,
+                          float* __restrict__ logp_out, float* __restrict__ entropy_out,
+                          int32_t* __restrict__ dev_status) {
+    const int lane = threadIdx.x & 31;
+    const int64_t t = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (t >= T) return;
+    const float4* row = partial + t * per_row;
+    float M = -INFINITY;
+    for (int c = lane; c < per_row; c += 32) M = fmaxf(M, row[c].x);
+    M = ord2f(__reduce_max_sync(0xffffffffu, f2ord(M)));
+    float S = 0.0f, U = 0.0f;
+    for (int c = lane; c < per_row; c += 32) {
+        const float4 e = row[c];
+        if (e.x == -INFINITY) continue;
+        const float dx = (e.x - M) * kLog2e;
+        const float f = ex2_approx(dx);
+        S += e.y * f;
+        if (f > 0.0f) U += f * fmaf(e.y, dx, e.z);
+    }
+    S = warp_sum(S);
+    U = warp_sum(U);
+    if (lane != 0) return;
+    const int32_t y = ids[t];
+    const bool bad = y < 0 || y >= V;
+    const float zy = bad ? 0.0f : __bfloat162float(logits[t * stride + y]);
+    const float lg2s = lg2_approx(S);
+    const float logp = (zy - M) - lg2s * kLn2;
+    const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) && (fabsf(logp) < INFINITY);
+    const float nan = __int_as_float(0x7fc00000);
+    logp_out[t] = (finite && !bad) ? logp : nan;
+    if (entropy_out) entropy_out[t] = finite ? (lg2s - U / S) * kLn2 : nan;
+    const int st = (bad ? RLF_DEV_BAD_TARGET : 0) | (finite ? 0 : RLF_DEV_NONFINITE);
+    if (st && dev_status) atomicOr(dev_status, st);
+}
+
+static int stream_chunks(int nvec) { return (nvec + kStreamThreads * kStreamNV - 1) / (kStreamThreads * kStreamNV); }
+size_t entropy_workspace_bytes(int64_t T, int32_t V) {
+    const size_t chunks = V >= 8 ? (size_t)stream_chunks(V >> 3) : 1;
+    return loss_workspace_bytes(T) + 16 * ws_tokens(T) * chunks * kStreamWarps + 256;
+}
+
 template <int THREADS>
 static FastKernel entropy_kernel_for_nv(int nv) {
     switch (nv) {
@@ -1154,14 +1333,34 @@ extern "C" rlf_status rlf_logp_entropy_fwd(const void* logits, rlf_dtype dt, int
     if (st != RLF_OK) return st;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
     char* ws = static_cast<char*>(workspace);
+    const bool fast_ok = dt == RLF_BF16 && (V % 8 == 0) && (row_stride % 8 == 0) && aligned(logits, 16) &&
+                         T < (1ll << 30);
+    if (fast_ok && workspace_bytes >= entropy_workspace_bytes(T, V)) {
+        // streaming form: chunk partials, then a per-row merge
+        const int smem = kStreamNV * kStreamThreads * 16;   // 40 KB: below the default dynamic limit
+        StreamParams sp;
+        sp.logits = static_cast<const __nv_bfloat16*>(logits);
+        sp.stride = row_stride;
+        sp.nvec = V >> 3;
+        sp.chunks = stream_chunks(sp.nvec);
+        sp.per_chunk_vec = (sp.nvec + sp.chunks - 1) / sp.chunks;
+        sp.units = (long long)T * sp.chunks;
+        sp.partial = reinterpret_cast<float4*>(ws + ((loss_workspace_bytes(T) + 255) & ~(size_t)255));
+        long long grid = (long long)sm_count() * kStreamCtasPerSm;
+        if (grid > sp.units) grid = sp.units;
+        if (entropy_out) logp_entropy_stream_kernel<true><<<(unsigned)grid, kStreamThreads, smem, s>>>(sp);
+        else logp_entropy_stream_kernel<false><<<(unsigned)grid, kStreamThreads, smem, s>>>(sp);
+        logp_entropy_merge_kernel<<<(unsigned)((T + 7) / 8), 256, 0, s>>>(
+            sp.partial, sp.chunks * kStreamWarps, sp.logits, row_stride, ids, T, V, logp_out, entropy_out, dev_status);
+        count_launch(2);
+        return cuda_ok(cudaGetLastError());
+    }
     long long* one = reinterpret_cast<long long*>(ws);
     float4* rec = reinterpret_cast<float4*>(ws + kWsRecordOff);
     ids_to_record_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(ids, T, V, rec, one, dev_status);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
 
-    const bool fast_ok = dt == RLF_BF16 && (V % 8 == 0) && (row_stride % 8 == 0) && aligned(logits, 16) &&
-                         T < (1ll << 30);
     FastShape sh;
     if (fast_ok && pick_shape(V >> 3, &sh)) {
         FastKernel k = sh.threads == 256 ? entropy_kernel_for_nv<256>(sh.nv)

@@ -13,9 +13,17 @@ DEV = "cuda"
 ENT_ATOL = 2e-3
 
 
+def _ws(b, form, T, V):
+    """`stream`: the entry's own workspace size (chunked streaming kernels); `cluster`: only the loss
+    workspace, which selects the row-per-cluster kernel."""
+    return b.new_workspace(b.FN_LOGP_ENTROPY if form == "stream" else b.FN_LOGP_LOSS, T, V, 0, b.RLF_BF16, DEV)
+
+
 @pytest.mark.parametrize("V,dtype,std", [(151936, "bf16", 3.0), (151936, "bf16", 0.5), (4096, "bf16", 8.0),
-                                          (1001, "bf16", 2.0), (1024, "f32", 2.0), (8, "bf16", 1.0)])
-def test_logp_and_entropy_match_oracle(V, dtype, std):
+                                          (1001, "bf16", 2.0), (1024, "f32", 2.0), (8, "bf16", 1.0),
+                                          (20480, "bf16", 3.0), (20488, "bf16", 3.0), (40968, "bf16", 3.0)])
+@pytest.mark.parametrize("form", ["stream", "cluster"])
+def test_logp_and_entropy_match_oracle(V, dtype, std, form):
     b = gc.binding()
     spec = synth.scaled(synth.SPECS[1], V=V, logits_dtype=dtype, logits_std=std, len_lo=12, len_hi=12, spans_lo=1,
                         spans_hi=1, obs_lo=2, obs_hi=3)
@@ -24,7 +32,7 @@ def test_logp_and_entropy_match_oracle(V, dtype, std):
     logits = synth.make_logits(spec, T, DEV)
     ids = torch.from_numpy(tok.ids).to(DEV)
     st = torch.zeros(1, dtype=torch.int32, device=DEV)
-    logp, ent = b.rlf_logp_entropy_fwd(logits, ids, dev_status=st)
+    logp, ent = b.rlf_logp_entropy_fwd(logits, ids, dev_status=st, workspace=_ws(b, form, T, V))
     torch.cuda.synchronize()
     assert st.item() == 0
     lp_o, h_o = orc.logp_entropy(gc.to_np(logits), tok.ids)
@@ -47,11 +55,13 @@ def test_every_launch_shape_and_special_rows():
     ids[2] = 1
     lp_o, h_o = orc.logp_entropy(gc.to_np(z), ids.cpu().numpy())
     assert abs(h_o[0] - np.log(V)) < 1e-9 and h_o[1] < 1e-20
-    for shape in [(0, 0), (8, 256), (8, 512), (4, 512), (2, 1024), (4, 1024)]:
-        b.tune_logits_kernel(shape[0], shape[1], -1)
+    for shape in ["stream", (0, 0), (8, 256), (8, 512), (4, 512), (2, 1024), (4, 1024)]:
+        form = "stream" if shape == "stream" else "cluster"
+        if form == "cluster":
+            b.tune_logits_kernel(shape[0], shape[1], -1)
         try:
             st = torch.zeros(1, dtype=torch.int32, device=DEV)
-            logp, ent = b.rlf_logp_entropy_fwd(z, ids, dev_status=st)
+            logp, ent = b.rlf_logp_entropy_fwd(z, ids, dev_status=st, workspace=_ws(b, form, T, V))
             torch.cuda.synchronize()
         finally:
             b.tune_logits_kernel(0, 0, -1)
@@ -66,8 +76,11 @@ def test_matches_the_training_entry_point_and_flags_bad_targets():
     batch = synth.make_batch(spec, DEV)
     full = gc.gpu_chain(batch, batch.logits, want_grad=False)
     logp, _ = b.rlf_logp_entropy_fwd(batch.logits, batch.ids, want_entropy=False)
+    logp_c, _ = b.rlf_logp_entropy_fwd(batch.logits, batch.ids, want_entropy=False,
+                                       workspace=_ws(b, "cluster", len(batch.ids), spec.V))
     torch.cuda.synchronize()
     assert (logp - full["logp"]).abs().max().item() <= 1e-5
+    assert (logp_c - full["logp"]).abs().max().item() <= 1e-5
     ids = batch.ids.clone()
     ids[3] = spec.V
     st = torch.zeros(1, dtype=torch.int32, device=DEV)
