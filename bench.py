@@ -89,7 +89,13 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3):
     out = {"workload": "%s: hidden [%d, %d] x W [151936, %d] bf16" % (spec.name, T, spec.D, spec.D), "T": T, "D": spec.D,
            "V": spec.V}
     burst, sustained, kind = _tensor_peaks()
-    for name, bwd, gemms, executed in (("fwd", False, 1, 1), ("fwd_bwd", True, 3, 4)):
+    # the backward contracts only over rows with a non-zero coefficient (here: the unmasked rows), so
+    # its flops are counted over those rows: useful = 2 GEMMs, executed = 3 (dZ is recomputed)
+    live = int(mask.sum().item())
+    out["live_rows"] = live
+    tvd = 2.0 * spec.V * spec.D
+    for name, bwd, useful_flops, executed_flops in (("fwd", False, tvd * T, tvd * T),
+                                                    ("fwd_bwd", True, tvd * (T + 2 * live), tvd * (T + 3 * live))):
         for _ in range(1 if tokens_per_response else 2):
             run(bwd)
         torch.cuda.synchronize()
@@ -102,9 +108,10 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3):
             torch.cuda.synchronize()
             ts.append(a.elapsed_time(b))
         ms = statistics.mean(ts)
-        useful = 2.0 * T * spec.V * spec.D * gemms / ms / 1e9
+        useful = useful_flops / ms / 1e9
         out[name] = {"ms": ms, "tokens_per_s": T / ms * 1e3, "useful_tflops": useful,
-                     "executed_tflops": 2.0 * T * spec.V * spec.D * executed / ms / 1e9,
+                     "executed_tflops": executed_flops / ms / 1e9,
+                     "dense_equivalent_tflops": tvd * T * (3 if bwd else 1) / ms / 1e9,
                      "roofline": {"bound": "tensor", "achieved": useful, "peak": burst, "unit": "TFLOP/s",
                                   "frac": useful / burst, "peak_kind": "of " + kind + " (burst)",
                                   "frac_of_sustained": useful / sustained, "frac_of_nominal_2250": useful / 2250.0,

@@ -62,6 +62,12 @@ struct GemmParams {
     long long out_stride;
     int accumulate;
     int32_t* dev_status;
+    // Token extent known only on the device (the backward runs over the compacted rows with a
+    // non-zero coefficient): when live_count is set, the token extent of this launch is
+    // clamp(*live_count - live_off, 0, M or K as built on the host).
+    const int* live_count;
+    int live_off;
+    const int32_t* row_index; // kGradHidden: output row of compact row r is row_index[live_off + r]
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -192,8 +198,17 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const bool sweep = p.mode == kLse || p.mode == kDz;     // a unit sweeps several vocabulary tiles
     // in pair form the scheduling unit covers two token tiles: this CTA takes tile 2 * mp + rank
     const int rank = PAIR ? (int)pair_rank() : 0;
-    const int m_units = PAIR ? (p.m_tiles + 1) / 2 : p.m_tiles;
-    const int units = sweep ? m_units * p.nsplit : m_units * p.n_tiles;
+    int M = p.M, m_tiles = p.m_tiles, k_slabs = p.k_slabs;
+    if (p.live_count) {
+        const int host_extent = p.mode == kGradW ? p.k_slabs * BK : p.M;
+        const int live = max(0, min(*p.live_count - p.live_off, host_extent));
+        if (p.mode == kGradW) k_slabs = (live + BK - 1) / BK;
+        else { M = live; m_tiles = (live + BM - 1) / BM; }
+    }
+    // no tokens under a grad_W tile: nothing to add; without accumulate the tile is still written (zeros)
+    const bool no_k = k_slabs == 0;
+    const int m_units = PAIR ? (m_tiles + 1) / 2 : m_tiles;
+    const int units = (no_k && p.accumulate) ? 0 : sweep ? m_units * p.nsplit : m_units * p.n_tiles;
     const int worker = PAIR ? blockIdx.x >> 1 : blockIdx.x;
     const int workers = PAIR ? gridDim.x >> 1 : gridDim.x;
 
@@ -248,13 +263,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int u = worker; u < units && ok; u += workers) {
+            for (int u = worker; u < units && ok && !no_k; u += workers) {
                 int m, n0, n1;
                 unit_range(u, m, n0, n1);
                 const int my_m = PAIR ? 2 * m + rank : m;
                 for (int n = n0; n < n1 && ok; ++n) {
                     const int b_row0 = n * BN + rank * C::kBRows;      // this CTA's rows of the B tile
-                    for (int kb = 0; kb < p.k_slabs; ++kb) {
+                    for (int kb = 0; kb < k_slabs; ++kb) {
                         if (!mbar_wait(smem_addr(&ctl->empty[stage]), phase ^ 1u, &ctl->abort_flag)) { ok = false; break; }
                         const uint32_t own_bar = smem_addr(&ctl->full[stage]);
                         const uint32_t bar = PAIR ? map_to_cta(own_bar, 0) : own_bar;   // the leader's barrier
@@ -292,14 +307,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             int buf = 0;
             uint32_t tphase[2] = {0, 0};
             bool ok = true;
-            for (int u = worker; u < units && ok; u += workers) {
+            for (int u = worker; u < units && ok && !no_k; u += workers) {
                 int m, n0, n1;
                 unit_range(u, m, n0, n1);
                 for (int n = n0; n < n1 && ok; ++n) {
                     if (!mbar_wait(smem_addr(&ctl->tmem_empty[buf]), tphase[buf] ^ 1u, &ctl->abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + (uint32_t)buf * BN;
-                    for (int kb = 0; kb < p.k_slabs; ++kb) {
+                    for (int kb = 0; kb < k_slabs; ++kb) {
                         if (!mbar_wait(smem_addr(&ctl->full[stage]), phase, &ctl->abort_flag)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t sa = tiles + stage * C::kStageBytes;
@@ -337,7 +352,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             int m, n0, n1;
             unit_range(u, m, n0, n1);
             const int row = (PAIR ? 2 * m + rank : m) * BM + row_in_tile;
-            const bool row_ok = row < p.M;
+            const bool row_ok = row < M;
             float run_m = -INFINITY, run_s = 0.0f;       // kLse
             float c2 = 0.0f, coef = 0.0f;                // kDz
             uint32_t sgn = 0;
@@ -351,8 +366,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 }
             }
             for (int n = n0; n < n1 && ok; ++n) {
-                if (!mbar_wait(smem_addr(&ctl->tmem_full[buf]), tphase[buf], &ctl->abort_flag)) { ok = false; break; }
-                tc_fence_after();
+                if (!no_k) {
+                    if (!mbar_wait(smem_addr(&ctl->tmem_full[buf]), tphase[buf], &ctl->abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                }
                 const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * BN;
                 const int col0 = n * BN;
 #pragma unroll 1
@@ -360,7 +377,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     const int cb = col0 + c * 32;
                     if (cb >= p.N) break;                // whole chunk beyond the valid columns (warp-uniform)
                     uint32_t v[32];
-                    tc_ld32(t_row + (uint32_t)(c * 32), v);
+                    if (no_k) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = 0u;
+                    } else {
+                        tc_ld32(t_row + (uint32_t)(c * 32), v);
+                    }
                     const int nvalid = min(32, p.N - cb);
                     if (p.mode == kLse) {
                         float cm = -INFINITY;
@@ -380,7 +402,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         }
                         run_s += s0 + s1;
                     } else if (p.mode == kDz) {
-                        if (row_ok) {
+                        // rows past the live extent (still inside this tile, which the scratch holds)
+                        // are stored as zeros: the grad_W contraction reads whole 64-row slabs
+                        {
                             uint32_t o[16];
                             if (coef == 0.0f) {
 #pragma unroll
@@ -423,7 +447,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         }
                     } else if (p.mode == kGradHidden) {
                         if (row_ok) {
-                            __nv_bfloat16* dst = p.out_bf16 + (long long)row * p.out_stride + cb;
+                            const long long orow = p.row_index ? (long long)p.row_index[p.live_off + row] : (long long)row;
+                            __nv_bfloat16* dst = p.out_bf16 + orow * p.out_stride + cb;
                             if (nvalid == 32) {
                                 uint32_t o[16];
 #pragma unroll
@@ -464,7 +489,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 // hand the accumulator buffer back to the MMA warp
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) {
+                if (lane == 0 && !no_k) {
                     if (PAIR) mbar_arrive_cluster(map_to_cta(smem_addr(&ctl->tmem_empty[buf]), 0));
                     else mbar_arrive(smem_addr(&ctl->tmem_empty[buf]));
                 }
@@ -555,6 +580,60 @@ combine_kernel(const float2* __restrict__ part, int nsplit, const float* __restr
     lse_out[t] = finite ? lse : 0.0f;
     coef_out[t] = coef;
     if (!finite && dev_status) atomicOr(dev_status, RLF_DEV_NONFINITE);
+}
+
+// Rows whose coefficient is zero (masked tokens, clipped tokens with beta = 0) contribute nothing to
+// either gradient, so the backward runs over the other rows only.  Stable compaction (token order is
+// kept, so results do not depend on timing): one CTA scans the T flags.
+__global__ void __launch_bounds__(1024)
+compact_live_kernel(const float* __restrict__ coef, int T, int32_t* __restrict__ live_idx, int* __restrict__ live_count) {
+    __shared__ int warp_tot[32];
+    __shared__ int base_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) base_s = 0;
+    __syncthreads();
+    for (int t0 = 0; t0 < T; t0 += 1024) {
+        const int t = t0 + tid;
+        const bool live = t < T && coef[t] != 0.0f;
+        const unsigned bal = __ballot_sync(0xffffffffu, live);
+        if (lane == 0) warp_tot[warp] = __popc(bal);
+        __syncthreads();
+        int before = 0, total = 0;
+        for (int w = 0; w < 32; ++w) {
+            const int c = warp_tot[w];
+            if (w < warp) before += c;
+            total += c;
+        }
+        const int base = base_s;
+        if (live) live_idx[base + before + __popc(bal & ((1u << lane) - 1u))] = t;
+        __syncthreads();
+        if (tid == 0) base_s = base + total;
+    }
+    __syncthreads();
+    if (tid == 0) *live_count = base_s;
+}
+
+// compact row r <- token live_idx[r]: hidden row, lse, coefficient, target id.  Rows from the live
+// count up to the next multiple of 256 are zero-filled (the contractions read whole tiles).
+__global__ void __launch_bounds__(128)
+gather_live_kernel(const __nv_bfloat16* __restrict__ hidden, int D, const float* __restrict__ lse,
+                   const float* __restrict__ coef, const int32_t* __restrict__ ids, const int32_t* __restrict__ live_idx,
+                   const int* __restrict__ live_count, __nv_bfloat16* __restrict__ hidden_c, float* __restrict__ lse_c,
+                   float* __restrict__ coef_c, int32_t* __restrict__ ids_c) {
+    const int n = *live_count;
+    const int r = blockIdx.x;
+    if (r >= ((n + 255) & ~255)) return;
+    uint4* dst = reinterpret_cast<uint4*>(hidden_c + (long long)r * D);
+    const int nv = D / 8;
+    if (r < n) {
+        const int t = live_idx[r];
+        const uint4* src = reinterpret_cast<const uint4*>(hidden + (long long)t * D);
+        for (int i = threadIdx.x; i < nv; i += blockDim.x) dst[i] = src[i];
+        if (threadIdx.x == 0) { lse_c[r] = lse[t]; coef_c[r] = coef[t]; ids_c[r] = ids[t]; }
+    } else {
+        for (int i = threadIdx.x; i < nv; i += blockDim.x) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (threadIdx.x == 0) { lse_c[r] = 0.0f; coef_c[r] = 0.0f; ids_c[r] = -1; }
+    }
 }
 
 // ---- host side ------------------------------------------------------------------------------
@@ -671,22 +750,28 @@ static int pick_split(int m_units, int n_tiles, int workers) {
 }
 
 struct LmWs {
-    size_t n_count, partial, rec, zy, lse, coef, part, dz, total;
+    size_t n_count, partial, rec, zy, lse, coef, part, live_idx, lse_c, coef_c, ids_c, hidden_c, dz, total;
 };
 static size_t up1k(size_t x) { return (x + 1023) & ~(size_t)1023; }
-static LmWs lm_workspace(int64_t T, int32_t V) {
+static LmWs lm_workspace(int64_t T, int32_t V, int32_t D) {
     LmWs w;
     size_t o = 0;
     const size_t Tn = (size_t)(T > 0 ? T : 0);
-    w.n_count = o; o += 1024;
+    const size_t Tp = (Tn + 255) & ~(size_t)255;     // compact arrays are padded to whole tile pairs
+    w.n_count = o; o += 1024;                        // [0] mask count, [64] live-row count
     w.partial = o; o += up1k(token_loss_partial_bytes());
     w.rec = o;     o += up1k(16 * Tn);
     w.zy = o;      o += up1k(4 * Tn);
     w.lse = o;     o += up1k(4 * Tn);
     w.coef = o;    o += up1k(4 * Tn);
     w.part = o;    o += up1k(8 * Tn * kMaxSplit);
+    w.live_idx = o; o += up1k(4 * Tp);
+    w.lse_c = o;   o += up1k(4 * Tp);
+    w.coef_c = o;  o += up1k(4 * Tp);
+    w.ids_c = o;   o += up1k(4 * Tp);
+    w.hidden_c = o; o += up1k(Tp * (size_t)(D > 0 ? D : 0) * 2);
     w.dz = o;
-    const size_t chunk = Tn < (size_t)kChunkTokens ? Tn : (size_t)kChunkTokens;
+    const size_t chunk = Tp < (size_t)kChunkTokens ? Tp : (size_t)kChunkTokens;
     o += up1k(chunk * (size_t)V * 2);
     w.total = o + 1024;
     return w;
@@ -695,9 +780,8 @@ static LmWs lm_workspace(int64_t T, int32_t V) {
 }  // namespace lm
 
 size_t lmhead_workspace_bytes(int64_t T, int32_t V, int32_t D) {
-    (void)D;
-    if (V < 1) return 0;
-    return lm::lm_workspace(T, V).total;
+    if (V < 1 || D < 1) return 0;
+    return lm::lm_workspace(T, V, D).total;
 }
 
 }  // namespace rlf
@@ -720,7 +804,7 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
     if (T > 0 && B == 0) return RLF_ERR_SHAPE;
     if (!aligned(hidden, 16) || !aligned(W, 16) || !aligned(grad_hidden, 16) || !aligned(grad_W, 16))
         return RLF_ERR_ALIGN;
-    const LmWs w = lm_workspace(T, V);
+    const LmWs w = lm_workspace(T, V, D);
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < w.total) return RLF_ERR_WORKSPACE;
     rlf_status st = check_arch();
     if (st != RLF_OK) return st;
@@ -781,26 +865,42 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
     if (st != RLF_OK) return st;
     if (!grad_hidden && !grad_W) return RLF_OK;
 
-    // backward by token chunks: dZ chunk -> grad_hidden rows of the chunk, grad_W += chunk's part
+    // backward over the rows with a non-zero coefficient only, compacted in token order; their number
+    // stays on the device (no host sync), so every chunk is launched and the kernels size themselves
+    int* live_count = reinterpret_cast<int*>(ws + w.n_count + 64);
+    int32_t* live_idx = reinterpret_cast<int32_t*>(ws + w.live_idx);
+    float* lse_c = reinterpret_cast<float*>(ws + w.lse_c);
+    float* coef_c = reinterpret_cast<float*>(ws + w.coef_c);
+    int32_t* ids_c = reinterpret_cast<int32_t*>(ws + w.ids_c);
+    __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(ws + w.hidden_c);
+    const int64_t Tp = (T + 255) & ~(int64_t)255;
+    compact_live_kernel<<<1, 1024, 0, s>>>(coef, (int)T, live_idx, live_count);
+    gather_live_kernel<<<(unsigned)Tp, 128, 0, s>>>(H, D, lse, coef, ids, live_idx, live_count, Hc, lse_c, coef_c, ids_c);
+    count_launch(2);
+    if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+    if (grad_hidden && cudaMemsetAsync(grad_hidden, 0, (size_t)T * D * 2, s) != cudaSuccess) return RLF_ERR_CUDA;
+
     for (int64_t t0 = 0; t0 < T; t0 += kChunkTokens) {
         const int64_t tc = (T - t0) < kChunkTokens ? (T - t0) : kChunkTokens;
         CUtensorMap mapHc;
-        if (!make_map(&mapHc, H + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
+        if (!make_map(&mapHc, Hc + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
         GemmParams z = g;
         z.mode = kDz;
         z.M = (int)tc;
         z.m_tiles = (int)((tc + BM - 1) / BM);
         z.nsplit = pick_split(pair ? (z.m_tiles + 1) / 2 : z.m_tiles, z.n_tiles, workers);
         z.n_tiles_per_split = (z.n_tiles + z.nsplit - 1) / z.nsplit;
-        z.lse = lse + t0;
-        z.coef = coef + t0;
-        z.ids = ids + t0;
+        z.lse = lse_c + t0;
+        z.coef = coef_c + t0;
+        z.ids = ids_c + t0;
         z.dz = dz;
         z.dz_stride = V;
+        z.live_count = live_count;
+        z.live_off = (int)t0;
         st = launch_gemm(mapHc, mapW, z, pair, s);
         if (st != RLF_OK) return st;
         if (grad_hidden) {
-            // grad_hidden[chunk] = dZ[chunk, V] W[V, D]
+            // grad_hidden[token of compact row] = dZ[chunk, V] W[V, D]
             CUtensorMap mapDzK, mapWn;
             if (!make_map(&mapDzK, dz, (uint64_t)tc, (uint64_t)V, (uint64_t)V, BK, BM)) return RLF_ERR_CUDA;
             if (!make_map(&mapWn, Wm, (uint64_t)V, (uint64_t)D, (uint64_t)D, 64, BK)) return RLF_ERR_CUDA;
@@ -811,9 +911,12 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
             h.m_tiles = (int)((tc + BM - 1) / BM);
             h.n_tiles = (D + BN - 1) / BN;
             h.k_slabs = (V + BK - 1) / BK;
-            h.out_bf16 = static_cast<__nv_bfloat16*>(grad_hidden) + t0 * D;
+            h.out_bf16 = static_cast<__nv_bfloat16*>(grad_hidden);
             h.out_stride = D;
             h.dev_status = dev_status;
+            h.live_count = live_count;
+            h.live_off = (int)t0;
+            h.row_index = live_idx;
             st = launch_gemm(mapDzK, mapWn, h, pair, s);
             if (st != RLF_OK) return st;
         }
@@ -821,7 +924,7 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
             // grad_W[V, D] (+)= dZ[chunk, V]^T hidden[chunk, D]
             CUtensorMap mapDzM, mapHn;
             if (!make_map(&mapDzM, dz, (uint64_t)tc, (uint64_t)V, (uint64_t)V, 64, BK)) return RLF_ERR_CUDA;
-            if (!make_map(&mapHn, H + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, 64, BK)) return RLF_ERR_CUDA;
+            if (!make_map(&mapHn, Hc + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, 64, BK)) return RLF_ERR_CUDA;
             GemmParams q = {};
             q.mode = kGradW;
             q.M = V;
@@ -833,6 +936,8 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
             q.out_stride = D;
             q.accumulate = (accumulate_grad_W || t0 > 0) ? 1 : 0;
             q.dev_status = dev_status;
+            q.live_count = live_count;
+            q.live_off = (int)t0;
             st = launch_gemm(mapDzM, mapHn, q, pair, s);
             if (st != RLF_OK) return st;
         }

@@ -184,3 +184,46 @@ def test_fused_micro_batches_with_global_denominator_accumulate():
     assert abs(total - full[1][0].item()) <= 1e-9 + 1e-6 * abs(full[1][0].item())
     scale = full[3].abs().max().item()
     assert (gw - full[3]).abs().max().item() <= 2.0 ** -7 * scale
+
+
+@pytest.mark.parametrize("n_live", [0, 1, 129])
+def test_fused_backward_runs_over_live_rows_only(n_live, form):
+    """The backward contracts over the rows with a non-zero coefficient only.  No live row at all:
+    grad_hidden is zero and grad_W is zero (or untouched when accumulating); one live row / one row
+    past a 128-row tile: the gradients equal the oracle's."""
+    b = gc.binding()
+    spec = synth.scaled(synth.SPECS[3], V=2048, D=128, w_std=0.3, **SMALL)
+    batch = synth.make_batch(spec, DEV)
+    T = len(batch.ids)
+    assert T > 129
+    mask_np = np.zeros(T, dtype=np.uint8)
+    mask_np[np.random.default_rng(5).permutation(T)[:n_live]] = 1
+    mask = torch.from_numpy(mask_np).to(DEV)
+    seq = torch.from_numpy(gc.oracle_chain(batch)["seq_id"]).to(DEV)
+    adv = b.rlf_group_advantage(batch.rewards, group_size=batch.tokens.group_size)
+    n = torch.tensor([max(n_live, 1)], dtype=torch.int64, device=DEV)
+    for accumulate in (False, True):
+        gw0 = torch.randn((spec.V, spec.D), device=DEV)
+        st = torch.zeros(1, dtype=torch.int32, device=DEV)
+        logp, loss, gh, gw = b.rlf_fused_lmhead_grpo(batch.hidden, batch.W, batch.ids, seq, adv, batch.old_logp,
+                                                     batch.ref_logp, mask, synth.EPS_CLIP, synth.BETA_KL, denom=n,
+                                                     grad_W=gw0.clone(), accumulate_grad_W=accumulate, dev_status=st)
+        torch.cuda.synchronize()
+        assert st.item() == 0
+        r = orc.fused_lmhead_grpo(synth.bf16_bits(batch.hidden), synth.bf16_bits(batch.W), batch.ids.cpu().numpy(),
+                                  seq.cpu().numpy(), adv.cpu().numpy().astype(np.float64),
+                                  batch.old_logp.cpu().numpy(), batch.ref_logp.cpu().numpy(), mask_np,
+                                  synth.EPS_CLIP, synth.BETA_KL, denom=int(n.item()))
+        got_w = (gw - gw0) if accumulate else gw
+        assert not gh[~mask.bool()].any()
+        if n_live == 0:
+            assert not got_w.any() and not gh.any()
+        elif accumulate:
+            # (gw0 + g) - gw0 keeps g only to fp32 rounding of gw0 ~ N(0, 1): absolute comparison
+            scale = np.abs(r["grad_W"]).max()
+            assert np.abs(got_w.cpu().numpy() - r["grad_W"]).max() <= 2.0 ** -7 * scale + 1e-6
+        else:
+            _close_tensor(got_w.cpu().numpy(), r["grad_W"], "grad_W")
+        if n_live:
+            live = np.flatnonzero(mask_np)
+            _close_tensor(gh.float().cpu().numpy()[live], r["grad_hidden"][live], "grad_hidden")
