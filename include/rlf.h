@@ -258,8 +258,8 @@ rlf_status rlf_grpo_logp_loss_fwd_bwd_static(const void *logits, rlf_dtype dt, i
 /*
  * Same loss with the logits formed on the fly, z = hidden W^T, so that they
  * never reach HBM.  (Paper Sec. 2.2: pi_theta is the language model's output
- * head; the fusion itself is this library's design.)  Backward recomputes the
- * logit tiles and returns
+ * head; the fusion itself is this library's design.)  The backward runs over the
+ * unmasked rows only (the others have zero gradient) and returns
  *     grad_hidden[t,:] = sum_v grad_z[t,v] W[v,:]       (bf16)
  *     grad_W[v,:]      = sum_t grad_z[t,v] hidden[t,:]  (fp32; added to the buffer if accumulate_grad_W)
  *
@@ -268,12 +268,16 @@ rlf_status rlf_grpo_logp_loss_fwd_bwd_static(const void *logits, rlf_dtype dt, i
  *   per-token arguments, denom, logp_out, loss_out: as for rlf_grpo_logp_loss_fwd_bwd
  *   grad_hidden [T, D] bf16 or NULL;  grad_W [V, D] fp32 or NULL (both NULL: forward only)
  *   workspace   rlf_workspace_bytes(RLF_FN_FUSED_LMHEAD, T, V, D, RLF_BF16) bytes, 256-byte aligned.
- *               It holds per-token records and partial sums and, for the backward, one chunk of
- *               dZ = grad_z as bf16, [min(T, 9472), V] (2.9 GB at V = 151936): the logits are never
- *               stored, this chunk of their gradient is, between the kernel that forms it and the
- *               two contractions that consume it.
+ *               It holds per-token records and partial sums and, for the backward, a copy of hidden
+ *               with the unmasked rows gathered first, and one chunk [min(T, 9472), V] of bf16
+ *               (2.9 GB at V = 151936): the forward sweep of a chunk of unmasked rows leaves
+ *               exp(z - max of the 256-column tile) there (never above 1, so no logit overflows
+ *               it), an elementwise pass rescales it in place into dZ = grad_z once the row's
+ *               log-sum-exp is known, and the two gradient contractions consume it.  The logits
+ *               themselves are never stored.
  * Tensor-core contractions are bf16 x bf16 with fp32 accumulation in tensor memory; grad_z is
- * rounded to bf16 before the two gradient contractions.  Waits inside the kernels are bounded: if
+ * rounded to bf16 (twice: the stored exponential, then its product with the row's scale) before
+ * the two gradient contractions.  Waits inside the kernels are bounded: if
  * one runs out, RLF_DEV_TIMEOUT is set in *dev_status and the outputs are not valid.
  */
 rlf_status rlf_fused_lmhead_grpo(const void *hidden, const void *W, int64_t T, int32_t D, int32_t V,

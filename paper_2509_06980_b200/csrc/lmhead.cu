@@ -2,9 +2,9 @@
 // (tcgen05.mma, operands staged in shared memory by TMA, accumulators in tensor memory) and consumed
 // by the softmax / loss epilogue straight from tensor memory, so they never reach HBM.
 //
-// One warp-specialised kernel template serves four contractions (all bf16 x bf16 -> fp32):
-//   LSE   z tile = H W^T, epilogue keeps a running (max, sum exp) per token      -> log-sum-exp
-//   DZ    z tile recomputed, epilogue turns it into dZ = c_t (softmax - onehot)  -> bf16 scratch
+// One warp-specialised kernel template serves three contractions (all bf16 x bf16 -> fp32):
+//   LSE   z tile = H W^T, epilogue keeps a running (max, sum exp) per token      -> log-sum-exp;
+//         for rows that take part in the backward it also stores e = exp(z - tile max) as bf16
 //   GH    grad_hidden = dZ W      (A = dZ K-major, B = W vocabulary-major rows: N-major operand)
 //   GW    grad_W     += dZ^T H    (both operands token-major rows: M-/N-major operands)
 // CTA = 192 threads: warp 0 issues TMA loads into a multi-stage ring, warp 1 issues the MMAs (one
@@ -13,8 +13,12 @@
 // is being multiplied.  Every mbarrier wait is bounded; a wait that runs out raises a CTA-wide
 // abort flag, all roles leave their loops, tensor memory is released and RLF_DEV_TIMEOUT is set.
 //
-// Backward is by token chunks: DZ writes a [chunk, V] bf16 scratch, GH and GW read it.  The
-// logits themselves are never stored; the dZ scratch is (stated in the entry point's contract).
+// Forward + backward: the tokens are partitioned into unmasked rows and the others (only the first
+// carry gradient).  Unmasked rows go by chunks: LSE with the exponentials stored in a [chunk, V] bf16
+// scratch, an elementwise pass that rescales them in place into dZ = c_t (softmax - onehot) once the
+// row's log-sum-exp is known, then GH and GW read the scratch: three contractions per unmasked
+// row, one per masked row, no recomputation.  The logits themselves are never stored; the bf16
+// scratch is (stated in the entry point's contract).
 #include <cuda.h>
 
 #include <atomic>
@@ -44,7 +48,7 @@ constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;
 constexpr int kSlabBytes = 64 * BK * 2;      // one 64-wide slab of an MN-major operand: 64 k-rows of 128 B
 
-enum Mode { kLse = 0, kDz = 1, kGradHidden = 2, kGradW = 3 };
+enum Mode { kLse = 0, kGradHidden = 2, kGradW = 3 };
 
 struct GemmParams {
     int mode;
@@ -52,18 +56,16 @@ struct GemmParams {
     int m_tiles, n_tiles, k_slabs;
     int nsplit, n_tiles_per_split;
     float2* part;             // kLse: [M][nsplit] (max, sum exp)
-    const float* lse;         // kDz: per row of this launch
-    const float* coef;
-    const int32_t* ids;
-    __nv_bfloat16* dz;        // kDz out, row stride dz_stride
+    __nv_bfloat16* dz;        // kLse (optional) out, row stride dz_stride: exp(z - tile max) as bf16
+    float* tmax;              // kLse with dz: [M][n_tiles] the tile maxima those exponentials refer to
     long long dz_stride;
     __nv_bfloat16* out_bf16;  // kGradHidden out [M][out_stride]
     float* out_f32;           // kGradW out [M][out_stride]
     long long out_stride;
     int accumulate;
     int32_t* dev_status;
-    // Token extent known only on the device (the backward runs over the compacted rows with a
-    // non-zero coefficient): when live_count is set, the token extent of this launch is
+    // Token extent known only on the device (launches over the gathered unmasked / masked rows):
+    // when live_count is set, the token extent of this launch is
     // clamp(*live_count - live_off, 0, M or K as built on the host).
     const int* live_count;
     int live_off;
@@ -195,7 +197,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool a_mn = p.mode == kGradW;
     const bool b_mn = p.mode == kGradHidden || p.mode == kGradW;
-    const bool sweep = p.mode == kLse || p.mode == kDz;     // a unit sweeps several vocabulary tiles
+    const bool sweep = p.mode == kLse;                      // a unit sweeps several vocabulary tiles
     // in pair form the scheduling unit covers two token tiles: this CTA takes tile 2 * mp + rank
     const int rank = PAIR ? (int)pair_rank() : 0;
     int M = p.M, m_tiles = p.m_tiles, k_slabs = p.k_slabs;
@@ -354,17 +356,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const int row = (PAIR ? 2 * m + rank : m) * BM + row_in_tile;
             const bool row_ok = row < M;
             float run_m = -INFINITY, run_s = 0.0f;       // kLse
-            float c2 = 0.0f, coef = 0.0f;                // kDz
-            uint32_t sgn = 0;
-            int y = -1;
-            if (p.mode == kDz && row_ok) {
-                coef = p.coef[row];
-                y = p.ids[row];
-                if (coef != 0.0f) {
-                    c2 = lg2_approx(fabsf(coef)) - p.lse[row] * kLog2e;
-                    sgn = coef < 0.0f ? 0x80008000u : 0u;
-                }
-            }
             for (int n = n0; n < n1 && ok; ++n) {
                 if (!no_k) {
                     if (!mbar_wait(smem_addr(&ctl->tmem_full[buf]), tphase[buf], &ctl->abort_flag)) { ok = false; break; }
@@ -372,6 +363,65 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 }
                 const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * BN;
                 const int col0 = n * BN;
+                if (p.mode == kLse && p.dz) {
+                    // Forward sweep that keeps the tile for the backward.  Pass 1 over the accumulator:
+                    // the row's maximum inside this tile; pass 2: e = exp(z - that maximum), summed for
+                    // the log-sum-exp and stored as bf16 (e <= 1: no overflow whatever the logits are;
+                    // the relative rounding error is that of a bf16 gradient entry).
+                    float tm = -INFINITY;
+#pragma unroll 1
+                    for (int c = 0; c < BN / 32; ++c) {
+                        const int cb = col0 + c * 32;
+                        if (cb >= p.N) break;
+                        uint32_t v[32];
+                        tc_ld32(t_row + (uint32_t)(c * 32), v);
+                        const int nvalid = min(32, p.N - cb);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (i < nvalid) tm = fmaxf(tm, __uint_as_float(v[i]));
+                    }
+                    const float tms = (tm == -INFINITY) ? 0.0f : tm;
+                    if (tm > run_m) {
+                        run_s *= ex2_approx((run_m - tm) * kLog2e);
+                        run_m = tm;
+                    }
+                    const float off = -tms * kLog2e;
+                    float ts0 = 0.0f, ts1 = 0.0f;
+#pragma unroll 1
+                    for (int c = 0; c < BN / 32; ++c) {
+                        const int cb = col0 + c * 32;
+                        if (cb >= p.N) break;
+                        uint32_t v[32];
+                        tc_ld32(t_row + (uint32_t)(c * 32), v);
+                        const int nvalid = min(32, p.N - cb);
+                        uint32_t o[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            float e0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), kLog2e, off));
+                            float e1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), kLog2e, off));
+                            if (2 * i >= nvalid) e0 = 0.0f;
+                            if (2 * i + 1 >= nvalid) e1 = 0.0f;
+                            ts0 += e0;
+                            ts1 += e1;
+                            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[i]) : "f"(e1), "f"(e0));
+                        }
+                        if (row_ok) {
+                            __nv_bfloat16* dst = p.dz + (long long)row * p.dz_stride + cb;
+                            if (nvalid == 32) {
+                                uint4* d4 = reinterpret_cast<uint4*>(dst);
+                                d4[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                                d4[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                                d4[2] = make_uint4(o[8], o[9], o[10], o[11]);
+                                d4[3] = make_uint4(o[12], o[13], o[14], o[15]);
+                            } else {
+                                for (int i = 0; i < nvalid; ++i)
+                                    dst[i] = __ushort_as_bfloat16((unsigned short)((i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xffffu)));
+                            }
+                        }
+                    }
+                    if (tm != -INFINITY) run_s += (ts0 + ts1) * ex2_approx((tm - run_m) * kLog2e);
+                    if (row_ok) p.tmax[(long long)row * p.n_tiles + n] = tms;
+                } else
 #pragma unroll 1
                 for (int c = 0; c < BN / 32; ++c) {
                     const int cb = col0 + c * 32;
@@ -401,50 +451,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                             if (i + 1 < nvalid) s1 += ex2_approx(fmaf(__uint_as_float(v[i + 1]), kLog2e, off));
                         }
                         run_s += s0 + s1;
-                    } else if (p.mode == kDz) {
-                        // rows past the live extent (still inside this tile, which the scratch holds)
-                        // are stored as zeros: the grad_W contraction reads whole 64-row slabs
-                        {
-                            uint32_t o[16];
-                            if (coef == 0.0f) {
-#pragma unroll
-                                for (int i = 0; i < 16; ++i) o[i] = 0u;
-                            } else {
-#pragma unroll
-                                for (int i = 0; i < 16; ++i) {
-                                    float g0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), kLog2e, c2));
-                                    float g1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), kLog2e, c2));
-                                    uint32_t pk;
-                                    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(g1), "f"(g0));
-                                    o[i] = pk ^ sgn;
-                                }
-                                if (y >= cb && y < cb + 32) {
-                                    // target column: c (p_y - 1), rounded once
-                                    const int e = y - cb;
-                                    float zy = 0.0f;
-#pragma unroll
-                                    for (int i = 0; i < 32; ++i)
-                                        if (i == e) zy = __uint_as_float(v[i]);
-                                    const float py = ex2_approx(fmaf(zy, kLog2e, -p.lse[row] * kLog2e));
-                                    const uint32_t gb = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(fmaf(coef, py, -coef)));
-#pragma unroll
-                                    for (int i = 0; i < 16; ++i)
-                                        if (i == (e >> 1))
-                                            o[i] = (e & 1) ? ((o[i] & 0x0000ffffu) | (gb << 16)) : ((o[i] & 0xffff0000u) | gb);
-                                }
-                            }
-                            __nv_bfloat16* dst = p.dz + (long long)row * p.dz_stride + cb;
-                            if (nvalid == 32) {
-                                uint4* d4 = reinterpret_cast<uint4*>(dst);
-                                d4[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                                d4[1] = make_uint4(o[4], o[5], o[6], o[7]);
-                                d4[2] = make_uint4(o[8], o[9], o[10], o[11]);
-                                d4[3] = make_uint4(o[12], o[13], o[14], o[15]);
-                            } else {
-                                for (int i = 0; i < nvalid; ++i)
-                                    dst[i] = __ushort_as_bfloat16((unsigned short)((i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xffffu)));
-                            }
-                        }
                     } else if (p.mode == kGradHidden) {
                         if (row_ok) {
                             const long long orow = p.row_index ? (long long)p.row_index[p.live_off + row] : (long long)row;
@@ -582,11 +588,13 @@ combine_kernel(const float2* __restrict__ part, int nsplit, const float* __restr
     if (!finite && dev_status) atomicOr(dev_status, RLF_DEV_NONFINITE);
 }
 
-// Rows whose coefficient is zero (masked tokens, clipped tokens with beta = 0) contribute nothing to
-// either gradient, so the backward runs over the other rows only.  Stable compaction (token order is
-// kept, so results do not depend on timing): one CTA scans the T flags.
+// Masked rows contribute nothing to either gradient, so the backward (and the part of the forward
+// that keeps logits for it) runs over the unmasked rows only.  Stable partition of the tokens by
+// the live bit of their record (token order is kept inside each part, so results do not depend on
+// timing): one CTA scans the T flags.  counts[0] = live rows, counts[1] = the others.
 __global__ void __launch_bounds__(1024)
-compact_live_kernel(const float* __restrict__ coef, int T, int32_t* __restrict__ live_idx, int* __restrict__ live_count) {
+partition_rows_kernel(const float4* __restrict__ rec, int T, int32_t* __restrict__ idx_live,
+                      int32_t* __restrict__ idx_dead, int* __restrict__ counts) {
     __shared__ int warp_tot[32];
     __shared__ int base_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -594,7 +602,7 @@ compact_live_kernel(const float* __restrict__ coef, int T, int32_t* __restrict__
     __syncthreads();
     for (int t0 = 0; t0 < T; t0 += 1024) {
         const int t = t0 + tid;
-        const bool live = t < T && coef[t] != 0.0f;
+        const bool live = t < T && __float_as_int(rec[t].w) < 0;
         const unsigned bal = __ballot_sync(0xffffffffu, live);
         if (lane == 0) warp_tot[warp] = __popc(bal);
         __syncthreads();
@@ -605,34 +613,117 @@ compact_live_kernel(const float* __restrict__ coef, int T, int32_t* __restrict__
             total += c;
         }
         const int base = base_s;
-        if (live) live_idx[base + before + __popc(bal & ((1u << lane) - 1u))] = t;
+        const int live_before = base + before + __popc(bal & ((1u << lane) - 1u));
+        if (live) idx_live[live_before] = t;
+        else if (t < T) idx_dead[t - live_before] = t;
         __syncthreads();
         if (tid == 0) base_s = base + total;
     }
     __syncthreads();
-    if (tid == 0) *live_count = base_s;
+    if (tid == 0) { counts[0] = base_s; counts[1] = T - base_s; }
 }
 
-// compact row r <- token live_idx[r]: hidden row, lse, coefficient, target id.  Rows from the live
-// count up to the next multiple of 256 are zero-filled (the contractions read whole tiles).
+// out row r <- hidden row idx[r] for r < *count; rows up to the next multiple of 256 are zero-filled
+// (the contractions read whole tiles)
 __global__ void __launch_bounds__(128)
-gather_live_kernel(const __nv_bfloat16* __restrict__ hidden, int D, const float* __restrict__ lse,
-                   const float* __restrict__ coef, const int32_t* __restrict__ ids, const int32_t* __restrict__ live_idx,
-                   const int* __restrict__ live_count, __nv_bfloat16* __restrict__ hidden_c, float* __restrict__ lse_c,
-                   float* __restrict__ coef_c, int32_t* __restrict__ ids_c) {
-    const int n = *live_count;
+gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden, int D, const int32_t* __restrict__ idx,
+                   const int* __restrict__ count, __nv_bfloat16* __restrict__ out) {
+    const int n = *count;
     const int r = blockIdx.x;
     if (r >= ((n + 255) & ~255)) return;
-    uint4* dst = reinterpret_cast<uint4*>(hidden_c + (long long)r * D);
+    uint4* dst = reinterpret_cast<uint4*>(out + (long long)r * D);
     const int nv = D / 8;
     if (r < n) {
-        const int t = live_idx[r];
-        const uint4* src = reinterpret_cast<const uint4*>(hidden + (long long)t * D);
+        const uint4* src = reinterpret_cast<const uint4*>(hidden + (long long)idx[r] * D);
         for (int i = threadIdx.x; i < nv; i += blockDim.x) dst[i] = src[i];
-        if (threadIdx.x == 0) { lse_c[r] = lse[t]; coef_c[r] = coef[t]; ids_c[r] = ids[t]; }
     } else {
         for (int i = threadIdx.x; i < nv; i += blockDim.x) dst[i] = make_uint4(0u, 0u, 0u, 0u);
-        if (threadIdx.x == 0) { lse_c[r] = 0.0f; coef_c[r] = 0.0f; ids_c[r] = -1; }
+    }
+}
+
+// combine_kernel for a launch over gathered rows: row r of the launch (partials part[r][.]) is token
+// idx[off + r]; logp goes to the token's place, lse / coefficient / target id to the gathered place
+__global__ void __launch_bounds__(256)
+combine_rows_kernel(const float2* __restrict__ part, int nsplit, int rows_max, const int32_t* __restrict__ idx,
+                    const int* __restrict__ count, int off, const float* __restrict__ zy,
+                    const float4* __restrict__ rec, const long long* __restrict__ denom, float eps_clip, float beta,
+                    float* __restrict__ logp_out, float* __restrict__ lse_g, float* __restrict__ coef_g,
+                    int32_t* __restrict__ y_g, int32_t* __restrict__ dev_status) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    const int n = max(0, min(*count - off, rows_max));
+    if (r >= n) return;
+    const int t = idx[off + r];
+    float M = -INFINITY;
+    for (int j = 0; j < nsplit; ++j) M = fmaxf(M, part[(long long)r * nsplit + j].x);
+    float S = 0.0f;
+    for (int j = 0; j < nsplit; ++j) {
+        const float2 ms = part[(long long)r * nsplit + j];
+        if (ms.x != -INFINITY) S += ms.y * expf(ms.x - M);
+    }
+    const float lse = M + logf(S);
+    const float logp = (zy[t] - M) - logf(S);
+    const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) && (fabsf(logp) < INFINITY);
+    const float4 rc = rec[t];
+    const bool live = (__float_as_int(rc.w) < 0) && finite;
+    float coef = 0.0f;
+    if (live) {
+        const long long N = *denom;
+        const float inv_n = 1.0f / (float)(N > 1 ? N : 1);
+        const float A = rc.z;
+        const float rho = expf(logp - rc.x);
+        const bool clipped = ((A > 0.0f) && (rho > 1.0f + eps_clip)) || ((A < 0.0f) && (rho < 1.0f - eps_clip));
+        const float dpg = clipped ? 0.0f : -A * rho;
+        coef = -inv_n * fmaf(beta, -expm1f(rc.y - logp), dpg);
+    }
+    logp_out[t] = finite ? logp : __int_as_float(0x7fc00000);
+    if (lse_g) {
+        lse_g[off + r] = finite ? lse : 0.0f;
+        coef_g[off + r] = coef;
+        y_g[off + r] = __float_as_int(rc.w) & 0x7fffffff;
+    }
+    if (!finite && dev_status) atomicOr(dev_status, RLF_DEV_NONFINITE);
+}
+
+// in place over one chunk of stored exponentials e = exp(z - tile max): dZ = coef (e exp(tile max - lse)
+// - [v == y]) as bf16; the target column takes the fp32 target logit.  Rows from the live extent up
+// to the next multiple of 256 become zeros.  One CTA per row.
+__global__ void __launch_bounds__(256)
+dz_from_e_kernel(__nv_bfloat16* __restrict__ ebuf, int V, int n_tiles, const float* __restrict__ tmax, int rows_max,
+                 const int* __restrict__ count, int off, const float* __restrict__ lse_g,
+                 const float* __restrict__ coef_g, const int32_t* __restrict__ y_g, const int32_t* __restrict__ idx,
+                 const float* __restrict__ zy) {
+    const int n = max(0, min(*count - off, rows_max));
+    const int r = blockIdx.x;
+    if (r >= ((n + 255) & ~255)) return;
+    uint4* row = reinterpret_cast<uint4*>(ebuf + (long long)r * V);
+    const int nv = V / 8;
+    const float coef = r < n ? coef_g[off + r] : 0.0f;
+    if (coef == 0.0f) {
+        for (int i = threadIdx.x; i < nv; i += 256) row[i] = make_uint4(0u, 0u, 0u, 0u);
+        return;
+    }
+    const float lse = lse_g[off + r];
+    const float c2 = lg2_approx(fabsf(coef)) - lse * kLog2e;
+    const float* tm = tmax + (long long)r * n_tiles;
+    for (int i = threadIdx.x; i < nv; i += 256) {
+        // signed scale of this vector's tile (BN = 256 columns = 32 vectors)
+        const float f = copysignf(ex2_approx(fmaf(tm[i >> 5], kLog2e, c2)), coef);
+        const uint4 z = row[i];
+        const uint32_t w[4] = {z.x, z.y, z.z, z.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[k])
+                : "f"(__uint_as_float(w[k] & 0xffff0000u) * f), "f"(__uint_as_float(w[k] << 16) * f));
+        row[i] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int y = y_g[off + r];
+        if (y >= 0 && y < V) {
+            const float py = ex2_approx((zy[idx[off + r]] - lse) * kLog2e);
+            ebuf[(long long)r * V + y] = __float2bfloat16_rn(fmaf(coef, py, -coef));
+        }
     }
 }
 
@@ -695,7 +786,7 @@ static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, co
             opted[dev] = true;
         }
     }
-    const bool sweep = p.mode == kLse || p.mode == kDz;
+    const bool sweep = p.mode == kLse;
     const int m_units = PAIR ? (p.m_tiles + 1) / 2 : p.m_tiles;
     const int units = sweep ? m_units * p.nsplit : m_units * p.n_tiles;
     if (units <= 0) return RLF_OK;
@@ -750,7 +841,7 @@ static int pick_split(int m_units, int n_tiles, int workers) {
 }
 
 struct LmWs {
-    size_t n_count, partial, rec, zy, lse, coef, part, live_idx, lse_c, coef_c, ids_c, hidden_c, dz, total;
+    size_t n_count, partial, rec, zy, lse, coef, part, idx_live, idx_dead, lse_g, coef_g, y_g, hidden_g, tmax, dz, total;
 };
 static size_t up1k(size_t x) { return (x + 1023) & ~(size_t)1023; }
 static LmWs lm_workspace(int64_t T, int32_t V, int32_t D) {
@@ -758,20 +849,22 @@ static LmWs lm_workspace(int64_t T, int32_t V, int32_t D) {
     size_t o = 0;
     const size_t Tn = (size_t)(T > 0 ? T : 0);
     const size_t Tp = (Tn + 255) & ~(size_t)255;     // compact arrays are padded to whole tile pairs
-    w.n_count = o; o += 1024;                        // [0] mask count, [64] live-row count
+    w.n_count = o; o += 1024;                        // [0] mask count, [64] live / other row counts
     w.partial = o; o += up1k(token_loss_partial_bytes());
     w.rec = o;     o += up1k(16 * Tn);
     w.zy = o;      o += up1k(4 * Tn);
     w.lse = o;     o += up1k(4 * Tn);
     w.coef = o;    o += up1k(4 * Tn);
     w.part = o;    o += up1k(8 * Tn * kMaxSplit);
-    w.live_idx = o; o += up1k(4 * Tp);
-    w.lse_c = o;   o += up1k(4 * Tp);
-    w.coef_c = o;  o += up1k(4 * Tp);
-    w.ids_c = o;   o += up1k(4 * Tp);
-    w.hidden_c = o; o += up1k(Tp * (size_t)(D > 0 ? D : 0) * 2);
-    w.dz = o;
+    w.idx_live = o; o += up1k(4 * Tp);
+    w.idx_dead = o; o += up1k(4 * Tp);
+    w.lse_g = o;   o += up1k(4 * Tp);
+    w.coef_g = o;  o += up1k(4 * Tp);
+    w.y_g = o;     o += up1k(4 * Tp);
+    w.hidden_g = o; o += 2 * up1k(Tp * (size_t)(D > 0 ? D : 0) * 2);   // live rows, then the others
     const size_t chunk = Tp < (size_t)kChunkTokens ? Tp : (size_t)kChunkTokens;
+    w.tmax = o;    o += up1k(4 * chunk * (size_t)((V + BN - 1) / BN));
+    w.dz = o;
     o += up1k(chunk * (size_t)V * 2);
     w.total = o + 1024;
     return w;
@@ -837,70 +930,83 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
 
-    // forward sweep: running (max, sum exp) per token and vocabulary split
     const bool pair = g_pair.load() != 0;
     const uint32_t b_rows = pair ? BN / 2 : BN;       // rows of a K-major B tile that one CTA stages
-    CUtensorMap mapH, mapW;
-    if (!make_map(&mapH, H, (uint64_t)T, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
+    const int workers = pair ? sm_count_lm() / 2 : sm_count_lm();
+    CUtensorMap mapW;
     if (!make_map(&mapW, Wm, (uint64_t)V, (uint64_t)D, (uint64_t)D, BK, b_rows)) return RLF_ERR_CUDA;
     GemmParams g = {};
     g.mode = kLse;
-    g.M = (int)T;
     g.N = V;
-    g.m_tiles = (int)((T + BM - 1) / BM);
     g.n_tiles = (V + BN - 1) / BN;
     g.k_slabs = D / BK;
-    const int workers = pair ? sm_count_lm() / 2 : sm_count_lm();
-    g.nsplit = pick_split(pair ? (g.m_tiles + 1) / 2 : g.m_tiles, g.n_tiles, workers);
-    g.n_tiles_per_split = (g.n_tiles + g.nsplit - 1) / g.nsplit;
     g.part = part;
     g.dev_status = dev_status;
-    st = launch_gemm(mapH, mapW, g, pair, s);
-    if (st != RLF_OK) return st;
-    combine_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(part, g.nsplit, zy, rec, T, dn, eps_clip, beta_kl, logp_out,
-                                                                lse, coef, dev_status);
-    count_launch();
-    if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
-    st = launch_token_loss(logp_out, rec, T, eps_clip, beta_kl, partial, dn, loss_out, s);
-    if (st != RLF_OK) return st;
-    if (!grad_hidden && !grad_W) return RLF_OK;
+    auto set_rows = [&](GemmParams& q, int64_t rows) {
+        q.M = (int)rows;
+        q.m_tiles = (int)((rows + BM - 1) / BM);
+        q.nsplit = pick_split(pair ? (q.m_tiles + 1) / 2 : q.m_tiles, q.n_tiles, workers);
+        q.n_tiles_per_split = (q.n_tiles + q.nsplit - 1) / q.nsplit;
+    };
 
-    // backward over the rows with a non-zero coefficient only, compacted in token order; their number
-    // stays on the device (no host sync), so every chunk is launched and the kernels size themselves
-    int* live_count = reinterpret_cast<int*>(ws + w.n_count + 64);
-    int32_t* live_idx = reinterpret_cast<int32_t*>(ws + w.live_idx);
-    float* lse_c = reinterpret_cast<float*>(ws + w.lse_c);
-    float* coef_c = reinterpret_cast<float*>(ws + w.coef_c);
-    int32_t* ids_c = reinterpret_cast<int32_t*>(ws + w.ids_c);
-    __nv_bfloat16* Hc = reinterpret_cast<__nv_bfloat16*>(ws + w.hidden_c);
+    if (!grad_hidden && !grad_W) {
+        // forward only: one sweep over all rows, running (max, sum exp) per token and vocabulary split
+        CUtensorMap mapH;
+        if (!make_map(&mapH, H, (uint64_t)T, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
+        set_rows(g, T);
+        st = launch_gemm(mapH, mapW, g, pair, s);
+        if (st != RLF_OK) return st;
+        combine_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(part, g.nsplit, zy, rec, T, dn, eps_clip, beta_kl,
+                                                                    logp_out, lse, coef, dev_status);
+        count_launch();
+        if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+        return launch_token_loss(logp_out, rec, T, eps_clip, beta_kl, partial, dn, loss_out, s);
+    }
+
+    // forward + backward.  The tokens are partitioned (stably) into unmasked rows and the others;
+    // their numbers stay on the device (no host sync), so every chunk is launched and the kernels
+    // size themselves.  Unmasked rows, by chunks: forward sweep that also keeps the chunk's
+    // exponentials (relative to tile maxima) as bf16 -> lse, logp, coefficient -> dZ in place -> grad_hidden rows, grad_W += chunk's part.
+    // The other rows only need their log-prob: one forward sweep.
+    int* counts = reinterpret_cast<int*>(ws + w.n_count + 64);
+    int32_t* idx_live = reinterpret_cast<int32_t*>(ws + w.idx_live);
+    int32_t* idx_dead = reinterpret_cast<int32_t*>(ws + w.idx_dead);
+    float* lse_g = reinterpret_cast<float*>(ws + w.lse_g);
+    float* coef_g = reinterpret_cast<float*>(ws + w.coef_g);
+    int32_t* y_g = reinterpret_cast<int32_t*>(ws + w.y_g);
     const int64_t Tp = (T + 255) & ~(int64_t)255;
-    compact_live_kernel<<<1, 1024, 0, s>>>(coef, (int)T, live_idx, live_count);
-    gather_live_kernel<<<(unsigned)Tp, 128, 0, s>>>(H, D, lse, coef, ids, live_idx, live_count, Hc, lse_c, coef_c, ids_c);
-    count_launch(2);
+    __nv_bfloat16* Hl = reinterpret_cast<__nv_bfloat16*>(ws + w.hidden_g);
+    __nv_bfloat16* Hd = reinterpret_cast<__nv_bfloat16*>(ws + w.hidden_g + up1k((size_t)Tp * D * 2));
+    partition_rows_kernel<<<1, 1024, 0, s>>>(rec, (int)T, idx_live, idx_dead, counts);
+    gather_rows_kernel<<<(unsigned)Tp, 128, 0, s>>>(H, D, idx_live, counts, Hl);
+    gather_rows_kernel<<<(unsigned)Tp, 128, 0, s>>>(H, D, idx_dead, counts + 1, Hd);
+    count_launch(3);
     if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
     if (grad_hidden && cudaMemsetAsync(grad_hidden, 0, (size_t)T * D * 2, s) != cudaSuccess) return RLF_ERR_CUDA;
 
     for (int64_t t0 = 0; t0 < T; t0 += kChunkTokens) {
         const int64_t tc = (T - t0) < kChunkTokens ? (T - t0) : kChunkTokens;
         CUtensorMap mapHc;
-        if (!make_map(&mapHc, Hc + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
+        if (!make_map(&mapHc, Hl + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
         GemmParams z = g;
-        z.mode = kDz;
-        z.M = (int)tc;
-        z.m_tiles = (int)((tc + BM - 1) / BM);
-        z.nsplit = pick_split(pair ? (z.m_tiles + 1) / 2 : z.m_tiles, z.n_tiles, workers);
-        z.n_tiles_per_split = (z.n_tiles + z.nsplit - 1) / z.nsplit;
-        z.lse = lse_c + t0;
-        z.coef = coef_c + t0;
-        z.ids = ids_c + t0;
+        set_rows(z, tc);
         z.dz = dz;
         z.dz_stride = V;
-        z.live_count = live_count;
+        z.tmax = reinterpret_cast<float*>(ws + w.tmax);
+        z.live_count = counts;
         z.live_off = (int)t0;
         st = launch_gemm(mapHc, mapW, z, pair, s);
         if (st != RLF_OK) return st;
+        combine_rows_kernel<<<(unsigned)((tc + 255) / 256), 256, 0, s>>>(part, z.nsplit, (int)tc, idx_live, counts, (int)t0,
+                                                                          zy, rec, dn, eps_clip, beta_kl, logp_out, lse_g,
+                                                                          coef_g, y_g, dev_status);
+        const int64_t tcp = (tc + 255) & ~(int64_t)255;
+        dz_from_e_kernel<<<(unsigned)tcp, 256, 0, s>>>(dz, V, z.n_tiles, z.tmax, (int)tc, counts, (int)t0, lse_g, coef_g, y_g,
+                                                        idx_live, zy);
+        count_launch(2);
+        if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
         if (grad_hidden) {
-            // grad_hidden[token of compact row] = dZ[chunk, V] W[V, D]
+            // grad_hidden[token of gathered row] = dZ[chunk, V] W[V, D]
             CUtensorMap mapDzK, mapWn;
             if (!make_map(&mapDzK, dz, (uint64_t)tc, (uint64_t)V, (uint64_t)V, BK, BM)) return RLF_ERR_CUDA;
             if (!make_map(&mapWn, Wm, (uint64_t)V, (uint64_t)D, (uint64_t)D, 64, BK)) return RLF_ERR_CUDA;
@@ -914,9 +1020,9 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
             h.out_bf16 = static_cast<__nv_bfloat16*>(grad_hidden);
             h.out_stride = D;
             h.dev_status = dev_status;
-            h.live_count = live_count;
+            h.live_count = counts;
             h.live_off = (int)t0;
-            h.row_index = live_idx;
+            h.row_index = idx_live;
             st = launch_gemm(mapDzK, mapWn, h, pair, s);
             if (st != RLF_OK) return st;
         }
@@ -924,7 +1030,7 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
             // grad_W[V, D] (+)= dZ[chunk, V]^T hidden[chunk, D]
             CUtensorMap mapDzM, mapHn;
             if (!make_map(&mapDzM, dz, (uint64_t)tc, (uint64_t)V, (uint64_t)V, 64, BK)) return RLF_ERR_CUDA;
-            if (!make_map(&mapHn, Hc + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, 64, BK)) return RLF_ERR_CUDA;
+            if (!make_map(&mapHn, Hl + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, 64, BK)) return RLF_ERR_CUDA;
             GemmParams q = {};
             q.mode = kGradW;
             q.M = V;
@@ -936,13 +1042,30 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
             q.out_stride = D;
             q.accumulate = (accumulate_grad_W || t0 > 0) ? 1 : 0;
             q.dev_status = dev_status;
-            q.live_count = live_count;
+            q.live_count = counts;
             q.live_off = (int)t0;
             st = launch_gemm(mapDzM, mapHn, q, pair, s);
             if (st != RLF_OK) return st;
         }
     }
-    return RLF_OK;
+
+    // the masked rows: log-prob only
+    {
+        CUtensorMap mapHd;
+        if (!make_map(&mapHd, Hd, (uint64_t)T, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
+        GemmParams d = g;
+        set_rows(d, T);
+        d.live_count = counts + 1;
+        d.live_off = 0;
+        st = launch_gemm(mapHd, mapW, d, pair, s);
+        if (st != RLF_OK) return st;
+        combine_rows_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(part, d.nsplit, (int)T, idx_dead, counts + 1, 0, zy,
+                                                                         rec, dn, eps_clip, beta_kl, logp_out, nullptr,
+                                                                         nullptr, nullptr, dev_status);
+        count_launch();
+        if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+    }
+    return launch_token_loss(logp_out, rec, T, eps_clip, beta_kl, partial, dn, loss_out, s);
 }
 
 extern "C" rlf_status rlf_tune_lmhead(int pair_ctas) {
