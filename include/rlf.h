@@ -115,6 +115,30 @@ rlf_status rlf_rule_reward(const float *scores, const float *weights, int32_t B,
                            float *reward_out, rlf_stream_t stream);
 
 /*
+ * KL penalty folded into the outcome reward instead of the loss (an objective variant of the GRPO /
+ * PPO-style update that the paper names in Sec. 2.3.1 and Sec. 2.3.2; the paper prints no formula,
+ * this is the usual form).  Call it between the reward and rlf_group_advantage, and run the loss with
+ * beta_kl = 0:
+ *     R'_b = R_b - beta * sum_{t in response b} mask[t] k(d_t),   d_t = old_logp[t] - ref_logp[t]
+ *     kl_kind RLF_KL_K1: k = d;   RLF_KL_K2: k = d^2 / 2;   RLF_KL_K3: k = exp(-d) + d - 1
+ * Sums are taken in fp64 in a fixed order (results are run-to-run identical).
+ *
+ *   rewards     [B] fp32;  old_logp, ref_logp [T] fp32;  mask [T] uint8
+ *   cu_seqlens  [B+1] int32: response b owns tokens cu_seqlens[b] .. cu_seqlens[b+1]-1
+ *   reward_out  [B] fp32 (may be the same buffer as rewards)
+ *   kl_seq_out  [B] fp32 or NULL: the summed estimate of each response
+ * A malformed cu_seqlens sets RLF_DEV_BAD_SEQ and the response is clipped to [0, T).  An unknown
+ * kl_kind returns RLF_ERR_UNSUPPORTED.  B = 0 and T = 0 are valid.
+ */
+#define RLF_KL_K1 0
+#define RLF_KL_K2 1
+#define RLF_KL_K3 2
+rlf_status rlf_kl_in_reward(const float *rewards, const float *old_logp, const float *ref_logp,
+                            const uint8_t *mask, const int32_t *cu_seqlens, int32_t B, int64_t T,
+                            float beta, int kl_kind, float *reward_out, float *kl_seq_out,
+                            int32_t *dev_status, rlf_stream_t stream);
+
+/*
  * Fused log-prob + clipped-ratio + k3-KL loss, forward and backward, over
  * materialised logits.  (Paper Sec. 2.2: the policy pi_theta(a | s_t); Sec.
  * 2.3.1: PPO-style update of the RL trainer; Sec. 2.3.2: GRPO with the loss

@@ -459,6 +459,48 @@ int orc_rule_reward(const float *scores, const float *weights, int32_t B, int32_
     return 0;
 }
 
+/*
+ * KL penalty folded into the reward instead of the loss (an objective variant; the paper names
+ * GRPO / a PPO-style update in Sec. 2.3 and prints no formula, so this is the common form of the
+ * RL trainers it builds on): the outcome reward of response b is reduced by beta times the summed
+ * per-token divergence estimate between the behaviour policy and the reference policy over the
+ * response's loss-carrying tokens,
+ *     R'_b = R_b - beta * sum_{t in b} mask_t k(old_logp_t, ref_logp_t),   d = old_logp_t - ref_logp_t
+ *     kind 0 (k1): k = d        kind 1 (k2): k = d^2 / 2        kind 2 (k3): k = exp(-d) + d - 1
+ * kl_seq[b] (optional) receives the summed estimate itself.  Tokens outside every response count
+ * for nothing.  Returns -3 for an unknown kind, -2 for a malformed cu_seqlens.
+ */
+int orc_kl_in_reward(const float *rewards, const float *old_logp, const float *ref_logp, const uint8_t *mask,
+                     const int32_t *cu_seqlens, int32_t B, int64_t T, double beta, int kind,
+                     double *reward_out, double *kl_seq)
+{
+    if (kind < 0 || kind > 2)
+        return -3;
+    for (int32_t b = 0; b < B; ++b) {
+        int64_t lo = cu_seqlens[b], hi = cu_seqlens[b + 1];
+        if (lo < 0 || hi < lo || hi > T)
+            return -2;
+        double acc = 0.0;
+        for (int64_t t = lo; t < hi; ++t) {
+            if (!mask[t])
+                continue;
+            double d = (double)old_logp[t] - (double)ref_logp[t];
+            double k;
+            if (kind == 0)
+                k = d;
+            else if (kind == 1)
+                k = 0.5 * d * d;
+            else
+                k = exp(-d) + d - 1.0;
+            acc += k;
+        }
+        if (kl_seq)
+            kl_seq[b] = acc;
+        reward_out[b] = (double)rewards[b] - beta * acc;
+    }
+    return 0;
+}
+
 int orc_num_threads(void)
 {
     int n = 1;

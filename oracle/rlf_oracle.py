@@ -207,3 +207,20 @@ def rule_reward(scores, weights):
     rc = lib().orc_rule_reward(_p(s), _p(w), ctypes.c_int32(B), ctypes.c_int32(n), _p(R))
     _check(rc, "rule_reward")
     return R
+
+
+def kl_in_reward(rewards, old_logp, ref_logp, mask, cu_seqlens, beta, kind=0):
+    """KL penalty folded into the outcome reward.  -> (R' f64[B], kl_seq f64[B])."""
+    r = _c(rewards, np.float32)
+    old_logp = _c(old_logp, np.float32)
+    ref_logp = _c(ref_logp, np.float32)
+    mask = _c(mask, np.uint8)
+    cu = _c(cu_seqlens, np.int32)
+    B = len(cu) - 1
+    T = len(mask)
+    out = np.zeros(B, np.float64)
+    kl = np.zeros(B, np.float64)
+    rc = lib().orc_kl_in_reward(_p(r), _p(old_logp), _p(ref_logp), _p(mask), _p(cu), ctypes.c_int32(B),
+                                ctypes.c_int64(T), ctypes.c_double(beta), ctypes.c_int(kind), _p(out), _p(kl))
+    _check(rc, "kl_in_reward")
+    return out, kl

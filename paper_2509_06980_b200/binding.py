@@ -18,7 +18,7 @@ FN_LOGP_LOSS, FN_FUSED_LMHEAD, FN_LOGP_ENTROPY = 3, 4, 5
 DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
 
 EXPORTS = [
-    "rlf_build_loss_mask", "rlf_group_advantage", "rlf_rule_reward", "rlf_grpo_logp_loss_fwd_bwd",
+    "rlf_build_loss_mask", "rlf_group_advantage", "rlf_rule_reward", "rlf_kl_in_reward", "rlf_grpo_logp_loss_fwd_bwd",
     "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_grpo_logp_loss_fwd_bwd_skip_masked", "rlf_grpo_logp_loss_fwd_bwd_obj", "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
     "rlf_tune_logits_kernel", "rlf_tune_lmhead", "rlf_launch_count", "rlf_status_string", "rlf_version",
 ]
@@ -167,6 +167,30 @@ def rlf_rule_reward(scores, weights, reward_out=None):
     _check(_lib.rlf_rule_reward(_ptr(scores, torch.float32), _ptr(weights, torch.float32), B, n,
                                 _ptr(reward_out, torch.float32), _stream()), "rlf_rule_reward")
     return reward_out
+
+
+KL_K1, KL_K2, KL_K3 = 0, 1, 2
+
+
+def rlf_kl_in_reward(rewards, old_logp, ref_logp, mask, cu_seqlens, beta, kl_kind=KL_K1, reward_out=None,
+                     kl_seq_out=None, dev_status=None):
+    """KL penalty folded into the outcome reward: R'_b = R_b - beta * sum_t mask_t k(old_t - ref_t).
+    -> (rewards fp32[B], summed estimate per response fp32[B])."""
+    B = cu_seqlens.shape[0] - 1
+    T = mask.shape[0]
+    dev = rewards.device
+    if reward_out is None:
+        reward_out = torch.empty(B, dtype=torch.float32, device=dev)
+    if kl_seq_out is None:
+        kl_seq_out = torch.empty(B, dtype=torch.float32, device=dev)
+    _lib.rlf_kl_in_reward.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _int, _vp, _vp, _vp, _vp]
+    _lib.rlf_kl_in_reward.restype = _int
+    _check(_lib.rlf_kl_in_reward(_ptr(rewards, torch.float32), _ptr(old_logp, torch.float32),
+                                 _ptr(ref_logp, torch.float32), _ptr(mask, torch.uint8),
+                                 _ptr(cu_seqlens, torch.int32), B, T, float(beta), int(kl_kind),
+                                 _ptr(reward_out, torch.float32), _ptr(kl_seq_out, torch.float32),
+                                 _ptr(dev_status, torch.int32), _stream()), "rlf_kl_in_reward")
+    return reward_out, kl_seq_out
 
 
 def rlf_grpo_logp_loss_fwd_bwd(logits, ids, seq_id, adv, old_logp, ref_logp, mask, eps_clip, beta_kl,

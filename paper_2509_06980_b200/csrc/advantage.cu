@@ -105,3 +105,59 @@ extern "C" rlf_status rlf_rule_reward(const float* scores, const float* weights,
     count_launch();
     return cuda_ok(cudaGetLastError());
 }
+
+// ---------------------------------------------------------------------------------------------
+// KL penalty folded into the outcome reward: R'_b = R_b - beta * sum_{t in b} mask_t k(old_t, ref_t),
+// d = old_logp - ref_logp; kind 0: k = d, kind 1: k = d^2 / 2, kind 2: k = exp(-d) + d - 1.
+// One CTA per response; every thread sums its tokens (stride 256, index order) in fp64 and the
+// partial sums are combined by a fixed shuffle tree and a fixed loop over warps, so results are
+// run-to-run identical.  10 bytes per token: launch latency is what this costs.
+namespace rlf {
+__global__ void __launch_bounds__(256)
+kl_in_reward_kernel(const float* __restrict__ rewards, const float* __restrict__ old_logp,
+                    const float* __restrict__ ref_logp, const uint8_t* __restrict__ mask,
+                    const int32_t* __restrict__ cu_seqlens, int64_t T, float beta, int kind,
+                    float* __restrict__ reward_out, float* __restrict__ kl_seq_out, int32_t* __restrict__ dev_status) {
+    __shared__ double warp_part[8];
+    const int b = blockIdx.x;
+    long long lo = cu_seqlens[b], hi = cu_seqlens[b + 1];
+    if (lo < 0 || hi < lo || hi > T) {
+        if (threadIdx.x == 0 && dev_status) atomicOr(dev_status, RLF_DEV_BAD_SEQ);
+        lo = lo < 0 ? 0 : (lo > T ? T : lo);
+        hi = hi < lo ? lo : (hi > T ? T : hi);
+    }
+    double acc = 0.0;
+    for (long long t = lo + threadIdx.x; t < hi; t += 256) {
+        if (!mask[t]) continue;
+        const double d = (double)old_logp[t] - (double)ref_logp[t];
+        acc += kind == 0 ? d : kind == 1 ? 0.5 * d * d : exp(-d) + d - 1.0;
+    }
+    acc = warp_sum_f64(acc);
+    if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double s = 0.0;
+        for (int w = 0; w < 8; ++w) s += warp_part[w];
+        if (kl_seq_out) kl_seq_out[b] = (float)s;
+        reward_out[b] = (float)((double)rewards[b] - (double)beta * s);
+    }
+}
+}  // namespace rlf
+
+extern "C" rlf_status rlf_kl_in_reward(const float* rewards, const float* old_logp, const float* ref_logp,
+                                       const uint8_t* mask, const int32_t* cu_seqlens, int32_t B, int64_t T,
+                                       float beta, int kl_kind, float* reward_out, float* kl_seq_out,
+                                       int32_t* dev_status, rlf_stream_t stream) {
+    using namespace rlf;
+    if (B < 0 || T < 0) return RLF_ERR_SHAPE;
+    if (kl_kind < 0 || kl_kind > 2) return RLF_ERR_UNSUPPORTED;
+    if (B == 0) return RLF_OK;
+    if (!rewards || !reward_out || !cu_seqlens) return RLF_ERR_NULL;
+    if (T > 0 && (!old_logp || !ref_logp || !mask)) return RLF_ERR_NULL;
+    rlf_status st = check_arch();
+    if (st != RLF_OK) return st;
+    kl_in_reward_kernel<<<B, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+        rewards, old_logp, ref_logp, mask, cu_seqlens, T, beta, kl_kind, reward_out, kl_seq_out, dev_status);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}

@@ -90,6 +90,13 @@ def test_host_validation_rejects_bad_arguments_before_touching_a_device(lib):
     assert h(fake, None, 4, 0, 1e-6, 1, fake, None, None) == -2
     assert h(None, None, 4, 2, 1e-6, 1, fake, None, None) == -1
     assert h(fake, None, 0, 2, 1e-6, 1, fake, None, None) == 0
+    k = lib.rlf_kl_in_reward
+    k.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_int, vp, vp, vp, vp]
+    assert k(fake, fake, fake, fake, fake, 2, 8, 0.1, 5, fake, None, None, None) == -8
+    assert k(fake, fake, fake, fake, fake, -1, 8, 0.1, 0, fake, None, None, None) == -2
+    assert k(fake, fake, fake, fake, None, 2, 8, 0.1, 0, fake, None, None, None) == -1
+    assert k(fake, None, fake, fake, fake, 2, 8, 0.1, 0, fake, None, None, None) == -1
+    assert k(fake, fake, fake, fake, fake, 0, 8, 0.1, 0, fake, None, None, None) == 0
     t = lib.rlf_tune_logits_kernel
     t.argtypes = [ctypes.c_int] * 3
     assert t(3, 512, 0) == -2 and t(4, 500, 0) == -2 and t(0, 0, -1) == 0
