@@ -313,6 +313,29 @@ rlf_status rlf_fused_lmhead_grpo(const void *hidden, const void *W, int64_t T, i
                                  void *workspace, size_t workspace_bytes, int32_t *dev_status,
                                  rlf_stream_t stream);
 
+/*
+ * rlf_fused_lmhead_grpo under the objective variants of rlf_grpo_logp_loss_fwd_bwd_obj (same
+ * formulas; the paper names GRPO / a PPO-style update in Sec. 2.3 and prints no objective):
+ *   eps_clip_low, eps_clip_high   clip range (1 - eps_clip_low, 1 + eps_clip_high)
+ *   aggregation   0: masked token mean (denom, if given, counts tokens);
+ *                 1: mean over responses of each response's masked token mean (denom, if given,
+ *                    counts responses); needs B <= T + 1
+ *   skip_masked   1: rows with mask 0 are not multiplied at all, not even for their log-prob, which
+ *                 reads NaN (with 46 % of the tokens inside tool observations, as in the Qwen3-4B
+ *                 recipe, that is 46 % of the forward contraction); loss and gradients are unchanged.
+ *                 0: every row's log-prob is produced.
+ * Everything else (layouts, workspace, errors) as for rlf_fused_lmhead_grpo.
+ */
+rlf_status rlf_fused_lmhead_grpo_obj(const void *hidden, const void *W, int64_t T, int32_t D, int32_t V,
+                                     const int32_t *ids, const int32_t *seq_id, const float *adv,
+                                     int32_t B, const float *old_logp, const float *ref_logp,
+                                     const uint8_t *mask, float eps_clip_low, float eps_clip_high,
+                                     float beta_kl, int aggregation, int skip_masked,
+                                     const int64_t *denom, float *logp_out, double *loss_out,
+                                     void *grad_hidden, float *grad_W, int accumulate_grad_W,
+                                     void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                     rlf_stream_t stream);
+
 /* Bytes of workspace the given entry point needs for these sizes (0 for unknown selectors). */
 size_t rlf_workspace_bytes(int which_fn, int64_t T, int32_t V, int32_t D, rlf_dtype dt);
 

@@ -360,6 +360,46 @@ int orc_grpo_loss_obj(const void *logits, int dtype, int64_t T, int32_t V, int64
  * Materialises z and grad_z as [T,V] fp64: for small T only.
  * grad_hidden / grad_W may be NULL (skipped).  z_out (nullable) gets z.
  */
+/* z[t,v] = sum_k H[t,k] W[v,k], every product and sum in fp64 */
+static void head_logits(const uint16_t *hidden, const uint16_t *W, int64_t T, int32_t D, int32_t V, double *z)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t t = 0; t < T; ++t)
+        for (int32_t v = 0; v < V; ++v) {
+            double acc = 0.0;
+            for (int32_t k = 0; k < D; ++k)
+                acc += widen(hidden, ORC_BF16, t * (int64_t)D + k) *
+                       widen(W, ORC_BF16, v * (int64_t)D + k);
+            z[t * (int64_t)V + v] = acc;
+        }
+}
+
+/* chain rule through the contraction, given grad_z = gz */
+static void head_backward(const uint16_t *hidden, const uint16_t *W, int64_t T, int32_t D, int32_t V,
+                          const double *gz, double *grad_hidden, double *grad_W)
+{
+    if (grad_hidden) {
+#pragma omp parallel for schedule(dynamic, 1)
+        for (int64_t t = 0; t < T; ++t)
+            for (int32_t k = 0; k < D; ++k) {
+                double acc = 0.0;
+                for (int32_t v = 0; v < V; ++v)
+                    acc += gz[t * (int64_t)V + v] * widen(W, ORC_BF16, v * (int64_t)D + k);
+                grad_hidden[t * (int64_t)D + k] = acc;
+            }
+    }
+    if (grad_W) {
+#pragma omp parallel for schedule(dynamic, 16)
+        for (int32_t v = 0; v < V; ++v)
+            for (int32_t k = 0; k < D; ++k) {
+                double acc = 0.0;
+                for (int64_t t = 0; t < T; ++t)
+                    acc += gz[t * (int64_t)V + v] * widen(hidden, ORC_BF16, t * (int64_t)D + k);
+                grad_W[v * (int64_t)D + k] = acc;
+            }
+    }
+}
+
 int orc_fused_lmhead_grpo(const uint16_t *hidden, const uint16_t *W, int64_t T, int32_t D,
                           int32_t V, const int32_t *ids, const int32_t *seq_id,
                           const float *adv, const float *old_logp, const float *ref_logp,
@@ -373,39 +413,40 @@ int orc_fused_lmhead_grpo(const uint16_t *hidden, const uint16_t *W, int64_t T, 
     double *gz = need_g ? (double *)malloc(sizeof(double) * tv) : NULL;
     if (!z || (need_g && !gz)) return -7;
 
-#pragma omp parallel for schedule(dynamic, 1)
-    for (int64_t t = 0; t < T; ++t)
-        for (int32_t v = 0; v < V; ++v) {
-            double acc = 0.0;
-            for (int32_t k = 0; k < D; ++k)
-                acc += widen(hidden, ORC_BF16, t * (int64_t)D + k) *
-                       widen(W, ORC_BF16, v * (int64_t)D + k);
-            z[t * (int64_t)V + v] = acc;
-        }
-
+    head_logits(hidden, W, T, D, V, z);
     int rc = orc_grpo_loss(z, ORC_F64, T, V, V, ids, seq_id, adv, old_logp, ref_logp, mask,
                            eps_clip, beta_kl, denom, logp_out, loss_out, gz, NULL);
-    if (rc == 0 && grad_hidden) {
-#pragma omp parallel for schedule(dynamic, 1)
-        for (int64_t t = 0; t < T; ++t)
-            for (int32_t k = 0; k < D; ++k) {
-                double acc = 0.0;
-                for (int32_t v = 0; v < V; ++v)
-                    acc += gz[t * (int64_t)V + v] * widen(W, ORC_BF16, v * (int64_t)D + k);
-                grad_hidden[t * (int64_t)D + k] = acc;
-            }
-    }
-    if (rc == 0 && grad_W) {
-#pragma omp parallel for schedule(dynamic, 16)
-        for (int32_t v = 0; v < V; ++v)
-            for (int32_t k = 0; k < D; ++k) {
-                double acc = 0.0;
-                for (int64_t t = 0; t < T; ++t)
-                    acc += gz[t * (int64_t)V + v] * widen(hidden, ORC_BF16, t * (int64_t)D + k);
-                grad_W[v * (int64_t)D + k] = acc;
-            }
-    }
+    if (rc == 0)
+        head_backward(hidden, W, T, D, V, gz, grad_hidden, grad_W);
     if (!z_out) free(z);
+    free(gz);
+    return rc;
+}
+
+/*
+ * The fused LM-head variant under the objective variants: the same fp64 logits, then exactly
+ * orc_grpo_loss_obj on them (asymmetric clip range, token-mean or sequence-mean aggregation), then
+ * the same chain rule through the contraction.
+ */
+int orc_fused_lmhead_grpo_obj(const uint16_t *hidden, const uint16_t *W, int64_t T, int32_t D,
+                              int32_t V, const int32_t *ids, const int32_t *seq_id,
+                              const float *adv, int32_t num_seqs, const float *old_logp,
+                              const float *ref_logp, const uint8_t *mask, double eps_low,
+                              double eps_high, double beta_kl, int aggregation, int64_t denom,
+                              double *logp_out, double *loss_out, double *grad_hidden, double *grad_W)
+{
+    size_t tv = (size_t)(T > 0 ? T : 1) * (size_t)V;
+    double *z = (double *)malloc(sizeof(double) * tv);
+    int need_g = grad_hidden || grad_W;
+    double *gz = need_g ? (double *)malloc(sizeof(double) * tv) : NULL;
+    if (!z || (need_g && !gz)) return -7;
+
+    head_logits(hidden, W, T, D, V, z);
+    int rc = orc_grpo_loss_obj(z, ORC_F64, T, V, V, ids, seq_id, adv, num_seqs, old_logp, ref_logp, mask,
+                               eps_low, eps_high, beta_kl, aggregation, denom, logp_out, loss_out, gz, NULL);
+    if (rc == 0)
+        head_backward(hidden, W, T, D, V, gz, grad_hidden, grad_W);
+    free(z);
     free(gz);
     return rc;
 }

@@ -224,3 +224,32 @@ def kl_in_reward(rewards, old_logp, ref_logp, mask, cu_seqlens, beta, kind=0):
                                 ctypes.c_int64(T), ctypes.c_double(beta), ctypes.c_int(kind), _p(out), _p(kl))
     _check(rc, "kl_in_reward")
     return out, kl
+
+
+def fused_lmhead_grpo_obj(hidden, W, ids, seq_id, adv, old_logp, ref_logp, mask, eps_low, eps_high, beta_kl,
+                          aggregation=0, denom=None, want_grad_hidden=True, want_grad_W=True):
+    """The fused LM-head variant under the objective variants.  hidden [T,D], W [V,D]: bf16 bit patterns.
+    -> dict(logp, loss, grad_hidden f64[T,D] | None, grad_W f64[V,D] | None)."""
+    hidden = _c(hidden, np.uint16)
+    W = _c(W, np.uint16)
+    T, D = hidden.shape
+    V = W.shape[0]
+    assert W.shape[1] == D
+    ids = _c(ids, np.int32)
+    seq_id = _c(seq_id, np.int32)
+    adv = _c(adv, np.float32)
+    old_logp = _c(old_logp, np.float32)
+    ref_logp = _c(ref_logp, np.float32)
+    mask = _c(mask, np.uint8)
+    logp = np.zeros(T, np.float64)
+    loss = np.zeros(4, np.float64)
+    gh = np.zeros((T, D), np.float64) if want_grad_hidden else None
+    gw = np.zeros((V, D), np.float64) if want_grad_W else None
+    rc = lib().orc_fused_lmhead_grpo_obj(_p(hidden), _p(W), ctypes.c_int64(T), ctypes.c_int32(D), ctypes.c_int32(V),
+                                         _p(ids), _p(seq_id), _p(adv), ctypes.c_int32(len(adv)), _p(old_logp),
+                                         _p(ref_logp), _p(mask), ctypes.c_double(eps_low), ctypes.c_double(eps_high),
+                                         ctypes.c_double(beta_kl), ctypes.c_int(aggregation),
+                                         ctypes.c_int64(-1 if denom is None else int(denom)), _p(logp), _p(loss),
+                                         _p(gh), _p(gw))
+    _check(rc, "fused_lmhead_grpo_obj")
+    return dict(logp=logp, loss=loss, grad_hidden=gh, grad_W=gw)

@@ -19,7 +19,7 @@ DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
 
 EXPORTS = [
     "rlf_build_loss_mask", "rlf_group_advantage", "rlf_rule_reward", "rlf_kl_in_reward", "rlf_grpo_logp_loss_fwd_bwd",
-    "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_grpo_logp_loss_fwd_bwd_skip_masked", "rlf_grpo_logp_loss_fwd_bwd_obj", "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
+    "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_grpo_logp_loss_fwd_bwd_skip_masked", "rlf_grpo_logp_loss_fwd_bwd_obj", "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_fused_lmhead_grpo_obj", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
     "rlf_tune_logits_kernel", "rlf_tune_lmhead", "rlf_launch_count", "rlf_status_string", "rlf_version",
 ]
 
@@ -354,6 +354,41 @@ def rlf_fused_lmhead_grpo(hidden, W, ids, seq_id, adv, old_logp, ref_logp, mask,
         _ptr(grad_hidden, torch.bfloat16), _ptr(grad_W, torch.float32), 1 if accumulate_grad_W else 0,
         workspace.data_ptr(), workspace.numel(), _ptr(dev_status, torch.int32), _stream()),
         "rlf_fused_lmhead_grpo")
+    return logp_out, loss_out, grad_hidden, grad_W
+
+
+def rlf_fused_lmhead_grpo_obj(hidden, W, ids, seq_id, adv, old_logp, ref_logp, mask, eps_clip_low, eps_clip_high,
+                              beta_kl, aggregation=0, skip_masked=False, denom=None, want_grad_hidden=True,
+                              want_grad_W=True, grad_hidden=None, grad_W=None, accumulate_grad_W=False,
+                              logp_out=None, loss_out=None, workspace=None, dev_status=None):
+    """The fused LM-head call with an asymmetric clip range, token- or sequence-mean aggregation and
+    the option of not multiplying masked rows at all (their log-prob is NaN).
+    -> (logp fp32[T], loss fp64[4], grad_hidden bf16[T,D] | None, grad_W fp32[V,D] | None)."""
+    T, D = hidden.shape
+    V = W.shape[0]
+    dev = hidden.device
+    if grad_hidden is None and want_grad_hidden:
+        grad_hidden = torch.empty((T, D), dtype=torch.bfloat16, device=dev)
+    if grad_W is None and want_grad_W:
+        grad_W = torch.zeros((V, D), dtype=torch.float32, device=dev)
+    if logp_out is None:
+        logp_out = torch.empty(T, dtype=torch.float32, device=dev)
+    if loss_out is None:
+        loss_out = torch.empty(4, dtype=torch.float64, device=dev)
+    if workspace is None:
+        workspace = new_workspace(FN_FUSED_LMHEAD, T, V, D, RLF_BF16, dev)
+    _lib.rlf_fused_lmhead_grpo_obj.argtypes = [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _f32,
+                                               _f32, _f32, _int, _int, _vp, _vp, _vp, _vp, _vp, _int, _vp, _sz,
+                                               _vp, _vp]
+    _lib.rlf_fused_lmhead_grpo_obj.restype = _int
+    _check(_lib.rlf_fused_lmhead_grpo_obj(
+        _ptr(hidden, torch.bfloat16), _ptr(W, torch.bfloat16), T, D, V, _ptr(ids, torch.int32),
+        _ptr(seq_id, torch.int32), _ptr(adv, torch.float32), adv.shape[0], _ptr(old_logp, torch.float32),
+        _ptr(ref_logp, torch.float32), _ptr(mask, torch.uint8), float(eps_clip_low), float(eps_clip_high),
+        float(beta_kl), int(aggregation), 1 if skip_masked else 0, _ptr(denom, torch.int64),
+        _ptr(logp_out, torch.float32), _ptr(loss_out, torch.float64), _ptr(grad_hidden, torch.bfloat16),
+        _ptr(grad_W, torch.float32), 1 if accumulate_grad_W else 0, workspace.data_ptr(), workspace.numel(),
+        _ptr(dev_status, torch.int32), _stream()), "rlf_fused_lmhead_grpo_obj")
     return logp_out, loss_out, grad_hidden, grad_W
 
 

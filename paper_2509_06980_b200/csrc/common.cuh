@@ -22,6 +22,14 @@ rlf_status launch_token_prep(const int32_t* ids, const int32_t* seq_id, const fl
 rlf_status launch_token_loss(const float* logp, const void* rec, int64_t T, float eps_clip, float beta,
                              double* partial, const long long* denom, double* loss_out, cudaStream_t s);
 size_t token_loss_partial_bytes();
+// the same with an asymmetric clip range and optional per-token weights (weighted sums are already means)
+rlf_status launch_token_loss_w(const float* logp, const void* rec, int64_t T, float eps_lo, float eps_hi, float beta,
+                               const float* wtok, double* partial, const long long* denom, double* loss_out,
+                               cudaStream_t s);
+// sequence-mean aggregation: wtok[t] = live_t / (n_b * S); cnt [B] ints and s_slot [1] are scratch
+rlf_status launch_seq_weights(const void* rec, const int32_t* seq_id, int64_t T, int32_t B,
+                              const long long* denom_or_null, int* cnt, long long* s_slot, float* wtok,
+                              cudaStream_t s);
 
 inline rlf_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? RLF_OK : RLF_ERR_CUDA; }
 

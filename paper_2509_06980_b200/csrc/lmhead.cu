@@ -556,8 +556,8 @@ target_logit_kernel(const __nv_bfloat16* __restrict__ hidden, const __nv_bfloat1
 __global__ void __launch_bounds__(256)
 combine_kernel(const float2* __restrict__ part, int nsplit, const float* __restrict__ zy,
                const float4* __restrict__ rec, int64_t T, const long long* __restrict__ denom, float eps_clip,
-               float beta, float* __restrict__ logp_out, float* __restrict__ lse_out, float* __restrict__ coef_out,
-               int32_t* __restrict__ dev_status) {
+               float eps_hi, const float* __restrict__ wtok, float beta, float* __restrict__ logp_out,
+               float* __restrict__ lse_out, float* __restrict__ coef_out, int32_t* __restrict__ dev_status) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= T) return;
     float M = -INFINITY;
@@ -575,10 +575,10 @@ combine_kernel(const float2* __restrict__ part, int nsplit, const float* __restr
     float coef = 0.0f;
     if (live) {
         const long long N = *denom;
-        const float inv_n = 1.0f / (float)(N > 1 ? N : 1);
+        const float inv_n = wtok ? wtok[t] : 1.0f / (float)(N > 1 ? N : 1);
         const float A = r.z;
         const float rho = expf(logp - r.x);
-        const bool clipped = ((A > 0.0f) && (rho > 1.0f + eps_clip)) || ((A < 0.0f) && (rho < 1.0f - eps_clip));
+        const bool clipped = ((A > 0.0f) && (rho > 1.0f + eps_hi)) || ((A < 0.0f) && (rho < 1.0f - eps_clip));
         const float dpg = clipped ? 0.0f : -A * rho;
         coef = -inv_n * fmaf(beta, -expm1f(r.y - logp), dpg);
     }
@@ -641,14 +641,21 @@ gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden, int D, const int32_
     }
 }
 
+// skip-masked form: the rows without loss weight are not multiplied at all; their log-prob reads NaN
+__global__ void __launch_bounds__(256)
+fill_nan_rows_kernel(const int32_t* __restrict__ idx, const int* __restrict__ count, float* __restrict__ logp_out) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < *count) logp_out[idx[r]] = __int_as_float(0x7fc00000);
+}
+
 // combine_kernel for a launch over gathered rows: row r of the launch (partials part[r][.]) is token
 // idx[off + r]; logp goes to the token's place, lse / coefficient / target id to the gathered place
 __global__ void __launch_bounds__(256)
 combine_rows_kernel(const float2* __restrict__ part, int nsplit, int rows_max, const int32_t* __restrict__ idx,
                     const int* __restrict__ count, int off, const float* __restrict__ zy,
-                    const float4* __restrict__ rec, const long long* __restrict__ denom, float eps_clip, float beta,
-                    float* __restrict__ logp_out, float* __restrict__ lse_g, float* __restrict__ coef_g,
-                    int32_t* __restrict__ y_g, int32_t* __restrict__ dev_status) {
+                    const float4* __restrict__ rec, const long long* __restrict__ denom, float eps_clip, float eps_hi,
+                    const float* __restrict__ wtok, float beta, float* __restrict__ logp_out, float* __restrict__ lse_g,
+                    float* __restrict__ coef_g, int32_t* __restrict__ y_g, int32_t* __restrict__ dev_status) {
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     const int n = max(0, min(*count - off, rows_max));
     if (r >= n) return;
@@ -668,10 +675,10 @@ combine_rows_kernel(const float2* __restrict__ part, int nsplit, int rows_max, c
     float coef = 0.0f;
     if (live) {
         const long long N = *denom;
-        const float inv_n = 1.0f / (float)(N > 1 ? N : 1);
+        const float inv_n = wtok ? wtok[t] : 1.0f / (float)(N > 1 ? N : 1);
         const float A = rc.z;
         const float rho = expf(logp - rc.x);
-        const bool clipped = ((A > 0.0f) && (rho > 1.0f + eps_clip)) || ((A < 0.0f) && (rho < 1.0f - eps_clip));
+        const bool clipped = ((A > 0.0f) && (rho > 1.0f + eps_hi)) || ((A < 0.0f) && (rho < 1.0f - eps_clip));
         const float dpg = clipped ? 0.0f : -A * rho;
         coef = -inv_n * fmaf(beta, -expm1f(rc.y - logp), dpg);
     }
@@ -822,26 +829,20 @@ static rlf_status launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, cons
 constexpr int kChunkTokens = 74 * BM;
 constexpr int kMaxSplit = 64;               // most vocabulary splits a sweep may use (sizes the partials)
 
-// Number of vocabulary splits for a sweep over m_units row units and n_tiles column tiles on
-// `workers` CTAs (or CTA pairs): the smallest count >= 4 whose m_units * splits work units fill
-// whole waves best, each split keeping at least 8 column tiles.
-static int pick_split(int m_units, int n_tiles, int workers) {
-    int best = 1;
-    double best_eff = 0.0;
-    for (int sp = 1; sp <= kMaxSplit; ++sp) {
-        const int per = (n_tiles + sp - 1) / sp;
-        if (sp > 1 && per < 8) break;
-        const int used = (n_tiles + per - 1) / per;            // splits that actually hold tiles
-        const long long units = (long long)m_units * used;
-        const long long waves = (units + workers - 1) / workers;
-        const double eff = (double)units / (double)(waves * workers) * ((double)n_tiles / (double)(per * used));
-        if (eff > best_eff + 0.02) { best_eff = eff; best = sp; }
-    }
-    return best;
+// Number of vocabulary splits of a sweep.  A work unit is (pair of token tiles, split); the units are
+// dealt round-robin to the persistent CTAs, which keep their load / multiply / drain pipelines
+// running across units, so small units cost nothing, while large ones leave a ragged last wave
+// (the number of rows that take part is only known on the device).  Splits of at least 8 column
+// tiles, at most kMaxSplit of them; concurrently running CTAs still work on the same few splits, so
+// the head's rows are shared in L2.
+static int pick_split(int n_tiles) {
+    int per = (n_tiles + kMaxSplit - 1) / kMaxSplit;
+    if (per < 8) per = 8;
+    return (n_tiles + per - 1) / per;
 }
 
 struct LmWs {
-    size_t n_count, partial, rec, zy, lse, coef, part, idx_live, idx_dead, lse_g, coef_g, y_g, hidden_g, tmax, dz, total;
+    size_t n_count, partial, rec, zy, lse, coef, wtok, seqcnt, part, idx_live, idx_dead, lse_g, coef_g, y_g, hidden_g, tmax, dz, total;
 };
 static size_t up1k(size_t x) { return (x + 1023) & ~(size_t)1023; }
 static LmWs lm_workspace(int64_t T, int32_t V, int32_t D) {
@@ -855,6 +856,8 @@ static LmWs lm_workspace(int64_t T, int32_t V, int32_t D) {
     w.zy = o;      o += up1k(4 * Tn);
     w.lse = o;     o += up1k(4 * Tn);
     w.coef = o;    o += up1k(4 * Tn);
+    w.wtok = o;    o += up1k(4 * Tn);                // sequence-mean aggregation: per-token weights
+    w.seqcnt = o;  o += up1k(4 * (Tn + 1));          //   and unmasked tokens per response (B <= T + 1)
     w.part = o;    o += up1k(8 * Tn * kMaxSplit);
     w.idx_live = o; o += up1k(4 * Tp);
     w.idx_dead = o; o += up1k(4 * Tp);
@@ -879,16 +882,23 @@ size_t lmhead_workspace_bytes(int64_t T, int32_t V, int32_t D) {
 
 }  // namespace rlf
 
-extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, int64_t T, int32_t D, int32_t V,
-                                            const int32_t* ids, const int32_t* seq_id, const float* adv, int32_t B,
-                                            const float* old_logp, const float* ref_logp, const uint8_t* mask,
-                                            float eps_clip, float beta_kl, const int64_t* denom, float* logp_out,
-                                            double* loss_out, void* grad_hidden, float* grad_W,
-                                            int accumulate_grad_W, void* workspace, size_t workspace_bytes,
-                                            int32_t* dev_status, rlf_stream_t stream) {
-    using namespace rlf;
-    using namespace rlf::lm;
+namespace rlf {
+namespace lm {
+
+// eps_clip is the lower clip width, eps_hi the upper one; aggregation 0 = token mean (denom counts
+// tokens), 1 = sequence mean (denom counts responses); skip_masked: rows without loss weight are not
+// multiplied at all and their log-prob reads NaN
+static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T, int32_t D, int32_t V,
+                                    const int32_t* ids, const int32_t* seq_id, const float* adv, int32_t B,
+                                    const float* old_logp, const float* ref_logp, const uint8_t* mask,
+                                    float eps_clip, float eps_hi, float beta_kl, int aggregation, int skip_masked,
+                                    const int64_t* denom, float* logp_out,
+                                    double* loss_out, void* grad_hidden, float* grad_W,
+                                    int accumulate_grad_W, void* workspace, size_t workspace_bytes,
+                                    int32_t* dev_status, rlf_stream_t stream) {
     if (T < 0 || V < 1 || D < 1 || B < 0) return RLF_ERR_SHAPE;
+    if (aggregation != 0 && aggregation != 1) return RLF_ERR_SHAPE;
+    if (aggregation == 1 && (int64_t)B > T + 1) return RLF_ERR_SHAPE;
     if (D % 64 != 0 || V % 8 != 0) return RLF_ERR_SHAPE;
     if (T >= (1ll << 30)) return RLF_ERR_UNSUPPORTED;
     if (!loss_out) return RLF_ERR_NULL;
@@ -916,23 +926,35 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
     const __nv_bfloat16* H = static_cast<const __nv_bfloat16*>(hidden);
     const __nv_bfloat16* Wm = static_cast<const __nv_bfloat16*>(W);
 
-    const long long* dn = reinterpret_cast<const long long*>(denom);
-    if (dn == nullptr) {
+    // token mean: dn is the token count (given, or counted by the record kernel); sequence mean: the
+    // per-token weights carry the whole normalisation and dn is only a valid address to read
+    const long long* dn = aggregation == 0 ? reinterpret_cast<const long long*>(denom) : nullptr;
+    const bool count_here = dn == nullptr;
+    if (count_here) {
         if (cudaMemsetAsync(n_count, 0, sizeof(long long), s) != cudaSuccess) return RLF_ERR_CUDA;
         dn = n_count;
     }
-    if (T == 0) return launch_token_loss(logp_out, rec, 0, eps_clip, beta_kl, partial, dn, loss_out, s);
+    float* wtok = nullptr;
+    auto token_loss = [&](int64_t rows) {
+        return launch_token_loss_w(logp_out, rec, rows, eps_clip, eps_hi, beta_kl, wtok, partial, dn, loss_out, s);
+    };
+    if (T == 0) return token_loss(0);
 
-    st = launch_token_prep(ids, seq_id, adv, old_logp, ref_logp, mask, T, V, B, rec, denom == nullptr ? n_count : nullptr,
+    st = launch_token_prep(ids, seq_id, adv, old_logp, ref_logp, mask, T, V, B, rec, count_here ? n_count : nullptr,
                            dev_status, s);
     if (st != RLF_OK) return st;
+    if (aggregation == 1) {
+        wtok = reinterpret_cast<float*>(ws + w.wtok);
+        st = launch_seq_weights(rec, seq_id, T, B, reinterpret_cast<const long long*>(denom),
+                                reinterpret_cast<int*>(ws + w.seqcnt), n_count + 4, wtok, s);
+        if (st != RLF_OK) return st;
+    }
     target_logit_kernel<<<(unsigned)((T + 7) / 8), 256, 0, s>>>(H, Wm, rec, T, D, zy);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
 
     const bool pair = g_pair.load() != 0;
     const uint32_t b_rows = pair ? BN / 2 : BN;       // rows of a K-major B tile that one CTA stages
-    const int workers = pair ? sm_count_lm() / 2 : sm_count_lm();
     CUtensorMap mapW;
     if (!make_map(&mapW, Wm, (uint64_t)V, (uint64_t)D, (uint64_t)D, BK, b_rows)) return RLF_ERR_CUDA;
     GemmParams g = {};
@@ -945,22 +967,22 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
     auto set_rows = [&](GemmParams& q, int64_t rows) {
         q.M = (int)rows;
         q.m_tiles = (int)((rows + BM - 1) / BM);
-        q.nsplit = pick_split(pair ? (q.m_tiles + 1) / 2 : q.m_tiles, q.n_tiles, workers);
+        q.nsplit = pick_split(q.n_tiles);
         q.n_tiles_per_split = (q.n_tiles + q.nsplit - 1) / q.nsplit;
     };
 
-    if (!grad_hidden && !grad_W) {
+    if (!grad_hidden && !grad_W && !skip_masked) {
         // forward only: one sweep over all rows, running (max, sum exp) per token and vocabulary split
         CUtensorMap mapH;
         if (!make_map(&mapH, H, (uint64_t)T, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
         set_rows(g, T);
         st = launch_gemm(mapH, mapW, g, pair, s);
         if (st != RLF_OK) return st;
-        combine_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(part, g.nsplit, zy, rec, T, dn, eps_clip, beta_kl,
-                                                                    logp_out, lse, coef, dev_status);
+        combine_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(part, g.nsplit, zy, rec, T, dn, eps_clip, eps_hi, wtok,
+                                                                    beta_kl, logp_out, lse, coef, dev_status);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
-        return launch_token_loss(logp_out, rec, T, eps_clip, beta_kl, partial, dn, loss_out, s);
+        return token_loss(T);
     }
 
     // forward + backward.  The tokens are partitioned (stably) into unmasked rows and the others;
@@ -979,31 +1001,36 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
     __nv_bfloat16* Hd = reinterpret_cast<__nv_bfloat16*>(ws + w.hidden_g + up1k((size_t)Tp * D * 2));
     partition_rows_kernel<<<1, 1024, 0, s>>>(rec, (int)T, idx_live, idx_dead, counts);
     gather_rows_kernel<<<(unsigned)Tp, 128, 0, s>>>(H, D, idx_live, counts, Hl);
-    gather_rows_kernel<<<(unsigned)Tp, 128, 0, s>>>(H, D, idx_dead, counts + 1, Hd);
-    count_launch(3);
+    if (!skip_masked) gather_rows_kernel<<<(unsigned)Tp, 128, 0, s>>>(H, D, idx_dead, counts + 1, Hd);
+    count_launch(skip_masked ? 2 : 3);
     if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
     if (grad_hidden && cudaMemsetAsync(grad_hidden, 0, (size_t)T * D * 2, s) != cudaSuccess) return RLF_ERR_CUDA;
 
+    const bool bwd = grad_hidden || grad_W;
     for (int64_t t0 = 0; t0 < T; t0 += kChunkTokens) {
         const int64_t tc = (T - t0) < kChunkTokens ? (T - t0) : kChunkTokens;
         CUtensorMap mapHc;
         if (!make_map(&mapHc, Hl + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
         GemmParams z = g;
         set_rows(z, tc);
-        z.dz = dz;
-        z.dz_stride = V;
-        z.tmax = reinterpret_cast<float*>(ws + w.tmax);
+        if (bwd) {
+            z.dz = dz;
+            z.dz_stride = V;
+            z.tmax = reinterpret_cast<float*>(ws + w.tmax);
+        }
         z.live_count = counts;
         z.live_off = (int)t0;
         st = launch_gemm(mapHc, mapW, z, pair, s);
         if (st != RLF_OK) return st;
         combine_rows_kernel<<<(unsigned)((tc + 255) / 256), 256, 0, s>>>(part, z.nsplit, (int)tc, idx_live, counts, (int)t0,
-                                                                          zy, rec, dn, eps_clip, beta_kl, logp_out, lse_g,
-                                                                          coef_g, y_g, dev_status);
+                                                                          zy, rec, dn, eps_clip, eps_hi, wtok, beta_kl,
+                                                                          logp_out, lse_g, coef_g, y_g, dev_status);
+        count_launch();
+        if (!bwd) continue;
         const int64_t tcp = (tc + 255) & ~(int64_t)255;
         dz_from_e_kernel<<<(unsigned)tcp, 256, 0, s>>>(dz, V, z.n_tiles, z.tmax, (int)tc, counts, (int)t0, lse_g, coef_g, y_g,
                                                         idx_live, zy);
-        count_launch(2);
+        count_launch();
         if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
         if (grad_hidden) {
             // grad_hidden[token of gathered row] = dZ[chunk, V] W[V, D]
@@ -1050,7 +1077,11 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
     }
 
     // the masked rows: log-prob only
-    {
+    if (skip_masked) {
+        fill_nan_rows_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(idx_dead, counts + 1, logp_out);
+        count_launch();
+        if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+    } else {
         CUtensorMap mapHd;
         if (!make_map(&mapHd, Hd, (uint64_t)T, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
         GemmParams d = g;
@@ -1060,13 +1091,44 @@ extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, i
         st = launch_gemm(mapHd, mapW, d, pair, s);
         if (st != RLF_OK) return st;
         combine_rows_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(part, d.nsplit, (int)T, idx_dead, counts + 1, 0, zy,
-                                                                         rec, dn, eps_clip, beta_kl, logp_out, nullptr,
-                                                                         nullptr, nullptr, dev_status);
+                                                                         rec, dn, eps_clip, eps_hi, wtok, beta_kl, logp_out,
+                                                                         nullptr, nullptr, nullptr, dev_status);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
     }
-    return launch_token_loss(logp_out, rec, T, eps_clip, beta_kl, partial, dn, loss_out, s);
+    return token_loss(T);
 }
+
+}  // namespace lm
+}  // namespace rlf
+
+extern "C" rlf_status rlf_fused_lmhead_grpo(const void* hidden, const void* W, int64_t T, int32_t D, int32_t V,
+                                            const int32_t* ids, const int32_t* seq_id, const float* adv, int32_t B,
+                                            const float* old_logp, const float* ref_logp, const uint8_t* mask,
+                                            float eps_clip, float beta_kl, const int64_t* denom, float* logp_out,
+                                            double* loss_out, void* grad_hidden, float* grad_W,
+                                            int accumulate_grad_W, void* workspace, size_t workspace_bytes,
+                                            int32_t* dev_status, rlf_stream_t stream) {
+    return rlf::lm::fused_lmhead_impl(hidden, W, T, D, V, ids, seq_id, adv, B, old_logp, ref_logp, mask, eps_clip,
+                                      eps_clip, beta_kl, 0, 0, denom, logp_out, loss_out, grad_hidden, grad_W,
+                                      accumulate_grad_W, workspace, workspace_bytes, dev_status, stream);
+}
+
+extern "C" rlf_status rlf_fused_lmhead_grpo_obj(const void* hidden, const void* W, int64_t T, int32_t D, int32_t V,
+                                                const int32_t* ids, const int32_t* seq_id, const float* adv, int32_t B,
+                                                const float* old_logp, const float* ref_logp, const uint8_t* mask,
+                                                float eps_clip_low, float eps_clip_high, float beta_kl, int aggregation,
+                                                int skip_masked, const int64_t* denom, float* logp_out,
+                                                double* loss_out, void* grad_hidden, float* grad_W,
+                                                int accumulate_grad_W, void* workspace, size_t workspace_bytes,
+                                                int32_t* dev_status, rlf_stream_t stream) {
+    if (skip_masked != 0 && skip_masked != 1) return RLF_ERR_SHAPE;
+    return rlf::lm::fused_lmhead_impl(hidden, W, T, D, V, ids, seq_id, adv, B, old_logp, ref_logp, mask, eps_clip_low,
+                                      eps_clip_high, beta_kl, aggregation, skip_masked, denom, logp_out, loss_out,
+                                      grad_hidden, grad_W, accumulate_grad_W, workspace, workspace_bytes, dev_status,
+                                      stream);
+}
+
 
 extern "C" rlf_status rlf_tune_lmhead(int pair_ctas) {
     if (pair_ctas != 0 && pair_ctas != 1) return RLF_ERR_SHAPE;

@@ -1599,6 +1599,36 @@ rlf_status launch_token_loss(const float* logp, const void* rec, int64_t T, floa
     return cuda_ok(cudaGetLastError());
 }
 
+rlf_status launch_token_loss_w(const float* logp, const void* rec, int64_t T, float eps_lo, float eps_hi, float beta,
+                               const float* wtok, double* partial, const long long* denom, double* loss_out,
+                               cudaStream_t s) {
+    int num_partials = 0;
+    if (T > 0) {
+        const int64_t blocks = (T + kLossThreads - 1) / kLossThreads;
+        num_partials = (int)(blocks < kMaxPartials ? blocks : kMaxPartials);
+        token_loss_kernel<<<num_partials, kLossThreads, 0, s>>>(logp, static_cast<const float4*>(rec), T, eps_lo,
+                                                               eps_hi, wtok, partial);
+        count_launch();
+        if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+    }
+    finalize_loss_kernel<<<1, 32, 0, s>>>(partial, num_partials, denom, beta, wtok != nullptr, loss_out);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
+rlf_status launch_seq_weights(const void* rec, const int32_t* seq_id, int64_t T, int32_t B,
+                              const long long* denom_or_null, int* cnt, long long* s_slot, float* wtok,
+                              cudaStream_t s) {
+    if (T <= 0) return RLF_OK;
+    const int64_t blocks = (T + 255) / 256;
+    if (cudaMemsetAsync(cnt, 0, sizeof(int) * (size_t)B, s) != cudaSuccess) return RLF_ERR_CUDA;
+    seq_count_kernel<<<(unsigned)blocks, 256, 0, s>>>(static_cast<const float4*>(rec), seq_id, T, cnt);
+    seq_live_kernel<<<1, 1024, 0, s>>>(cnt, B, denom_or_null, s_slot);
+    seq_weight_kernel<<<(unsigned)blocks, 256, 0, s>>>(static_cast<const float4*>(rec), seq_id, T, cnt, s_slot, wtok);
+    count_launch(3);
+    return cuda_ok(cudaGetLastError());
+}
+
 size_t token_loss_partial_bytes() { return sizeof(double) * 4 * kMaxPartials; }
 
 }  // namespace rlf

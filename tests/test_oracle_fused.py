@@ -86,3 +86,47 @@ def test_finite_differences_through_the_head():
         Wp, Wm = W.copy(), W.copy()
         Wp[v, k] += h; Wm[v, k] -= h
         assert abs((L(H, Wp) - L(H, Wm)) / (2 * h) - r["grad_W"][v, k]) < 1e-8
+
+
+def test_objective_variant_of_the_head_reduces_and_composes():
+    Hb, H, Wb, W, ids, seq, adv, old, ref, mask = _problem(4)
+    base = orc.fused_lmhead_grpo(Hb, Wb, ids, seq, adv, old, ref, mask, 0.2, 0.05)
+    same = orc.fused_lmhead_grpo_obj(Hb, Wb, ids, seq, adv, old, ref, mask, 0.2, 0.2, 0.05, aggregation=0)
+    for k in ("logp", "loss", "grad_hidden", "grad_W"):
+        assert np.allclose(base[k], same[k], atol=1e-15), k
+    # composition with the logits-path variant on the fp64 contraction (numpy matmul as the library step)
+    for agg in (0, 1):
+        r = orc.fused_lmhead_grpo_obj(Hb, Wb, ids, seq, adv, old, ref, mask, 0.1, 0.3, 0.05, aggregation=agg)
+        g = orc.grpo_loss_obj(H @ W.T, ids, seq, adv, old, ref, mask, 0.1, 0.3, 0.05, aggregation=agg)
+        assert np.allclose(r["loss"], g["loss"], atol=1e-13) and np.allclose(r["logp"], g["logp"], atol=1e-13)
+        assert np.allclose(r["grad_hidden"], g["grad"] @ W, atol=1e-14)
+        assert np.allclose(r["grad_W"], g["grad"].T @ H, atol=1e-14)
+
+
+def test_objective_variant_of_the_head_matches_torch_autograd_fp64():
+    """Asymmetric clip range with the sequence mean: L = (1/S) sum_b (1/n_b) sum_{t in b} mask_t l_t."""
+    Hb, H, Wb, W, ids, seq, adv, old, ref, mask = _problem(5, T=16, B=4)
+    lo, hi, beta = 0.15, 0.4, 0.07
+    r = orc.fused_lmhead_grpo_obj(Hb, Wb, ids, seq, adv, old, ref, mask, lo, hi, beta, aggregation=1)
+    Ht = torch.tensor(H, requires_grad=True)
+    Wt = torch.tensor(W, requires_grad=True)
+    logp = torch.log_softmax(Ht @ Wt.t(), -1).gather(1, torch.tensor(ids, dtype=torch.int64)[:, None])[:, 0]
+    seq_t = torch.tensor(seq, dtype=torch.int64)
+    A = torch.tensor(adv, dtype=torch.float64)[seq_t]
+    rho = torch.exp(logp - torch.tensor(old, dtype=torch.float64))
+    pg = -torch.minimum(rho * A, torch.clamp(rho, 1 - lo, 1 + hi) * A)
+    d = torch.tensor(ref, dtype=torch.float64) - logp
+    m = torch.tensor(mask, dtype=torch.float64)
+    tok = m * (pg + beta * (torch.exp(d) - d - 1))
+    L = 0.0
+    S = 0
+    for b in range(4):
+        sel = seq_t == b
+        if m[sel].sum() > 0:
+            L = L + tok[sel].sum() / m[sel].sum()
+            S += 1
+    L = L / S
+    L.backward()
+    assert abs(r["loss"][0] - L.item()) < 1e-13
+    assert np.abs(r["grad_hidden"] - Ht.grad.numpy()).max() < 1e-14
+    assert np.abs(r["grad_W"] - Wt.grad.numpy()).max() < 1e-14

@@ -29,6 +29,9 @@ MUTATIONS = [
     ("grad_W_uses_wrong_operand", "acc += gz[t * (int64_t)V + v] * widen(hidden, ORC_BF16, t * (int64_t)D + k);", "acc += gz[t * (int64_t)V + v] * widen(hidden, ORC_BF16, t * (int64_t)D + (D - 1 - k));", "test_oracle_fused.py"),
     ("asymmetric_clip_uses_low_for_both", "1.0 - eps_low, 1.0 + eps_high, &pg", "1.0 - eps_low, 1.0 + eps_low, &pg", "test_oracle_objective.py"),
     ("sequence_mean_weighs_by_batch_count", "w[t] = mask[t] ? 1.0 / ((double)nb[seq_id[t]] * sd) : 0.0;", "w[t] = mask[t] ? 1.0 / ((double)T * sd) : 0.0;", "test_oracle_objective.py"),
+    ("kl_reward_counts_masked_tokens", "            if (!mask[t])\n                continue;\n            double d = (double)old_logp[t]", "            double d = (double)old_logp[t]", "test_oracle_kl_reward.py"),
+    ("kl_reward_k3_direction", "k = exp(-d) + d - 1.0;", "k = exp(d) - d - 1.0;", "test_oracle_kl_reward.py"),
+    ("kl_reward_penalty_sign", "reward_out[b] = (double)rewards[b] - beta * acc;", "reward_out[b] = (double)rewards[b] + beta * acc;", "test_oracle_kl_reward.py"),
     ("entropy_sign", "if (pv > 0.0) h -= pv * lp;", "if (pv > 0.0) h += pv * lp;", "test_oracle_entropy.py"),
 ]
 
