@@ -58,12 +58,14 @@ def _tensor_peaks():
     return 1590.0, 1400.0, "fallback"
 
 
-def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3):
+def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3, responses=0):
     """The fused LM-head variant on the Qwen3-4B head (T = 32768, D = 2560, V = 151936): forward
     (log-probs and loss, logits never stored) and forward + backward (grad_hidden, grad_W)."""
     spec = synth.SPECS[cfg]
     if tokens_per_response:
         spec = synth.scaled(spec, len_lo=tokens_per_response, len_hi=tokens_per_response)
+    if responses:
+        spec = synth.scaled(spec, num_prompts=1, group_size=responses)     # fewer full-length responses
     tok = synth.make_tokens(spec)
     T = len(tok.ids)
     ids = torch.from_numpy(tok.ids).to(dev)
@@ -96,7 +98,7 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3):
     tvd = 2.0 * spec.V * spec.D
     for name, bwd, useful_flops, executed_flops in (("fwd", False, tvd * T, tvd * T),
                                                     ("fwd_bwd", True, tvd * (T + 2 * live), tvd * (T + 2 * live))):
-        for _ in range(1 if tokens_per_response else 2):
+        for _ in range(1 if (tokens_per_response or responses) else 2):
             run(bwd)
         torch.cuda.synchronize()
         ts = []
@@ -116,9 +118,44 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3):
                                   "frac": useful / burst, "peak_kind": "of " + kind + " (burst)",
                                   "frac_of_sustained": useful / sustained, "frac_of_nominal_2250": useful / 2250.0,
                                   "traffic": None}}
+    # the same call without multiplying the masked rows at all (their log-prob is not produced)
+    def run_skip():
+        rlf.rlf_fused_lmhead_grpo_obj(H, W, ids, seq, adv, old, ref, mask, synth.EPS_CLIP, synth.EPS_CLIP,
+                                      synth.BETA_KL, skip_masked=True, denom=n, grad_hidden=gh, grad_W=gw,
+                                      logp_out=logp, loss_out=loss, workspace=ws, dev_status=st)
+    run_skip()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        run_skip()
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    ms = statistics.mean(ts)
+    out["fwd_bwd_skip_masked"] = {"entry": "rlf_fused_lmhead_grpo_obj(skip_masked=1)", "ms": ms,
+                                  "tokens_per_s": T / ms * 1e3, "executed_tflops": tvd * 3 * live / ms / 1e9}
     if st.item() != 0:
         out["device_status"] = int(st.item())
     out["loss"] = float(loss[0].item())
+    if not tokens_per_response and not responses:
+        # context: the library GEMM of the forward's shape on this GPU, in the same state (back to back,
+        # logits written to HBM as bf16): what an unfused path pays for the contraction alone
+        z = torch.empty((T, spec.V), dtype=torch.bfloat16, device=dev)
+        for _ in range(2):
+            torch.matmul(H, W.t(), out=z)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            torch.matmul(H, W.t(), out=z)
+        b.record()
+        torch.cuda.synchronize()
+        lib_ms = a.elapsed_time(b) / steps
+        out["library_gemm_same_shape"] = {"what": "torch.matmul(H, W^T) -> bf16 [T, V], not part of the path",
+                                          "ms": lib_ms, "tflops": tvd * T / lib_ms / 1e9}
+        del z
     return out
 
 
@@ -288,7 +325,8 @@ def run_fused_only(args):
     """Only the fused LM-head variant, optionally at a reduced token count (profiling captures)."""
     from paper_2509_06980_b200 import binding as rlf
     torch.cuda.set_device(0)
-    out = time_fused_lmhead(rlf, torch.device("cuda", 0), max(1, args.steps), args.tokens_per_response)
+    out = time_fused_lmhead(rlf, torch.device("cuda", 0), max(1, args.steps), args.tokens_per_response,
+                            responses=args.responses)
     print(json.dumps({"fused_lmhead": out, "gpu_launches": rlf.launch_count()}))
 
 
@@ -592,6 +630,8 @@ def main():
                     help="time cfg 2 (ragged, in place) and cfg 4 (micro-batched; both paths) instead (rank 0)")
     ap.add_argument("--tokens-per-response", type=int, default=0,
                     help="smaller micro-batch of the same recipe (profiling captures); 0 = the full 2048")
+    ap.add_argument("--responses", type=int, default=0,
+                    help="with --fused-only: one group of this many full-length responses (profiling captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -55,6 +55,7 @@ struct GemmParams {
     int M, N;                 // extent of the output tile grid in rows / columns (valid elements)
     int m_tiles, n_tiles, k_slabs;
     int nsplit, n_tiles_per_split;
+    int m_block;              // kLse: row units per scheduling block
     float2* part;             // kLse: [M][nsplit] (max, sum exp)
     __nv_bfloat16* dz;        // kLse (optional) out, row stride dz_stride: exp(z - tile max) as bf16
     float* tmax;              // kLse with dz: [M][n_tiles] the tile maxima those exponentials refer to
@@ -246,8 +247,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     // unit -> (m unit, first n tile, one-past-last n tile)
     auto unit_range = [&](int u, int& m, int& n0, int& n1) {
         if (sweep) {
-            m = u % m_units;
-            const int sp = u / m_units;
+            // blocks of m_block row units; inside a block, units run over its row units first, then
+            // over the splits: the CTAs running at one time share both the rows of the head they
+            // sweep and a set of token tiles small enough to stay in L2
+            const int per_block = p.m_block * p.nsplit;
+            const int blk = u / per_block, within = u - blk * per_block;
+            const int rows_here = min(p.m_block, m_units - blk * p.m_block);
+            const int sp = within / rows_here;
+            m = blk * p.m_block + (within - sp * rows_here);
             n0 = sp * p.n_tiles_per_split;
             n1 = min(p.n_tiles, n0 + p.n_tiles_per_split);
         } else {
@@ -358,7 +365,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             float run_m = -INFINITY, run_s = 0.0f;       // kLse
             for (int n = n0; n < n1 && ok; ++n) {
                 if (!no_k) {
-                    if (!mbar_wait(smem_addr(&ctl->tmem_full[buf]), tphase[buf], &ctl->abort_flag)) { ok = false; break; }
+                    // one lane polls for the warp (128 polling threads would only burn issue slots and
+                    // power while the tile is being multiplied); the shuffle hands its result to the others
+                    int got = 0;
+                    if (lane == 0) got = mbar_wait(smem_addr(&ctl->tmem_full[buf]), tphase[buf], &ctl->abort_flag) ? 1 : 0;
+                    got = __shfl_sync(0xffffffffu, got, 0);
+                    if (!got) { ok = false; break; }
                     tc_fence_after();
                 }
                 const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * BN;
@@ -503,7 +515,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 buf ^= 1;
             }
             if (p.mode == kLse && row_ok && ok) {
-                const int sp = u / m_units;
+                const int sp = n0 / p.n_tiles_per_split;
                 p.part[(long long)row * p.nsplit + sp] = make_float2(run_m, run_s);
             }
         }
@@ -798,6 +810,12 @@ static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, co
     const int units = sweep ? m_units * p.nsplit : m_units * p.n_tiles;
     if (units <= 0) return RLF_OK;
     int workers = PAIR ? sm_count_lm() / 2 : sm_count_lm();
+    // Sweep schedule: the CTAs (or pairs) running at one time cover workers / 2 row units x 2 splits,
+    // in lockstep.  Their token tiles (1.3 MB per pair at D = 2560) are re-read for every column tile
+    // and must stay in L2 next to the streaming head: with all 74 pairs on different row units
+    // (97 MB) they did not, and the same launch drew its 1 kW at 1.06 GHz instead of 1.39 GHz.
+    GemmParams q = p;
+    q.m_block = workers / 2 > 0 ? workers / 2 : 1;
     if (workers > units) workers = units;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(PAIR ? 2 * workers : workers);
@@ -811,7 +829,7 @@ static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, co
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, umma_gemm_kernel<PAIR>, ma, mb, p) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, umma_gemm_kernel<PAIR>, ma, mb, q) != cudaSuccess) {
         cudaGetLastError();
         return RLF_ERR_CUDA;
     }

@@ -48,8 +48,14 @@ def test_fused_objective_variants_match_oracle(V, D, lo, hi, agg, skip):
     else:
         assert np.abs(lp - r["logp"]).max() <= gc.LOGP_ATOL
     lg = loss.cpu().numpy()
+    # The surrogate's mean nearly cancels here (zero-mean advantages, ratios near 1), so a tolerance
+    # relative to its value alone would ask for more than fp32 log-probs can give: a log-prob error e
+    # moves a token's term by |A| rho e.  Floor of the scale: the mean |A| of the unmasked tokens times the
+    # log-prob tolerance.
+    a_tok = np.abs(adv.cpu().numpy()[seq.cpu().numpy()])[m == 1]
+    floor = gc.LOGP_ATOL * float(a_tok.mean()) if a_tok.size else 1e-6
     for k in range(3):
-        assert loss_close(lg[k], r["loss"][k], 1e-6, gc.LOSS_RTOL), (k, lg, r["loss"])
+        assert loss_close(lg[k], r["loss"][k], floor if k < 2 else 1e-6, gc.LOSS_RTOL), (k, lg, r["loss"])
     assert abs(lg[3] - r["loss"][3]) <= 2.0 / max(int(m.sum()), 1)
     _close_tensor(gh.float().cpu().numpy(), r["grad_hidden"], "grad_hidden")
     _close_tensor(gw.cpu().numpy(), r["grad_W"], "grad_W")
