@@ -20,7 +20,7 @@ DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
 EXPORTS = [
     "rlf_build_loss_mask", "rlf_group_advantage", "rlf_rule_reward", "rlf_kl_in_reward", "rlf_grpo_logp_loss_fwd_bwd",
     "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_grpo_logp_loss_fwd_bwd_skip_masked", "rlf_grpo_logp_loss_fwd_bwd_obj", "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_fused_lmhead_grpo_obj", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
-    "rlf_tune_logits_kernel", "rlf_tune_lmhead", "rlf_launch_count", "rlf_status_string", "rlf_version",
+    "rlf_tune_logits_kernel", "rlf_tune_lmhead", "rlf_tune_lmhead_schedule", "rlf_launch_count", "rlf_status_string", "rlf_version",
 ]
 
 if not os.path.exists(_LIB_PATH):
@@ -123,6 +123,12 @@ def tune_lmhead(pair_ctas=1):
     _lib.rlf_tune_lmhead.argtypes = [_int]
     _lib.rlf_tune_lmhead.restype = _int
     _check(_lib.rlf_tune_lmhead(int(pair_ctas)), "rlf_tune_lmhead")
+
+
+def tune_lmhead_schedule(m_block=0):
+    _lib.rlf_tune_lmhead_schedule.argtypes = [_int]
+    _lib.rlf_tune_lmhead_schedule.restype = _int
+    _check(_lib.rlf_tune_lmhead_schedule(int(m_block)), "rlf_tune_lmhead_schedule")
 
 
 def rlf_build_loss_mask(ids, cu_seqlens, open_id, close_id, valid=None, mask_out=None, seq_id_out=None,

@@ -787,6 +787,7 @@ static int sm_count_lm() {
 }
 
 static std::atomic<int> g_pair{1};       // 1: cta_group::2 pair form, 0: single-CTA form
+static std::atomic<int> g_m_block{0};    // row units per scheduling block of the sweep; 0: automatic
 
 template <bool PAIR>
 static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, cudaStream_t s) {
@@ -816,6 +817,7 @@ static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, co
     // (97 MB) they did not, and the same launch drew its 1 kW at 1.06 GHz instead of 1.39 GHz.
     GemmParams q = p;
     q.m_block = workers / 2 > 0 ? workers / 2 : 1;
+    if (g_m_block.load() > 0) q.m_block = g_m_block.load();
     if (workers > units) workers = units;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(PAIR ? 2 * workers : workers);
@@ -1151,5 +1153,11 @@ extern "C" rlf_status rlf_fused_lmhead_grpo_obj(const void* hidden, const void* 
 extern "C" rlf_status rlf_tune_lmhead(int pair_ctas) {
     if (pair_ctas != 0 && pair_ctas != 1) return RLF_ERR_SHAPE;
     rlf::lm::g_pair = pair_ctas;
+    return RLF_OK;
+}
+
+extern "C" rlf_status rlf_tune_lmhead_schedule(int m_block) {
+    if (m_block < 0 || m_block > (1 << 20)) return RLF_ERR_SHAPE;
+    rlf::lm::g_m_block = m_block;
     return RLF_OK;
 }
