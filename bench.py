@@ -398,6 +398,28 @@ def run_other_configs(args):
     del logits, grad, ws
     torch.cuda.empty_cache()
     out["cfg4_fused_lmhead"] = time_fused_lmhead(rlf, dev, 2, 0, cfg=4)
+    torch.cuda.empty_cache()
+
+    # cfg 4, fused path as the recipe words it: 8 calls of one 8192-token response each, the batch's
+    # token count as denominator, grad_W accumulated over the calls
+    H, W = synth.make_hidden_and_head(spec, T, dev)
+    ws = rlf.new_workspace(rlf.FN_FUSED_LMHEAD, mb, spec.V, spec.D, rlf.RLF_BF16, dev)
+    gh = torch.empty((T, spec.D), dtype=torch.bfloat16, device=dev)
+    gw = torch.empty((spec.V, spec.D), dtype=torch.float32, device=dev)
+    logp_all = torch.empty(T, dtype=torch.float32, device=dev)
+    old = torch.full((T,), -11.9, device=dev)
+
+    def fused_micro():
+        for i in range(T // mb):
+            sl = slice(i * mb, (i + 1) * mb)
+            rlf.rlf_fused_lmhead_grpo(H[sl], W, ids[sl], seq[sl], adv, old[sl], old[sl], mask[sl], synth.EPS_CLIP,
+                                      synth.BETA_KL, denom=n, grad_hidden=gh[sl], grad_W=gw, accumulate_grad_W=i > 0,
+                                      logp_out=logp_all[sl], loss_out=loss, workspace=ws)
+    ms = timed(fused_micro, 2)
+    live = int(mask.sum().item())
+    out["cfg4_fused_lmhead_8_microbatches"] = {
+        "T": T, "ms": ms, "tokens_per_s": T / ms * 1e3,
+        "executed_tflops": 2.0 * spec.V * spec.D * (T + 2 * live) / ms / 1e9}
     print(json.dumps({"other_configs": out, "gpu_launches": rlf.launch_count()}))
 
 

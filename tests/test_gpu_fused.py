@@ -148,6 +148,22 @@ def test_cfg3_full_size_sampled_rows_and_invariants():
     col = gw.double().sum(dim=0).abs().max().item()
     assert col <= 1e-3 * gw.double().abs().sum(dim=0).max().item()
 
+    # the same size without the masked rows: identical loss and gradients, NaN log-probs where masked
+    logp2, loss2, gh2, gw2 = b.rlf_fused_lmhead_grpo_obj(batch.hidden, batch.W, batch.ids, seq, adv, batch.old_logp,
+                                                         batch.ref_logp, mask, synth.EPS_CLIP, synth.EPS_CLIP,
+                                                         synth.BETA_KL, skip_masked=True, denom=n, dev_status=st)
+    # and the forward-only sweep over all rows in one launch
+    logp3, loss3, _, _ = b.rlf_fused_lmhead_grpo(batch.hidden, batch.W, batch.ids, seq, adv, batch.old_logp,
+                                                 batch.ref_logp, mask, synth.EPS_CLIP, synth.BETA_KL, denom=n,
+                                                 want_grad_hidden=False, want_grad_W=False, dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    livem = mask.bool()
+    assert torch.equal(gh, gh2) and torch.equal(gw, gw2) and torch.equal(loss, loss2)
+    assert torch.equal(logp[livem], logp2[livem]) and torch.isnan(logp2[~livem]).all()
+    assert (logp3 - logp).abs().max().item() <= 1e-4
+    assert loss_close(loss3[0].item(), want, 1e-6, gc.LOSS_RTOL)
+
 
 def test_cfg4_head_shape_reduced_T():
     """Qwen3-8B head (D = 4096 = 64 k-slabs, V = 151936) at 8 x 8 tokens, all outputs in full."""
