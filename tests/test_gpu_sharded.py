@@ -1,0 +1,84 @@
+"""The sharded single-batch step with the CUDA kernels on one GPU: the two ranks' shards are run one
+after the other (no kernel waits on another), the token counts are summed as the all-reduce would, and
+the parts must add up to the unsharded call: loss scalars, row gradients (bit-identical: a row's
+gradient depends on the row and the global count only) and the weight gradient."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2509_06980_b200 import sharded, synth
+import gpu_common as gc
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _shard_inputs(batch, responses, with_head):
+    tok = {"ids": batch.ids.cpu().numpy(), "old": batch.old_logp.cpu().numpy(), "ref": batch.ref_logp.cpu().numpy(),
+           "rows": np.arange(batch.T)}
+    cu, t, r = sharded.take_shard(responses, batch.cu_seqlens.cpu().numpy(), tok, {"rewards": batch.rewards.cpu().numpy()})
+    rows = torch.from_numpy(t["rows"]).to(DEV)
+    d = dict(ids=torch.from_numpy(t["ids"]).to(DEV), cu=torch.from_numpy(cu).to(DEV),
+             rewards=torch.from_numpy(r["rewards"]).to(DEV), old=torch.from_numpy(t["old"]).to(DEV),
+             ref=torch.from_numpy(t["ref"]).to(DEV), rows=rows)
+    if with_head:
+        d["hidden"] = batch.hidden[rows].contiguous()
+    else:
+        d["logits"] = batch.logits[rows].contiguous()
+    return d
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_logits_path_shards_add_up(world):
+    spec = synth.scaled(synth.SPECS[2], V=4096, num_prompts=4, group_size=4, len_lo=10, len_hi=80, spans_lo=1,
+                        spans_hi=2, cover_lo=0.2, cover_hi=0.5)
+    batch = synth.make_batch(spec, DEV)
+    full = sharded.sharded_grpo_step(batch.ids, batch.cu_seqlens, batch.rewards, spec.group_size, batch.old_logp,
+                                     batch.ref_logp, spec.open_id, spec.close_id, synth.EPS_CLIP, synth.BETA_KL,
+                                     logits=batch.logits)                      # world of one: no exchange
+    ref = gc.gpu_chain(batch, batch.logits)
+    assert torch.equal(full["loss"], ref["loss"]) and torch.equal(full["grad_logits"], ref["grad"])
+    plan = sharded.plan_shards(batch.cu_seqlens.cpu().numpy(), spec.group_size, world)
+    parts = [_shard_inputs(batch, p, False) for p in plan]
+    counted = [sharded.count_phase(p["ids"], p["cu"], spec.open_id, spec.close_id) for p in parts]
+    n_global = sum(c[2] for c in counted)                                       # what the all-reduce yields
+    assert n_global.item() == ref["n"].item()
+    loss = torch.zeros(4, dtype=torch.float64, device=DEV)
+    for p, (mask, seq, _) in zip(parts, counted):
+        o = sharded.loss_phase(n_global, mask, seq, p["ids"], p["rewards"], spec.group_size, p["old"], p["ref"],
+                               synth.EPS_CLIP, synth.BETA_KL, logits=p["logits"])
+        torch.cuda.synchronize()
+        loss += o["loss"]
+        assert torch.equal(o["grad_logits"], ref["grad"][p["rows"]])
+        assert torch.equal(o["logp"], ref["logp"][p["rows"]])
+        assert torch.equal(o["adv"], ref["adv"][torch.from_numpy(plan[parts.index(p)]).to(DEV)])
+    assert torch.allclose(loss, ref["loss"], rtol=1e-12, atol=1e-15)
+
+
+def test_fused_path_shards_add_up():
+    b = gc.binding()
+    spec = synth.scaled(synth.SPECS[3], V=4096 + 264, D=192, w_std=0.3, num_prompts=4, group_size=2, len_lo=24, len_hi=40,
+                        spans_lo=1, spans_hi=2, obs_lo=2, obs_hi=4)
+    batch = synth.make_batch(spec, DEV)
+    mask, seq, n = b.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, spec.open_id, spec.close_id)
+    adv = b.rlf_group_advantage(batch.rewards, group_size=spec.group_size)
+    lp, ls, gh, gw = b.rlf_fused_lmhead_grpo(batch.hidden, batch.W, batch.ids, seq, adv, batch.old_logp, batch.ref_logp,
+                                             mask, synth.EPS_CLIP, synth.BETA_KL, denom=n)
+    plan = sharded.plan_shards(batch.cu_seqlens.cpu().numpy(), spec.group_size, 2)
+    parts = [_shard_inputs(batch, p, True) for p in plan]
+    counted = [sharded.count_phase(p["ids"], p["cu"], spec.open_id, spec.close_id) for p in parts]
+    n_global = sum(c[2] for c in counted)
+    loss = torch.zeros(4, dtype=torch.float64, device=DEV)
+    gw_sum = torch.zeros_like(gw)
+    for p, (m, s, _) in zip(parts, counted):
+        o = sharded.loss_phase(n_global, m, s, p["ids"], p["rewards"], spec.group_size, p["old"], p["ref"], synth.EPS_CLIP,
+                               synth.BETA_KL, hidden=p["hidden"], W=batch.W)
+        torch.cuda.synchronize()
+        loss += o["loss"]
+        gw_sum += o["grad_W"]                                                    # the all-reduce's sum
+        # a row's log-prob and grad_hidden come out of other tiles than in the unsharded call: equal to rounding
+        assert (o["logp"] - lp[p["rows"]]).abs().max().item() <= 1e-5
+        scale = gh.float().abs().max().item()
+        assert (o["grad_hidden"].float() - gh[p["rows"]].float()).abs().max().item() <= 2.0 ** -7 * scale
+    assert torch.allclose(loss, ls, rtol=1e-6, atol=1e-12)
+    assert (gw_sum - gw).abs().max().item() <= 2.0 ** -7 * gw.abs().max().item()
