@@ -44,14 +44,14 @@ def test_logits_path_shards_add_up(world):
     n_global = sum(c[2] for c in counted)                                       # what the all-reduce yields
     assert n_global.item() == ref["n"].item()
     loss = torch.zeros(4, dtype=torch.float64, device=DEV)
-    for p, (mask, seq, _) in zip(parts, counted):
+    for k, (p, (mask, seq, _)) in enumerate(zip(parts, counted)):
         o = sharded.loss_phase(n_global, mask, seq, p["ids"], p["rewards"], spec.group_size, p["old"], p["ref"],
                                synth.EPS_CLIP, synth.BETA_KL, logits=p["logits"])
         torch.cuda.synchronize()
         loss += o["loss"]
         assert torch.equal(o["grad_logits"], ref["grad"][p["rows"]])
         assert torch.equal(o["logp"], ref["logp"][p["rows"]])
-        assert torch.equal(o["adv"], ref["adv"][torch.from_numpy(plan[parts.index(p)]).to(DEV)])
+        assert torch.equal(o["adv"], ref["adv"][torch.from_numpy(plan[k]).to(DEV)])
     assert torch.allclose(loss, ref["loss"], rtol=1e-12, atol=1e-15)
 
 
