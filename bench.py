@@ -159,6 +159,20 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3, responses=0
     return out
 
 
+# the same for the forward-only log-prob + entropy pass (profiles/logp_entropy_stream_kernel_T4096_ncu_full.md)
+NCU_TRAFFIC_ENTROPY = {"section_sha1": "cec2eff0a14f99f71358242b527710b41589d7d1", "dram_bytes_per_token": 307100.3}
+
+
+def _entropy_section_sha1():
+    """Hash of the forward-only section of logits_loss.cu (streaming and merge kernels, entry point)."""
+    p = os.path.join(ROOT, "paper_2509_06980_b200", "csrc", "logits_loss.cu")
+    with open(p, "rb") as f:
+        text = f.read()
+    a = text.find(b"// Forward-only log-prob (+ entropy) of given target ids")
+    b = text.find(b"// Skip-masked variant:")
+    return hashlib.sha1(text[a:b] if 0 <= a < b else text).hexdigest()
+
+
 def _kernel_sha1():
     """Hash of the row kernel's source text (from its section header to the general kernel's)."""
     p = os.path.join(ROOT, "paper_2509_06980_b200", "csrc", "logits_loss.cu")
@@ -558,7 +572,9 @@ def run_cuda(args):
         fwd_only = {"entry": "rlf_logp_entropy_fwd", "ms": fms, "tokens_per_s": T / fms * 1e3,
                     "roofline": {"bound": "hbm", "achieved": T * V * 2 / fms / 1e6, "peak": hbm_peak, "unit": "GB/s",
                                  "frac": T * V * 2 / fms / 1e6 / hbm_peak, "peak_kind": "of " + hbm_kind,
-                                 "traffic": None, "algorithmic_bytes": T * V * 2}}
+                                 "traffic": NCU_TRAFFIC_ENTROPY["dram_bytes_per_token"] * T
+                                 if NCU_TRAFFIC_ENTROPY["section_sha1"] == _entropy_section_sha1() else None,
+                                 "algorithmic_bytes": T * V * 2}}
 
     # skip-masked variant on the same batch: rows without loss weight are neither read nor computed
     skip_masked = None
