@@ -340,7 +340,7 @@ def run_fused_only(args):
     from paper_2509_06980_b200 import binding as rlf
     torch.cuda.set_device(0)
     out = time_fused_lmhead(rlf, torch.device("cuda", 0), max(1, args.steps), args.tokens_per_response,
-                            responses=args.responses)
+                            cfg=args.fused_cfg, responses=args.responses)
     print(json.dumps({"fused_lmhead": out, "gpu_launches": rlf.launch_count()}))
 
 
@@ -668,6 +668,8 @@ def main():
                     help="time cfg 2 (ragged, in place) and cfg 4 (micro-batched; both paths) instead (rank 0)")
     ap.add_argument("--tokens-per-response", type=int, default=0,
                     help="smaller micro-batch of the same recipe (profiling captures); 0 = the full 2048")
+    ap.add_argument("--fused-cfg", type=int, default=3, choices=[3, 4],
+                    help="with --fused-only: the Qwen3-4B head (3) or the Qwen3-8B head (4)")
     ap.add_argument("--responses", type=int, default=0,
                     help="with --fused-only: one group of this many full-length responses (profiling captures)")
     args = ap.parse_args()

@@ -374,12 +374,14 @@ rlf_status rlf_tune_logits_kernel(int cluster_ctas, int threads_per_cta, int one
  * Results are identical up to fp32 summation order. */
 rlf_status rlf_tune_lmhead(int pair_ctas);
 
-/* Scheduling block of the fused forward sweep for later calls in this process: the persistent CTAs
- * (or CTA pairs) that run at one time cover m_block row units (256 tokens in pair form) times as
- * many vocabulary splits as it takes to occupy them all.  0 restores the built-in choice (half the
- * number of CTA pairs).  Smaller blocks keep less of the hidden states in L2 at a time and stream
- * the head more often.  Results do not depend on it. */
-rlf_status rlf_tune_lmhead_schedule(int m_block);
+/* Scheduling of the fused contractions for later calls in this process.  m_block: the persistent
+ * CTAs (or CTA pairs) of the forward sweep that run at one time cover m_block row units (256 tokens
+ * in pair form) times as many vocabulary splits as it takes to occupy them all; smaller blocks keep
+ * less of the hidden states in L2 at a time and stream the head more often.  max_workers: upper
+ * bound on the persistent CTAs (pairs) of every contraction launch.  0 restores the built-in choice
+ * (m_block = half the number of workers; one worker per SM or pair of SMs).  Results do not depend
+ * on either. */
+rlf_status rlf_tune_lmhead_schedule(int m_block, int max_workers);
 
 /* Number of kernels this library has launched in this process (for accounting). */
 int64_t rlf_launch_count(void);

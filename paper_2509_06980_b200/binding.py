@@ -125,10 +125,10 @@ def tune_lmhead(pair_ctas=1):
     _check(_lib.rlf_tune_lmhead(int(pair_ctas)), "rlf_tune_lmhead")
 
 
-def tune_lmhead_schedule(m_block=0):
-    _lib.rlf_tune_lmhead_schedule.argtypes = [_int]
+def tune_lmhead_schedule(m_block=0, max_workers=0):
+    _lib.rlf_tune_lmhead_schedule.argtypes = [_int, _int]
     _lib.rlf_tune_lmhead_schedule.restype = _int
-    _check(_lib.rlf_tune_lmhead_schedule(int(m_block)), "rlf_tune_lmhead_schedule")
+    _check(_lib.rlf_tune_lmhead_schedule(int(m_block), int(max_workers)), "rlf_tune_lmhead_schedule")
 
 
 def rlf_build_loss_mask(ids, cu_seqlens, open_id, close_id, valid=None, mask_out=None, seq_id_out=None,

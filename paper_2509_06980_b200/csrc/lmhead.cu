@@ -788,6 +788,7 @@ static int sm_count_lm() {
 
 static std::atomic<int> g_pair{1};       // 1: cta_group::2 pair form, 0: single-CTA form
 static std::atomic<int> g_m_block{0};    // row units per scheduling block of the sweep; 0: automatic
+static std::atomic<int> g_max_workers{0};   // persistent CTAs (or pairs) per launch; 0: one per SM (pair of SMs)
 
 template <bool PAIR>
 static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, cudaStream_t s) {
@@ -815,6 +816,7 @@ static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, co
     // in lockstep.  Their token tiles (1.3 MB per pair at D = 2560) are re-read for every column tile
     // and must stay in L2 next to the streaming head: with all 74 pairs on different row units
     // (97 MB) they did not, and the same launch drew its 1 kW at 1.06 GHz instead of 1.39 GHz.
+    if (g_max_workers.load() > 0 && g_max_workers.load() < workers) workers = g_max_workers.load();
     GemmParams q = p;
     q.m_block = workers / 2 > 0 ? workers / 2 : 1;
     if (g_m_block.load() > 0) q.m_block = g_m_block.load();
@@ -1158,8 +1160,9 @@ extern "C" rlf_status rlf_tune_lmhead(int pair_ctas) {
     return RLF_OK;
 }
 
-extern "C" rlf_status rlf_tune_lmhead_schedule(int m_block) {
-    if (m_block < 0 || m_block > (1 << 20)) return RLF_ERR_SHAPE;
+extern "C" rlf_status rlf_tune_lmhead_schedule(int m_block, int max_workers) {
+    if (m_block < 0 || m_block > (1 << 20) || max_workers < 0) return RLF_ERR_SHAPE;
     rlf::lm::g_m_block = m_block;
+    rlf::lm::g_max_workers = max_workers;
     return RLF_OK;
 }
