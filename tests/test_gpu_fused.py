@@ -243,3 +243,40 @@ def test_fused_backward_runs_over_live_rows_only(n_live, form):
         if n_live:
             live = np.flatnonzero(mask_np)
             _close_tensor(gh.float().cpu().numpy()[live], r["grad_hidden"][live], "grad_hidden")
+
+
+def test_fused_malformed_rows_are_neutralised_and_reported():
+    """A target id outside the vocabulary or a response index outside [0, B) cannot be seen by the
+    host: the row gets weight 0 and a zero gradient, a status bit is set, every other row is
+    unaffected, and the denominator still counts the mask as given."""
+    b = gc.binding()
+    spec = synth.scaled(synth.SPECS[3], V=2048, D=128, w_std=0.3, **SMALL)
+    batch = synth.make_batch(spec, DEV)
+    mask, seq, n = b.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, spec.open_id, spec.close_id)
+    adv = b.rlf_group_advantage(batch.rewards, group_size=batch.tokens.group_size)
+    live = torch.nonzero(mask).flatten().cpu().numpy()
+    bad_id_rows, bad_seq_row = live[[3, 40]], live[77]
+    ids = batch.ids.clone()
+    ids[int(bad_id_rows[0])] = spec.V + 5
+    ids[int(bad_id_rows[1])] = -1
+    seq2 = seq.clone()
+    seq2[int(bad_seq_row)] = adv.shape[0]
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    logp, loss, gh, gw = b.rlf_fused_lmhead_grpo(batch.hidden, batch.W, ids, seq2, adv, batch.old_logp, batch.ref_logp,
+                                                 mask, synth.EPS_CLIP, synth.BETA_KL, denom=n, dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == (b.DEV_BAD_TARGET | b.DEV_BAD_SEQ)
+    bad = np.concatenate([bad_id_rows, [bad_seq_row]])
+    assert not gh[torch.as_tensor(bad, device=DEV)].any()
+    m2 = mask.cpu().numpy().copy()
+    m2[bad] = 0
+    ids_ok = batch.ids.cpu().numpy().copy()
+    seq_ok = seq.cpu().numpy()
+    r = orc.fused_lmhead_grpo(synth.bf16_bits(batch.hidden), synth.bf16_bits(batch.W), ids_ok, seq_ok,
+                              adv.cpu().numpy(), batch.old_logp.cpu().numpy(), batch.ref_logp.cpu().numpy(), m2,
+                              synth.EPS_CLIP, synth.BETA_KL, denom=int(n.item()))
+    good = np.setdiff1d(np.arange(len(ids_ok)), bad_id_rows)
+    assert np.abs(logp.cpu().numpy()[good] - r["logp"][good]).max() <= gc.LOGP_ATOL
+    assert loss_close(loss[0].item(), r["loss"][0], 1e-6, gc.LOSS_RTOL)
+    _close_tensor(gh.float().cpu().numpy(), r["grad_hidden"], "grad_hidden")
+    _close_tensor(gw.cpu().numpy(), r["grad_W"], "grad_W")
