@@ -568,8 +568,22 @@ def run_cuda(args):
             torch.cuda.synchronize()
             fe.append(a.elapsed_time(b))
         fms = statistics.mean(fe)
+        # log-prob alone (no entropy output): what the old / reference policy pass needs at the least
+        for _ in range(2):
+            rlf.rlf_logp_entropy_fwd(batch.logits, batch.ids, want_entropy=False, logp_out=logp, workspace=ws_ent)
+        torch.cuda.synchronize()
+        fl = []
+        for _ in range(max(3, min(args.steps, 10))):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            rlf.rlf_logp_entropy_fwd(batch.logits, batch.ids, want_entropy=False, logp_out=logp, workspace=ws_ent)
+            b.record()
+            torch.cuda.synchronize()
+            fl.append(a.elapsed_time(b))
+        lms = statistics.mean(fl)
         hbm_peak, hbm_kind = _peaks()
         fwd_only = {"entry": "rlf_logp_entropy_fwd", "ms": fms, "tokens_per_s": T / fms * 1e3,
+                    "logp_only": {"ms": lms, "gbs": T * V * 2 / lms / 1e6, "frac": T * V * 2 / lms / 1e6 / hbm_peak},
                     "roofline": {"bound": "hbm", "achieved": T * V * 2 / fms / 1e6, "peak": hbm_peak, "unit": "GB/s",
                                  "frac": T * V * 2 / fms / 1e6 / hbm_peak, "peak_kind": "of " + hbm_kind,
                                  "traffic": NCU_TRAFFIC_ENTROPY["dram_bytes_per_token"] * T
