@@ -139,6 +139,23 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3, responses=0
     if st.item() != 0:
         out["device_status"] = int(st.item())
     out["loss"] = float(loss[0].item())
+    # forward-only log-prob + entropy from hidden states (the old / reference policy pass)
+    ws_lp = rlf.new_workspace(rlf.FN_FUSED_LOGP_ENTROPY, T, spec.V, spec.D, rlf.RLF_BF16, dev)
+    ent = torch.empty(T, dtype=torch.float32, device=dev)
+    run_lp = lambda: rlf.rlf_fused_lmhead_logp_entropy(H, W, ids, logp_out=logp, entropy_out=ent, workspace=ws_lp)
+    run_lp()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        run_lp()
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    ms = statistics.mean(ts)
+    out["fwd_logp_entropy"] = {"entry": "rlf_fused_lmhead_logp_entropy", "ms": ms, "tokens_per_s": T / ms * 1e3,
+                               "executed_tflops": tvd * T / ms / 1e9}
     if not tokens_per_response and not responses:
         # context: the library GEMM of the forward's shape on this GPU, in the same state (back to back,
         # logits written to HBM as bf16): what an unfused path pays for the contraction alone

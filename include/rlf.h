@@ -60,6 +60,7 @@ typedef enum { RLF_BF16 = 0, RLF_F32 = 1 } rlf_dtype;
 #define RLF_FN_LOGP_LOSS 3
 #define RLF_FN_FUSED_LMHEAD 4
 #define RLF_FN_LOGP_ENTROPY 5
+#define RLF_FN_FUSED_LOGP_ENTROPY 6
 
 typedef struct CUstream_st *rlf_stream_t;
 
@@ -336,6 +337,24 @@ rlf_status rlf_fused_lmhead_grpo_obj(const void *hidden, const void *W, int64_t 
                                      void *workspace, size_t workspace_bytes, int32_t *dev_status,
                                      rlf_stream_t stream);
 
+/*
+ * Forward-only log-prob and entropy with the logits formed on the fly from the hidden states: the
+ * pass that produces old_logp / ref_logp (the behaviour and reference policies of the PPO-style
+ * update, paper Sec. 2.3.1; pi_theta of Sec. 2.2 is the language model's output head) without ever
+ * writing [T, V] logits.
+ *     z[t,:] = hidden[t,:] W^T;   logp[t] = z[t, ids[t]] - lse_t;   entropy[t] = lse_t - sum_v p_v z[t,v]
+ *   hidden [T, D] bf16, W [V, D] bf16 (16-byte aligned; D a multiple of 64, V of 8);  ids [T] int32
+ *   logp_out [T] fp32;  entropy_out [T] fp32 or NULL
+ *   workspace  rlf_workspace_bytes(RLF_FN_FUSED_LOGP_ENTROPY, T, 0, 0, RLF_BF16) bytes, 256-byte aligned
+ * An id outside [0, V) gives NaN log-prob (entropy is still produced) and RLF_DEV_BAD_TARGET; a
+ * non-finite row gives NaN and RLF_DEV_NONFINITE.  Same contraction kernel, waits and tuning knobs as
+ * rlf_fused_lmhead_grpo.  T = 0 is valid.
+ */
+rlf_status rlf_fused_lmhead_logp_entropy(const void *hidden, const void *W, int64_t T, int32_t D, int32_t V,
+                                         const int32_t *ids, float *logp_out, float *entropy_out,
+                                         void *workspace, size_t workspace_bytes, int32_t *dev_status,
+                                         rlf_stream_t stream);
+
 /* Bytes of workspace the given entry point needs for these sizes (0 for unknown selectors). */
 size_t rlf_workspace_bytes(int which_fn, int64_t T, int32_t V, int32_t D, rlf_dtype dt);
 
@@ -378,10 +397,12 @@ rlf_status rlf_tune_lmhead(int pair_ctas);
  * CTAs (or CTA pairs) of the forward sweep that run at one time cover m_block row units (256 tokens
  * in pair form) times as many vocabulary splits as it takes to occupy them all; smaller blocks keep
  * less of the hidden states in L2 at a time and stream the head more often.  max_workers: upper
- * bound on the persistent CTAs (pairs) of every contraction launch.  0 restores the built-in choice
- * (m_block = half the number of workers; one worker per SM or pair of SMs).  Results do not depend
- * on either. */
-rlf_status rlf_tune_lmhead_schedule(int m_block, int max_workers);
+ * bound on the persistent CTAs (pairs) of every contraction launch.  chunk_tiles: 128-token tiles
+ * per chunk of the backward (even; at most the 148 the workspace is sized for).  0 restores the
+ * built-in choice (m_block = half the number of workers; one worker per SM or pair of SMs; 148
+ * tiles).  Results do not depend on m_block or max_workers; the chunk size changes the order in
+ * which grad_W is accumulated (fp32 rounding only). */
+rlf_status rlf_tune_lmhead_schedule(int m_block, int max_workers, int chunk_tiles);
 
 /* Number of kernels this library has launched in this process (for accounting). */
 int64_t rlf_launch_count(void);

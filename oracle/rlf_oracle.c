@@ -487,6 +487,21 @@ int orc_logp_entropy(const void *logits, int dtype, int64_t T, int32_t V, int64_
     return bad ? -2 : 0;
 }
 
+/*
+ * Forward-only log-prob and entropy with the logits formed from the head: z = H W^T in fp64
+ * (head_logits), then exactly orc_logp_entropy on them.  entropy_out may be NULL.
+ */
+int orc_fused_lmhead_logp_entropy(const uint16_t *hidden, const uint16_t *W, int64_t T, int32_t D, int32_t V,
+                                  const int32_t *ids, double *logp_out, double *entropy_out)
+{
+    double *z = (double *)malloc(sizeof(double) * (size_t)(T > 0 ? T : 1) * (size_t)V);
+    if (!z) return -7;
+    head_logits(hidden, W, T, D, V, z);
+    int rc = orc_logp_entropy(z, ORC_F64, T, V, V, ids, logp_out, entropy_out);
+    free(z);
+    return rc;
+}
+
 /* Rule reward, Eq. 1: R = sum_i w_i r_i over n rule scores, for each of B responses.
  * scores is [B, n] row-major. */
 int orc_rule_reward(const float *scores, const float *weights, int32_t B, int32_t n, double *R)

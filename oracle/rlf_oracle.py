@@ -253,3 +253,19 @@ def fused_lmhead_grpo_obj(hidden, W, ids, seq_id, adv, old_logp, ref_logp, mask,
                                          _p(gh), _p(gw))
     _check(rc, "fused_lmhead_grpo_obj")
     return dict(logp=logp, loss=loss, grad_hidden=gh, grad_W=gw)
+
+
+def fused_lmhead_logp_entropy(hidden, W, ids, want_entropy=True):
+    """hidden [T,D], W [V,D]: bf16 bit patterns -> (logp f64[T], entropy f64[T] | None)."""
+    hidden = _c(hidden, np.uint16)
+    W = _c(W, np.uint16)
+    T, D = hidden.shape
+    V = W.shape[0]
+    assert W.shape[1] == D
+    ids = _c(ids, np.int32)
+    logp = np.zeros(T, np.float64)
+    ent = np.zeros(T, np.float64) if want_entropy else None
+    rc = lib().orc_fused_lmhead_logp_entropy(_p(hidden), _p(W), ctypes.c_int64(T), ctypes.c_int32(D),
+                                             ctypes.c_int32(V), _p(ids), _p(logp), _p(ent))
+    _check(rc, "fused_lmhead_logp_entropy")
+    return logp, ent

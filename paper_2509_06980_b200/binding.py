@@ -14,12 +14,12 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "librlf.so")
 
 RLF_BF16, RLF_F32 = 0, 1
-FN_LOGP_LOSS, FN_FUSED_LMHEAD, FN_LOGP_ENTROPY = 3, 4, 5
+FN_LOGP_LOSS, FN_FUSED_LMHEAD, FN_LOGP_ENTROPY, FN_FUSED_LOGP_ENTROPY = 3, 4, 5, 6
 DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
 
 EXPORTS = [
     "rlf_build_loss_mask", "rlf_group_advantage", "rlf_rule_reward", "rlf_kl_in_reward", "rlf_grpo_logp_loss_fwd_bwd",
-    "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_grpo_logp_loss_fwd_bwd_skip_masked", "rlf_grpo_logp_loss_fwd_bwd_obj", "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_fused_lmhead_grpo_obj", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
+    "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_grpo_logp_loss_fwd_bwd_skip_masked", "rlf_grpo_logp_loss_fwd_bwd_obj", "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_fused_lmhead_grpo_obj", "rlf_fused_lmhead_logp_entropy", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
     "rlf_tune_logits_kernel", "rlf_tune_lmhead", "rlf_tune_lmhead_schedule", "rlf_launch_count", "rlf_status_string", "rlf_version",
 ]
 
@@ -125,10 +125,11 @@ def tune_lmhead(pair_ctas=1):
     _check(_lib.rlf_tune_lmhead(int(pair_ctas)), "rlf_tune_lmhead")
 
 
-def tune_lmhead_schedule(m_block=0, max_workers=0):
-    _lib.rlf_tune_lmhead_schedule.argtypes = [_int, _int]
+def tune_lmhead_schedule(m_block=0, max_workers=0, chunk_tiles=0):
+    _lib.rlf_tune_lmhead_schedule.argtypes = [_int, _int, _int]
     _lib.rlf_tune_lmhead_schedule.restype = _int
-    _check(_lib.rlf_tune_lmhead_schedule(int(m_block), int(max_workers)), "rlf_tune_lmhead_schedule")
+    _check(_lib.rlf_tune_lmhead_schedule(int(m_block), int(max_workers), int(chunk_tiles)),
+           "rlf_tune_lmhead_schedule")
 
 
 def rlf_build_loss_mask(ids, cu_seqlens, open_id, close_id, valid=None, mask_out=None, seq_id_out=None,
@@ -396,6 +397,27 @@ def rlf_fused_lmhead_grpo_obj(hidden, W, ids, seq_id, adv, old_logp, ref_logp, m
         _ptr(grad_W, torch.float32), 1 if accumulate_grad_W else 0, workspace.data_ptr(), workspace.numel(),
         _ptr(dev_status, torch.int32), _stream()), "rlf_fused_lmhead_grpo_obj")
     return logp_out, loss_out, grad_hidden, grad_W
+
+
+def rlf_fused_lmhead_logp_entropy(hidden, W, ids, want_entropy=True, logp_out=None, entropy_out=None,
+                                  workspace=None, dev_status=None):
+    """Forward only, from hidden states: -> (logp fp32[T], entropy fp32[T] | None); logits are never stored."""
+    T, D = hidden.shape
+    V = W.shape[0]
+    dev = hidden.device
+    if logp_out is None:
+        logp_out = torch.empty(T, dtype=torch.float32, device=dev)
+    if entropy_out is None and want_entropy:
+        entropy_out = torch.empty(T, dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = new_workspace(FN_FUSED_LOGP_ENTROPY, T, V, D, RLF_BF16, dev)
+    _lib.rlf_fused_lmhead_logp_entropy.argtypes = [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+    _lib.rlf_fused_lmhead_logp_entropy.restype = _int
+    _check(_lib.rlf_fused_lmhead_logp_entropy(
+        _ptr(hidden, torch.bfloat16) if T > 0 else None, _ptr(W, torch.bfloat16), T, D, V, _ptr(ids, torch.int32),
+        _ptr(logp_out, torch.float32), _ptr(entropy_out, torch.float32), workspace.data_ptr(), workspace.numel(),
+        _ptr(dev_status, torch.int32), _stream()), "rlf_fused_lmhead_logp_entropy")
+    return logp_out, entropy_out
 
 
 def step_arena_bytes(T, V, B, dt=RLF_BF16):

@@ -28,6 +28,7 @@ rlf_status check_arch() {
 size_t loss_workspace_bytes(int64_t T);                          // logits_loss.cu
 size_t lmhead_workspace_bytes(int64_t T, int32_t V, int32_t D);  // lmhead.cu
 size_t entropy_workspace_bytes(int64_t T, int32_t V);             // logits_loss.cu
+size_t lmhead_logp_workspace_bytes(int64_t T);                    // lmhead.cu
 
 static size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
 
@@ -83,6 +84,7 @@ extern "C" size_t rlf_workspace_bytes(int which_fn, int64_t T, int32_t V, int32_
     if (which_fn == RLF_FN_LOGP_LOSS) return rlf::loss_workspace_bytes(T);
     if (which_fn == RLF_FN_FUSED_LMHEAD) return rlf::lmhead_workspace_bytes(T, V, D);
     if (which_fn == RLF_FN_LOGP_ENTROPY) return rlf::entropy_workspace_bytes(T, V);
+    if (which_fn == RLF_FN_FUSED_LOGP_ENTROPY) return rlf::lmhead_logp_workspace_bytes(T);
     return 0;
 }
 

@@ -57,6 +57,7 @@ struct GemmParams {
     int nsplit, n_tiles_per_split;
     int m_block;              // kLse: row units per scheduling block
     float2* part;             // kLse: [M][nsplit] (max, sum exp)
+    float* part_u;            // kLse (optional): [M][nsplit] sum of 2^x x, x the base-2 exponent against that max
     __nv_bfloat16* dz;        // kLse (optional) out, row stride dz_stride: exp(z - tile max) as bf16
     float* tmax;              // kLse with dz: [M][n_tiles] the tile maxima those exponentials refer to
     long long dz_stride;
@@ -363,6 +364,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const int row = (PAIR ? 2 * m + rank : m) * BM + row_in_tile;
             const bool row_ok = row < M;
             float run_m = -INFINITY, run_s = 0.0f;       // kLse
+            float run_u = 0.0f;                          // kLse with entropy: sum of 2^x x against run_m
             for (int n = n0; n < n1 && ok; ++n) {
                 if (!no_k) {
                     // one lane polls for the warp (128 polling threads would only burn issue slots and
@@ -452,15 +454,38 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         for (int i = 0; i < 32; ++i)
                             if (i < nvalid) cm = fmaxf(cm, __uint_as_float(v[i]));
                         if (cm > run_m) {
-                            run_s *= ex2_approx((run_m - cm) * kLog2e);   // exp2(-inf) = 0 on the first chunk
+                            // a larger maximum shifts every exponent so far by dx <= 0:
+                            // s -> 2^dx s,  u -> 2^dx (u + dx s)
+                            const float dx = (run_m - cm) * kLog2e;       // -inf on the first chunk
+                            const float f = ex2_approx(dx);               // exp2(-inf) = 0 on the first chunk
+                            if (p.part_u) run_u = (run_m == -INFINITY) ? 0.0f : f * fmaf(dx, run_s, run_u);
+                            run_s *= f;
                             run_m = cm;
                         }
                         const float off = -run_m * kLog2e;
                         float s0 = 0.0f, s1 = 0.0f;
+                        if (p.part_u) {
+                            float u0 = 0.0f, u1 = 0.0f;
 #pragma unroll
-                        for (int i = 0; i < 32; i += 2) {
-                            if (i < nvalid) s0 += ex2_approx(fmaf(__uint_as_float(v[i]), kLog2e, off));
-                            if (i + 1 < nvalid) s1 += ex2_approx(fmaf(__uint_as_float(v[i + 1]), kLog2e, off));
+                            for (int i = 0; i < 32; i += 2) {
+                                if (i < nvalid) {
+                                    const float x = fmaf(__uint_as_float(v[i]), kLog2e, off), e = ex2_approx(x);
+                                    s0 += e;
+                                    u0 = fmaf(e, x, u0);
+                                }
+                                if (i + 1 < nvalid) {
+                                    const float x = fmaf(__uint_as_float(v[i + 1]), kLog2e, off), e = ex2_approx(x);
+                                    s1 += e;
+                                    u1 = fmaf(e, x, u1);
+                                }
+                            }
+                            run_u += u0 + u1;
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 2) {
+                                if (i < nvalid) s0 += ex2_approx(fmaf(__uint_as_float(v[i]), kLog2e, off));
+                                if (i + 1 < nvalid) s1 += ex2_approx(fmaf(__uint_as_float(v[i + 1]), kLog2e, off));
+                            }
                         }
                         run_s += s0 + s1;
                     } else if (p.mode == kGradHidden) {
@@ -517,6 +542,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             if (p.mode == kLse && row_ok && ok) {
                 const int sp = n0 / p.n_tiles_per_split;
                 p.part[(long long)row * p.nsplit + sp] = make_float2(run_m, run_s);
+                if (p.part_u) p.part_u[(long long)row * p.nsplit + sp] = run_u;
             }
         }
     }
@@ -597,6 +623,67 @@ combine_kernel(const float2* __restrict__ part, int nsplit, const float* __restr
     logp_out[t] = finite ? logp : __int_as_float(0x7fc00000);
     lse_out[t] = finite ? lse : 0.0f;
     coef_out[t] = coef;
+    if (!finite && dev_status) atomicOr(dev_status, RLF_DEV_NONFINITE);
+}
+
+// forward-only pass from target ids alone: z_target per token (NaN and a status bit for an id outside
+// the vocabulary), one warp per token
+__global__ void __launch_bounds__(256)
+target_logit_ids_kernel(const __nv_bfloat16* __restrict__ hidden, const __nv_bfloat16* __restrict__ W,
+                        const int32_t* __restrict__ ids, int64_t T, int32_t D, int32_t V, float* __restrict__ zy,
+                        int32_t* __restrict__ dev_status) {
+    const int64_t t = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (t >= T) return;
+    const int lane = threadIdx.x & 31;
+    const int y = ids[t];
+    if (y < 0 || y >= V) {
+        if (lane == 0) {
+            zy[t] = __int_as_float(0x7fc00000);
+            if (dev_status) atomicOr(dev_status, RLF_DEV_BAD_TARGET);
+        }
+        return;
+    }
+    const uint4* h = reinterpret_cast<const uint4*>(hidden + t * (int64_t)D);
+    const uint4* w = reinterpret_cast<const uint4*>(W + (int64_t)y * D);
+    float acc = 0.0f;
+    for (int i = lane; i < D / 8; i += 32) {
+        const uint4 a = h[i], b = w[i];
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            acc = fmaf(__uint_as_float(aw[k] << 16), __uint_as_float(bw[k] << 16), acc);
+            acc = fmaf(__uint_as_float(aw[k] & 0xffff0000u), __uint_as_float(bw[k] & 0xffff0000u), acc);
+        }
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) zy[t] = acc;
+}
+
+// merge the per-split (max, s, u) triples of every token: logp = z_y - lse, H = ln S - ln2 U / S with
+// S = sum_k s_k 2^dx_k, U = sum_k 2^dx_k (u_k + s_k dx_k), dx_k the split's base against the row maximum
+__global__ void __launch_bounds__(256)
+combine_logp_entropy_kernel(const float2* __restrict__ part, const float* __restrict__ part_u, int nsplit,
+                            const float* __restrict__ zy, int64_t T, float* __restrict__ logp_out,
+                            float* __restrict__ entropy_out, int32_t* __restrict__ dev_status) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    float M = -INFINITY;
+    for (int j = 0; j < nsplit; ++j) M = fmaxf(M, part[t * nsplit + j].x);
+    float S = 0.0f, U = 0.0f;
+    for (int j = 0; j < nsplit; ++j) {
+        const float2 ms = part[t * nsplit + j];
+        if (ms.x == -INFINITY) continue;
+        const float dx = (ms.x - M) * kLog2e;
+        const float f = exp2f(dx);
+        S += ms.y * f;
+        if (part_u && f > 0.0f) U += f * fmaf(ms.y, dx, part_u[t * nsplit + j]);
+    }
+    const float lnS = logf(S);
+    const float logp = (zy[t] - M) - lnS;
+    const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY);
+    const float nan = __int_as_float(0x7fc00000);
+    logp_out[t] = (finite && fabsf(logp) < INFINITY) ? logp : nan;      // NaN z_y (bad target id) stays NaN
+    if (entropy_out) entropy_out[t] = finite ? lnS - kLn2 * U / S : nan;
     if (!finite && dev_status) atomicOr(dev_status, RLF_DEV_NONFINITE);
 }
 
@@ -789,6 +876,7 @@ static int sm_count_lm() {
 static std::atomic<int> g_pair{1};       // 1: cta_group::2 pair form, 0: single-CTA form
 static std::atomic<int> g_m_block{0};    // row units per scheduling block of the sweep; 0: automatic
 static std::atomic<int> g_max_workers{0};   // persistent CTAs (or pairs) per launch; 0: one per SM (pair of SMs)
+static std::atomic<int> g_chunk_tiles{0};   // token tiles per backward chunk; 0: the most the workspace holds
 
 template <bool PAIR>
 static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, cudaStream_t s) {
@@ -898,6 +986,11 @@ static LmWs lm_workspace(int64_t T, int32_t V, int32_t D) {
 }
 
 }  // namespace lm
+
+size_t lmhead_logp_workspace_bytes(int64_t T) {
+    const size_t Tn = (size_t)(T > 0 ? T : 0);
+    return 1024 + lm::up1k(4 * Tn) + lm::up1k(8 * Tn * lm::kMaxSplit) + lm::up1k(4 * Tn * lm::kMaxSplit) + 1024;
+}
 
 size_t lmhead_workspace_bytes(int64_t T, int32_t V, int32_t D) {
     if (V < 1 || D < 1) return 0;
@@ -1031,8 +1124,10 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
     if (grad_hidden && cudaMemsetAsync(grad_hidden, 0, (size_t)T * D * 2, s) != cudaSuccess) return RLF_ERR_CUDA;
 
     const bool bwd = grad_hidden || grad_W;
-    for (int64_t t0 = 0; t0 < T; t0 += kChunkTokens) {
-        const int64_t tc = (T - t0) < kChunkTokens ? (T - t0) : kChunkTokens;
+    const int tuned_tiles = g_chunk_tiles.load();
+    const int64_t chunk_tokens = (tuned_tiles > 0 && tuned_tiles * BM < kChunkTokens) ? tuned_tiles * BM : kChunkTokens;
+    for (int64_t t0 = 0; t0 < T; t0 += chunk_tokens) {
+        const int64_t tc = (T - t0) < chunk_tokens ? (T - t0) : chunk_tokens;
         CUtensorMap mapHc;
         if (!make_map(&mapHc, Hl + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
         GemmParams z = g;
@@ -1154,15 +1249,66 @@ extern "C" rlf_status rlf_fused_lmhead_grpo_obj(const void* hidden, const void* 
 }
 
 
+extern "C" rlf_status rlf_fused_lmhead_logp_entropy(const void* hidden, const void* W, int64_t T, int32_t D, int32_t V,
+                                                    const int32_t* ids, float* logp_out, float* entropy_out,
+                                                    void* workspace, size_t workspace_bytes, int32_t* dev_status,
+                                                    rlf_stream_t stream) {
+    using namespace rlf;
+    using namespace rlf::lm;
+    if (T < 0 || V < 1 || D < 1) return RLF_ERR_SHAPE;
+    if (D % 64 != 0 || V % 8 != 0) return RLF_ERR_SHAPE;
+    if (T >= (1ll << 30)) return RLF_ERR_UNSUPPORTED;
+    if (T == 0) return RLF_OK;
+    if (!hidden || !W || !ids || !logp_out) return RLF_ERR_NULL;
+    if (!aligned(hidden, 16) || !aligned(W, 16)) return RLF_ERR_ALIGN;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < lmhead_logp_workspace_bytes(T))
+        return RLF_ERR_WORKSPACE;
+    rlf_status st = check_arch();
+    if (st != RLF_OK) return st;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    char* ws = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(workspace) + 1023) & ~(uintptr_t)1023);
+    float* zy = reinterpret_cast<float*>(ws);
+    float2* part = reinterpret_cast<float2*>(ws + up1k(4 * (size_t)T));
+    float* part_u = reinterpret_cast<float*>(ws + up1k(4 * (size_t)T) + up1k(8 * (size_t)T * kMaxSplit));
+    const __nv_bfloat16* H = static_cast<const __nv_bfloat16*>(hidden);
+    const __nv_bfloat16* Wm = static_cast<const __nv_bfloat16*>(W);
+    target_logit_ids_kernel<<<(unsigned)((T + 7) / 8), 256, 0, s>>>(H, Wm, ids, T, D, V, zy, dev_status);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+    const bool pair = g_pair.load() != 0;
+    CUtensorMap mapH, mapW;
+    if (!make_map(&mapH, H, (uint64_t)T, (uint64_t)D, (uint64_t)D, BK, BM)) return RLF_ERR_CUDA;
+    if (!make_map(&mapW, Wm, (uint64_t)V, (uint64_t)D, (uint64_t)D, BK, pair ? BN / 2 : BN)) return RLF_ERR_CUDA;
+    GemmParams g = {};
+    g.mode = kLse;
+    g.M = (int)T;
+    g.N = V;
+    g.m_tiles = (int)((T + BM - 1) / BM);
+    g.n_tiles = (V + BN - 1) / BN;
+    g.k_slabs = D / BK;
+    g.nsplit = pick_split(g.n_tiles);
+    g.n_tiles_per_split = (g.n_tiles + g.nsplit - 1) / g.nsplit;
+    g.part = part;
+    g.part_u = entropy_out ? part_u : nullptr;
+    g.dev_status = dev_status;
+    st = launch_gemm(mapH, mapW, g, pair, s);
+    if (st != RLF_OK) return st;
+    combine_logp_entropy_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(part, g.part_u, g.nsplit, zy, T, logp_out,
+                                                                             entropy_out, dev_status);
+    count_launch();
+    return cuda_ok(cudaGetLastError());
+}
+
 extern "C" rlf_status rlf_tune_lmhead(int pair_ctas) {
     if (pair_ctas != 0 && pair_ctas != 1) return RLF_ERR_SHAPE;
     rlf::lm::g_pair = pair_ctas;
     return RLF_OK;
 }
 
-extern "C" rlf_status rlf_tune_lmhead_schedule(int m_block, int max_workers) {
-    if (m_block < 0 || m_block > (1 << 20) || max_workers < 0) return RLF_ERR_SHAPE;
+extern "C" rlf_status rlf_tune_lmhead_schedule(int m_block, int max_workers, int chunk_tiles) {
+    if (m_block < 0 || m_block > (1 << 20) || max_workers < 0 || chunk_tiles < 0 || (chunk_tiles & 1)) return RLF_ERR_SHAPE;
     rlf::lm::g_m_block = m_block;
     rlf::lm::g_max_workers = max_workers;
+    rlf::lm::g_chunk_tiles = chunk_tiles;
     return RLF_OK;
 }

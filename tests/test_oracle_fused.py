@@ -130,3 +130,25 @@ def test_objective_variant_of_the_head_matches_torch_autograd_fp64():
     assert abs(r["loss"][0] - L.item()) < 1e-13
     assert np.abs(r["grad_hidden"] - Ht.grad.numpy()).max() < 1e-14
     assert np.abs(r["grad_W"] - Wt.grad.numpy()).max() < 1e-14
+
+
+def test_forward_only_head_log_prob_and_entropy():
+    import math
+    Hb, H, Wb, W, ids, seq, adv, old, ref, mask = _problem(6, T=9, D=6, V=13)
+    logp, ent = orc.fused_lmhead_logp_entropy(Hb, Wb, ids)
+    # composition with the logits-path function on numpy's fp64 contraction
+    lp2, ent2 = orc.logp_entropy(H @ W.T, ids)
+    assert np.allclose(logp, lp2, atol=1e-13) and np.allclose(ent, ent2, atol=1e-13)
+    # fp64 torch
+    z = torch.tensor(H) @ torch.tensor(W).t()
+    ls = torch.log_softmax(z, -1)
+    assert np.allclose(logp, ls.gather(1, torch.tensor(ids, dtype=torch.int64)[:, None])[:, 0].numpy(), atol=1e-13)
+    assert np.allclose(ent, -(ls.exp() * ls).sum(-1).numpy(), atol=1e-13)
+    # a zero head gives the uniform distribution: log-prob -ln V, entropy ln V, whatever the hidden states
+    Zb, _ = _bf16(np.zeros((13, 6)))
+    logp0, ent0 = orc.fused_lmhead_logp_entropy(Hb, Zb, ids)
+    assert np.allclose(logp0, -math.log(13), atol=1e-15) and np.allclose(ent0, math.log(13), atol=1e-15)
+    # agreement with the training path's log-prob
+    r = orc.fused_lmhead_grpo(Hb, Wb, ids, seq, adv, old, ref, mask, 0.2, 0.05, want_grad_hidden=False, want_grad_W=False)
+    assert np.allclose(r["logp"], logp, atol=1e-13)
+    assert orc.fused_lmhead_logp_entropy(Hb, Wb, ids, want_entropy=False)[1] is None
