@@ -96,11 +96,23 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3, responses=0
     live = int(mask.sum().item())
     out["live_rows"] = live
     tvd = 2.0 * spec.V * spec.D
+    # Tensor-core work is power-bound here: a kernel timed in the first second after an idle spell runs
+    # at clocks it cannot hold.  Every variant is therefore looped for warm_s seconds before it is timed
+    # (profiling captures at reduced size skip this: they take their figures from the counters).
+    warm_s = 0.0 if (tokens_per_response or responses) else 1.5
+
+    def warm(fn):
+        fn()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        while time.perf_counter() - t0 < warm_s:
+            for _ in range(4):
+                fn()
+            torch.cuda.synchronize()
+
     for name, bwd, useful_flops, executed_flops in (("fwd", False, tvd * T, tvd * T),
                                                     ("fwd_bwd", True, tvd * (T + 2 * live), tvd * (T + 2 * live))):
-        for _ in range(1 if (tokens_per_response or responses) else 2):
-            run(bwd)
-        torch.cuda.synchronize()
+        warm(lambda: run(bwd))
         ts = []
         for _ in range(steps):
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -123,8 +135,7 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3, responses=0
         rlf.rlf_fused_lmhead_grpo_obj(H, W, ids, seq, adv, old, ref, mask, synth.EPS_CLIP, synth.EPS_CLIP,
                                       synth.BETA_KL, skip_masked=True, denom=n, grad_hidden=gh, grad_W=gw,
                                       logp_out=logp, loss_out=loss, workspace=ws, dev_status=st)
-    run_skip()
-    torch.cuda.synchronize()
+    warm(run_skip)
     ts = []
     for _ in range(steps):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -143,8 +154,7 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3, responses=0
     ws_lp = rlf.new_workspace(rlf.FN_FUSED_LOGP_ENTROPY, T, spec.V, spec.D, rlf.RLF_BF16, dev)
     ent = torch.empty(T, dtype=torch.float32, device=dev)
     run_lp = lambda: rlf.rlf_fused_lmhead_logp_entropy(H, W, ids, logp_out=logp, entropy_out=ent, workspace=ws_lp)
-    run_lp()
-    torch.cuda.synchronize()
+    warm(run_lp)
     ts = []
     for _ in range(steps):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -160,9 +170,7 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3, responses=0
         # context: the library GEMM of the forward's shape on this GPU, in the same state (back to back,
         # logits written to HBM as bf16): what an unfused path pays for the contraction alone
         z = torch.empty((T, spec.V), dtype=torch.bfloat16, device=dev)
-        for _ in range(2):
-            torch.matmul(H, W.t(), out=z)
-        torch.cuda.synchronize()
+        warm(lambda: torch.matmul(H, W.t(), out=z))
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         for _ in range(steps):

@@ -294,8 +294,8 @@ rlf_status rlf_grpo_logp_loss_fwd_bwd_static(const void *logits, rlf_dtype dt, i
  *   grad_hidden [T, D] bf16 or NULL;  grad_W [V, D] fp32 or NULL (both NULL: forward only)
  *   workspace   rlf_workspace_bytes(RLF_FN_FUSED_LMHEAD, T, V, D, RLF_BF16) bytes, 256-byte aligned.
  *               It holds per-token records and partial sums and, for the backward, a copy of hidden
- *               with the unmasked rows gathered first, and one chunk [min(T, 18944), V] of bf16
- *               (5.8 GB at V = 151936): the forward sweep of a chunk of unmasked rows leaves
+ *               with the unmasked rows gathered first, and one chunk [min(T, 9472), V] of bf16
+ *               (2.9 GB at V = 151936): the forward sweep of a chunk of unmasked rows leaves
  *               exp(z - max of the 256-column tile) there (never above 1, so no logit overflows
  *               it), an elementwise pass rescales it in place into dZ = grad_z once the row's
  *               log-sum-exp is known, and the two gradient contractions consume it.  The logits
@@ -398,8 +398,8 @@ rlf_status rlf_tune_lmhead(int pair_ctas);
  * in pair form) times as many vocabulary splits as it takes to occupy them all; smaller blocks keep
  * less of the hidden states in L2 at a time and stream the head more often.  max_workers: upper
  * bound on the persistent CTAs (pairs) of every contraction launch.  chunk_tiles: 128-token tiles
- * per chunk of the backward (even; at most the 148 the workspace is sized for).  0 restores the
- * built-in choice (m_block = half the number of workers; one worker per SM or pair of SMs; 148
+ * per chunk of the backward (even; at most the 74 the workspace is sized for).  0 restores the
+ * built-in choice (m_block = half the number of workers; one worker per SM or pair of SMs; 74
  * tiles).  Results do not depend on m_block or max_workers; the chunk size changes the order in
  * which grad_W is accumulated (fp32 rounding only). */
 rlf_status rlf_tune_lmhead_schedule(int m_block, int max_workers, int chunk_tiles);

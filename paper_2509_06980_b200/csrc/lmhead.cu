@@ -934,11 +934,12 @@ static rlf_status launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, cons
     return pair ? launch_gemm_t<true>(ma, mb, p, s) : launch_gemm_t<false>(ma, mb, p, s);
 }
 
-// rows of dZ held in scratch at a time: 148 token tiles = 74 pair units (two scheduling blocks of the
-// sweep; 74 x D/256 whole waves of the grad_hidden contraction on 74 CTA pairs).  Fewer, larger chunks
-// stream the head fewer times and accumulate into grad_W fewer times: 9472 -> 18944 rows took the
-// Qwen3-4B-head step from 47 to 43 ms; the scratch is 5.8 GB at V = 151936.
-constexpr int kChunkTokens = 148 * BM;
+// rows of dZ held in scratch at a time: 74 token tiles = 37 pair units (one scheduling block of the
+// sweep; 37 x D/256 whole waves of the grad_hidden contraction on 74 CTA pairs); 2.9 GB at
+// V = 151936.  Twice the chunk halves the passes over the head and the accumulations into grad_W, but
+// measured under sustained load (3 s loops at the power cap) it is slower: 48.6 against 46.8 ms for
+// the Qwen3-4B-head step, at 1.16 against 1.25 GHz.
+constexpr int kChunkTokens = 74 * BM;
 constexpr int kMaxSplit = 64;               // most vocabulary splits a sweep may use (sizes the partials)
 
 // Number of vocabulary splits of a sweep.  A work unit is (pair of token tiles, split); the units are
