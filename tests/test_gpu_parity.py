@@ -146,7 +146,10 @@ def test_extreme_logits_and_targets_at_the_ends():
 def test_bad_rows_are_neutralised_and_flagged():
     b = gc.binding()
     V, T = 1024, 5
-    z = (torch.randn((T, V), device=DEV) * 2).to(torch.bfloat16)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(12)
+    z = (torch.randn((T, V), device=DEV, generator=g) * 2).to(torch.bfloat16)
+    z[0, 3] = 0.0                      # row 0's ratio stays below the clip bound: its gradient is non-zero
     z[3, 10] = float("inf")
     z[4, :] = float("-inf")
     ids = torch.tensor([3, -1, V, 4, 4], dtype=torch.int32, device=DEV)
