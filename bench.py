@@ -644,6 +644,26 @@ def run_cuda(args):
                                                                "algorithmic_bytes": moved, "gbs": moved / sms / 1e6}
         del g2
 
+    # context for the roofline fraction: the same STREAM-style copy that produced the recorded peak,
+    # taken on this GPU in this run (GPUs of one pool differ by a few per cent)
+    copy_gbs = None
+    if rank == 0 and world == 1 and not args.tokens_per_response:
+        src = torch.empty(1 << 30, dtype=torch.bfloat16, device=dev)
+        dst = torch.empty_like(src)
+        src.zero_()
+        best = None
+        for i in range(12):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            dst.copy_(src)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 2:
+                best = a.elapsed_time(b) if best is None else min(best, a.elapsed_time(b))
+        copy_gbs = 2 * src.numel() * 2 / best / 1e6
+        del src, dst
+        torch.cuda.empty_cache()
+
     fused = None
     if rank == 0 and world == 1 and not args.skip_fused:
         fused = time_fused_lmhead(rlf, dev, max(2, min(args.steps, 5)))
@@ -673,7 +693,9 @@ def run_cuda(args):
                      "peak_kind": "of " + peak_kind, "frac_of_nominal_8tbs": achieved / 8000.0, "traffic": traffic,
                      "kernel": "grpo_row_cluster_kernel (timed as the rlf_grpo_logp_loss_fwd_bwd call: "
                                "row kernel + 3 sub-10us kernels)",
-                     "kernel_ms": k_ms, "kernel_ms_min": min(kernel_ms), "algorithmic_bytes": alg_bytes},
+                     "kernel_ms": k_ms, "kernel_ms_min": min(kernel_ms), "algorithmic_bytes": alg_bytes,
+                     "copy_gbs_this_gpu": copy_gbs,
+                     "frac_of_copy_this_gpu": (achieved / copy_gbs) if copy_gbs else None},
         "gpu_launches": int(launches),
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                    "samples": clocks["samples"]},
