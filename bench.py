@@ -392,6 +392,47 @@ def run_other_configs(args):
             ts.append(a.elapsed_time(b))
         return statistics.mean(ts)
 
+    # cfg 0 (tiny, latency-bound): the whole step launched call by call and replayed from a CUDA graph
+    spec0 = synth.SPECS[0]
+    b0 = synth.make_batch(spec0, dev)
+    o = dict(mask=torch.empty(b0.T, dtype=torch.uint8, device=dev), seq=torch.empty(b0.T, dtype=torch.int32, device=dev),
+             n=torch.empty(1, dtype=torch.int64, device=dev), adv=torch.empty(b0.rewards.shape[0], device=dev),
+             logp=torch.empty(b0.T, device=dev), loss=torch.empty(4, dtype=torch.float64, device=dev),
+             grad=torch.empty_like(b0.logits), ws=rlf.new_workspace(rlf.FN_LOGP_LOSS, b0.T, spec0.V, 0, rlf.RLF_F32, dev))
+
+    def step0():
+        rlf.rlf_build_loss_mask(b0.ids, b0.cu_seqlens, spec0.open_id, spec0.close_id, mask_out=o["mask"],
+                                seq_id_out=o["seq"], n_out=o["n"])
+        rlf.rlf_group_advantage(b0.rewards, group_size=spec0.group_size, adv_out=o["adv"])
+        rlf.rlf_grpo_logp_loss_fwd_bwd(b0.logits, b0.ids, o["seq"], o["adv"], b0.old_logp, b0.ref_logp, o["mask"],
+                                       synth.EPS_CLIP, synth.BETA_KL, denom=o["n"], grad_logits=o["grad"],
+                                       logp_out=o["logp"], loss_out=o["loss"], workspace=o["ws"])
+
+    def per_step_us(fn, reps=200):
+        for _ in range(10):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / reps
+    eager_us = per_step_us(step0)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step0()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step0()
+    out["cfg0_tiny_step_latency"] = {"T": b0.T, "V": spec0.V, "launches_per_step": 6, "eager_us": eager_us,
+                                     "cuda_graph_us": per_step_us(graph.replay)}
+    del b0, o, graph
+
     # cfg 2: in place over the whole packed batch (the gradient overwrites the logits, so every timed
     # call sees the previous call's output as its logits: same bytes moved, values irrelevant to time)
     spec = synth.SPECS[2]
