@@ -238,7 +238,7 @@ class ClockSampler:
             self.proc.kill()
         self.tmp.flush()
         self.tmp.seek(0)
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.tmp.read().splitlines():
             c = [x.strip() for x in line.split(",")]
@@ -249,6 +249,10 @@ class ClockSampler:
                 mx.append(float(c[2]))
             except ValueError:
                 continue
+            try:
+                pw.append(float(c[3]))
+            except ValueError:
+                pass
             for name, v in zip(names, c[5:9]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
@@ -256,6 +260,11 @@ class ClockSampler:
         os.unlink(self.tmp.name)
         if sm:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+            # settled part of the run only (the first third still carries the previous state's clocks)
+            tail = sm[len(sm) // 3:]
+            out["sm_mhz_settled"] = statistics.median(tail)
+            if pw:
+                out["power_w_settled"] = statistics.median(pw[len(pw) // 3:])
         return out
 
 
@@ -367,6 +376,73 @@ def run_fused_only(args):
     out = time_fused_lmhead(rlf, torch.device("cuda", 0), max(1, args.steps), args.tokens_per_response,
                             cfg=args.fused_cfg, responses=args.responses)
     print(json.dumps({"fused_lmhead": out, "gpu_launches": rlf.launch_count()}))
+
+
+def run_fused_phases(args):
+    """Sustained cost of the fused LM-head call by phase (cfg 3 or 4): each variant is looped for
+    --phase-seconds with the SM clock and board power sampled, so that what the power cap costs each
+    phase shows.  Variants differ by one phase at a time (forward sweep over the unmasked rows; plus
+    grad_hidden; plus grad_W; plus both; plus the masked rows' log-probs).  Prints one JSON line."""
+    from paper_2509_06980_b200 import binding as rlf
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    spec = synth.SPECS[args.fused_cfg]
+    tok = synth.make_tokens(spec)
+    T = len(tok.ids)
+    ids = torch.from_numpy(tok.ids).to(dev)
+    cu = torch.from_numpy(tok.cu_seqlens).to(dev)
+    H, W = synth.make_hidden_and_head(spec, T, dev)
+    mask, seq, n = rlf.rlf_build_loss_mask(ids, cu, spec.open_id, spec.close_id)
+    adv = rlf.rlf_group_advantage(torch.from_numpy(tok.rewards).to(dev), group_size=spec.group_size)
+    center = synth.center_logp_from_head(H, W, ids)
+    old, ref = synth.perturbed_logps(spec, center)
+    del center
+    ws = rlf.new_workspace(rlf.FN_FUSED_LMHEAD, T, spec.V, spec.D, rlf.RLF_BF16, dev)
+    gh = torch.empty((T, spec.D), dtype=torch.bfloat16, device=dev)
+    gw = torch.empty((spec.V, spec.D), dtype=torch.float32, device=dev)
+    logp = torch.empty(T, dtype=torch.float32, device=dev)
+    loss = torch.empty(4, dtype=torch.float64, device=dev)
+    z = torch.empty((T, spec.V), dtype=torch.bfloat16, device=dev)
+    live = int(mask.sum().item())
+
+    def call(skip, want_gh, want_gw):
+        rlf.rlf_fused_lmhead_grpo_obj(H, W, ids, seq, adv, old, ref, mask, synth.EPS_CLIP, synth.EPS_CLIP, synth.BETA_KL,
+                                      skip_masked=skip, denom=n, want_grad_hidden=want_gh, want_grad_W=want_gw,
+                                      grad_hidden=gh if want_gh else None, grad_W=gw if want_gw else None,
+                                      logp_out=logp, loss_out=loss, workspace=ws)
+    tvd = 2.0 * spec.V * spec.D
+    variants = [
+        ("library_gemm_all_rows", lambda: torch.matmul(H, W.t(), out=z), tvd * T),
+        ("sweep_all_rows", lambda: call(False, False, False), tvd * T),
+        ("sweep_unmasked_rows", lambda: call(True, False, False), tvd * live),
+        ("sweep_unmasked_plus_grad_hidden", lambda: call(True, True, False), tvd * 2 * live),
+        ("sweep_unmasked_plus_grad_W", lambda: call(True, False, True), tvd * 2 * live),
+        ("sweep_unmasked_plus_both_gradients", lambda: call(True, True, True), tvd * 3 * live),
+        ("full_call_all_log_probs_both_gradients", lambda: call(False, True, True), tvd * (T + 2 * live)),
+    ]
+    out = {"workload": "%s: hidden [%d, %d] x W [%d, %d] bf16" % (spec.name, T, spec.D, spec.V, spec.D),
+           "unmasked_rows": live, "seconds_per_variant": args.phase_seconds, "variants": {}}
+    for name, fn, flops in variants:
+        fn()
+        torch.cuda.synchronize()
+        sampler = ClockSampler(0)
+        sampler.start()
+        t0 = time.perf_counter()
+        k = 0
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        while time.perf_counter() - t0 < args.phase_seconds:
+            for _ in range(4):
+                fn()
+            k += 4
+            torch.cuda.synchronize()
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / k
+        clocks = sampler.stop()
+        out["variants"][name] = {"ms": ms, "executed_tflops": flops / ms / 1e9, "sm_mhz": clocks.get("sm_mhz_settled"),
+                                 "power_w": clocks.get("power_w_settled"), "reasons": clocks["reasons"]}
+    print(json.dumps({"fused_phases": out, "gpu_launches": rlf.launch_count()}))
 
 
 def run_other_configs(args):
@@ -507,6 +583,10 @@ def run_cuda(args):
     rank, world, local = dist_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    if args.fused_phases:
+        if dist_env()[0] == 0:
+            run_fused_phases(args)
+        return
     if args.fused_only or args.other_configs:
         if rank == 0:
             run_other_configs(args) if args.other_configs else run_fused_only(args)
@@ -770,6 +850,9 @@ def main():
                     help="time cfg 2 (ragged, in place) and cfg 4 (micro-batched; both paths) instead (rank 0)")
     ap.add_argument("--tokens-per-response", type=int, default=0,
                     help="smaller micro-batch of the same recipe (profiling captures); 0 = the full 2048")
+    ap.add_argument("--fused-phases", action="store_true",
+                    help="sustained cost of the fused LM-head call by phase, with clocks and power (rank 0)")
+    ap.add_argument("--phase-seconds", type=float, default=3.0)
     ap.add_argument("--fused-cfg", type=int, default=3, choices=[3, 4],
                     help="with --fused-only: the Qwen3-4B head (3) or the Qwen3-8B head (4)")
     ap.add_argument("--responses", type=int, default=0,
