@@ -97,6 +97,25 @@ def test_host_validation_rejects_bad_arguments_before_touching_a_device(lib):
     assert k(fake, fake, fake, fake, None, 2, 8, 0.1, 0, fake, None, None, None) == -1
     assert k(fake, None, fake, fake, fake, 2, 8, 0.1, 0, fake, None, None, None) == -1
     assert k(fake, fake, fake, fake, fake, 0, 8, 0.1, 0, fake, None, None, None) == 0
+    e = lib.rlf_fused_lmhead_logp_entropy
+    e.argtypes = [vp, vp, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, vp, vp, vp, vp, ctypes.c_size_t, vp, vp]
+    assert e(fake, fake, 8, 100, 64, fake, fake, None, fake, 1 << 30, None, None) == -2      # D not a multiple of 64
+    assert e(fake, fake, 8, 128, 63, fake, fake, None, fake, 1 << 30, None, None) == -2      # V not a multiple of 8
+    assert e(None, fake, 8, 128, 64, fake, fake, None, fake, 1 << 30, None, None) == -1
+    assert e(fake, fake, 8, 128, 64, fake, None, None, fake, 1 << 30, None, None) == -1
+    assert e(4104, fake, 8, 128, 64, fake, fake, None, fake, 1 << 30, None, None) == -3      # hidden not 16-byte aligned
+    assert e(fake, fake, 8, 128, 64, fake, fake, None, fake, 16, None, None) == -5
+    assert e(fake, fake, 0, 128, 64, None, None, None, None, 0, None, None) == 0             # T = 0: nothing to do
+    o = lib.rlf_fused_lmhead_grpo_obj
+    o.argtypes = [vp, vp, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, vp, vp, vp, ctypes.c_int32, vp, vp, vp,
+                  ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_int, ctypes.c_int, vp, vp, vp, vp, vp,
+                  ctypes.c_int, vp, ctypes.c_size_t, vp, vp]
+    oargs = lambda agg=0, skip=0, B=1: [fake, fake, 8, 128, 64, fake, fake, fake, B, fake, fake, fake, 0.2, 0.3, 0.0, agg,
+                                        skip, None, fake, fake, None, None, 0, fake, 1 << 30, None, None]
+    assert o(*oargs(agg=2)) == -2 and o(*oargs(skip=2)) == -2 and o(*oargs(agg=1, B=100)) == -2
+    s = lib.rlf_tune_lmhead_schedule
+    s.argtypes = [ctypes.c_int] * 3
+    assert s(-1, 0, 0) == -2 and s(0, -1, 0) == -2 and s(0, 0, 3) == -2 and s(0, 0, 0) == 0
     t = lib.rlf_tune_logits_kernel
     t.argtypes = [ctypes.c_int] * 3
     assert t(3, 512, 0) == -2 and t(4, 500, 0) == -2 and t(0, 0, -1) == 0
