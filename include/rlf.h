@@ -388,6 +388,14 @@ size_t rlf_step_arena_bytes(int64_t T, int32_t V, int32_t B, rlf_dtype dt);
  * beyond fp32 summation order (and, for one_exp, one extra bf16 rounding of the gradient). */
 rlf_status rlf_tune_logits_kernel(int cluster_ctas, int threads_per_cta, int one_exp);
 
+/* Grid sizing of the logits kernels for later calls in this process.  rows_per_cluster: a cluster of
+ * the row kernels (training, skip-masked, row-per-cluster forward) handles about this many rows and
+ * retires, so that several generations of clusters pass through the device during one launch (never
+ * fewer clusters than fit at once); units_per_cta: the same for the CTAs of the streaming forward
+ * pass, in row chunks.  0 restores the built-in choice (24 rows; 8 units).  Results do not depend
+ * on either. */
+rlf_status rlf_tune_logits_grid(int rows_per_cluster, int units_per_cta);
+
 /* Form of the fused LM-head contractions for later calls in this process: 1 = pairs of CTAs share a
  * 256 x 256 tile (tcgen05 cta_group::2; the built-in choice), 0 = one CTA per 128 x 256 tile.
  * Results are identical up to fp32 summation order. */

@@ -20,7 +20,7 @@ DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
 EXPORTS = [
     "rlf_build_loss_mask", "rlf_group_advantage", "rlf_rule_reward", "rlf_kl_in_reward", "rlf_grpo_logp_loss_fwd_bwd",
     "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_grpo_logp_loss_fwd_bwd_skip_masked", "rlf_grpo_logp_loss_fwd_bwd_obj", "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_fused_lmhead_grpo_obj", "rlf_fused_lmhead_logp_entropy", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
-    "rlf_tune_logits_kernel", "rlf_tune_lmhead", "rlf_tune_lmhead_schedule", "rlf_launch_count", "rlf_status_string", "rlf_version",
+    "rlf_tune_logits_kernel", "rlf_tune_logits_grid", "rlf_tune_lmhead", "rlf_tune_lmhead_schedule", "rlf_launch_count", "rlf_status_string", "rlf_version",
 ]
 
 if not os.path.exists(_LIB_PATH):
@@ -117,6 +117,12 @@ def new_workspace(which_fn, T, V, D=0, dt=RLF_BF16, device="cuda"):
 
 def tune_logits_kernel(cluster_ctas=0, threads_per_cta=0, one_exp=-1):
     _check(_lib.rlf_tune_logits_kernel(cluster_ctas, threads_per_cta, one_exp), "rlf_tune_logits_kernel")
+
+
+def tune_logits_grid(rows_per_cluster=0, units_per_cta=0):
+    _lib.rlf_tune_logits_grid.argtypes = [_int, _int]
+    _lib.rlf_tune_logits_grid.restype = _int
+    _check(_lib.rlf_tune_logits_grid(int(rows_per_cluster), int(units_per_cta)), "rlf_tune_logits_grid")
 
 
 def tune_lmhead(pair_ctas=1):
