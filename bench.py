@@ -38,7 +38,7 @@ WORKLOAD = "cfg1_qwen3_4b_microbatch: 16 responses x 2048 tokens, V=151936 bf16 
 
 # DRAM bytes of one row-kernel launch from the ncu capture summarised under profiles/, as bytes per
 # token; valid only for the row kernel's source text it was taken from (else reported as null).
-NCU_TRAFFIC = {"logits_loss_cu_sha1": "beae1f6cbc292ea9da59db4c5f59b105793ed141", "dram_bytes_per_token": 596259.0}
+NCU_TRAFFIC = {"logits_loss_cu_sha1": "beae1f6cbc292ea9da59db4c5f59b105793ed141", "dram_bytes_per_token": 594787.0}
 
 
 def _peaks():
@@ -185,7 +185,7 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3, responses=0
 
 
 # the same for the forward-only log-prob + entropy pass (profiles/logp_entropy_stream_kernel_T4096_ncu_full.md)
-NCU_TRAFFIC_ENTROPY = {"section_sha1": "cec2eff0a14f99f71358242b527710b41589d7d1", "dram_bytes_per_token": 307100.3}
+NCU_TRAFFIC_ENTROPY = {"section_sha1": "16eaba301a844ad26f759e3b7a762daf505bb851", "dram_bytes_per_token": 305667.0}
 
 
 def _entropy_section_sha1():

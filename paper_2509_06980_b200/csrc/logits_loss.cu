@@ -897,6 +897,15 @@ static int clusters_for(int resident, int64_t rows) {
     return (int)nc;
 }
 
+// CTAs of the general (one CTA per row) kernel: a few rows per CTA, for the same reason
+static int general_grid(int64_t rows) {
+    int64_t g = (rows + 3) / 4;
+    if (g < (int64_t)sm_count() * 8) g = (int64_t)sm_count() * 8;
+    if (g > rows) g = rows;
+    if (g > (1 << 30)) g = 1 << 30;
+    return (int)g;
+}
+
 struct LossArgs {
     const void* logits;
     void* grad;
@@ -1028,8 +1037,7 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
             p.rec = rec; p.denom = denom; p.logp_out = a.logp_out; p.dev_status = a.dev_status;
             p.eps_clip = a.eps_clip; p.eps_hi = a.eps_hi; p.beta = a.beta; p.entropy_out = nullptr; p.fwd_only = 0;
             p.wtok = wtok;
-            int grid = sm_count() * 8;
-            if ((int64_t)grid > a.T) grid = (int)a.T;
+            int grid = general_grid(a.T);
             if (a.dt == RLF_BF16) grpo_row_general_kernel<__nv_bfloat16><<<grid, kGenThreads, 0, s>>>(p);
             else grpo_row_general_kernel<float><<<grid, kGenThreads, 0, s>>>(p);
             count_launch();
@@ -1439,8 +1447,7 @@ extern "C" rlf_status rlf_logp_entropy_fwd(const void* logits, rlf_dtype dt, int
     g.logp_out = logp_out; g.entropy_out = entropy_out; g.dev_status = dev_status; g.eps_clip = 0.0f; g.beta = 0.0f;
     g.eps_hi = 0.0f; g.wtok = nullptr;
     g.fwd_only = 1;
-    int grid = sm_count() * 8;
-    if ((int64_t)grid > T) grid = (int)T;
+    int grid = general_grid(T);
     if (dt == RLF_BF16) grpo_row_general_kernel<__nv_bfloat16><<<grid, kGenThreads, 0, s>>>(g);
     else grpo_row_general_kernel<float><<<grid, kGenThreads, 0, s>>>(g);
     count_launch();
