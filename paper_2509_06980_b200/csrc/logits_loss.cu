@@ -708,16 +708,19 @@ token_loss_kernel(const float* __restrict__ logp, const float4* __restrict__ rec
     }
 }
 
-// per-block partial sums -> loss_out[4], added in index order by one thread per quantity
-__global__ void finalize_loss_kernel(const double* __restrict__ partial, int num_partials,
-                                     const long long* __restrict__ denom, float beta, int weighted,
-                                     double* __restrict__ loss_out) {
+// per-block partial sums -> loss_out[4].  One warp per quantity: each lane adds its partials (stride 32,
+// index order), then a fixed shuffle tree: the same order on every launch, so results are run-to-run
+// identical.  Launched with 96 threads.
+__global__ void __launch_bounds__(96)
+finalize_loss_kernel(const double* __restrict__ partial, int num_partials, const long long* __restrict__ denom,
+                     float beta, int weighted, double* __restrict__ loss_out) {
     __shared__ double s[3];
-    if (threadIdx.x < 3) {
-        double a = 0.0;
-        for (int i = 0; i < num_partials; ++i) a += partial[4 * i + threadIdx.x];
-        s[threadIdx.x] = a;
-    }
+    const int q = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    double a = 0.0;
+    for (int i = lane; i < num_partials; i += 32) a += partial[4 * i + q];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if (lane == 0) s[q] = a;
     __syncthreads();
     if (threadIdx.x == 0) {
         const long long N = *denom;
@@ -1049,7 +1052,7 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
     }
-    finalize_loss_kernel<<<1, 32, 0, s>>>(partial, num_partials, denom, a.beta, wtok != nullptr, a.loss_out);
+    finalize_loss_kernel<<<1, 96, 0, s>>>(partial, num_partials, denom, a.beta, wtok != nullptr, a.loss_out);
     count_launch();
     return cuda_ok(cudaGetLastError());
 }
@@ -1547,7 +1550,7 @@ extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd_skip_masked(
                                                     workspace, workspace_bytes, dev_status, stream);
         if (st0 != RLF_OK || T == 0) return st0;
         const float4* rec0 = reinterpret_cast<const float4*>(static_cast<char*>(workspace) + kWsRecordOff);
-        fill_dead_rows_kernel<float><<<sm_count() * 4, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+        fill_dead_rows_kernel<float><<<general_grid(T), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
             rec0, T, V, row_stride, nullptr, 0, logp_out);
         count_launch();
         return cuda_ok(cudaGetLastError());
@@ -1569,7 +1572,7 @@ extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd_skip_masked(
     if (st != RLF_OK) return st;
     compact_live_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(rec, T, row_list, rec_c, n_live);
     count_launch();
-    fill_dead_rows_kernel<__nv_bfloat16><<<sm_count() * 4, 256, 0, s>>>(
+    fill_dead_rows_kernel<__nv_bfloat16><<<general_grid(T), 256, 0, s>>>(
         rec, T, V, row_stride, static_cast<__nv_bfloat16*>(grad_logits), zero_masked_grad, logp_out);
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
@@ -1637,7 +1640,7 @@ rlf_status launch_token_loss(const float* logp, const void* rec, int64_t T, floa
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
     }
-    finalize_loss_kernel<<<1, 32, 0, s>>>(partial, num_partials, denom, beta, 0, loss_out);
+    finalize_loss_kernel<<<1, 96, 0, s>>>(partial, num_partials, denom, beta, 0, loss_out);
     count_launch();
     return cuda_ok(cudaGetLastError());
 }
@@ -1654,7 +1657,7 @@ rlf_status launch_token_loss_w(const float* logp, const void* rec, int64_t T, fl
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
     }
-    finalize_loss_kernel<<<1, 32, 0, s>>>(partial, num_partials, denom, beta, wtok != nullptr, loss_out);
+    finalize_loss_kernel<<<1, 96, 0, s>>>(partial, num_partials, denom, beta, wtok != nullptr, loss_out);
     count_launch();
     return cuda_ok(cudaGetLastError());
 }
