@@ -8,6 +8,7 @@ import torch
 from oracle import rlf_oracle as orc
 from paper_2509_06980_b200 import synth
 import gpu_common as gc
+from util import loss_close
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -315,3 +316,44 @@ def test_rule_reward_eq1_feeds_the_advantage():
     assert np.abs(got.cpu().numpy() - want).max() <= 1e-7 * np.abs(want).max()
     want_adv = orc.group_advantage(got.cpu().numpy(), group_size=8)
     assert np.allclose(adv.cpu().numpy(), want_adv, rtol=2e-7, atol=1e-30)
+
+
+@pytest.mark.parametrize("T", [1, 7, 74, 75, 1775, 1776, 1777, 3600])
+def test_results_do_not_depend_on_the_grid(T):
+    """A launch runs several generations of short-lived clusters (CTAs); how many is a tuning choice.
+    Row counts around the generation boundaries, and the extreme settings (one row per cluster / one
+    chunk per CTA; a single persistent generation): every output is bit-identical, and equal to the
+    oracle within the usual tolerances."""
+    b = gc.binding()
+    V = 4096 + 264
+    g = torch.Generator(device=DEV)
+    g.manual_seed(100 + T)
+    z = (torch.randn((T, V), device=DEV, generator=g) * 3).to(torch.bfloat16)
+    ids = torch.randint(0, V, (T,), device=DEV, generator=g).to(torch.int32)
+    seq = (torch.arange(T, device=DEV) % 4).to(torch.int32)
+    adv = torch.tensor([0.7, -1.1, 0.2, 1.4], device=DEV)
+    mask = (torch.rand(T, device=DEV, generator=g) < 0.6).to(torch.uint8)
+    old = torch.full((T,), -9.0, device=DEV) + 0.1 * torch.randn(T, device=DEV, generator=g)
+    ref = old + 0.05
+    outs = []
+    try:
+        for rows_per_cluster, units_per_cta in ((0, 0), (1, 1), (1 << 30, 1 << 30), (5, 3)):
+            b.tune_logits_grid(rows_per_cluster, units_per_cta)
+            logp, loss, grad = b.rlf_grpo_logp_loss_fwd_bwd(z, ids, seq, adv, old, ref, mask, 0.2, 0.01)
+            lp2, ent = b.rlf_logp_entropy_fwd(z, ids)
+            lp3, l3, g3 = b.rlf_grpo_logp_loss_fwd_bwd_skip_masked(z, ids, seq, adv, old, ref, mask, 0.2, 0.01)
+            torch.cuda.synchronize()
+            outs.append((logp, loss, grad, lp2, ent, l3, g3))
+    finally:
+        b.tune_logits_grid(0, 0)
+    for o in outs[1:]:
+        for a, c in zip(outs[0], o):
+            assert torch.equal(a, c)
+    r = orc.grpo_loss(gc.to_np(z), ids.cpu().numpy(), seq.cpu().numpy(), adv.cpu().numpy(), old.cpu().numpy(),
+                      ref.cpu().numpy(), mask.cpu().numpy(), 0.2, 0.01, want_coef=True)
+    logp, loss, grad = outs[0][:3]
+    assert np.abs(logp.cpu().numpy() - r["logp"]).max() <= gc.LOGP_ATOL
+    assert loss_close(loss[0].item(), r["loss"][0], 1e-6, gc.LOSS_RTOL)
+    guard = gc.near_clip_bound(r["logp"], old.cpu().numpy(), None)
+    ulps = gc.grad_ulps(gc.grad_to_f64(grad)[~guard], r["grad"][~guard], ids.cpu().numpy()[~guard], r["coef"][~guard])
+    assert ulps.size == 0 or ulps.max() <= gc.GRAD_ULPS
