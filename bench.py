@@ -665,6 +665,23 @@ def run_cuda(args):
     ms_total_max = max_over_ranks(ms_total, world, dev)
     value = aggregate(T * args.steps, world, ms_total_max / 1e3)
 
+    # the same step looped back to back for about a second: the row kernel keeps the SMs busy enough to
+    # reach the board's power cap, and what it holds then is lower than over 20 steps from a rested GPU
+    sustained = None
+    if rank == 0 and world == 1 and not args.tokens_per_response:
+        n_sus = 300
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(n_sus // 2):
+            step()
+        s0.record()
+        for _ in range(n_sus):
+            step()
+        s1.record()
+        torch.cuda.synchronize()
+        sus_ms = s0.elapsed_time(s1) / n_sus
+        sustained = {"steps": n_sus, "after_untimed_steps": n_sus // 2, "ms_per_step": sus_ms,
+                     "tokens_per_s": T / sus_ms * 1e3, "logits_gbs_whole_step": T * V * 4 / sus_ms / 1e6}
+
     # end to end through the host-buffer entry point: inputs start in pinned host memory, the loss
     # (and per-token log-probs) come back to the host, every step
     e2e = None
@@ -821,6 +838,7 @@ def run_cuda(args):
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                    "samples": clocks["samples"]},
         "loss": float(loss[0].item()),
+        "sustained": sustained,
     }
     if e2e is not None:
         line["e2e"] = e2e
