@@ -294,8 +294,9 @@ rlf_status rlf_grpo_logp_loss_fwd_bwd_static(const void *logits, rlf_dtype dt, i
  *   grad_hidden [T, D] bf16 or NULL;  grad_W [V, D] fp32 or NULL (both NULL: forward only)
  *   workspace   rlf_workspace_bytes(RLF_FN_FUSED_LMHEAD, T, V, D, RLF_BF16) bytes, 256-byte aligned.
  *               It holds per-token records and partial sums and, for the backward, a copy of hidden
- *               with the unmasked rows gathered first, and one chunk [min(T, 9472), V] of bf16
- *               (2.9 GB at V = 151936): the forward sweep of a chunk of unmasked rows leaves
+ *               with the unmasked rows gathered first, and one chunk of min(T, 9472) rows by V
+ *               (rounded up to whole 256-column tiles) of bf16, stored in blocks of 128 rows x 64
+ *               columns (2.9 GB at V = 151936): the forward sweep of a chunk of unmasked rows leaves
  *               exp(z - max of the 256-column tile) there (never above 1, so no logit overflows
  *               it), an elementwise pass rescales it in place into dZ = grad_z once the row's
  *               log-sum-exp is known, and the two gradient contractions consume it.  The logits

@@ -50,6 +50,18 @@ constexpr int kSlabBytes = 64 * BK * 2;      // one 64-wide slab of an MN-major 
 
 enum Mode { kLse = 0, kGradHidden = 2, kGradW = 3 };
 
+// The [rows, V] scratch that carries a chunk's exponentials, then its dZ, is stored in blocks of
+// 128 token rows x 64 vocabulary columns (16 KB, rows of 128 bytes), blocks of one token tile side by
+// side: element (row, col) sits at ((row / 128 * nc + col / 64) * 128 + row % 128) * 64 + col % 64,
+// nc = 4 x the number of 256-column tiles.  Every operand box the two gradient contractions fetch
+// (128 or 64 rows of 128 bytes) is then one contiguous piece of memory, and so is what a warp of the
+// sweep's epilogue stores; with plain rows of 2 V bytes each of those touched 64 - 128 DRAM pages for
+// 128 bytes apiece.
+constexpr int kDzBlockRows = 128, kDzBlockCols = 64;
+__host__ __device__ __forceinline__ long long dz_offset(long long row, int col, int nc) {
+    return (((row >> 7) * nc + (col >> 6)) * kDzBlockRows + (row & 127)) * kDzBlockCols + (col & 63);
+}
+
 struct GemmParams {
     int mode;
     int M, N;                 // extent of the output tile grid in rows / columns (valid elements)
@@ -58,9 +70,10 @@ struct GemmParams {
     int m_block;              // kLse: row units per scheduling block
     float2* part;             // kLse: [M][nsplit] (max, sum exp)
     float* part_u;            // kLse (optional): [M][nsplit] sum of 2^x x, x the base-2 exponent against that max
-    __nv_bfloat16* dz;        // kLse (optional) out, row stride dz_stride: exp(z - tile max) as bf16
+    __nv_bfloat16* dz;        // kLse (optional) out, blocked scratch (see dz_offset): exp(z - tile max) as bf16
     float* tmax;              // kLse with dz: [M][n_tiles] the tile maxima those exponentials refer to
-    long long dz_stride;
+    int dz_nc;                // 64-column blocks per token tile of the blocked scratch; also set for the
+                              // gradient contractions, whose A operand is that scratch
     __nv_bfloat16* out_bf16;  // kGradHidden out [M][out_stride]
     float* out_f32;           // kGradW out [M][out_stride]
     long long out_stride;
@@ -291,10 +304,16 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                             if (PAIR) tma_load_2d_pair(dst, map, bar, x, y);
                             else tma_load_2d(dst, map, bar, x, y);
                         };
-                        if (!a_mn) {
-                            load(sa, &map_a, kb * BK, my_m * BM);
+                        if (p.mode == kGradHidden) {
+                            // dZ block (token tile my_m, vocabulary block kb): 128 rows of 128 bytes
+                            load(sa, &map_a, 0, (my_m * p.dz_nc + kb) * kDzBlockRows);
+                        } else if (p.mode == kGradW) {
+                            // dZ^T: vocabulary blocks 2 my_m + j, the 64 token rows of k-slab kb
+                            for (int j = 0; j < BM / 64; ++j)
+                                load(sa + j * kSlabBytes, &map_a, 0,
+                                     ((kb >> 1) * p.dz_nc + (my_m * 2 + j)) * kDzBlockRows + (kb & 1) * 64);
                         } else {
-                            for (int j = 0; j < BM / 64; ++j) load(sa + j * kSlabBytes, &map_a, my_m * BM + j * 64, kb * BK);
+                            load(sa, &map_a, kb * BK, my_m * BM);
                         }
                         if (!b_mn) {
                             load(sb, &map_b, kb * BK, b_row0);
@@ -403,34 +422,34 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     float ts0 = 0.0f, ts1 = 0.0f;
 #pragma unroll 1
                     for (int c = 0; c < BN / 32; ++c) {
+                        // every column block of the tile is written: the scratch covers whole tiles and
+                        // the columns past the vocabulary must read as zeros (warp-uniform conditions)
                         const int cb = col0 + c * 32;
-                        if (cb >= p.N) break;
-                        uint32_t v[32];
-                        tc_ld32(t_row + (uint32_t)(c * 32), v);
-                        const int nvalid = min(32, p.N - cb);
+                        const int nvalid = max(0, min(32, p.N - cb));
                         uint32_t o[16];
+                        if (nvalid > 0) {
+                            uint32_t v[32];
+                            tc_ld32(t_row + (uint32_t)(c * 32), v);
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            float e0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), kLog2e, off));
-                            float e1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), kLog2e, off));
-                            if (2 * i >= nvalid) e0 = 0.0f;
-                            if (2 * i + 1 >= nvalid) e1 = 0.0f;
-                            ts0 += e0;
-                            ts1 += e1;
-                            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[i]) : "f"(e1), "f"(e0));
+                            for (int i = 0; i < 16; ++i) {
+                                float e0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), kLog2e, off));
+                                float e1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), kLog2e, off));
+                                if (2 * i >= nvalid) e0 = 0.0f;
+                                if (2 * i + 1 >= nvalid) e1 = 0.0f;
+                                ts0 += e0;
+                                ts1 += e1;
+                                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[i]) : "f"(e1), "f"(e0));
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) o[i] = 0u;
                         }
                         if (row_ok) {
-                            __nv_bfloat16* dst = p.dz + (long long)row * p.dz_stride + cb;
-                            if (nvalid == 32) {
-                                uint4* d4 = reinterpret_cast<uint4*>(dst);
-                                d4[0] = make_uint4(o[0], o[1], o[2], o[3]);
-                                d4[1] = make_uint4(o[4], o[5], o[6], o[7]);
-                                d4[2] = make_uint4(o[8], o[9], o[10], o[11]);
-                                d4[3] = make_uint4(o[12], o[13], o[14], o[15]);
-                            } else {
-                                for (int i = 0; i < nvalid; ++i)
-                                    dst[i] = __ushort_as_bfloat16((unsigned short)((i & 1) ? (o[i >> 1] >> 16) : (o[i >> 1] & 0xffffu)));
-                            }
+                            uint4* d4 = reinterpret_cast<uint4*>(p.dz + dz_offset(row, cb, p.dz_nc));
+                            d4[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                            d4[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                            d4[2] = make_uint4(o[8], o[9], o[10], o[11]);
+                            d4[3] = make_uint4(o[12], o[13], o[14], o[15]);
                         }
                     }
                     if (tm != -INFINITY) run_s += (ts0 + ts1) * ex2_approx((tm - run_m) * kLog2e);
@@ -792,43 +811,57 @@ combine_rows_kernel(const float2* __restrict__ part, int nsplit, int rows_max, c
 
 // in place over one chunk of stored exponentials e = exp(z - tile max): dZ = coef (e exp(tile max - lse)
 // - [v == y]) as bf16; the target column takes the fp32 target logit.  Rows from the live extent up
-// to the next multiple of 256 become zeros.  One CTA per row.
+// to the next multiple of 256 become zeros.  One CTA per (token tile, 256-column tile): four adjacent
+// blocks of the scratch, 64 KB of contiguous memory.
 __global__ void __launch_bounds__(256)
 dz_from_e_kernel(__nv_bfloat16* __restrict__ ebuf, int V, int n_tiles, const float* __restrict__ tmax, int rows_max,
                  const int* __restrict__ count, int off, const float* __restrict__ lse_g,
                  const float* __restrict__ coef_g, const int32_t* __restrict__ y_g, const int32_t* __restrict__ idx,
                  const float* __restrict__ zy) {
+    __shared__ float f_s[kDzBlockRows];          // signed scale of each row for this column tile
+    __shared__ int live_s[kDzBlockRows];
     const int n = max(0, min(*count - off, rows_max));
-    const int r = blockIdx.x;
-    if (r >= ((n + 255) & ~255)) return;
-    uint4* row = reinterpret_cast<uint4*>(ebuf + (long long)r * V);
-    const int nv = V / 8;
-    const float coef = r < n ? coef_g[off + r] : 0.0f;
-    if (coef == 0.0f) {
-        for (int i = threadIdx.x; i < nv; i += 256) row[i] = make_uint4(0u, 0u, 0u, 0u);
-        return;
+    const int tt = blockIdx.x, jt = blockIdx.y;
+    if (tt * kDzBlockRows >= ((n + 255) & ~255)) return;
+    const int nc = 4 * n_tiles;
+    if (threadIdx.x < kDzBlockRows) {
+        const int r = tt * kDzBlockRows + threadIdx.x;
+        const float coef = r < n ? coef_g[off + r] : 0.0f;
+        float f = 0.0f;
+        if (coef != 0.0f) {
+            const float c2 = lg2_approx(fabsf(coef)) - lse_g[off + r] * kLog2e;
+            f = copysignf(ex2_approx(fmaf(tmax[(long long)r * n_tiles + jt], kLog2e, c2)), coef);
+        }
+        f_s[threadIdx.x] = f;
+        live_s[threadIdx.x] = coef != 0.0f;
     }
-    const float lse = lse_g[off + r];
-    const float c2 = lg2_approx(fabsf(coef)) - lse * kLog2e;
-    const float* tm = tmax + (long long)r * n_tiles;
-    for (int i = threadIdx.x; i < nv; i += 256) {
-        // signed scale of this vector's tile (BN = 256 columns = 32 vectors)
-        const float f = copysignf(ex2_approx(fmaf(tm[i >> 5], kLog2e, c2)), coef);
-        const uint4 z = row[i];
+    __syncthreads();
+    uint4* base = reinterpret_cast<uint4*>(ebuf + dz_offset((long long)tt * kDzBlockRows, jt * BN, nc));
+    // 4 blocks x 128 rows x 8 vectors of 16 bytes
+    for (int i = threadIdx.x; i < 4 * kDzBlockRows * 8; i += 256) {
+        const int rr = (i >> 3) & (kDzBlockRows - 1);
+        if (!live_s[rr]) {
+            base[i] = make_uint4(0u, 0u, 0u, 0u);
+            continue;
+        }
+        const float f = f_s[rr];
+        const uint4 z = base[i];
         const uint32_t w[4] = {z.x, z.y, z.z, z.w};
         uint32_t o[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k)
             asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[k])
                 : "f"(__uint_as_float(w[k] & 0xffff0000u) * f), "f"(__uint_as_float(w[k] << 16) * f));
-        row[i] = make_uint4(o[0], o[1], o[2], o[3]);
+        base[i] = make_uint4(o[0], o[1], o[2], o[3]);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (threadIdx.x < kDzBlockRows && live_s[threadIdx.x]) {
+        const int r = tt * kDzBlockRows + threadIdx.x;
         const int y = y_g[off + r];
-        if (y >= 0 && y < V) {
-            const float py = ex2_approx((zy[idx[off + r]] - lse) * kLog2e);
-            ebuf[(long long)r * V + y] = __float2bfloat16_rn(fmaf(coef, py, -coef));
+        if (y >= jt * BN && y < jt * BN + BN && y < V) {
+            const float coef = coef_g[off + r];
+            const float py = ex2_approx((zy[idx[off + r]] - lse_g[off + r]) * kLog2e);
+            ebuf[dz_offset(r, y, nc)] = __float2bfloat16_rn(fmaf(coef, py, -coef));
         }
     }
 }
@@ -981,7 +1014,7 @@ static LmWs lm_workspace(int64_t T, int32_t V, int32_t D) {
     const size_t chunk = Tp < (size_t)kChunkTokens ? Tp : (size_t)kChunkTokens;
     w.tmax = o;    o += up1k(4 * chunk * (size_t)((V + BN - 1) / BN));
     w.dz = o;
-    o += up1k(chunk * (size_t)V * 2);
+    o += up1k(chunk * (size_t)((V + BN - 1) / BN) * BN * 2);     // blocked: whole 256-column tiles
     w.total = o + 1024;
     return w;
 }
@@ -1135,7 +1168,7 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
         set_rows(z, tc);
         if (bwd) {
             z.dz = dz;
-            z.dz_stride = V;
+            z.dz_nc = 4 * z.n_tiles;
             z.tmax = reinterpret_cast<float*>(ws + w.tmax);
         }
         z.live_count = counts;
@@ -1148,14 +1181,16 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
         count_launch();
         if (!bwd) continue;
         const int64_t tcp = (tc + 255) & ~(int64_t)255;
-        dz_from_e_kernel<<<(unsigned)tcp, 256, 0, s>>>(dz, V, z.n_tiles, z.tmax, (int)tc, counts, (int)t0, lse_g, coef_g, y_g,
-                                                        idx_live, zy);
+        dz_from_e_kernel<<<dim3((unsigned)(tcp / kDzBlockRows), (unsigned)z.n_tiles), 256, 0, s>>>(
+            dz, V, z.n_tiles, z.tmax, (int)tc, counts, (int)t0, lse_g, coef_g, y_g, idx_live, zy);
+        // the scratch as the contractions see it: rows of 64 columns, 128 rows per block
+        const uint64_t dz_rows = (uint64_t)(tcp / kDzBlockRows) * (uint64_t)(4 * z.n_tiles) * kDzBlockRows;
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
         if (grad_hidden) {
             // grad_hidden[token of gathered row] = dZ[chunk, V] W[V, D]
             CUtensorMap mapDzK, mapWn;
-            if (!make_map(&mapDzK, dz, (uint64_t)tc, (uint64_t)V, (uint64_t)V, BK, BM)) return RLF_ERR_CUDA;
+            if (!make_map(&mapDzK, dz, dz_rows, kDzBlockCols, kDzBlockCols, BK, BM)) return RLF_ERR_CUDA;
             if (!make_map(&mapWn, Wm, (uint64_t)V, (uint64_t)D, (uint64_t)D, 64, BK)) return RLF_ERR_CUDA;
             GemmParams h = {};
             h.mode = kGradHidden;
@@ -1163,7 +1198,8 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
             h.N = D;
             h.m_tiles = (int)((tc + BM - 1) / BM);
             h.n_tiles = (D + BN - 1) / BN;
-            h.k_slabs = (V + BK - 1) / BK;
+            h.k_slabs = 4 * z.n_tiles;                     // every block of the scratch (zeros past the vocabulary)
+            h.dz_nc = 4 * z.n_tiles;
             h.out_bf16 = static_cast<__nv_bfloat16*>(grad_hidden);
             h.out_stride = D;
             h.dev_status = dev_status;
@@ -1176,7 +1212,7 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
         if (grad_W) {
             // grad_W[V, D] (+)= dZ[chunk, V]^T hidden[chunk, D]
             CUtensorMap mapDzM, mapHn;
-            if (!make_map(&mapDzM, dz, (uint64_t)tc, (uint64_t)V, (uint64_t)V, 64, BK)) return RLF_ERR_CUDA;
+            if (!make_map(&mapDzM, dz, dz_rows, kDzBlockCols, kDzBlockCols, 64, BK)) return RLF_ERR_CUDA;
             if (!make_map(&mapHn, Hl + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, 64, BK)) return RLF_ERR_CUDA;
             GemmParams q = {};
             q.mode = kGradW;
@@ -1185,6 +1221,7 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
             q.m_tiles = (V + BM - 1) / BM;
             q.n_tiles = (D + BN - 1) / BN;
             q.k_slabs = (int)((tc + BK - 1) / BK);
+            q.dz_nc = 4 * z.n_tiles;
             q.out_f32 = grad_W;
             q.out_stride = D;
             q.accumulate = (accumulate_grad_W || t0 > 0) ? 1 : 0;
