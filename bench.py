@@ -665,6 +665,27 @@ def run_cuda(args):
     ms_total_max = max_over_ranks(ms_total, world, dev)
     value = aggregate(T * args.steps, world, ms_total_max / 1e3)
 
+    # the two launch-latency-bound calls of the step, each looped on its own (5 bytes per token; B floats)
+    small_us = None
+    if rank == 0 and world == 1:
+        def loop_us(fn, reps=200):
+            for _ in range(10):
+                fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(reps):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) * 1e3 / reps
+        small_us = {
+            "rlf_build_loss_mask": loop_us(lambda: rlf.rlf_build_loss_mask(
+                batch.ids, batch.cu_seqlens, spec.open_id, spec.close_id, mask_out=mask, seq_id_out=seq_id, n_out=n_tok,
+                dev_status=status)),
+            "rlf_group_advantage": loop_us(lambda: rlf.rlf_group_advantage(
+                batch.rewards, group_size=G, eps=1e-6, adv_out=adv, dev_status=status)),
+            "what": "microseconds per call, 200 calls back to back (launch-latency bound)"}
+
     # the same step looped back to back for about a second: the row kernel keeps the SMs busy enough to
     # reach the board's power cap, and what it holds then is lower than over 20 steps from a rested GPU
     sustained = None
@@ -839,6 +860,7 @@ def run_cuda(args):
                    "samples": clocks["samples"]},
         "loss": float(loss[0].item()),
         "sustained": sustained,
+        "small_calls_us": small_us,
     }
     if e2e is not None:
         line["e2e"] = e2e
