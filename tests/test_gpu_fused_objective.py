@@ -104,3 +104,31 @@ def test_fused_objective_all_rows_masked_and_bad_arguments():
     with pytest.raises(Exception):
         b.rlf_fused_lmhead_grpo_obj(batch.hidden, batch.W, batch.ids, seq, adv, batch.old_logp, batch.ref_logp, mask,
                                     0.2, 0.3, 0.01, aggregation=2)
+
+
+def test_fused_results_do_not_depend_on_the_schedule():
+    """Scheduling block, worker cap and backward chunk are tuning choices: log-probs, loss and
+    grad_hidden are bit-identical for every setting; grad_W is bit-identical unless the chunking
+    changes (then the chunks' contributions are added in another order: fp32 rounding only)."""
+    b, spec, batch, mask, seq, n, adv = _setup(4096 + 264, 192)
+    # enough rows for several token tiles and, with 2-tile chunks, several chunks
+    spec = synth.scaled(spec, len_lo=60, len_hi=60)
+    batch = synth.make_batch(spec, DEV)
+    mask, seq, n = b.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, spec.open_id, spec.close_id)
+    adv = b.rlf_group_advantage(batch.rewards, group_size=batch.tokens.group_size)
+    args = (batch.hidden, batch.W, batch.ids, seq, adv, batch.old_logp, batch.ref_logp, mask, synth.EPS_CLIP, synth.BETA_KL)
+    outs = {}
+    try:
+        for key in ((0, 0, 0), (1, 0, 0), (3, 5, 0), (1000, 1, 0), (0, 0, 2), (2, 7, 4)):
+            b.tune_lmhead_schedule(*key)
+            outs[key] = b.rlf_fused_lmhead_grpo(*args, denom=n)
+            torch.cuda.synchronize()
+    finally:
+        b.tune_lmhead_schedule(0, 0, 0)
+    ref = outs[(0, 0, 0)]
+    for key, o in outs.items():
+        assert torch.equal(o[0], ref[0]) and torch.equal(o[1], ref[1]) and torch.equal(o[2], ref[2]), key
+        if key[2] == 0:
+            assert torch.equal(o[3], ref[3]), key
+        else:
+            assert (o[3] - ref[3]).abs().max().item() <= 1e-5 * ref[3].abs().max().item(), key
