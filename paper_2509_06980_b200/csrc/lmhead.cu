@@ -609,6 +609,40 @@ target_logit_kernel(const __nv_bfloat16* __restrict__ hidden, const __nv_bfloat1
     if (lane == 0) zy[t] = acc;
 }
 
+// One token's row statistics from its per-split (max, sum exp) partials, and its gradient coefficient
+// c_t = -(w_t) (dpg/dlogp + beta (1 - exp(ref - logp))), w_t = the token's loss weight.
+struct TokenStats {
+    float lse, logp, coef;
+    bool finite;
+};
+__device__ __forceinline__ TokenStats token_stats(const float2* __restrict__ parts, int nsplit, float zy, const float4 rec,
+                                                  const float* __restrict__ wtok, int64_t t,
+                                                  const long long* __restrict__ denom, float eps_clip, float eps_hi,
+                                                  float beta) {
+    float M = -INFINITY;
+    for (int j = 0; j < nsplit; ++j) M = fmaxf(M, parts[j].x);
+    float S = 0.0f;
+    for (int j = 0; j < nsplit; ++j) {
+        const float2 ms = parts[j];
+        if (ms.x != -INFINITY) S += ms.y * expf(ms.x - M);
+    }
+    TokenStats o;
+    o.lse = M + logf(S);
+    o.logp = (zy - M) - logf(S);
+    o.finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) && (fabsf(o.logp) < INFINITY);
+    o.coef = 0.0f;
+    if ((__float_as_int(rec.w) < 0) && o.finite) {
+        const long long N = *denom;
+        const float inv_n = wtok ? wtok[t] : 1.0f / (float)(N > 1 ? N : 1);
+        const float A = rec.z;
+        const float rho = expf(o.logp - rec.x);
+        const bool clipped = ((A > 0.0f) && (rho > 1.0f + eps_hi)) || ((A < 0.0f) && (rho < 1.0f - eps_clip));
+        const float dpg = clipped ? 0.0f : -A * rho;
+        o.coef = -inv_n * fmaf(beta, -expm1f(rec.y - o.logp), dpg);
+    }
+    return o;
+}
+
 // merge the per-split (max, sum exp) pairs of every token into lse, logp and the gradient coefficient
 __global__ void __launch_bounds__(256)
 combine_kernel(const float2* __restrict__ part, int nsplit, const float* __restrict__ zy,
@@ -617,32 +651,11 @@ combine_kernel(const float2* __restrict__ part, int nsplit, const float* __restr
                float* __restrict__ lse_out, float* __restrict__ coef_out, int32_t* __restrict__ dev_status) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= T) return;
-    float M = -INFINITY;
-    for (int j = 0; j < nsplit; ++j) M = fmaxf(M, part[t * nsplit + j].x);
-    float S = 0.0f;
-    for (int j = 0; j < nsplit; ++j) {
-        const float2 ms = part[t * nsplit + j];
-        if (ms.x != -INFINITY) S += ms.y * expf(ms.x - M);
-    }
-    const float lse = M + logf(S);
-    const float logp = (zy[t] - M) - logf(S);
-    const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) && (fabsf(logp) < INFINITY);
-    const float4 r = rec[t];
-    const bool live = (__float_as_int(r.w) < 0) && finite;
-    float coef = 0.0f;
-    if (live) {
-        const long long N = *denom;
-        const float inv_n = wtok ? wtok[t] : 1.0f / (float)(N > 1 ? N : 1);
-        const float A = r.z;
-        const float rho = expf(logp - r.x);
-        const bool clipped = ((A > 0.0f) && (rho > 1.0f + eps_hi)) || ((A < 0.0f) && (rho < 1.0f - eps_clip));
-        const float dpg = clipped ? 0.0f : -A * rho;
-        coef = -inv_n * fmaf(beta, -expm1f(r.y - logp), dpg);
-    }
-    logp_out[t] = finite ? logp : __int_as_float(0x7fc00000);
-    lse_out[t] = finite ? lse : 0.0f;
-    coef_out[t] = coef;
-    if (!finite && dev_status) atomicOr(dev_status, RLF_DEV_NONFINITE);
+    const TokenStats ts = token_stats(part + t * nsplit, nsplit, zy[t], rec[t], wtok, t, denom, eps_clip, eps_hi, beta);
+    logp_out[t] = ts.finite ? ts.logp : __int_as_float(0x7fc00000);
+    lse_out[t] = ts.finite ? ts.lse : 0.0f;
+    coef_out[t] = ts.coef;
+    if (!ts.finite && dev_status) atomicOr(dev_status, RLF_DEV_NONFINITE);
 }
 
 // forward-only pass from target ids alone: z_target per token (NaN and a status bit for an id outside
@@ -778,35 +791,16 @@ combine_rows_kernel(const float2* __restrict__ part, int nsplit, int rows_max, c
     const int n = max(0, min(*count - off, rows_max));
     if (r >= n) return;
     const int t = idx[off + r];
-    float M = -INFINITY;
-    for (int j = 0; j < nsplit; ++j) M = fmaxf(M, part[(long long)r * nsplit + j].x);
-    float S = 0.0f;
-    for (int j = 0; j < nsplit; ++j) {
-        const float2 ms = part[(long long)r * nsplit + j];
-        if (ms.x != -INFINITY) S += ms.y * expf(ms.x - M);
-    }
-    const float lse = M + logf(S);
-    const float logp = (zy[t] - M) - logf(S);
-    const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) && (fabsf(logp) < INFINITY);
     const float4 rc = rec[t];
-    const bool live = (__float_as_int(rc.w) < 0) && finite;
-    float coef = 0.0f;
-    if (live) {
-        const long long N = *denom;
-        const float inv_n = wtok ? wtok[t] : 1.0f / (float)(N > 1 ? N : 1);
-        const float A = rc.z;
-        const float rho = expf(logp - rc.x);
-        const bool clipped = ((A > 0.0f) && (rho > 1.0f + eps_hi)) || ((A < 0.0f) && (rho < 1.0f - eps_clip));
-        const float dpg = clipped ? 0.0f : -A * rho;
-        coef = -inv_n * fmaf(beta, -expm1f(rc.y - logp), dpg);
-    }
-    logp_out[t] = finite ? logp : __int_as_float(0x7fc00000);
+    const TokenStats ts = token_stats(part + (long long)r * nsplit, nsplit, zy[t], rc, wtok, t, denom, eps_clip, eps_hi,
+                                      beta);
+    logp_out[t] = ts.finite ? ts.logp : __int_as_float(0x7fc00000);
     if (lse_g) {
-        lse_g[off + r] = finite ? lse : 0.0f;
-        coef_g[off + r] = coef;
+        lse_g[off + r] = ts.finite ? ts.lse : 0.0f;
+        coef_g[off + r] = ts.coef;
         y_g[off + r] = __float_as_int(rc.w) & 0x7fffffff;
     }
-    if (!finite && dev_status) atomicOr(dev_status, RLF_DEV_NONFINITE);
+    if (!ts.finite && dev_status) atomicOr(dev_status, RLF_DEV_NONFINITE);
 }
 
 // in place over one chunk of stored exponentials e = exp(z - tile max): dZ = coef (e exp(tile max - lse)
