@@ -585,16 +585,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 }
 
 // ---- small kernels around it ----------------------------------------------------------------
-// z_target[t] = <hidden[t, :], W[ids[t], :]> in fp32: one warp per token
-__global__ void __launch_bounds__(256)
-target_logit_kernel(const __nv_bfloat16* __restrict__ hidden, const __nv_bfloat16* __restrict__ W,
-                    const float4* __restrict__ rec, int64_t T, int32_t D, float* __restrict__ zy) {
-    const int64_t t = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (t >= T) return;
-    const int lane = threadIdx.x & 31;
-    const int y = __float_as_int(rec[t].w) & 0x7fffffff;
-    const uint4* h = reinterpret_cast<const uint4*>(hidden + t * (int64_t)D);
-    const uint4* w = reinterpret_cast<const uint4*>(W + (int64_t)y * D);
+// <h, w> over D bf16 elements by one warp, fp32 accumulation (every lane gets the sum)
+__device__ __forceinline__ float warp_dot_bf16(const uint4* __restrict__ h, const uint4* __restrict__ w, int D, int lane) {
     float acc = 0.0f;
     for (int i = lane; i < D / 8; i += 32) {
         const uint4 a = h[i], b = w[i];
@@ -605,7 +597,20 @@ target_logit_kernel(const __nv_bfloat16* __restrict__ hidden, const __nv_bfloat1
             acc = fmaf(__uint_as_float(aw[k] & 0xffff0000u), __uint_as_float(bw[k] & 0xffff0000u), acc);
         }
     }
-    acc = warp_sum(acc);
+    return warp_sum(acc);
+}
+
+// z_target[t] = <hidden[t, :], W[ids[t], :]> in fp32: one warp per token
+__global__ void __launch_bounds__(256)
+target_logit_kernel(const __nv_bfloat16* __restrict__ hidden, const __nv_bfloat16* __restrict__ W,
+                    const float4* __restrict__ rec, int64_t T, int32_t D, float* __restrict__ zy) {
+    const int64_t t = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (t >= T) return;
+    const int lane = threadIdx.x & 31;
+    const int y = __float_as_int(rec[t].w) & 0x7fffffff;
+    const uint4* h = reinterpret_cast<const uint4*>(hidden + t * (int64_t)D);
+    const uint4* w = reinterpret_cast<const uint4*>(W + (int64_t)y * D);
+    const float acc = warp_dot_bf16(h, w, D, lane);
     if (lane == 0) zy[t] = acc;
 }
 
@@ -677,17 +682,7 @@ target_logit_ids_kernel(const __nv_bfloat16* __restrict__ hidden, const __nv_bfl
     }
     const uint4* h = reinterpret_cast<const uint4*>(hidden + t * (int64_t)D);
     const uint4* w = reinterpret_cast<const uint4*>(W + (int64_t)y * D);
-    float acc = 0.0f;
-    for (int i = lane; i < D / 8; i += 32) {
-        const uint4 a = h[i], b = w[i];
-        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            acc = fmaf(__uint_as_float(aw[k] << 16), __uint_as_float(bw[k] << 16), acc);
-            acc = fmaf(__uint_as_float(aw[k] & 0xffff0000u), __uint_as_float(bw[k] & 0xffff0000u), acc);
-        }
-    }
-    acc = warp_sum(acc);
+    const float acc = warp_dot_bf16(h, w, D, lane);
     if (lane == 0) zy[t] = acc;
 }
 
