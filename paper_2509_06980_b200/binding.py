@@ -52,8 +52,25 @@ _lib.rlf_launch_count.restype = _i64
 _lib.rlf_status_string.argtypes = [_int]
 _lib.rlf_status_string.restype = ctypes.c_char_p
 _lib.rlf_version.restype = _int
-for _n in ("rlf_build_loss_mask", "rlf_group_advantage", "rlf_grpo_logp_loss_fwd_bwd",
-           "rlf_fused_lmhead_grpo", "rlf_grpo_step_host", "rlf_tune_logits_kernel"):
+_lib.rlf_tune_logits_grid.argtypes = [_int, _int]
+_lib.rlf_tune_lmhead.argtypes = [_int]
+_lib.rlf_tune_lmhead_schedule.argtypes = [_int, _int, _int]
+_lib.rlf_rule_reward.argtypes = [_vp, _vp, _i32, _i32, _vp, _vp]
+_lib.rlf_kl_in_reward.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _int, _vp, _vp, _vp, _vp]
+_lib.rlf_grpo_logp_loss_fwd_bwd_obj.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _f32,
+                                                _f32, _f32, _int, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+_lib.rlf_grpo_logp_loss_fwd_bwd_skip_masked.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _i32, _vp, _vp, _vp,
+                                                        _f32, _f32, _vp, _vp, _vp, _vp, _int, _vp, _sz, _vp, _vp]
+_lib.rlf_logp_entropy_fwd.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+_lib.rlf_fused_lmhead_grpo_obj.argtypes = [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _f32, _f32,
+                                           _f32, _int, _int, _vp, _vp, _vp, _vp, _vp, _int, _vp, _sz, _vp, _vp]
+_lib.rlf_fused_lmhead_logp_entropy.argtypes = [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+# every entry point that returns an rlf_status
+for _n in ("rlf_build_loss_mask", "rlf_group_advantage", "rlf_rule_reward", "rlf_kl_in_reward",
+           "rlf_grpo_logp_loss_fwd_bwd", "rlf_grpo_logp_loss_fwd_bwd_obj", "rlf_grpo_logp_loss_fwd_bwd_skip_masked",
+           "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_fused_lmhead_grpo_obj",
+           "rlf_fused_lmhead_logp_entropy", "rlf_grpo_step_host", "rlf_tune_logits_kernel", "rlf_tune_logits_grid",
+           "rlf_tune_lmhead", "rlf_tune_lmhead_schedule"):
     getattr(_lib, _n).restype = _int
 
 
@@ -120,20 +137,14 @@ def tune_logits_kernel(cluster_ctas=0, threads_per_cta=0, one_exp=-1):
 
 
 def tune_logits_grid(rows_per_cluster=0, units_per_cta=0):
-    _lib.rlf_tune_logits_grid.argtypes = [_int, _int]
-    _lib.rlf_tune_logits_grid.restype = _int
     _check(_lib.rlf_tune_logits_grid(int(rows_per_cluster), int(units_per_cta)), "rlf_tune_logits_grid")
 
 
 def tune_lmhead(pair_ctas=1):
-    _lib.rlf_tune_lmhead.argtypes = [_int]
-    _lib.rlf_tune_lmhead.restype = _int
     _check(_lib.rlf_tune_lmhead(int(pair_ctas)), "rlf_tune_lmhead")
 
 
 def tune_lmhead_schedule(m_block=0, max_workers=0, chunk_tiles=0):
-    _lib.rlf_tune_lmhead_schedule.argtypes = [_int, _int, _int]
-    _lib.rlf_tune_lmhead_schedule.restype = _int
     _check(_lib.rlf_tune_lmhead_schedule(int(m_block), int(max_workers), int(chunk_tiles)),
            "rlf_tune_lmhead_schedule")
 
@@ -175,8 +186,6 @@ def rlf_rule_reward(scores, weights, reward_out=None):
     B, n = scores.shape
     if reward_out is None:
         reward_out = torch.empty(B, dtype=torch.float32, device=scores.device)
-    _lib.rlf_rule_reward.argtypes = [_vp, _vp, _i32, _i32, _vp, _vp]
-    _lib.rlf_rule_reward.restype = _int
     _check(_lib.rlf_rule_reward(_ptr(scores, torch.float32), _ptr(weights, torch.float32), B, n,
                                 _ptr(reward_out, torch.float32), _stream()), "rlf_rule_reward")
     return reward_out
@@ -196,8 +205,6 @@ def rlf_kl_in_reward(rewards, old_logp, ref_logp, mask, cu_seqlens, beta, kl_kin
         reward_out = torch.empty(B, dtype=torch.float32, device=dev)
     if kl_seq_out is None:
         kl_seq_out = torch.empty(B, dtype=torch.float32, device=dev)
-    _lib.rlf_kl_in_reward.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _int, _vp, _vp, _vp, _vp]
-    _lib.rlf_kl_in_reward.restype = _int
     _check(_lib.rlf_kl_in_reward(_ptr(rewards, torch.float32), _ptr(old_logp, torch.float32),
                                  _ptr(ref_logp, torch.float32), _ptr(mask, torch.uint8),
                                  _ptr(cu_seqlens, torch.int32), B, T, float(beta), int(kl_kind),
@@ -255,9 +262,6 @@ def rlf_grpo_logp_loss_fwd_bwd_obj(logits, ids, seq_id, adv, old_logp, ref_logp,
     if workspace is None:
         workspace = new_workspace(FN_LOGP_LOSS, T, V, 0, dt, dev)
     f = _lib.rlf_grpo_logp_loss_fwd_bwd_obj
-    f.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _f32, _f32, _f32, _int, _vp, _vp, _vp,
-                  _vp, _vp, _sz, _vp, _vp]
-    f.restype = _int
     _check(f(logits.data_ptr() if T > 0 else None, dt, T, V, stride, _ptr(ids, torch.int32), _ptr(seq_id, torch.int32),
              _ptr(adv, torch.float32), adv.shape[0], _ptr(old_logp, torch.float32), _ptr(ref_logp, torch.float32),
              _ptr(mask, torch.uint8), float(eps_clip_low), float(eps_clip_high), float(beta_kl), int(aggregation),
@@ -285,9 +289,6 @@ def rlf_grpo_logp_loss_fwd_bwd_skip_masked(logits, ids, seq_id, adv, old_logp, r
     if workspace is None:
         workspace = new_workspace(FN_LOGP_LOSS, T, V, 0, dt, dev)
     f = _lib.rlf_grpo_logp_loss_fwd_bwd_skip_masked
-    f.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _f32, _f32, _vp, _vp, _vp, _vp, _int,
-                  _vp, _sz, _vp, _vp]
-    f.restype = _int
     _check(f(logits.data_ptr() if T > 0 else None, dt, T, V, stride, _ptr(ids, torch.int32), _ptr(seq_id, torch.int32),
              _ptr(adv, torch.float32), adv.shape[0], _ptr(old_logp, torch.float32), _ptr(ref_logp, torch.float32),
              _ptr(mask, torch.uint8), float(eps_clip), float(beta_kl), _ptr(denom, torch.int64),
@@ -311,8 +312,6 @@ def rlf_logp_entropy_fwd(logits, ids, want_entropy=True, logp_out=None, entropy_
     dt = _dt(logits)
     if workspace is None:
         workspace = new_workspace(FN_LOGP_ENTROPY, T, V, 0, dt, dev)
-    _lib.rlf_logp_entropy_fwd.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
-    _lib.rlf_logp_entropy_fwd.restype = _int
     _check(_lib.rlf_logp_entropy_fwd(logits.data_ptr() if T > 0 else None, dt, T, V, stride, _ptr(ids, torch.int32),
                                      _ptr(logp_out, torch.float32), _ptr(entropy_out, torch.float32),
                                      workspace.data_ptr(), workspace.numel(), _ptr(dev_status, torch.int32),
@@ -390,10 +389,6 @@ def rlf_fused_lmhead_grpo_obj(hidden, W, ids, seq_id, adv, old_logp, ref_logp, m
         loss_out = torch.empty(4, dtype=torch.float64, device=dev)
     if workspace is None:
         workspace = new_workspace(FN_FUSED_LMHEAD, T, V, D, RLF_BF16, dev)
-    _lib.rlf_fused_lmhead_grpo_obj.argtypes = [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _f32,
-                                               _f32, _f32, _int, _int, _vp, _vp, _vp, _vp, _vp, _int, _vp, _sz,
-                                               _vp, _vp]
-    _lib.rlf_fused_lmhead_grpo_obj.restype = _int
     _check(_lib.rlf_fused_lmhead_grpo_obj(
         _ptr(hidden, torch.bfloat16), _ptr(W, torch.bfloat16), T, D, V, _ptr(ids, torch.int32),
         _ptr(seq_id, torch.int32), _ptr(adv, torch.float32), adv.shape[0], _ptr(old_logp, torch.float32),
@@ -417,8 +412,6 @@ def rlf_fused_lmhead_logp_entropy(hidden, W, ids, want_entropy=True, logp_out=No
         entropy_out = torch.empty(T, dtype=torch.float32, device=dev)
     if workspace is None:
         workspace = new_workspace(FN_FUSED_LOGP_ENTROPY, T, V, D, RLF_BF16, dev)
-    _lib.rlf_fused_lmhead_logp_entropy.argtypes = [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
-    _lib.rlf_fused_lmhead_logp_entropy.restype = _int
     _check(_lib.rlf_fused_lmhead_logp_entropy(
         _ptr(hidden, torch.bfloat16) if T > 0 else None, _ptr(W, torch.bfloat16), T, D, V, _ptr(ids, torch.int32),
         _ptr(logp_out, torch.float32), _ptr(entropy_out, torch.float32), workspace.data_ptr(), workspace.numel(),
