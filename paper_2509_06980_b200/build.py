@@ -41,7 +41,7 @@ def build(force=False, verbose=False):
             sys.stderr.write(out)
     if force or procs or _stale(LIB, objs):
         tmp = LIB + ".tmp%d" % os.getpid()
-        subprocess.check_call([nvcc, "-shared", "-o", tmp] + objs)
+        subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp] + objs)
         os.replace(tmp, LIB)
     return LIB
 
