@@ -185,7 +185,7 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3, responses=0
 
 
 # the same for the forward-only log-prob + entropy pass (profiles/logp_entropy_stream_kernel_T4096_ncu_full.md)
-NCU_TRAFFIC_ENTROPY = {"section_sha1": "16eaba301a844ad26f759e3b7a762daf505bb851", "dram_bytes_per_token": 305667.0}
+NCU_TRAFFIC_ENTROPY = {"section_sha1": "301958076486f234067b1a04b5a95e4254d97c46", "dram_bytes_per_token": 305667.0}
 
 
 def _entropy_section_sha1():

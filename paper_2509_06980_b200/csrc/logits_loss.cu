@@ -34,6 +34,7 @@
 // General row kernel (fp32 logits, odd V, unaligned rows): one CTA per row, three sweeps with
 // scalar loads (max, sum, gradient); later sweeps of a row are served by L2 when the row fits.
 #include <atomic>
+#include <type_traits>
 #include <mutex>
 
 #include "common.cuh"
@@ -1239,10 +1240,10 @@ struct StreamParams {
     float4* partial;            // [units][kStreamWarps] (max, sum, usum, -)
 };
 
-template <bool WANT_U>
+template <bool WANT_U, int NV>
 __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm)
 logp_entropy_stream_kernel(const StreamParams p) {
-    constexpr int NV = kStreamNV, THREADS = kStreamThreads;
+    constexpr int THREADS = kStreamThreads;
     extern __shared__ __align__(16) uint4 stage[];      // [NV][THREADS], slot (i, tid) private to thread tid
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -1337,7 +1338,26 @@ logp_entropy_merge_kernel(const float4* __restrict__ partial, int per_row, const
     if (st && dev_status) atomicOr(dev_status, st);
 }
 
-static int stream_chunks(int nvec) { return (nvec + kStreamThreads * kStreamNV - 1) / (kStreamThreads * kStreamNV); }
+// Vectors per thread of a unit.  A row is cut into equal chunks of at most 256 x NV vectors; with NV = 10
+// a row of 1024 vectors (V = 8192) would fill 40 % of its unit's staging slots and leave the rest of the
+// in-flight capacity unused.  The largest NV among 10, 8, 6, 5, 4 that fills at least 85 % of the slots
+// is taken (large units have the least per-unit overhead), else the one that fills the most.
+static int stream_nv(int nvec) {
+    static const int choices[] = {10, 8, 6, 5, 4};
+    int best = kStreamNV;
+    double best_fill = -1.0;
+    for (int nv : choices) {
+        const int chunks = (nvec + kStreamThreads * nv - 1) / (kStreamThreads * nv);
+        const double fill = (double)nvec / ((double)chunks * kStreamThreads * nv);
+        if (fill >= 0.85) return nv;
+        if (fill > best_fill) { best_fill = fill; best = nv; }
+    }
+    return best;
+}
+static int stream_chunks(int nvec) {
+    const int nv = stream_nv(nvec);
+    return (nvec + kStreamThreads * nv - 1) / (kStreamThreads * nv);
+}
 size_t entropy_workspace_bytes(int64_t T, int32_t V) {
     const size_t chunks = V >= 8 ? (size_t)stream_chunks(V >> 3) : 1;
     return loss_workspace_bytes(T) + 16 * ws_tokens(T) * chunks * kStreamWarps + 256;
@@ -1380,7 +1400,8 @@ extern "C" rlf_status rlf_logp_entropy_fwd(const void* logits, rlf_dtype dt, int
                          T < (1ll << 30);
     if (fast_ok && workspace_bytes >= entropy_workspace_bytes(T, V)) {
         // streaming form: chunk partials, then a per-row merge
-        const int smem = kStreamNV * kStreamThreads * 16;   // 40 KB: below the default dynamic limit
+        const int snv = stream_nv(V >> 3);
+        const int smem = snv * kStreamThreads * 16;         // at most 40 KB: below the default dynamic limit
         StreamParams sp;
         sp.logits = static_cast<const __nv_bfloat16*>(logits);
         sp.stride = row_stride;
@@ -1395,8 +1416,18 @@ extern "C" rlf_status rlf_logp_entropy_fwd(const void* logits, rlf_dtype dt, int
         if ((sp.units + upc - 1) / upc > grid) grid = (sp.units + upc - 1) / upc;
         if (grid > sp.units) grid = sp.units;
         if (grid > (1ll << 30)) grid = 1ll << 30;
-        if (entropy_out) logp_entropy_stream_kernel<true><<<(unsigned)grid, kStreamThreads, smem, s>>>(sp);
-        else logp_entropy_stream_kernel<false><<<(unsigned)grid, kStreamThreads, smem, s>>>(sp);
+        auto launch = [&](auto want_u) {
+            constexpr bool U = decltype(want_u)::value;
+            switch (snv) {
+                case 4: logp_entropy_stream_kernel<U, 4><<<(unsigned)grid, kStreamThreads, smem, s>>>(sp); break;
+                case 5: logp_entropy_stream_kernel<U, 5><<<(unsigned)grid, kStreamThreads, smem, s>>>(sp); break;
+                case 6: logp_entropy_stream_kernel<U, 6><<<(unsigned)grid, kStreamThreads, smem, s>>>(sp); break;
+                case 8: logp_entropy_stream_kernel<U, 8><<<(unsigned)grid, kStreamThreads, smem, s>>>(sp); break;
+                default: logp_entropy_stream_kernel<U, 10><<<(unsigned)grid, kStreamThreads, smem, s>>>(sp); break;
+            }
+        };
+        if (entropy_out) launch(std::true_type{});
+        else launch(std::false_type{});
         logp_entropy_merge_kernel<<<(unsigned)((T + 7) / 8), 256, 0, s>>>(
             sp.partial, sp.chunks * kStreamWarps, sp.logits, row_stride, ids, T, V, logp_out, entropy_out, dev_status);
         count_launch(2);

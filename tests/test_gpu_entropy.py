@@ -21,7 +21,10 @@ def _ws(b, form, T, V):
 
 @pytest.mark.parametrize("V,dtype,std", [(151936, "bf16", 3.0), (151936, "bf16", 0.5), (4096, "bf16", 8.0),
                                           (1001, "bf16", 2.0), (1024, "f32", 2.0), (8, "bf16", 1.0),
-                                          (20480, "bf16", 3.0), (20488, "bf16", 3.0), (40968, "bf16", 3.0)])
+                                          (20480, "bf16", 3.0), (20488, "bf16", 3.0), (40968, "bf16", 3.0),
+                                          # unit shapes of the streaming form: 4, 5, 6, 8 vectors per thread
+                                          (8192, "bf16", 3.0), (50304, "bf16", 3.0), (12288, "bf16", 3.0),
+                                          (32000, "bf16", 3.0)])
 @pytest.mark.parametrize("form", ["stream", "cluster"])
 def test_logp_and_entropy_match_oracle(V, dtype, std, form):
     b = gc.binding()
