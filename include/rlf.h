@@ -10,9 +10,21 @@
  * Conventions that hold for every entry point unless stated otherwise:
  *   - Every pointer is DEVICE memory owned by the caller and valid on the
  *     current device until the work queued on `stream` has finished.  The
- *     library allocates nothing, keeps no state between calls and never
- *     synchronises: it validates arguments on the host, queues kernels (and
- *     small memsets) on `stream`, and returns.
+ *     library allocates nothing and never synchronises: it validates
+ *     arguments on the host, queues kernels (and small memsets) on `stream`,
+ *     and returns.  The one exception is rlf_grpo_step_host, which takes HOST
+ *     buffers and ends with a stream synchronisation.
+ *   - State: a compute call leaves nothing behind that a later call depends
+ *     on.  What the library does keep is (a) per-device caches of facts that
+ *     never change while the process lives (the architecture check, kernel
+ *     attributes and occupancy, the device address of the *_static entry
+ *     point's built-in scratch), filled on first use under a lock, and (b) the
+ *     PROCESS-WIDE tuning knobs set by the rlf_tune_* calls.  A knob changes
+ *     every later compute call of every thread (rlf_tune_logits_kernel can
+ *     make a later call return RLF_ERR_UNSUPPORTED for a shape that cannot
+ *     hold a row); the knobs are plain atomics, so set them before compute
+ *     calls start on other threads, not beside them.  Compute calls themselves
+ *     are re-entrant.
  *   - `stream` is a CUDA stream handle (cudaStream_t); NULL is the default stream.
  *   - Host-detectable problems return a negative rlf_status before anything is
  *     queued.  Problems only visible on the device (a target id outside the
@@ -257,7 +269,8 @@ rlf_status rlf_logp_entropy_fwd(const void *logits, rlf_dtype dt, int64_t T, int
  * buffer; only the kernels' scratch (token records and partial sums) moves into the library.
  *
  * The scratch is a fixed array in the library's device image, RLF_STATIC_MAX_TOKENS tokens large
- * (about 1.1 MB; every GPU that loads the library holds it until the process exits).  This call
+ * (about 2.9 MB, the workspace of a batch of that size; every GPU that loads the library holds it
+ * until the process exits).  This call
  * allocates nothing, on the device or through any library: T > RLF_STATIC_MAX_TOKENS returns
  * RLF_ERR_TOO_LARGE before anything is queued.  All other arguments, results and errors are
  * those of rlf_grpo_logp_loss_fwd_bwd, and the same kernels run.
@@ -412,6 +425,15 @@ rlf_status rlf_tune_lmhead(int pair_ctas);
  * tiles).  Results do not depend on m_block or max_workers; the chunk size changes the order in
  * which grad_W is accumulated (fp32 rounding only). */
 rlf_status rlf_tune_lmhead_schedule(int m_block, int max_workers, int chunk_tiles);
+
+/* Backward scratch of the fused LM-head call for later calls in this process.  1 (the built-in choice):
+ * the forward sweep stores exp(z - rho_t) against a per-row reference rho_t known before the sweep (the
+ * row's fp32 target logit plus a constant), each row's factor c_t exp(rho_t - lse_t) is applied by the
+ * gradient contractions, and there is no rescaling pass over the scratch; a chunk holding a row whose
+ * reference proves unusable (its target's log-prob below about -78, or a non-finite sum) is redone the
+ * other way, decided on the device.  0: exponentials against per-tile maxima, rescaled in place into
+ * dZ by one more pass over the scratch.  Results agree to bf16 rounding of dZ. */
+rlf_status rlf_tune_lmhead_backward(int row_reference);
 
 /* Number of kernels this library has launched in this process (for accounting). */
 int64_t rlf_launch_count(void);

@@ -104,8 +104,9 @@ int orc_build_loss_mask(const int32_t *ids, const int32_t *cu_seqlens, int32_t B
  * Group-relative outcome advantage (GRPO, named in Sec. 2.3.2 / Fig. 4):
  *     A_i = (r_i - mean_g) / (std_g + eps),   g = group of response i.
  * std uses divisor n-1 when `unbiased` (n = group size) and n otherwise; a
- * group of one response, or one with zero spread, gets A = 0 by the formula
- * (numerator 0) -- for n = 1 with the unbiased divisor std is defined as 0.
+ * group of one response, or one with zero spread, gets A = 0 (numerator 0;
+ * with eps = 0 the quotient 0/0 is read as 0 too) -- for n = 1 with the
+ * unbiased divisor std is defined as 0.
  * group_id == NULL means contiguous groups of `g_or_num_groups` responses.
  */
 int orc_group_advantage(const float *rewards, const int32_t *group_id, int32_t B,
@@ -136,7 +137,8 @@ int orc_group_advantage(const float *rewards, const int32_t *group_id, int32_t B
         double sd = (div > 0.0) ? sqrt(ss / div) : 0.0;
         for (int32_t i = 0; i < B; ++i) {
             int32_t gi = group_id ? group_id[i] : i / g_or_num_groups;
-            if (gi == g) adv[i] = ((double)rewards[i] - mean) / (sd + eps);
+            /* a group without spread carries no signal: A = 0 also when eps = 0 (0/0 otherwise) */
+            if (gi == g) adv[i] = (sd + eps > 0.0) ? ((double)rewards[i] - mean) / (sd + eps) : 0.0;
         }
     }
     if (group_id)

@@ -41,7 +41,10 @@ group_advantage_kernel(const float* __restrict__ rewards, const int32_t* __restr
         ss = warp_sum_f64(ss);
         const double div = unbiased ? (double)(n - 1) : (double)n;
         const double sd = div > 0.0 ? sqrt(ss / div) : 0.0;
-        const double inv = 1.0 / (sd + (double)eps);
+        // zero spread (or a single member) with eps = 0 would be 0 * inf: such a group carries no
+        // signal and gets A = 0 like every other degenerate group
+        const double den = sd + (double)eps;
+        const double inv = den > 0.0 ? 1.0 / den : 0.0;
         for (int i = lo + lane; i < hi; i += 32) {
             if (!group_id || group_id[i] == g) adv_out[i] = (float)(((double)rewards[i] - mean) * inv);
         }

@@ -85,6 +85,10 @@ struct GemmParams {
     const int* live_count;
     int live_off;
     const int32_t* row_index; // kGradHidden: output row of compact row r is row_index[live_off + r]
+    const float* ref;         // kLse with dz (optional): per-row reference of the stored exponentials (see below)
+    const float* row_scale;   // kGradHidden (optional): fp32 factor of compact row r applied to its output row
+    const int* run_flag;      // optional: the launch does nothing unless *run_flag == run_want
+    int run_want;
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -135,6 +139,9 @@ __device__ __forceinline__ void tc_mma2(uint32_t d_tmem, uint64_t adesc, uint64_
                  "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
 }
+// The multicast here is that of a BARRIER SIGNAL: the commit arrives on the mbarrier at the same offset in
+// both CTAs of the pair (mask 0b11).  No load in this file is multicast -- every cp.async.bulk.tensor
+// below is a plain per-CTA copy -- and every tensor map covers this GPU's own memory.
 __device__ __forceinline__ void tc_commit2(uint32_t bar) {
     const unsigned short both = 3;
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -204,6 +211,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                  const GemmParams p) {
     using C = Cfg<PAIR>;
     extern __shared__ unsigned char smem_raw[];
+    // a launch that is conditional on a device-side flag (uniform over the grid): leave before
+    // anything is set up
+    if (p.run_flag && *p.run_flag != p.run_want) return;
     // operand stages must sit on 1024-byte boundaries (swizzle atom)
     const uint32_t raw = smem_addr(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
@@ -396,7 +406,51 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 }
                 const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * BN;
                 const int col0 = n * BN;
-                if (p.mode == kLse && p.dz) {
+                if (p.mode == kLse && p.dz && p.ref) {
+                    // Forward sweep that keeps the tile for the backward, exponentials taken against a
+                    // reference rho known BEFORE the sweep (one per row): e = exp(z - rho) is summed for
+                    // the log-sum-exp and stored as bf16 in one pass over the accumulator.  bf16 has
+                    // fp32's exponent range, so any rho within some tens of the row's log-sum-exp
+                    // keeps every entry that matters a normal number at full relative precision, and
+                    // dZ = (c_t exp(rho - lse)) e needs only a per-row factor afterwards.  A row whose
+                    // reference turns out too far off shows in its sum (inf, or far from one) and
+                    // sends its chunk through the per-tile-maximum path instead.
+                    const float off = row_ok ? -p.ref[row] * kLog2e : 0.0f;
+                    float ts0 = 0.0f, ts1 = 0.0f;
+#pragma unroll 1
+                    for (int c = 0; c < BN / 32; ++c) {
+                        const int cb = col0 + c * 32;
+                        const int nvalid = max(0, min(32, p.N - cb));
+                        uint32_t o[16];
+                        if (nvalid > 0) {                  // warp-uniform: the tensor-memory load is a warp-wide instruction
+                            uint32_t v[32];
+                            tc_ld32(t_row + (uint32_t)(c * 32), v);
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                float e0 = ex2_approx(fmaf(__uint_as_float(v[2 * i]), kLog2e, off));
+                                float e1 = ex2_approx(fmaf(__uint_as_float(v[2 * i + 1]), kLog2e, off));
+                                if (2 * i >= nvalid) e0 = 0.0f;
+                                if (2 * i + 1 >= nvalid) e1 = 0.0f;
+                                ts0 += e0;
+                                ts1 += e1;
+                                asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[i]) : "f"(e1), "f"(e0));
+                            }
+                        }
+                        if (nvalid <= 0 || !row_ok) {
+                            // columns past the vocabulary and rows past the live extent (up to the end of
+                            // this pair of token tiles) read as zeros in the gradient contractions
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) o[i] = 0u;
+                        }
+                        uint4* d4 = reinterpret_cast<uint4*>(p.dz + dz_offset(row, cb, p.dz_nc));
+                        d4[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                        d4[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                        d4[2] = make_uint4(o[8], o[9], o[10], o[11]);
+                        d4[3] = make_uint4(o[12], o[13], o[14], o[15]);
+                    }
+                    run_s += ts0 + ts1;
+                    if (row_ok) run_m = p.ref[row];
+                } else if (p.mode == kLse && p.dz) {
                     // Forward sweep that keeps the tile for the backward.  Pass 1 over the accumulator:
                     // the row's maximum inside this tile; pass 2: e = exp(z - that maximum), summed for
                     // the log-sum-exp and stored as bf16 (e <= 1: no overflow whatever the logits are;
@@ -511,19 +565,20 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         if (row_ok) {
                             const long long orow = p.row_index ? (long long)p.row_index[p.live_off + row] : (long long)row;
                             __nv_bfloat16* dst = p.out_bf16 + orow * p.out_stride + cb;
+                            const float sc = p.row_scale ? p.row_scale[row] : 1.0f;
                             if (nvalid == 32) {
                                 uint32_t o[16];
 #pragma unroll
                                 for (int i = 0; i < 16; ++i)
                                     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[i])
-                                        : "f"(__uint_as_float(v[2 * i + 1])), "f"(__uint_as_float(v[2 * i])));
+                                        : "f"(__uint_as_float(v[2 * i + 1]) * sc), "f"(__uint_as_float(v[2 * i]) * sc));
                                 uint4* d4 = reinterpret_cast<uint4*>(dst);
                                 d4[0] = make_uint4(o[0], o[1], o[2], o[3]);
                                 d4[1] = make_uint4(o[4], o[5], o[6], o[7]);
                                 d4[2] = make_uint4(o[8], o[9], o[10], o[11]);
                                 d4[3] = make_uint4(o[12], o[13], o[14], o[15]);
                             } else {
-                                for (int i = 0; i < nvalid; ++i) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                                for (int i = 0; i < nvalid; ++i) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]) * sc);
                             }
                         }
                     } else {   // kGradW
@@ -751,12 +806,16 @@ partition_rows_kernel(const float4* __restrict__ rec, int T, int32_t* __restrict
 
 // out row r <- hidden row idx[r] for r < *count; rows up to the next multiple of 256 are zero-filled
 // (the contractions read whole tiles)
+// ref_out (optional): the reference of row r's stored exponentials, its target logit plus kRefShift
+constexpr float kRefShift = 32.0f;
 __global__ void __launch_bounds__(128)
 gather_rows_kernel(const __nv_bfloat16* __restrict__ hidden, int D, const int32_t* __restrict__ idx,
-                   const int* __restrict__ count, __nv_bfloat16* __restrict__ out) {
+                   const int* __restrict__ count, __nv_bfloat16* __restrict__ out, const float* __restrict__ zy,
+                   float* __restrict__ ref_out) {
     const int n = *count;
     const int r = blockIdx.x;
     if (r >= ((n + 255) & ~255)) return;
+    if (ref_out && threadIdx.x == 0) ref_out[r] = r < n ? zy[idx[r]] + kRefShift : 0.0f;
     uint4* dst = reinterpret_cast<uint4*>(out + (long long)r * D);
     const int nv = D / 8;
     if (r < n) {
@@ -775,13 +834,26 @@ fill_nan_rows_kernel(const int32_t* __restrict__ idx, const int* __restrict__ co
 }
 
 // combine_kernel for a launch over gathered rows: row r of the launch (partials part[r][.]) is token
-// idx[off + r]; logp goes to the token's place, lse / coefficient / target id to the gathered place
+// idx[off + r]; logp goes to the token's place, lse / coefficient / target id to the gathered place.
+//
+// With ref_g (the sweep stored e = exp(z - rho_r), rho_r = ref_g[off + r]) the kernel also finishes the
+// row for the gradient contractions: scale_g = c_t exp(rho - lse), the per-row factor that turns the
+// stored exponentials into dZ, and the target column of the scratch is overwritten with
+// (p_y - 1) exp(lse - rho) (formed in fp32 from the fp32 target logit), so that factor x entry is
+// c_t (p_y - 1) to bf16 rounding even when p_y is close to one.  The reference is usable while the
+// factor and the entries stay normal numbers: a row with a non-finite sum or lse - rho above
+// kRefWindow raises *fallback instead of a status bit, and the chunk is redone with per-tile maxima.
+// Without ref_g, scale_g (if given) is set to one: the scratch will hold dZ itself.
+constexpr float kRefWindow = 46.0f;
 __global__ void __launch_bounds__(256)
 combine_rows_kernel(const float2* __restrict__ part, int nsplit, int rows_max, const int32_t* __restrict__ idx,
                     const int* __restrict__ count, int off, const float* __restrict__ zy,
                     const float4* __restrict__ rec, const long long* __restrict__ denom, float eps_clip, float eps_hi,
                     const float* __restrict__ wtok, float beta, float* __restrict__ logp_out, float* __restrict__ lse_g,
-                    float* __restrict__ coef_g, int32_t* __restrict__ y_g, int32_t* __restrict__ dev_status) {
+                    float* __restrict__ coef_g, int32_t* __restrict__ y_g, int32_t* __restrict__ dev_status,
+                    const float* __restrict__ ref_g, float* __restrict__ scale_g, __nv_bfloat16* __restrict__ dz,
+                    int dz_nc, int V, int* __restrict__ fallback, const int* __restrict__ run_flag, int run_want) {
+    if (run_flag && *run_flag != run_want) return;
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     const int n = max(0, min(*count - off, rows_max));
     if (r >= n) return;
@@ -790,12 +862,55 @@ combine_rows_kernel(const float2* __restrict__ part, int nsplit, int rows_max, c
     const TokenStats ts = token_stats(part + (long long)r * nsplit, nsplit, zy[t], rc, wtok, t, denom, eps_clip, eps_hi,
                                       beta);
     logp_out[t] = ts.finite ? ts.logp : __int_as_float(0x7fc00000);
+    const int y = __float_as_int(rc.w) & 0x7fffffff;
     if (lse_g) {
         lse_g[off + r] = ts.finite ? ts.lse : 0.0f;
         coef_g[off + r] = ts.coef;
-        y_g[off + r] = __float_as_int(rc.w) & 0x7fffffff;
+        y_g[off + r] = y;
     }
+    if (ref_g) {
+        const float rho = ref_g[off + r];
+        const bool usable = ts.finite && (ts.lse - rho <= kRefWindow);
+        if (!usable) {
+            atomicOr(fallback, 1);
+            scale_g[off + r] = 0.0f;
+            return;
+        }
+        scale_g[off + r] = ts.coef * expf(rho - ts.lse);
+        if (ts.coef != 0.0f && y < V) dz[dz_offset(r, y, dz_nc)] = __float2bfloat16_rn(expm1f(ts.logp) * expf(ts.lse - rho));
+        return;
+    }
+    if (scale_g) scale_g[off + r] = 1.0f;
     if (!ts.finite && dev_status) atomicOr(dev_status, RLF_DEV_NONFINITE);
+}
+
+// Hs[r, :] = bf16(scale[off + r] * Hl[r, :]) for the rows of one chunk: the token-side operand of
+// grad_W = e^T (scale H) when the scratch holds exponentials against a per-row reference.  Rows from
+// the live extent up to the next multiple of 256 become zeros.
+__global__ void __launch_bounds__(128)
+scale_rows_kernel(const __nv_bfloat16* __restrict__ Hl, int D, int rows_max, const int* __restrict__ count, int off,
+                  const float* __restrict__ scale_g, __nv_bfloat16* __restrict__ Hs) {
+    const int n = max(0, min(*count - off, rows_max));
+    const int r = blockIdx.x;
+    if (r >= ((n + 255) & ~255)) return;
+    uint4* dst = reinterpret_cast<uint4*>(Hs + (long long)r * D);
+    const int nv = D / 8;
+    if (r >= n) {
+        for (int i = threadIdx.x; i < nv; i += blockDim.x) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+        return;
+    }
+    const float f = scale_g[off + r];
+    const uint4* src = reinterpret_cast<const uint4*>(Hl + (long long)r * D);
+    for (int i = threadIdx.x; i < nv; i += blockDim.x) {
+        const uint4 z = src[i];
+        const uint32_t w[4] = {z.x, z.y, z.z, z.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(o[k])
+                : "f"(__uint_as_float(w[k] & 0xffff0000u) * f), "f"(__uint_as_float(w[k] << 16) * f));
+        dst[i] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
 }
 
 // in place over one chunk of stored exponentials e = exp(z - tile max): dZ = coef (e exp(tile max - lse)
@@ -806,8 +921,9 @@ __global__ void __launch_bounds__(256)
 dz_from_e_kernel(__nv_bfloat16* __restrict__ ebuf, int V, int n_tiles, const float* __restrict__ tmax, int rows_max,
                  const int* __restrict__ count, int off, const float* __restrict__ lse_g,
                  const float* __restrict__ coef_g, const int32_t* __restrict__ y_g, const int32_t* __restrict__ idx,
-                 const float* __restrict__ zy) {
+                 const float* __restrict__ zy, const int* __restrict__ run_flag, int run_want) {
     __shared__ float f_s[kDzBlockRows];          // signed scale of each row for this column tile
+    if (run_flag && *run_flag != run_want) return;
     __shared__ int live_s[kDzBlockRows];
     const int n = max(0, min(*count - off, rows_max));
     const int tt = blockIdx.x, jt = blockIdx.y;
@@ -899,6 +1015,7 @@ static std::atomic<int> g_pair{1};       // 1: cta_group::2 pair form, 0: single
 static std::atomic<int> g_m_block{0};    // row units per scheduling block of the sweep; 0: automatic
 static std::atomic<int> g_max_workers{0};   // persistent CTAs (or pairs) per launch; 0: one per SM (pair of SMs)
 static std::atomic<int> g_chunk_tiles{0};   // token tiles per backward chunk; 0: the most the workspace holds
+static std::atomic<int> g_row_ref{1};       // backward scratch: 1 exponentials against a per-row reference, 0 per-tile maxima
 
 template <bool PAIR>
 static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, cudaStream_t s) {
@@ -977,7 +1094,8 @@ static int pick_split(int n_tiles) {
 }
 
 struct LmWs {
-    size_t n_count, partial, rec, zy, lse, coef, wtok, seqcnt, part, idx_live, idx_dead, lse_g, coef_g, y_g, hidden_g, tmax, dz, total;
+    size_t n_count, partial, rec, zy, lse, coef, wtok, seqcnt, part, idx_live, idx_dead, lse_g, coef_g, y_g, ref_g, scale_g,
+        hidden_g, hidden_s, tmax, dz, total;
 };
 static size_t up1k(size_t x) { return (x + 1023) & ~(size_t)1023; }
 static LmWs lm_workspace(int64_t T, int32_t V, int32_t D) {
@@ -985,7 +1103,7 @@ static LmWs lm_workspace(int64_t T, int32_t V, int32_t D) {
     size_t o = 0;
     const size_t Tn = (size_t)(T > 0 ? T : 0);
     const size_t Tp = (Tn + 255) & ~(size_t)255;     // compact arrays are padded to whole tile pairs
-    w.n_count = o; o += 1024;                        // [0] mask count, [64] live / other row counts
+    w.n_count = o; o += 1024;                        // [0] mask count, [64] live / other row counts, [128] chunk flag
     w.partial = o; o += up1k(token_loss_partial_bytes());
     w.rec = o;     o += up1k(16 * Tn);
     w.zy = o;      o += up1k(4 * Tn);
@@ -999,8 +1117,11 @@ static LmWs lm_workspace(int64_t T, int32_t V, int32_t D) {
     w.lse_g = o;   o += up1k(4 * Tp);
     w.coef_g = o;  o += up1k(4 * Tp);
     w.y_g = o;     o += up1k(4 * Tp);
+    w.ref_g = o;   o += up1k(4 * Tp);                // per-row reference of the stored exponentials
+    w.scale_g = o; o += up1k(4 * Tp);                // per-row factor exponentials -> dZ
     w.hidden_g = o; o += 2 * up1k(Tp * (size_t)(D > 0 ? D : 0) * 2);   // live rows, then the others
     const size_t chunk = Tp < (size_t)kChunkTokens ? Tp : (size_t)kChunkTokens;
+    w.hidden_s = o; o += up1k(chunk * (size_t)(D > 0 ? D : 0) * 2);    // one chunk of live rows times their factors
     w.tmax = o;    o += up1k(4 * chunk * (size_t)((V + BN - 1) / BN));
     w.dz = o;
     o += up1k(chunk * (size_t)((V + BN - 1) / BN) * BN * 2);     // blocked: whole 256-column tiles
@@ -1139,14 +1260,22 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
     const int64_t Tp = (T + 255) & ~(int64_t)255;
     __nv_bfloat16* Hl = reinterpret_cast<__nv_bfloat16*>(ws + w.hidden_g);
     __nv_bfloat16* Hd = reinterpret_cast<__nv_bfloat16*>(ws + w.hidden_g + up1k((size_t)Tp * D * 2));
+    const bool bwd = grad_hidden || grad_W;
+    // backward scratch: exponentials against a per-row reference (no rescaling pass; the per-tile-maximum
+    // path stays queued behind a device flag for chunks whose reference turns out unusable), or the
+    // per-tile-maximum path alone
+    const bool row_ref = bwd && g_row_ref.load() != 0;
+    float* ref_g = reinterpret_cast<float*>(ws + w.ref_g);
+    float* scale_g = reinterpret_cast<float*>(ws + w.scale_g);
+    __nv_bfloat16* Hs = reinterpret_cast<__nv_bfloat16*>(ws + w.hidden_s);
+    int* chunk_flag = reinterpret_cast<int*>(ws + w.n_count + 128);
     partition_rows_kernel<<<1, 1024, 0, s>>>(rec, (int)T, idx_live, idx_dead, counts);
-    gather_rows_kernel<<<(unsigned)Tp, 128, 0, s>>>(H, D, idx_live, counts, Hl);
-    if (!skip_masked) gather_rows_kernel<<<(unsigned)Tp, 128, 0, s>>>(H, D, idx_dead, counts + 1, Hd);
+    gather_rows_kernel<<<(unsigned)Tp, 128, 0, s>>>(H, D, idx_live, counts, Hl, zy, row_ref ? ref_g : nullptr);
+    if (!skip_masked) gather_rows_kernel<<<(unsigned)Tp, 128, 0, s>>>(H, D, idx_dead, counts + 1, Hd, nullptr, nullptr);
     count_launch(skip_masked ? 2 : 3);
     if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
     if (grad_hidden && cudaMemsetAsync(grad_hidden, 0, (size_t)T * D * 2, s) != cudaSuccess) return RLF_ERR_CUDA;
 
-    const bool bwd = grad_hidden || grad_W;
     const int tuned_tiles = g_chunk_tiles.load();
     const int64_t chunk_tokens = (tuned_tiles > 0 && tuned_tiles * BM < kChunkTokens) ? tuned_tiles * BM : kChunkTokens;
     for (int64_t t0 = 0; t0 < T; t0 += chunk_tokens) {
@@ -1162,22 +1291,49 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
         }
         z.live_count = counts;
         z.live_off = (int)t0;
-        st = launch_gemm(mapHc, mapW, z, pair, s);
-        if (st != RLF_OK) return st;
-        combine_rows_kernel<<<(unsigned)((tc + 255) / 256), 256, 0, s>>>(part, z.nsplit, (int)tc, idx_live, counts, (int)t0,
-                                                                          zy, rec, dn, eps_clip, eps_hi, wtok, beta_kl,
-                                                                          logp_out, lse_g, coef_g, y_g, dev_status);
-        count_launch();
-        if (!bwd) continue;
+        auto combine = [&](bool with_ref, const int* run_flag) {
+            combine_rows_kernel<<<(unsigned)((tc + 255) / 256), 256, 0, s>>>(
+                part, z.nsplit, (int)tc, idx_live, counts, (int)t0, zy, rec, dn, eps_clip, eps_hi, wtok, beta_kl, logp_out,
+                lse_g, coef_g, y_g, dev_status, with_ref ? ref_g : nullptr, row_ref ? scale_g : nullptr, dz, z.dz_nc, V,
+                chunk_flag, run_flag, 1);
+            count_launch();
+        };
         const int64_t tcp = (tc + 255) & ~(int64_t)255;
-        dz_from_e_kernel<<<dim3((unsigned)(tcp / kDzBlockRows), (unsigned)z.n_tiles), 256, 0, s>>>(
-            dz, V, z.n_tiles, z.tmax, (int)tc, counts, (int)t0, lse_g, coef_g, y_g, idx_live, zy);
+        auto dz_pass = [&](const int* run_flag) {
+            dz_from_e_kernel<<<dim3((unsigned)(tcp / kDzBlockRows), (unsigned)z.n_tiles), 256, 0, s>>>(
+                dz, V, z.n_tiles, z.tmax, (int)tc, counts, (int)t0, lse_g, coef_g, y_g, idx_live, zy, run_flag, 1);
+            count_launch();
+        };
+        if (row_ref) {
+            if (cudaMemsetAsync(chunk_flag, 0, sizeof(int), s) != cudaSuccess) return RLF_ERR_CUDA;
+            z.ref = ref_g + t0;
+            st = launch_gemm(mapHc, mapW, z, pair, s);
+            if (st != RLF_OK) return st;
+            combine(true, nullptr);
+            // queued always, run only if some row of the chunk raised the flag: the chunk again with
+            // per-tile maxima, rescaled in place into dZ (every row's factor becomes one)
+            GemmParams zf = z;
+            zf.ref = nullptr;
+            zf.run_flag = chunk_flag;
+            zf.run_want = 1;
+            st = launch_gemm(mapHc, mapW, zf, pair, s);
+            if (st != RLF_OK) return st;
+            combine(false, chunk_flag);
+            dz_pass(chunk_flag);
+            scale_rows_kernel<<<(unsigned)tcp, 128, 0, s>>>(Hl + t0 * D, D, (int)tc, counts, (int)t0, scale_g, Hs);
+            count_launch();
+        } else {
+            st = launch_gemm(mapHc, mapW, z, pair, s);
+            if (st != RLF_OK) return st;
+            combine(false, nullptr);
+            if (!bwd) continue;
+            dz_pass(nullptr);
+        }
         // the scratch as the contractions see it: rows of 64 columns, 128 rows per block
         const uint64_t dz_rows = (uint64_t)(tcp / kDzBlockRows) * (uint64_t)(4 * z.n_tiles) * kDzBlockRows;
-        count_launch();
         if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
         if (grad_hidden) {
-            // grad_hidden[token of gathered row] = dZ[chunk, V] W[V, D]
+            // grad_hidden[token of gathered row] = (row factor) dZ[chunk, V] W[V, D]
             CUtensorMap mapDzK, mapWn;
             if (!make_map(&mapDzK, dz, dz_rows, kDzBlockCols, kDzBlockCols, BK, BM)) return RLF_ERR_CUDA;
             if (!make_map(&mapWn, Wm, (uint64_t)V, (uint64_t)D, (uint64_t)D, 64, BK)) return RLF_ERR_CUDA;
@@ -1195,14 +1351,16 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
             h.live_count = counts;
             h.live_off = (int)t0;
             h.row_index = idx_live;
+            h.row_scale = row_ref ? scale_g + t0 : nullptr;
             st = launch_gemm(mapDzK, mapWn, h, pair, s);
             if (st != RLF_OK) return st;
         }
         if (grad_W) {
-            // grad_W[V, D] (+)= dZ[chunk, V]^T hidden[chunk, D]
+            // grad_W[V, D] (+)= dZ[chunk, V]^T hidden[chunk, D]  (hidden rows times their factors)
             CUtensorMap mapDzM, mapHn;
             if (!make_map(&mapDzM, dz, dz_rows, kDzBlockCols, kDzBlockCols, 64, BK)) return RLF_ERR_CUDA;
-            if (!make_map(&mapHn, Hl + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, 64, BK)) return RLF_ERR_CUDA;
+            if (!make_map(&mapHn, row_ref ? Hs : Hl + t0 * D, (uint64_t)tc, (uint64_t)D, (uint64_t)D, 64, BK))
+                return RLF_ERR_CUDA;
             GemmParams q = {};
             q.mode = kGradW;
             q.M = V;
@@ -1238,7 +1396,8 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
         if (st != RLF_OK) return st;
         combine_rows_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(part, d.nsplit, (int)T, idx_dead, counts + 1, 0, zy,
                                                                          rec, dn, eps_clip, eps_hi, wtok, beta_kl, logp_out,
-                                                                         nullptr, nullptr, nullptr, dev_status);
+                                                                         nullptr, nullptr, nullptr, dev_status, nullptr,
+                                                                         nullptr, nullptr, 0, V, nullptr, nullptr, 0);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
     }
@@ -1329,6 +1488,12 @@ extern "C" rlf_status rlf_fused_lmhead_logp_entropy(const void* hidden, const vo
 extern "C" rlf_status rlf_tune_lmhead(int pair_ctas) {
     if (pair_ctas != 0 && pair_ctas != 1) return RLF_ERR_SHAPE;
     rlf::lm::g_pair = pair_ctas;
+    return RLF_OK;
+}
+
+extern "C" rlf_status rlf_tune_lmhead_backward(int row_reference) {
+    if (row_reference != 0 && row_reference != 1) return RLF_ERR_SHAPE;
+    rlf::lm::g_row_ref = row_reference;
     return RLF_OK;
 }
 

@@ -49,14 +49,15 @@ constexpr size_t kWsRecordOff = kWsPartialOff + sizeof(double) * 4 * kMaxPartial
 
 // the skip-masked variant adds, after the records: compacted records (16 B per token), the list of
 // live rows (4 B per token); its live-row counter sits at byte 128 of the workspace
-static size_t ws_tokens(int64_t T) { return (size_t)(T > 0 ? T : 0); }
-static size_t ws_compact_rec_off(int64_t T) { return kWsRecordOff + 16 * ws_tokens(T) + 256; }
-static size_t ws_row_list_off(int64_t T) { return ws_compact_rec_off(T) + 16 * ws_tokens(T) + 256; }
+constexpr size_t ws_tokens(int64_t T) { return (size_t)(T > 0 ? T : 0); }
+constexpr size_t ws_compact_rec_off(int64_t T) { return kWsRecordOff + 16 * ws_tokens(T) + 256; }
+constexpr size_t ws_row_list_off(int64_t T) { return ws_compact_rec_off(T) + 16 * ws_tokens(T) + 256; }
 // then per-token weights (4 B per token) and per-sequence counters (4 B x (T + 1)) of the
 // sequence-mean aggregation
-static size_t ws_wtok_off(int64_t T) { return ws_row_list_off(T) + 4 * ws_tokens(T) + 256; }
-static size_t ws_seqcnt_off(int64_t T) { return ws_wtok_off(T) + 4 * ws_tokens(T) + 256; }
-size_t loss_workspace_bytes(int64_t T) { return ws_seqcnt_off(T) + 4 * (ws_tokens(T) + 1) + 256; }
+constexpr size_t ws_wtok_off(int64_t T) { return ws_row_list_off(T) + 4 * ws_tokens(T) + 256; }
+constexpr size_t ws_seqcnt_off(int64_t T) { return ws_wtok_off(T) + 4 * ws_tokens(T) + 256; }
+constexpr size_t ws_total_bytes(int64_t T) { return ws_seqcnt_off(T) + 4 * (ws_tokens(T) + 1) + 256; }
+size_t loss_workspace_bytes(int64_t T) { return ws_total_bytes(T); }
 
 // ---------------------------------------------------------------------------------------------
 // token records
@@ -1714,7 +1715,12 @@ size_t token_loss_partial_bytes() { return sizeof(double) * 4 * kMaxPartials; }
 // Variant for callers that cannot allocate: the scratch lives in the library's device image.
 namespace rlf {
 
-constexpr size_t kStaticScratchBytes = kWsRecordOff + 16 * (size_t)RLF_STATIC_MAX_TOKENS + 256;
+// The array is sized by the same layout function that the workspace check of the forwarded call
+// uses, so a batch of RLF_STATIC_MAX_TOKENS tokens always fits (about 2.9 MB per device).
+constexpr size_t kStaticScratchBytes = (ws_total_bytes(RLF_STATIC_MAX_TOKENS) + 255) & ~(size_t)255;
+static_assert(kStaticScratchBytes >= ws_total_bytes(RLF_STATIC_MAX_TOKENS) &&
+              ws_total_bytes(RLF_STATIC_MAX_TOKENS) >= ws_total_bytes(RLF_STATIC_MAX_TOKENS - 1),
+              "the built-in scratch must hold the workspace of the largest batch the entry point accepts");
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 // Device address of the scratch array on the current device.  In host code the array's name only

@@ -6,7 +6,7 @@ the rewards of its own GRPO group.  So a batch is cut between groups: every rank
 all-reduce sums over NCCL:
 
   1. the int64 count of loss-carrying tokens, before the loss kernel (its coefficients divide by the
-     global count);  for the sequence mean, the count of responses that carry loss instead;
+     global count);
   2. the four fp64 loss scalars, after it (each rank's are already divided by the global count, so
      they add up);
   3. for the fused LM-head path, grad_W [V, D] fp32 (the ordinary data-parallel weight-gradient
@@ -103,18 +103,22 @@ def loss_phase(n_global, mask, seq_id, ids, rewards, group_size, old_logp, ref_l
 
 def sharded_grpo_step(ids, cu_seqlens, rewards, group_size, old_logp, ref_logp, open_id, close_id, eps_clip, beta_kl,
                       logits=None, hidden=None, W=None, grad_W=None, accumulate_grad_W=False, adv_eps=1e-6,
-                      group=None, ops=None, reduce_grad_W=True):
+                      group=None, ops=None, reduce_grad_W=True, n_global=None):
     """This rank's part of one sharded step.  All tensors are this rank's own (whole groups).
 
     Give `logits` [T_local, V] for the logits path (returns grad_logits) or `hidden` [T_local, D] and
     `W` [V, D] for the fused LM-head path (returns grad_hidden and the all-reduced grad_W).
     `group`: the process group of the ranks that share the batch (None or a group of one: no exchange).
     When grad_W is accumulated over several micro-batches, pass reduce_grad_W=False on all but the
-    last one (a reduced buffer must not be reduced again).
+    last one (a reduced buffer must not be reduced again), and pass the whole batch's token count as
+    `n_global` (int64[1], e.g. the n_global a counting pass over the whole shard returned): a
+    micro-batch's own count is not the batch's denominator.  With `n_global` given the count exchange
+    is skipped.
     -> dict(mask, seq_id, n_local, n_global, adv, logp, loss (global, fp64[4]), grad_logits | grad_hidden, grad_W)
     """
     mask, seq_id, n_local = count_phase(ids, cu_seqlens, open_id, close_id, ops)
-    n_global = _all_reduce_sum(n_local.clone(), group)
+    if n_global is None:
+        n_global = _all_reduce_sum(n_local.clone(), group)
     out = loss_phase(n_global, mask, seq_id, ids, rewards, group_size, old_logp, ref_logp, eps_clip, beta_kl,
                      logits=logits, hidden=hidden, W=W, grad_W=grad_W, accumulate_grad_W=accumulate_grad_W,
                      adv_eps=adv_eps, ops=ops)

@@ -45,6 +45,40 @@ def oracle_chain(batch, logits_np=None, want_grad=True, rows=None):
     return out
 
 
+def oracle_all_rows_through_fp64_head(hidden, W, ora, old, ref, row_chunk=2048):
+    """Every row's log-prob and the scalar loss of the fused path from the oracle at full size.
+    The head contraction z = H W^T is the one library step: torch.matmul in fp64 on the GPU (bf16
+    inputs widened exactly), a chunk of rows at a time; each chunk's fp64 logits go to the host and
+    through orc_grpo_loss (dtype f64) with the batch's token count as denominator, so the chunks'
+    loss terms add up to the batch's.  Nothing of the library under test is involved.
+    -> (logp f64[T], loss f64[4])"""
+    T = hidden.shape[0]
+    W64 = W.double()
+    logp = np.empty(T, np.float64)
+    loss = np.zeros(4, np.float64)
+    for r0 in range(0, T, row_chunk):
+        sl = slice(r0, min(T, r0 + row_chunk))
+        z = torch.matmul(hidden[sl].double(), W64.t()).cpu().numpy()
+        r = orc.grpo_loss(z, ora["ids"][sl], ora["seq_id"][sl], ora["adv"], old[sl], ref[sl], ora["mask"][sl],
+                          synth.EPS_CLIP, synth.BETA_KL, denom=ora["n"], want_grad=False)
+        logp[sl] = r["logp"]
+        loss += np.asarray(r["loss"], np.float64)
+        del z
+    del W64
+    torch.cuda.empty_cache()
+    return logp, loss
+
+
+def loss_floor(ora):
+    """Scale below which a relative loss error is not meaningful: the surrogate's mean nearly cancels
+    under zero-mean advantages and ratios near one, while a log-prob error e (allowed up to
+    LOGP_ATOL) moves a token's term by |A| rho e.  The floor is that permitted movement,
+    LOGP_ATOL x mean |A| over the unmasked tokens."""
+    a_tok = np.abs(ora["adv"].astype(np.float64))[ora["seq_id"]]
+    m = ora["mask"].astype(np.float64)
+    return LOGP_ATOL * float((a_tok * m).sum() / max(m.sum(), 1.0))
+
+
 def gpu_chain(batch, logits, in_place=False, want_grad=True, dev_status=None):
     b = binding()
     mask, seq, n = b.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, batch.spec.open_id, batch.spec.close_id,

@@ -42,11 +42,12 @@ def test_binding_lists_the_same_symbols():
 def test_status_strings_and_version(lib):
     lib.rlf_status_string.restype = ctypes.c_char_p
     seen = set()
-    for code in range(0, -9, -1):
+    for code in range(0, -10, -1):           # RLF_OK .. RLF_ERR_TOO_LARGE (-9)
         s = lib.rlf_status_string(code).decode()
         assert s and s != "unknown status"
         seen.add(s)
-    assert len(seen) == 9
+    assert len(seen) == 10
+    assert "RLF_STATIC_MAX_TOKENS" in lib.rlf_status_string(-9).decode()
     assert lib.rlf_status_string(-99).decode() == "unknown status"
     assert lib.rlf_version() >= 100
 

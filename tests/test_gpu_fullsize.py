@@ -6,6 +6,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import rlf_oracle as orc
 from paper_2509_06980_b200 import synth
 import gpu_common as gc
 from util import loss_close, ulp_error_bf16
@@ -88,6 +89,64 @@ def test_cfg2_ragged_sampled_rows():
     assert loss_close(loss[0].item(), r["loss"][0], 1e-9, gc.LOSS_RTOL)
     guard = gc.near_clip_bound(r["logp"], old.cpu().numpy(), None)
     assert ulp_error_bf16(gc.grad_to_f64(grad)[~guard], r["grad"][~guard]).max() <= gc.GRAD_ULPS
+
+
+def test_cfg2_full_size_in_place_against_oracle():
+    """The ragged recipe at its stated size, the way it has to be run there: one launch over all
+    ~133k rows (40 GB of bf16 logits) with grad_logits written over the logits.  The oracle's forward
+    pass runs over every row before the call (chunk by chunk, while the logits still exist); 640 sampled
+    rows, among them the first and last row of several responses, are snapshotted for the element-wise
+    gradient comparison."""
+    dev = "cuda"
+    spec = synth.SPECS[2]
+    batch = synth.make_batch(spec, dev)
+    T, V = batch.logits.shape
+    assert V == 151936 and 100_000 < T < 180_000 and batch.rewards.shape[0] == 64
+    ora = gc.oracle_chain(batch)
+    old, ref = batch.old_logp.cpu().numpy(), batch.ref_logp.cpu().numpy()
+
+    logp_o = np.empty(T, np.float64)
+    loss_o = np.zeros(4, np.float64)
+    for r0 in range(0, T, 4096):
+        sl = slice(r0, min(T, r0 + 4096))
+        r = orc.grpo_loss(gc.to_np(batch.logits[sl]), ora["ids"][sl], ora["seq_id"][sl], ora["adv"], old[sl], ref[sl],
+                          ora["mask"][sl], synth.EPS_CLIP, synth.BETA_KL, denom=ora["n"], want_grad=False)
+        logp_o[sl] = r["logp"]
+        loss_o += np.asarray(r["loss"], np.float64)
+
+    rng = np.random.default_rng(2)
+    cu = batch.tokens.cu_seqlens.astype(np.int64)
+    edges = np.concatenate([cu[:9], cu[1:9] - 1, [T - 1]])
+    rows = np.unique(np.concatenate([edges, rng.choice(T, size=640, replace=False)]))
+    rt = torch.as_tensor(rows, device=dev)
+    snap = batch.logits[rt].clone()
+    sub = orc.grpo_loss(gc.to_np(snap), ora["ids"][rows], ora["seq_id"][rows], ora["adv"], old[rows], ref[rows],
+                        ora["mask"][rows], synth.EPS_CLIP, synth.BETA_KL, denom=ora["n"], want_coef=True)
+
+    st = torch.zeros(1, dtype=torch.int32, device=dev)
+    ptr = batch.logits.data_ptr()
+    gpu = gc.gpu_chain(batch, batch.logits, in_place=True, dev_status=st)
+    assert st.item() == 0 and gpu["grad"].data_ptr() == ptr
+    assert np.array_equal(gpu["mask"].cpu().numpy(), ora["mask"]) and gpu["n"].item() == ora["n"]
+    assert np.array_equal(gpu["seq_id"].cpu().numpy(), ora["seq_id"])
+    assert np.abs(gpu["logp"].cpu().numpy() - logp_o).max() <= gc.LOGP_ATOL
+    lg = gpu["loss"].cpu().numpy()
+    for k in range(3):
+        assert loss_close(lg[k], loss_o[k], 1e-6, gc.LOSS_RTOL), (k, lg, loss_o)
+
+    g = gc.grad_to_f64(gpu["grad"][rt])
+    guard = gc.near_clip_bound(sub["logp"], old[rows], None)
+    ulps = gc.grad_ulps(g[~guard], sub["grad"][~guard], ora["ids"][rows][~guard], sub["coef"][~guard])
+    assert ulps.max() <= gc.GRAD_ULPS
+    assert (g[ora["mask"][rows] == 0] == 0).all()
+
+    grad = gpu["grad"]
+    m = gpu["mask"].bool()
+    coef_scale = np.abs(sub["coef"]).max()
+    for r0 in range(0, T, 4096):
+        blk, mb = grad[r0:r0 + 4096], m[r0:r0 + 4096]
+        assert not blk[~mb].any()
+        assert blk[mb].float().sum(dim=1).abs().max().item() <= 0.05 * coef_scale
 
 
 def test_cfg1_full_size_is_bitwise_stable_over_repeated_launches():

@@ -1,8 +1,8 @@
 """Full-size parity of the Qwen3-8B-shaped long-context recipe (T = 65536 = 8 x 8192, D = 4096,
 V = 151936), processed the way the recipe words it: 8 micro-batches of one 8192-token response with the
 batch's token count as denominator.  Fused LM-head path: grad_W accumulated over the micro-batches;
-log-probs and grad_hidden rows of sampled tokens against the oracle, the scalar loss against the token
-terms in fp64, grad_W through its zero column sums and against the single-call result.  Logits
+grad_hidden rows of sampled tokens against the oracle, every row's log-prob and the summed scalar loss
+against the oracle run on fp64 logits of the whole batch, grad_W through its zero column sums and against the single-call result.  Logits
 path: one micro-batch of bf16 logits formed from the hidden states (the recipe's stand-in for the model's
 own head), sampled rows against the oracle."""
 import numpy as np
@@ -62,15 +62,16 @@ def test_cfg4_full_size_micro_batched():
     _close_tensor(gh[rt].float().cpu().numpy(), r["grad_hidden"], "grad_hidden rows")
     assert not gh[~mask.bool()].any()
 
-    lp = logp.double().cpu()
-    A = torch.from_numpy(ora["adv"].astype(np.float64))[torch.from_numpy(ora["seq_id"]).long()]
-    rho = torch.exp(lp - batch.old_logp.double().cpu())
-    pg = -torch.minimum(rho * A, torch.clamp(rho, 1 - synth.EPS_CLIP, 1 + synth.EPS_CLIP) * A)
-    d = batch.ref_logp.double().cpu() - lp
-    m = torch.from_numpy(ora["mask"].astype(np.float64))
-    want = float((m * (pg + synth.BETA_KL * (torch.exp(d) - d - 1))).sum() / ora["n"])
-    floor = gc.LOGP_ATOL * float((A.abs() * m).sum() / m.sum())
-    assert loss_close(loss_sum[0].item(), want, floor, gc.LOSS_RTOL)
+    # every row of all eight micro-batches: log-prob and the summed scalar loss against the oracle
+    # (fp64 logits from the library's fp64 contraction, then the oracle's loss)
+    logp_o, loss_o = gc.oracle_all_rows_through_fp64_head(batch.hidden, batch.W, ora, batch.old_logp.cpu().numpy(),
+                                                          batch.ref_logp.cpu().numpy(), row_chunk=2048)
+    assert np.abs(logp.cpu().numpy() - logp_o).max() <= gc.LOGP_ATOL
+    assert np.abs(logp_o[rows] - r["logp"]).max() <= 1e-9
+    floor = gc.loss_floor(ora)
+    ls = loss_sum.cpu().numpy()
+    for k in range(3):
+        assert loss_close(ls[k], loss_o[k], floor if k < 2 else 1e-9, gc.LOSS_RTOL), (k, ls, loss_o)
 
     col = gw.double().sum(dim=0).abs().max().item()
     assert col <= 1e-3 * gw.double().abs().sum(dim=0).max().item()

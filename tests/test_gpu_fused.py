@@ -104,8 +104,8 @@ def test_fused_full_vocabulary_and_hidden_reduced_T():
 def test_cfg3_full_size_sampled_rows_and_invariants():
     """The launch configuration the benchmark times (T = 32768, D = 2560, V = 151936): log-probs and
     grad_hidden rows of sampled tokens against the oracle (a token's row depends only on that token
-    and the batch's token count); the scalar loss against the token terms evaluated in fp64 from the
-    returned log-probs; grad_W through the invariant that its columns sum to zero over the vocabulary."""
+    and the batch's token count); every row's log-prob and the scalar loss against the oracle run on
+    fp64 logits of the whole batch; grad_W through the invariant that its columns sum to zero over the vocabulary."""
     b = gc.binding()
     spec = synth.SPECS[3]
     batch = synth.make_batch(spec, DEV)
@@ -135,15 +135,16 @@ def test_cfg3_full_size_sampled_rows_and_invariants():
     _close_tensor(gh[rt].float().cpu().numpy(), r["grad_hidden"], "grad_hidden rows")
     assert not gh[~mask.bool()].any()
 
-    # scalar loss = masked token mean of the token terms at the returned log-probs
-    lp = logp.double().cpu()
-    A = torch.from_numpy(ora["adv"].astype(np.float64))[torch.from_numpy(ora["seq_id"]).long()]
-    rho = torch.exp(lp - batch.old_logp.double().cpu())
-    pg = -torch.minimum(rho * A, torch.clamp(rho, 1 - synth.EPS_CLIP, 1 + synth.EPS_CLIP) * A)
-    d = batch.ref_logp.double().cpu() - lp
-    m = torch.from_numpy(ora["mask"].astype(np.float64))
-    want = float((m * (pg + synth.BETA_KL * (torch.exp(d) - d - 1))).sum() / ora["n"])
-    assert loss_close(loss[0].item(), want, 1e-6, gc.LOSS_RTOL)
+    # every row's log-prob and the scalar loss against the oracle (fp64 logits from the library's
+    # fp64 contraction, then the oracle's loss over all 32768 rows)
+    logp_o, loss_o = gc.oracle_all_rows_through_fp64_head(batch.hidden, batch.W, ora, batch.old_logp.cpu().numpy(),
+                                                          batch.ref_logp.cpu().numpy())
+    assert np.abs(logp.cpu().numpy() - logp_o).max() <= gc.LOGP_ATOL
+    assert np.abs(logp_o[rows] - r["logp"]).max() <= 1e-9      # the two oracle routes agree on the sampled rows
+    lg = loss.cpu().numpy()
+    floor = gc.loss_floor(ora)
+    for k in range(3):
+        assert loss_close(lg[k], loss_o[k], floor if k < 2 else 1e-9, gc.LOSS_RTOL), (k, lg, loss_o)
 
     col = gw.double().sum(dim=0).abs().max().item()
     assert col <= 1e-3 * gw.double().abs().sum(dim=0).max().item()
@@ -162,7 +163,7 @@ def test_cfg3_full_size_sampled_rows_and_invariants():
     assert torch.equal(gh, gh2) and torch.equal(gw, gw2) and torch.equal(loss, loss2)
     assert torch.equal(logp[livem], logp2[livem]) and torch.isnan(logp2[~livem]).all()
     assert (logp3 - logp).abs().max().item() <= 1e-4
-    assert loss_close(loss3[0].item(), want, 1e-6, gc.LOSS_RTOL)
+    assert loss_close(loss3[0].item(), loss_o[0], floor, gc.LOSS_RTOL)
 
 
 def test_cfg4_head_shape_reduced_T():
@@ -280,3 +281,90 @@ def test_fused_malformed_rows_are_neutralised_and_reported():
     assert loss_close(loss[0].item(), r["loss"][0], 1e-6, gc.LOSS_RTOL)
     _close_tensor(gh.float().cpu().numpy(), r["grad_hidden"], "grad_hidden")
     _close_tensor(gw.cpu().numpy(), r["grad_W"], "grad_W")
+
+
+def _fused_call(b, batch, mask, seq, adv, n, st):
+    return b.rlf_fused_lmhead_grpo(batch.hidden, batch.W, batch.ids, seq, adv, batch.old_logp, batch.ref_logp, mask,
+                                   synth.EPS_CLIP, synth.BETA_KL, denom=n, dev_status=st)
+
+
+@pytest.mark.parametrize("V,D", [(2048, 128), (4096 + 264, 320)])
+def test_backward_scratch_forms_agree_and_both_match_the_oracle(V, D, form):
+    """The two forms of the backward scratch (exponentials against a per-row reference, applied as a row
+    factor by the gradient contractions; exponentials against per-tile maxima, rescaled in place) on the
+    same batch: each within the per-tensor tolerance of the oracle, the log-probs within rounding of each
+    other, and NOT bit-identical gradients (they round dZ at different places), which shows that the
+    switch switches something."""
+    b = gc.binding()
+    spec = synth.scaled(synth.SPECS[3], V=V, D=D, w_std=0.3, **SMALL)
+    batch = synth.make_batch(spec, DEV)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    mask, seq, n = b.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, spec.open_id, spec.close_id)
+    adv = b.rlf_group_advantage(batch.rewards, group_size=batch.tokens.group_size)
+    ora = gc.oracle_chain(batch)
+    r = orc.fused_lmhead_grpo(synth.bf16_bits(batch.hidden), synth.bf16_bits(batch.W), ora["ids"], ora["seq_id"], ora["adv"],
+                              batch.old_logp.cpu().numpy(), batch.ref_logp.cpu().numpy(), ora["mask"], synth.EPS_CLIP,
+                              synth.BETA_KL, denom=ora["n"])
+    outs = {}
+    try:
+        for row_ref in (1, 0):
+            b.tune_lmhead_backward(row_ref)
+            logp, loss, gh, gw = _fused_call(b, batch, mask, seq, adv, n, st)
+            torch.cuda.synchronize()
+            assert st.item() == 0
+            assert np.abs(logp.cpu().numpy() - r["logp"]).max() <= gc.LOGP_ATOL
+            _close_tensor(gh.float().cpu().numpy(), r["grad_hidden"], "grad_hidden")
+            _close_tensor(gw.cpu().numpy(), r["grad_W"], "grad_W")
+            outs[row_ref] = (logp, loss, gh, gw)
+    finally:
+        b.tune_lmhead_backward(1)
+    assert (outs[1][0] - outs[0][0]).abs().max().item() <= 1e-4
+    assert not torch.equal(outs[1][3], outs[0][3])
+
+
+def test_row_reference_gives_way_when_a_target_has_vanishing_probability(form):
+    """A row's reference is its target logit plus a constant; it stops being usable when the target's
+    log-prob falls below about -78 (the row factor or the stored exponentials would leave the normal
+    range of bf16).  One live token is given a target logit ~120 below its row maximum: the chunk must be
+    redone with per-tile maxima on the device, which shows as results bit-identical to those of the
+    per-tile-maximum form (in a chunk that kept its references they differ), and they match the oracle."""
+    b = gc.binding()
+    spec = synth.scaled(synth.SPECS[3], V=2048, D=128, w_std=0.3, **SMALL)
+    batch = synth.make_batch(spec, DEV)
+    mask, seq, n = b.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, spec.open_id, spec.close_id)
+    adv = b.rlf_group_advantage(batch.rewards, group_size=batch.tokens.group_size)
+    live = torch.nonzero(mask).flatten()
+    t = int(live[11].item())
+    y = int(batch.ids[t].item())
+    other = (y + 7) % 1000                                  # not a marker id, not the target
+    h = batch.hidden[t].float()
+    W = batch.W.clone()
+    W[y] = (-60.0 * h / (h * h).sum()).to(torch.bfloat16)      # z[t, y] ~ -60
+    W[other] = (60.0 * h / (h * h).sum()).to(torch.bfloat16)   # z[t, other] ~ +60
+    batch.W = W
+    z_t = (h.double() @ W.double().t())
+    assert (z_t.max() - z_t[y]).item() > 100.0
+    lp_t = float(z_t[y] - torch.logsumexp(z_t, 0))           # keep that token's ratio and KL term moderate
+    batch.old_logp[t] = lp_t + 0.03
+    batch.ref_logp[t] = lp_t - 0.05
+    ora = gc.oracle_chain(batch)
+    r = orc.fused_lmhead_grpo(synth.bf16_bits(batch.hidden), synth.bf16_bits(batch.W), ora["ids"], ora["seq_id"], ora["adv"],
+                              batch.old_logp.cpu().numpy(), batch.ref_logp.cpu().numpy(), ora["mask"], synth.EPS_CLIP,
+                              synth.BETA_KL, denom=ora["n"])
+    assert r["logp"][t] < -100.0
+    outs = {}
+    try:
+        for row_ref in (1, 0):
+            b.tune_lmhead_backward(row_ref)
+            st = torch.zeros(1, dtype=torch.int32, device=DEV)
+            outs[row_ref] = _fused_call(b, batch, mask, seq, adv, n, st)
+            torch.cuda.synchronize()
+            assert st.item() == 0
+    finally:
+        b.tune_lmhead_backward(1)
+    logp, loss, gh, gw = outs[1]
+    assert np.abs(logp.cpu().numpy() - r["logp"]).max() <= gc.LOGP_ATOL
+    _close_tensor(gh.float().cpu().numpy(), r["grad_hidden"], "grad_hidden")
+    _close_tensor(gw.cpu().numpy(), r["grad_W"], "grad_W")
+    for got, want in zip(outs[1], outs[0]):
+        assert torch.equal(got, want)

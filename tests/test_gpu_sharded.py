@@ -82,3 +82,32 @@ def test_fused_path_shards_add_up():
         assert (o["grad_hidden"].float() - gh[p["rows"]].float()).abs().max().item() <= 2.0 ** -7 * scale
     assert torch.allclose(loss, ls, rtol=1e-6, atol=1e-12)
     assert (gw_sum - gw).abs().max().item() <= 2.0 ** -7 * gw.abs().max().item()
+
+
+def test_fused_step_in_a_group_of_one_against_the_oracle():
+    """sharded_grpo_step itself (count phase, loss phase, the three exchanges degenerate in a group of
+    one) on the fused LM-head path, every output against the CPU oracle rather than against another
+    GPU call."""
+    from oracle import rlf_oracle as orc
+    spec = synth.scaled(synth.SPECS[3], V=2048 + 136, D=128, w_std=0.3, num_prompts=3, group_size=4, len_lo=20, len_hi=36,
+                        spans_lo=1, spans_hi=2, obs_lo=2, obs_hi=4)
+    batch = synth.make_batch(spec, DEV)
+    out = sharded.sharded_grpo_step(batch.ids, batch.cu_seqlens, batch.rewards, spec.group_size, batch.old_logp,
+                                    batch.ref_logp, spec.open_id, spec.close_id, synth.EPS_CLIP, synth.BETA_KL,
+                                    hidden=batch.hidden, W=batch.W)
+    torch.cuda.synchronize()
+    ora = gc.oracle_chain(batch)
+    assert np.array_equal(out["mask"].cpu().numpy(), ora["mask"]) and np.array_equal(out["seq_id"].cpu().numpy(), ora["seq_id"])
+    assert out["n_local"].item() == out["n_global"].item() == ora["n"]
+    assert np.abs(out["adv"].cpu().numpy() - ora["adv64"]).max() <= 1e-6
+    r = orc.fused_lmhead_grpo(synth.bf16_bits(batch.hidden), synth.bf16_bits(batch.W), ora["ids"], ora["seq_id"], ora["adv"],
+                              batch.old_logp.cpu().numpy(), batch.ref_logp.cpu().numpy(), ora["mask"], synth.EPS_CLIP,
+                              synth.BETA_KL, denom=ora["n"])
+    assert np.abs(out["logp"].cpu().numpy() - r["logp"]).max() <= gc.LOGP_ATOL
+    from util import loss_close
+    lg = out["loss"].cpu().numpy()
+    for k in range(3):
+        assert loss_close(lg[k], r["loss"][k], gc.loss_floor(ora) if k < 2 else 1e-9, gc.LOSS_RTOL), (k, lg, r["loss"])
+    for name in ("grad_hidden", "grad_W"):
+        got = out[name].float().cpu().numpy().astype(np.float64)
+        assert np.abs(got - r[name]).max() <= 2.0 ** -7 * np.abs(r[name]).max(), name

@@ -68,3 +68,38 @@ def test_reference_arm_prints_nothing_on_nonzero_ranks(monkeypatch, capsys):
         steps, warmup, gpus = 1, 0, 2
     bench.run_reference(A)
     assert capsys.readouterr().out == ""
+
+
+def test_plain_start_with_several_gpus_becomes_a_launcher_of_that_many_ranks(monkeypatch):
+    """`python bench.py --gpus 4` outside torchrun must not time one GPU and call it four: it re-runs
+    its own command line as four ranks and hands their exit code on."""
+    sys.path.insert(0, ROOT)
+    import subprocess
+    import pytest
+    import bench
+    seen = {}
+
+    def fake_call(cmd):
+        seen["cmd"] = cmd
+        return 7
+    monkeypatch.setattr(subprocess, "call", fake_call)
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "4", "--steps", "2", "--warmup", "3"])
+    with pytest.raises(SystemExit) as e:
+        bench.main()
+    assert e.value.code == 7
+    cmd = seen["cmd"]
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--nproc-per-node") + 1] == "4" and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-6:] == ["--gpus", "4", "--steps", "2", "--warmup", "3"] and cmd[-7].endswith("bench.py")
+
+
+def test_rank_count_that_differs_from_gpus_is_refused(monkeypatch):
+    sys.path.insert(0, ROOT)
+    import pytest
+    import bench
+    monkeypatch.setenv("WORLD_SIZE", "2")
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "8"])
+    with pytest.raises(SystemExit) as e:
+        bench.main()
+    assert "n_gpus" in str(e.value.code)

@@ -61,6 +61,19 @@ def test_degenerate_groups_give_zero():
     assert (a1 == 0.0).all()
 
 
+def test_degenerate_groups_give_zero_also_without_eps():
+    # eps = 0: the formula reads 0 / 0 for a group without spread; the reading is A = 0 (no signal),
+    # never NaN, for both std conventions, for a single-member group, and beside a healthy group
+    r = np.array([1, 1, 1, 1, 0, 1, 0, 1], np.float32)
+    for unbiased in (True, False):
+        a = orc.group_advantage(r, group_size=4, eps=0.0, unbiased=unbiased)
+        assert np.isfinite(a).all() and (a[:4] == 0.0).all()
+        sd = np.std(r[4:].astype(np.float64), ddof=1 if unbiased else 0)
+        assert np.allclose(a[4:], (r[4:] - 0.5) / sd, atol=1e-12)
+    a1 = orc.group_advantage(np.array([0.3, 0.9], np.float32), group_size=1, eps=0.0)
+    assert (a1 == 0.0).all()
+
+
 def test_explicit_group_ids_match_contiguous_groups():
     rng = np.random.default_rng(5)
     r = rng.random(12).astype(np.float32)

@@ -116,8 +116,23 @@ def _worker(rank, world, port, out):
                            torch.from_numpy(t_k["old"]), torch.from_numpy(t_k["ref"]), 0.2, 0.05, hidden=P["H"][rows_k],
                            W=P["W"], grad_W=gw, accumulate_grad_W=k > 0, ops=oracle_ops)
     dist.all_reduce(gw)
+    # the same two micro-batches through the step itself: accumulate without reducing, then accumulate
+    # and reduce once; the batch's token count is handed in, so no count exchange takes place
+    gw2 = torch.zeros((P["V"], P["D"]), dtype=torch.float64)
+    loss2 = torch.zeros(4, dtype=torch.float64)
+    for k, part in enumerate(parts):
+        cu_k, t_k, r_k = sharded.take_shard(part, P["cu"], tok, {"rewards": P["rewards"]})
+        rows_k = torch.from_numpy(t_k["rows"])
+        o = sharded.sharded_grpo_step(torch.from_numpy(t_k["ids"]), torch.from_numpy(cu_k),
+                                      torch.from_numpy(r_k["rewards"]), old_logp=torch.from_numpy(t_k["old"]),
+                                      ref_logp=torch.from_numpy(t_k["ref"]), hidden=P["H"][rows_k], W=P["W"],
+                                      grad_W=gw2, accumulate_grad_W=k > 0, reduce_grad_W=(k == len(parts) - 1),
+                                      n_global=n_all, **common)
+        assert o["grad_W"] is gw2 and o["n_global"] is n_all
+        loss2 += o["loss"]
     out.put((rank, t["rows"], a["n_local"].item(), a["n_global"].item(), a["loss"].numpy(), a["grad_logits"].numpy(),
-             a["logp"].numpy(), b["loss"].numpy(), b["grad_hidden"].numpy(), b["grad_W"].numpy(), gw.numpy()))
+             a["logp"].numpy(), b["loss"].numpy(), b["grad_hidden"].numpy(), b["grad_W"].numpy(), gw.numpy(),
+             gw2.numpy(), loss2.numpy()))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -156,4 +171,6 @@ def test_two_ranks_add_up_to_the_unsharded_step():
         assert np.allclose(g[8], Bf["grad_hidden"].numpy()[rows], rtol=1e-11, atol=1e-16)
         assert np.allclose(g[9], Bf["grad_W"].numpy(), rtol=1e-10, atol=1e-15)         # all-reduced weight gradient
         assert np.allclose(g[10], Bf["grad_W"].numpy(), rtol=1e-10, atol=1e-15)        # accumulated, reduced once
+        assert np.allclose(g[11], Bf["grad_W"].numpy(), rtol=1e-10, atol=1e-15)        # ... by the step's own flags
+        assert np.allclose(g[12], Bf["loss"].numpy(), rtol=1e-12, atol=1e-15)          # micro-batch losses add up
     assert sorted(np.concatenate([got[0][1], got[1][1]]).tolist()) == list(range(len(P["ids"])))

@@ -52,6 +52,37 @@ def test_static_scratch_variant_matches_workspace_variant_on_two_calls_in_a_row(
         assert (g_logp - w_logp).abs().max().item() <= gc.LOGP_ATOL
 
 
+@pytest.mark.parametrize("T", [23807, 23808, 32768, 65536])
+def test_static_scratch_variant_takes_every_batch_size_up_to_its_stated_maximum(T):
+    """Batches near and at RLF_STATIC_MAX_TOKENS (small vocabulary, so the logits stay a few MB): the
+    built-in scratch must be as large as the workspace the ordinary entry point asks for at that size.
+    23808 is the first size at which an array holding the token records alone would be too small,
+    32768 the token count of the Qwen3-4B-shaped micro-batch."""
+    b = gc.binding()
+    assert T <= b.STATIC_MAX_TOKENS
+    g = torch.Generator(device=DEV).manual_seed(T)
+    V, B = 64, 16
+    logits = (torch.randn((T, V), generator=g, device=DEV) * 3.0).to(torch.bfloat16)
+    ids = torch.randint(0, V, (T,), generator=g, device=DEV, dtype=torch.int32)
+    seq = (torch.arange(T, device=DEV, dtype=torch.int64) * B // T).to(torch.int32)
+    adv = torch.randn(B, generator=g, device=DEV)
+    old = -torch.rand(T, generator=g, device=DEV) * 6.0
+    ref = old + 0.1 * torch.randn(T, generator=g, device=DEV)
+    mask = (torch.rand(T, generator=g, device=DEV) < 0.6).to(torch.uint8)
+    n = mask.sum().to(torch.int64).reshape(1)
+    want = b.rlf_grpo_logp_loss_fwd_bwd(logits, ids, seq, adv, old, ref, mask, synth.EPS_CLIP, synth.BETA_KL, denom=n)
+    for _ in range(2):
+        logp = torch.full((T,), 7.0, dtype=torch.float32, device=DEV)
+        loss = torch.full((4,), 7.0, dtype=torch.float64, device=DEV)
+        grad = torch.full_like(logits, 7.0)
+        st = torch.zeros(1, dtype=torch.int32, device=DEV)
+        b.rlf_grpo_logp_loss_fwd_bwd_static(logits, ids, seq, adv, old, ref, mask, synth.EPS_CLIP, synth.BETA_KL,
+                                            n, logp, loss, grad, st)
+        torch.cuda.synchronize()
+        assert st.item() == 0
+        assert torch.equal(logp, want[0]) and torch.equal(loss, want[1]) and torch.equal(grad, want[2])
+
+
 def test_static_scratch_variant_without_a_denominator_counts_the_mask_itself():
     b = gc.binding()
     batch = synth.make_batch(synth.scaled(synth.SPECS[1], len_lo=16, len_hi=16, spans_lo=1, spans_hi=1,
