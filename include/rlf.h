@@ -420,8 +420,8 @@ rlf_status rlf_tune_lmhead(int pair_ctas);
  * in pair form) times as many vocabulary splits as it takes to occupy them all; smaller blocks keep
  * less of the hidden states in L2 at a time and stream the head more often.  max_workers: upper
  * bound on the persistent CTAs (pairs) of every contraction launch.  chunk_tiles: 128-token tiles
- * per chunk of the backward (even; at most the 74 the workspace is sized for).  0 restores the
- * built-in choice (m_block = half the number of workers; one worker per SM or pair of SMs; 74
+ * per chunk of the backward (even; at most the 148 the workspace is sized for).  0 restores the
+ * built-in choice (m_block = half the number of workers; one worker per SM or pair of SMs; 148
  * tiles).  Results do not depend on m_block or max_workers; the chunk size changes the order in
  * which grad_W is accumulated (fp32 rounding only). */
 rlf_status rlf_tune_lmhead_schedule(int m_block, int max_workers, int chunk_tiles);
@@ -432,8 +432,12 @@ rlf_status rlf_tune_lmhead_schedule(int m_block, int max_workers, int chunk_tile
  * gradient contractions, and there is no rescaling pass over the scratch; a chunk holding a row whose
  * reference proves unusable (its target's log-prob below about -78, or a non-finite sum) is redone the
  * other way, decided on the device.  0: exponentials against per-tile maxima, rescaled in place into
- * dZ by one more pass over the scratch.  Results agree to bf16 rounding of dZ. */
-rlf_status rlf_tune_lmhead_backward(int row_reference);
+ * dZ by one more pass over the scratch.  Results agree to bf16 rounding of dZ.
+ * two_accumulators (pair form only): 1 (built-in) = in the two gradient contractions a CTA pair
+ * multiplies two 256-row tiles against each 256-column slab it stages (three quarters of the
+ * shared-memory fill per flop, half the passes over the head or the hidden states); 0 = one tile per
+ * pair with a double-buffered accumulator, as in the forward sweep.  Results are bit-identical. */
+rlf_status rlf_tune_lmhead_backward(int row_reference, int two_accumulators);
 
 /* Number of kernels this library has launched in this process (for accounting). */
 int64_t rlf_launch_count(void);

@@ -55,7 +55,7 @@ _lib.rlf_version.restype = _int
 _lib.rlf_tune_logits_grid.argtypes = [_int, _int]
 _lib.rlf_tune_lmhead.argtypes = [_int]
 _lib.rlf_tune_lmhead_schedule.argtypes = [_int, _int, _int]
-_lib.rlf_tune_lmhead_backward.argtypes = [_int]
+_lib.rlf_tune_lmhead_backward.argtypes = [_int, _int]
 _lib.rlf_rule_reward.argtypes = [_vp, _vp, _i32, _i32, _vp, _vp]
 _lib.rlf_kl_in_reward.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _int, _vp, _vp, _vp, _vp]
 _lib.rlf_grpo_logp_loss_fwd_bwd_obj.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _f32,
@@ -145,8 +145,8 @@ def tune_lmhead(pair_ctas=1):
     _check(_lib.rlf_tune_lmhead(int(pair_ctas)), "rlf_tune_lmhead")
 
 
-def tune_lmhead_backward(row_reference=1):
-    _check(_lib.rlf_tune_lmhead_backward(int(row_reference)), "rlf_tune_lmhead_backward")
+def tune_lmhead_backward(row_reference=1, two_accumulators=1):
+    _check(_lib.rlf_tune_lmhead_backward(int(row_reference), int(two_accumulators)), "rlf_tune_lmhead_backward")
 
 
 def tune_lmhead_schedule(m_block=0, max_workers=0, chunk_tiles=0):

@@ -36,11 +36,20 @@ constexpr int BM = 128, BN = 256, BK = 64;
 // each CTA's tensor memory receives its own 128 rows of the accumulator.  Per flop the pair form
 // moves two thirds of the shared-memory bytes of the single form.
 constexpr int kABytes = BM * BK * 2;
-template <bool PAIR> struct Cfg {
-    static constexpr int kStages = PAIR ? 6 : 4;
+// Two-accumulator pair form (ACC2, the two gradient contractions): a pair works on TWO 256-row tiles
+// against the same 256 columns, each CTA staging two A tiles beside its half of B (48 KB per stage, 4
+// stages), so every B slab that crosses L2 -> shared memory is used for 512 rows: three quarters of
+// the shared-memory fill bytes per flop of the plain pair form, and half the passes over the B
+// matrix.  The two accumulators take all 512 TMEM columns, so the drain of a unit does not overlap the
+// next unit's multiplies; with K running over the whole vocabulary or a whole chunk of tokens the
+// drain is a per cent or two of a unit.
+template <bool PAIR, bool ACC2 = false> struct Cfg {
+    static_assert(PAIR || !ACC2, "two accumulators per CTA exist in pair form only");
+    static constexpr int kAcc = ACC2 ? 2 : 1;
+    static constexpr int kStages = ACC2 ? 4 : (PAIR ? 6 : 4);
     static constexpr int kBRows = PAIR ? BN / 2 : BN;
     static constexpr int kBBytes = kBRows * BK * 2;
-    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kStageBytes = kAcc * kABytes + kBBytes;
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
 };
 constexpr int kMaxStages = 6;
@@ -205,11 +214,12 @@ struct SmemCtl {
 };
 
 // ---- the kernel -----------------------------------------------------------------------------
-template <bool PAIR>
+template <bool PAIR, bool ACC2>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const GemmParams p) {
-    using C = Cfg<PAIR>;
+    using C = Cfg<PAIR, ACC2>;
+    constexpr int NACC = C::kAcc;
     extern __shared__ unsigned char smem_raw[];
     // a launch that is conditional on a device-side flag (uniform over the grid): leave before
     // anything is set up
@@ -234,7 +244,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     }
     // no tokens under a grad_W tile: nothing to add; without accumulate the tile is still written (zeros)
     const bool no_k = k_slabs == 0;
-    const int m_units = PAIR ? (m_tiles + 1) / 2 : m_tiles;
+    // token (or vocabulary) tiles per scheduling unit: 1, 2 in pair form, 4 with two accumulators; this
+    // CTA's tile for accumulator a of unit m is kTilesPerUnit * m + 2 * a + rank
+    constexpr int kTilesPerUnit = (PAIR ? 2 : 1) * NACC;
+    const int m_units = (m_tiles + kTilesPerUnit - 1) / kTilesPerUnit;
     const int units = (no_k && p.accumulate) ? 0 : sweep ? m_units * p.nsplit : m_units * p.n_tiles;
     const int worker = PAIR ? blockIdx.x >> 1 : blockIdx.x;
     const int workers = PAIR ? gridDim.x >> 1 : gridDim.x;
@@ -299,31 +312,35 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             for (int u = worker; u < units && ok && !no_k; u += workers) {
                 int m, n0, n1;
                 unit_range(u, m, n0, n1);
-                const int my_m = PAIR ? 2 * m + rank : m;
                 for (int n = n0; n < n1 && ok; ++n) {
                     const int b_row0 = n * BN + rank * C::kBRows;      // this CTA's rows of the B tile
                     for (int kb = 0; kb < k_slabs; ++kb) {
                         if (!mbar_wait(smem_addr(&ctl->empty[stage]), phase ^ 1u, &ctl->abort_flag)) { ok = false; break; }
                         const uint32_t own_bar = smem_addr(&ctl->full[stage]);
                         const uint32_t bar = PAIR ? map_to_cta(own_bar, 0) : own_bar;   // the leader's barrier
-                        const uint32_t sa = tiles + stage * C::kStageBytes;
-                        const uint32_t sb = sa + kABytes;
+                        const uint32_t sa0 = tiles + stage * C::kStageBytes;
+                        const uint32_t sb = sa0 + NACC * kABytes;
                         if (!PAIR) mbar_expect_tx(own_bar, C::kStageBytes);
                         else if (rank == 0) mbar_expect_tx(own_bar, 2 * C::kStageBytes);
                         auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
                             if (PAIR) tma_load_2d_pair(dst, map, bar, x, y);
                             else tma_load_2d(dst, map, bar, x, y);
                         };
-                        if (p.mode == kGradHidden) {
-                            // dZ block (token tile my_m, vocabulary block kb): 128 rows of 128 bytes
-                            load(sa, &map_a, 0, (my_m * p.dz_nc + kb) * kDzBlockRows);
-                        } else if (p.mode == kGradW) {
-                            // dZ^T: vocabulary blocks 2 my_m + j, the 64 token rows of k-slab kb
-                            for (int j = 0; j < BM / 64; ++j)
-                                load(sa + j * kSlabBytes, &map_a, 0,
-                                     ((kb >> 1) * p.dz_nc + (my_m * 2 + j)) * kDzBlockRows + (kb & 1) * 64);
-                        } else {
-                            load(sa, &map_a, kb * BK, my_m * BM);
+#pragma unroll
+                        for (int a = 0; a < NACC; ++a) {
+                            const int my_m = kTilesPerUnit * m + 2 * a + rank;
+                            const uint32_t sa = sa0 + a * kABytes;
+                            if (p.mode == kGradHidden) {
+                                // dZ block (token tile my_m, vocabulary block kb): 128 rows of 128 bytes
+                                load(sa, &map_a, 0, (my_m * p.dz_nc + kb) * kDzBlockRows);
+                            } else if (p.mode == kGradW) {
+                                // dZ^T: vocabulary blocks 2 my_m + j, the 64 token rows of k-slab kb
+                                for (int j = 0; j < BM / 64; ++j)
+                                    load(sa + j * kSlabBytes, &map_a, 0,
+                                         ((kb >> 1) * p.dz_nc + (my_m * 2 + j)) * kDzBlockRows + (kb & 1) * 64);
+                            } else {
+                                load(sa, &map_a, kb * BK, my_m * BM);
+                            }
                         }
                         if (!b_mn) {
                             load(sb, &map_b, kb * BK, b_row0);
@@ -358,11 +375,18 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         tc_fence_after();
                         const uint32_t sa = tiles + stage * C::kStageBytes;
                         const uint64_t adesc = smem_desc(sa, a_mn);
-                        const uint64_t bdesc = smem_desc(sa + kABytes, b_mn);
+                        const uint64_t bdesc = smem_desc(sa + NACC * kABytes, b_mn);
 #pragma unroll
                         for (int k = 0; k < BK / 16; ++k) {
-                            if (PAIR) tc_mma2(d_tmem, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc,
-                                              (kb | k) ? 1u : 0u);
+                            if (ACC2) {
+                                // accumulator a (TMEM columns a * 256 ..) takes A tile a; both share the B slab
+#pragma unroll
+                                for (int a = 0; a < NACC; ++a)
+                                    tc_mma2(tmem_base + (uint32_t)(a * BN),
+                                            adesc + (uint64_t)(a * (kABytes >> 4)) + (uint64_t)(k * a_kstep),
+                                            bdesc + (uint64_t)(k * b_kstep), idesc, (kb | k) ? 1u : 0u);
+                            } else if (PAIR) tc_mma2(d_tmem, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc,
+                                                     (kb | k) ? 1u : 0u);
                             else tc_mma(d_tmem, adesc + (uint64_t)(k * a_kstep), bdesc + (uint64_t)(k * b_kstep), idesc,
                                         (kb | k) ? 1u : 0u);
                         }
@@ -376,7 +400,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     if (PAIR) tc_commit2(smem_addr(&ctl->tmem_full[buf]));
                     else tc_commit(smem_addr(&ctl->tmem_full[buf]));
                     tphase[buf] ^= 1u;
-                    buf ^= 1;
+                    if (!ACC2) buf ^= 1;              // with two accumulators per unit there is one "buffer": both
                 }
             }
         }
@@ -390,7 +414,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         for (int u = worker; u < units && ok; u += workers) {
             int m, n0, n1;
             unit_range(u, m, n0, n1);
-            const int row = (PAIR ? 2 * m + rank : m) * BM + row_in_tile;
+            const int row = (kTilesPerUnit * m + rank) * BM + row_in_tile;     // accumulator 0's row
             const bool row_ok = row < M;
             float run_m = -INFINITY, run_s = 0.0f;       // kLse
             float run_u = 0.0f;                          // kLse with entropy: sum of 2^x x against run_m
@@ -510,15 +534,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     if (row_ok) p.tmax[(long long)row * p.n_tiles + n] = tms;
                 } else
 #pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
+                for (int ac = 0; ac < NACC * (BN / 32); ++ac) {
+                    // accumulator a of this unit: the token (vocabulary) tile 2 a further on, TMEM columns a * 256 ..
+                    const int a = ac / (BN / 32), c = ac - a * (BN / 32);
+                    const int row_a = row + a * 2 * BM;
+                    const bool row_ok_a = row_a < M;
                     const int cb = col0 + c * 32;
-                    if (cb >= p.N) break;                // whole chunk beyond the valid columns (warp-uniform)
+                    if (cb >= p.N) continue;             // whole chunk beyond the valid columns (warp-uniform)
                     uint32_t v[32];
                     if (no_k) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] = 0u;
                     } else {
-                        tc_ld32(t_row + (uint32_t)(c * 32), v);
+                        tc_ld32(t_row + (uint32_t)(a * BN + c * 32), v);
                     }
                     const int nvalid = min(32, p.N - cb);
                     if (p.mode == kLse) {
@@ -562,10 +590,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         }
                         run_s += s0 + s1;
                     } else if (p.mode == kGradHidden) {
-                        if (row_ok) {
-                            const long long orow = p.row_index ? (long long)p.row_index[p.live_off + row] : (long long)row;
+                        if (row_ok_a) {
+                            const long long orow = p.row_index ? (long long)p.row_index[p.live_off + row_a] : (long long)row_a;
                             __nv_bfloat16* dst = p.out_bf16 + orow * p.out_stride + cb;
-                            const float sc = p.row_scale ? p.row_scale[row] : 1.0f;
+                            const float sc = p.row_scale ? p.row_scale[row_a] : 1.0f;
                             if (nvalid == 32) {
                                 uint32_t o[16];
 #pragma unroll
@@ -582,19 +610,22 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                             }
                         }
                     } else {   // kGradW
-                        if (row_ok) {
-                            float* dst = p.out_f32 + (long long)row * p.out_stride + cb;
+                        if (row_ok_a) {
+                            float* dst = p.out_f32 + (long long)row_a * p.out_stride + cb;
                             if (nvalid == 32) {
                                 float4* d4 = reinterpret_cast<float4*>(dst);
 #pragma unroll
                                 for (int i = 0; i < 8; ++i) {
-                                    float4 a = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
-                                                           __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
-                                    if (p.accumulate) {
-                                        const float4 old = d4[i];
-                                        a.x += old.x; a.y += old.y; a.z += old.z; a.w += old.w;
-                                    }
-                                    d4[i] = a;
+                                    // accumulation is a fire-and-forget vector reduction at the memory side (no
+                                    // read round trip in the drain); each element gets exactly one addend per
+                                    // launch, so the result does not depend on timing
+                                    if (p.accumulate)
+                                        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
+                                                     :: "l"(d4 + i), "r"(v[4 * i]), "r"(v[4 * i + 1]), "r"(v[4 * i + 2]),
+                                                        "r"(v[4 * i + 3]) : "memory");
+                                    else
+                                        d4[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                                            __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
                                 }
                             } else {
                                 for (int i = 0; i < nvalid; ++i)
@@ -611,7 +642,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     else mbar_arrive(smem_addr(&ctl->tmem_empty[buf]));
                 }
                 tphase[buf] ^= 1u;
-                buf ^= 1;
+                if (!ACC2) buf ^= 1;
             }
             if (p.mode == kLse && row_ok && ok) {
                 const int sp = n0 / p.n_tiles_per_split;
@@ -1017,7 +1048,7 @@ static std::atomic<int> g_max_workers{0};   // persistent CTAs (or pairs) per la
 static std::atomic<int> g_chunk_tiles{0};   // token tiles per backward chunk; 0: the most the workspace holds
 static std::atomic<int> g_row_ref{1};       // backward scratch: 1 exponentials against a per-row reference, 0 per-tile maxima
 
-template <bool PAIR>
+template <bool PAIR, bool ACC2>
 static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, cudaStream_t s) {
     static std::mutex mu;
     static bool opted[64] = {};
@@ -1026,8 +1057,8 @@ static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, co
     {
         std::lock_guard<std::mutex> lock(mu);
         if (dev >= 0 && dev < 64 && !opted[dev]) {
-            if (cudaFuncSetAttribute((const void*)umma_gemm_kernel<PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     Cfg<PAIR>::kSmemBytes) != cudaSuccess) {
+            if (cudaFuncSetAttribute((const void*)umma_gemm_kernel<PAIR, ACC2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     Cfg<PAIR, ACC2>::kSmemBytes) != cudaSuccess) {
                 cudaGetLastError();
                 return RLF_ERR_CUDA;
             }
@@ -1035,7 +1066,8 @@ static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, co
         }
     }
     const bool sweep = p.mode == kLse;
-    const int m_units = PAIR ? (p.m_tiles + 1) / 2 : p.m_tiles;
+    constexpr int kTilesPerUnit = (PAIR ? 2 : 1) * (ACC2 ? 2 : 1);
+    const int m_units = (p.m_tiles + kTilesPerUnit - 1) / kTilesPerUnit;
     const int units = sweep ? m_units * p.nsplit : m_units * p.n_tiles;
     if (units <= 0) return RLF_OK;
     int workers = PAIR ? sm_count_lm() / 2 : sm_count_lm();
@@ -1051,7 +1083,7 @@ static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, co
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(PAIR ? 2 * workers : workers);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = Cfg<PAIR>::kSmemBytes;
+    cfg.dynamicSmemBytes = Cfg<PAIR, ACC2>::kSmemBytes;
     cfg.stream = s;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
@@ -1060,7 +1092,7 @@ static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, co
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, umma_gemm_kernel<PAIR>, ma, mb, q) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, umma_gemm_kernel<PAIR, ACC2>, ma, mb, q) != cudaSuccess) {
         cudaGetLastError();
         return RLF_ERR_CUDA;
     }
@@ -1068,17 +1100,19 @@ static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, co
     return RLF_OK;
 }
 
+static std::atomic<int> g_acc2{1};          // gradient contractions in pair form: 1 two accumulators per CTA, 0 one
 static rlf_status launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const GemmParams& p, bool pair,
                               cudaStream_t s) {
-    return pair ? launch_gemm_t<true>(ma, mb, p, s) : launch_gemm_t<false>(ma, mb, p, s);
+    if (!pair) return launch_gemm_t<false, false>(ma, mb, p, s);
+    if (p.mode != kLse && g_acc2.load() != 0) return launch_gemm_t<true, true>(ma, mb, p, s);
+    return launch_gemm_t<true, false>(ma, mb, p, s);
 }
 
-// rows of dZ held in scratch at a time: 74 token tiles = 37 pair units (one scheduling block of the
-// sweep; 37 x D/256 whole waves of the grad_hidden contraction on 74 CTA pairs); 2.9 GB at
-// V = 151936.  Twice the chunk halves the passes over the head and the accumulations into grad_W, but
-// measured under sustained load (3 s loops at the power cap) it is slower: 48.6 against 46.8 ms for
-// the Qwen3-4B-head step, at 1.16 against 1.25 GHz.
-constexpr int kChunkTokens = 74 * BM;
+// Rows of dZ held in scratch at a time: up to 148 token tiles = 37 units of the two-accumulator
+// gradient contractions (37 x D/256 = 370 units at D = 2560: five whole waves on 74 CTA pairs) = two
+// scheduling blocks of the sweep; 5.8 GB at V = 151936.  Larger chunks mean fewer passes over the head
+// in grad_hidden and fewer accumulations into grad_W.
+constexpr int kChunkTokens = 148 * BM;
 constexpr int kMaxSplit = 64;               // most vocabulary splits a sweep may use (sizes the partials)
 
 // Number of vocabulary splits of a sweep.  A work unit is (pair of token tiles, split); the units are
@@ -1491,9 +1525,10 @@ extern "C" rlf_status rlf_tune_lmhead(int pair_ctas) {
     return RLF_OK;
 }
 
-extern "C" rlf_status rlf_tune_lmhead_backward(int row_reference) {
-    if (row_reference != 0 && row_reference != 1) return RLF_ERR_SHAPE;
+extern "C" rlf_status rlf_tune_lmhead_backward(int row_reference, int two_accumulators) {
+    if ((row_reference != 0 && row_reference != 1) || (two_accumulators != 0 && two_accumulators != 1)) return RLF_ERR_SHAPE;
     rlf::lm::g_row_ref = row_reference;
+    rlf::lm::g_acc2 = two_accumulators;
     return RLF_OK;
 }
 

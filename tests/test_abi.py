@@ -117,6 +117,9 @@ def test_host_validation_rejects_bad_arguments_before_touching_a_device(lib):
     s = lib.rlf_tune_lmhead_schedule
     s.argtypes = [ctypes.c_int] * 3
     assert s(-1, 0, 0) == -2 and s(0, -1, 0) == -2 and s(0, 0, 3) == -2 and s(0, 0, 0) == 0
+    bw = lib.rlf_tune_lmhead_backward
+    bw.argtypes = [ctypes.c_int] * 2
+    assert bw(2, 1) == -2 and bw(1, -1) == -2 and bw(0, 0) == 0 and bw(1, 1) == 0
     t = lib.rlf_tune_logits_kernel
     t.argtypes = [ctypes.c_int] * 3
     assert t(3, 512, 0) == -2 and t(4, 500, 0) == -2 and t(0, 0, -1) == 0

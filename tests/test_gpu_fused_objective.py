@@ -132,3 +132,36 @@ def test_fused_results_do_not_depend_on_the_schedule():
             assert torch.equal(o[3], ref[3]), key
         else:
             assert (o[3] - ref[3]).abs().max().item() <= 1e-5 * ref[3].abs().max().item(), key
+
+
+@pytest.mark.parametrize("tokens", [24, 44, 60])
+def test_two_accumulator_gradient_contractions_are_bit_identical_to_the_one_accumulator_form(tokens):
+    """In pair form the two gradient contractions give each CTA pair two 256-row tiles per 256-column
+    slab.  Every output element is still one fp32 accumulation over the same k-slabs in the same order,
+    so both forms must agree bit for bit: at tile counts that leave the last unit with one, two or three
+    of its four tiles, with several chunks, and when grad_W is accumulated onto given values (a vector
+    reduction in one form's drain against a plain store in the first chunk)."""
+    b, spec, batch, mask, seq, n, adv = _setup(4096 + 264, 192)
+    spec = synth.scaled(spec, len_lo=tokens, len_hi=tokens)
+    batch = synth.make_batch(spec, DEV)
+    mask, seq, n = b.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, spec.open_id, spec.close_id)
+    adv = b.rlf_group_advantage(batch.rewards, group_size=batch.tokens.group_size)
+    args = (batch.hidden, batch.W, batch.ids, seq, adv, batch.old_logp, batch.ref_logp, mask, synth.EPS_CLIP, synth.BETA_KL)
+    gw0 = torch.randn((spec.V, spec.D), device=DEV)
+    outs = {}
+    try:
+        for acc2 in (1, 0):
+            for chunk in (0, 2, 6):
+                for accumulate in (False, True):
+                    b.tune_lmhead_backward(1, acc2)
+                    b.tune_lmhead_schedule(0, 0, chunk)
+                    outs[(acc2, chunk, accumulate)] = b.rlf_fused_lmhead_grpo(
+                        *args, denom=n, grad_W=gw0.clone() if accumulate else None, accumulate_grad_W=accumulate)
+                    torch.cuda.synchronize()
+    finally:
+        b.tune_lmhead_backward(1, 1)
+        b.tune_lmhead_schedule(0, 0, 0)
+    for (acc2, chunk, accumulate), o in outs.items():
+        ref = outs[(0, chunk, accumulate)]
+        for got, want in zip(o, ref):
+            assert torch.equal(got, want), (acc2, chunk, accumulate)
