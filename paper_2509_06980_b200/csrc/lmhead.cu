@@ -190,6 +190,27 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// the same load without its wait, and the wait: the registers pass through the wait as in/out operands
+// so that no use of them can be scheduled ahead of it
+__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                   "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                   "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                   "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_ld_wait(uint32_t (&v)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                   "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]),
+                   "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
+                   "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
+                 :: "memory");
+}
+
 // Shared-memory operand descriptor, 128-byte swizzle, descriptor version 1.
 //   K-major tile  (rows of 64 bf16 = 128 B, 8-row groups 1024 B apart): LBO 1, SBO 1024 B.
 //   MN-major tile (64-wide slabs, each 64 k-rows of 128 B): LBO = slab pitch 8192 B, SBO 1024 B.
@@ -532,21 +553,20 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     }
                     if (tm != -INFINITY) run_s += (ts0 + ts1) * ex2_approx((tm - run_m) * kLog2e);
                     if (row_ok) p.tmax[(long long)row * p.n_tiles + n] = tms;
-                } else
-#pragma unroll 1
-                for (int ac = 0; ac < NACC * (BN / 32); ++ac) {
+                } else {
+                // 32-column chunks of the accumulator(s), software-pipelined: the tensor-memory load of
+                // chunk ac + 1 is in flight while chunk ac is consumed (with two accumulators the drain is
+                // not hidden behind the next unit's multiplies, so its latency chain matters)
+                auto consume = [&](int ac, uint32_t (&v)[32]) {
                     // accumulator a of this unit: the token (vocabulary) tile 2 a further on, TMEM columns a * 256 ..
                     const int a = ac / (BN / 32), c = ac - a * (BN / 32);
                     const int row_a = row + a * 2 * BM;
                     const bool row_ok_a = row_a < M;
                     const int cb = col0 + c * 32;
-                    if (cb >= p.N) continue;             // whole chunk beyond the valid columns (warp-uniform)
-                    uint32_t v[32];
+                    if (cb >= p.N) return;               // whole chunk beyond the valid columns (warp-uniform)
                     if (no_k) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] = 0u;
-                    } else {
-                        tc_ld32(t_row + (uint32_t)(a * BN + c * 32), v);
                     }
                     const int nvalid = min(32, p.N - cb);
                     if (p.mode == kLse) {
@@ -606,7 +626,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                                 d4[2] = make_uint4(o[8], o[9], o[10], o[11]);
                                 d4[3] = make_uint4(o[12], o[13], o[14], o[15]);
                             } else {
-                                for (int i = 0; i < nvalid; ++i) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]) * sc);
+#pragma unroll
+                                for (int i = 0; i < 32; ++i)
+                                    if (i < nvalid) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]) * sc);
                             }
                         }
                     } else {   // kGradW
@@ -628,11 +650,30 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                                                             __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
                                 }
                             } else {
-                                for (int i = 0; i < nvalid; ++i)
-                                    dst[i] = __uint_as_float(v[i]) + (p.accumulate ? dst[i] : 0.0f);
+#pragma unroll
+                                for (int i = 0; i < 32; ++i)
+                                    if (i < nvalid) dst[i] = __uint_as_float(v[i]) + (p.accumulate ? dst[i] : 0.0f);
                             }
                         }
                     }
+                };
+                constexpr int kChunks = NACC * (BN / 32);
+                const uint32_t t_buf = t_row;
+                uint32_t va[32], vb[32];
+                if (!no_k) tc_ld32_issue(t_buf, va);
+#pragma unroll 1
+                for (int ac = 0; ac < kChunks; ac += 2) {
+                    if (!no_k) {
+                        tc_ld_wait(va);
+                        tc_ld32_issue(t_buf + (uint32_t)((ac + 1) * 32), vb);      // kChunks is even
+                    }
+                    consume(ac, va);
+                    if (!no_k) {
+                        tc_ld_wait(vb);
+                        if (ac + 2 < kChunks) tc_ld32_issue(t_buf + (uint32_t)((ac + 2) * 32), va);
+                    }
+                    consume(ac + 1, vb);
+                }
                 }
                 // hand the accumulator buffer back to the MMA warp
                 tc_fence_before();
@@ -1071,13 +1112,33 @@ static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, co
     const int units = sweep ? m_units * p.nsplit : m_units * p.n_tiles;
     if (units <= 0) return RLF_OK;
     int workers = PAIR ? sm_count_lm() / 2 : sm_count_lm();
-    // Sweep schedule: the CTAs (or pairs) running at one time cover workers / 2 row units x 2 splits,
-    // in lockstep.  Their token tiles (1.3 MB per pair at D = 2560) are re-read for every column tile
-    // and must stay in L2 next to the streaming head: with all 74 pairs on different row units
-    // (97 MB) they did not, and the same launch drew its 1 kW at 1.06 GHz instead of 1.39 GHz.
+    // Sweep schedule: the CTAs (or pairs) running at one time cover m_block row units x (workers / m_block)
+    // splits, in lockstep.  Their token tiles (256 x D bf16 per pair: 1.3 MB at D = 2560, 2 MB at 4096)
+    // are re-read for every column tile and must stay in L2 next to the streaming head: with all 74 pairs
+    // on different row units (97 MB at D = 2560) they did not, and the same launch drew its 1 kW at
+    // 1.06 GHz instead of 1.39 GHz.  So m_block is what keeps about 48 MB of token tiles live, at most half
+    // the workers, and a divisor of the worker count (blocks that leave the splits misaligned cost
+    // 4 - 10 %): when no nearby divisor exists a few workers are left out instead (D = 4096: 24 row
+    // units on 72 of the 74 pairs measured 5 % faster than 37 on 74; D = 2560 keeps 37 on 74).
     if (g_max_workers.load() > 0 && g_max_workers.load() < workers) workers = g_max_workers.load();
     GemmParams q = p;
     q.m_block = workers / 2 > 0 ? workers / 2 : 1;
+    if (sweep && g_m_block.load() == 0 && g_max_workers.load() == 0) {
+        const double unit_bytes = (double)(PAIR ? 2 : 1) * BM * (double)p.k_slabs * BK * 2.0;
+        const double target = 48.0 * 1024 * 1024 / unit_bytes;
+        int hi = (int)(target * 1.05);
+        if (hi > workers / 2) hi = workers / 2;
+        if (hi < 1) hi = 1;
+        int lo = (int)(target * 0.6);
+        if (lo < 1) lo = 1;
+        int best_mb = hi, best_w = workers / hi * hi;
+        for (int mb = hi - 1; mb >= lo; --mb) {
+            const int w = workers / mb * mb;
+            if (w > best_w) { best_w = w; best_mb = mb; }
+        }
+        q.m_block = best_mb;
+        workers = best_w;
+    }
     if (g_m_block.load() > 0) q.m_block = g_m_block.load();
     if (workers > units) workers = units;
     cudaLaunchConfig_t cfg = {};
