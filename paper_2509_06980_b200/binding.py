@@ -20,7 +20,7 @@ DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
 EXPORTS = [
     "rlf_build_loss_mask", "rlf_group_advantage", "rlf_rule_reward", "rlf_kl_in_reward", "rlf_grpo_logp_loss_fwd_bwd",
     "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_grpo_logp_loss_fwd_bwd_skip_masked", "rlf_grpo_logp_loss_fwd_bwd_obj", "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_fused_lmhead_grpo_obj", "rlf_fused_lmhead_logp_entropy", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
-    "rlf_tune_logits_kernel", "rlf_tune_logits_grid", "rlf_tune_lmhead", "rlf_tune_lmhead_schedule", "rlf_tune_lmhead_backward", "rlf_launch_count", "rlf_status_string", "rlf_version",
+    "rlf_tune_logits_kernel", "rlf_tune_logits_grid", "rlf_tune_lmhead", "rlf_tune_lmhead_schedule", "rlf_tune_lmhead_backward", "rlf_tune_lmhead_pacing", "rlf_launch_count", "rlf_status_string", "rlf_version",
 ]
 
 if not os.path.exists(_LIB_PATH):
@@ -56,6 +56,7 @@ _lib.rlf_tune_logits_grid.argtypes = [_int, _int]
 _lib.rlf_tune_lmhead.argtypes = [_int]
 _lib.rlf_tune_lmhead_schedule.argtypes = [_int, _int, _int]
 _lib.rlf_tune_lmhead_backward.argtypes = [_int, _int]
+_lib.rlf_tune_lmhead_pacing.argtypes = [_int]
 _lib.rlf_rule_reward.argtypes = [_vp, _vp, _i32, _i32, _vp, _vp]
 _lib.rlf_kl_in_reward.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _int, _vp, _vp, _vp, _vp]
 _lib.rlf_grpo_logp_loss_fwd_bwd_obj.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _i32, _vp, _vp, _vp, _f32,
@@ -71,7 +72,7 @@ for _n in ("rlf_build_loss_mask", "rlf_group_advantage", "rlf_rule_reward", "rlf
            "rlf_grpo_logp_loss_fwd_bwd", "rlf_grpo_logp_loss_fwd_bwd_obj", "rlf_grpo_logp_loss_fwd_bwd_skip_masked",
            "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_fused_lmhead_grpo_obj",
            "rlf_fused_lmhead_logp_entropy", "rlf_grpo_step_host", "rlf_tune_logits_kernel", "rlf_tune_logits_grid",
-           "rlf_tune_lmhead", "rlf_tune_lmhead_schedule", "rlf_tune_lmhead_backward"):
+           "rlf_tune_lmhead", "rlf_tune_lmhead_schedule", "rlf_tune_lmhead_backward", "rlf_tune_lmhead_pacing"):
     getattr(_lib, _n).restype = _int
 
 
@@ -147,6 +148,10 @@ def tune_lmhead(pair_ctas=1):
 
 def tune_lmhead_backward(row_reference=1, two_accumulators=1):
     _check(_lib.rlf_tune_lmhead_backward(int(row_reference), int(two_accumulators)), "rlf_tune_lmhead_backward")
+
+
+def tune_lmhead_pacing(on=1):
+    _check(_lib.rlf_tune_lmhead_pacing(int(on)), "rlf_tune_lmhead_pacing")
 
 
 def tune_lmhead_schedule(m_block=0, max_workers=0, chunk_tiles=0):

@@ -98,6 +98,13 @@ struct GemmParams {
     const float* row_scale;   // kGradHidden (optional): fp32 factor of compact row r applied to its output row
     const int* run_flag;      // optional: the launch does nothing unless *run_flag == run_want
     int run_want;
+    // Pacing (optional): a counter, zero at launch, on which the load-issuing threads of all workers meet at
+    // the start of each of their units and at pace_parts - 1 evenly spaced points inside it.  Workers that
+    // share operand slabs through L2 then request them within a short time of each other; left alone they
+    // drift apart over a few thousand k-slabs until each fetches its slabs from HBM on its own.  Waits
+    // are bounded and only delay loads: a worker that gives up runs on unpaced.
+    int* pace;
+    int pace_parts;
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -118,6 +125,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 constexpr int kWaitPolls = 1 << 22;
+constexpr int kPacePolls = 1 << 14;          // a pacing wait gives up after about 10 ms and is not taken again
 // bounded wait; on failure (or if another role already gave up) returns false
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     for (int i = 0; i < kWaitPolls; ++i) {
@@ -303,6 +311,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const uint32_t tmem_base = ctl->tmem_base;
 
     // unit -> (m unit, first n tile, one-past-last n tile)
+    const int split_base = sweep ? p.n_tiles / p.nsplit : 0, split_rem = sweep ? p.n_tiles % p.nsplit : 0;
     auto unit_range = [&](int u, int& m, int& n0, int& n1) {
         if (sweep) {
             // blocks of m_block row units; inside a block, units run over its row units first, then
@@ -313,8 +322,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const int rows_here = min(p.m_block, m_units - blk * p.m_block);
             const int sp = within / rows_here;
             m = blk * p.m_block + (within - sp * rows_here);
-            n0 = sp * p.n_tiles_per_split;
-            n1 = min(p.n_tiles, n0 + p.n_tiles_per_split);
+            // column tiles dealt evenly: the first split_rem splits hold one tile more than the others
+            n0 = sp * split_base + min(sp, split_rem);
+            n1 = n0 + split_base + (sp < split_rem ? 1 : 0);
         } else {
             // column tiles fastest: the CTAs running at the same time share their A slabs (the dZ
             // rows or columns) in L2 instead of each streaming the whole scratch from HBM
@@ -330,12 +340,32 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int u = worker; u < units && ok && !no_k; u += workers) {
+            // pacing: arrivals expected on the counter before this worker passes its next meeting point
+            long long pace_due = 0;
+            bool pace_wait = p.pace != nullptr;
+            int iter = 0;
+            for (int u = worker; u < units && ok && !no_k; u += workers, ++iter) {
                 int m, n0, n1;
                 unit_range(u, m, n0, n1);
+                const int with_me = min(workers, units - iter * workers);     // workers that have a unit number `iter`
+                const long long unit_slabs = (long long)(n1 - n0) * k_slabs;
+                long long pos = 0;
+                int next_meet = iter == 0 ? 1 : 0;                            // no meeting before the very first unit
                 for (int n = n0; n < n1 && ok; ++n) {
                     const int b_row0 = n * BN + rank * C::kBRows;      // this CTA's rows of the B tile
-                    for (int kb = 0; kb < k_slabs; ++kb) {
+                    for (int kb = 0; kb < k_slabs; ++kb, ++pos) {
+                        while (p.pace && next_meet < p.pace_parts && pos == next_meet * unit_slabs / p.pace_parts) {
+                            ++next_meet;
+                            pace_due += with_me;
+                            if (rank == 0) atomicAdd(p.pace, 1);
+                            if (pace_wait) {
+                                int polls = 0;
+                                while ((long long)*reinterpret_cast<volatile int*>(p.pace) < pace_due) {
+                                    if (++polls > kPacePolls) { pace_wait = false; break; }
+                                    __nanosleep(64);
+                                }
+                            }
+                        }
                         if (!mbar_wait(smem_addr(&ctl->empty[stage]), phase ^ 1u, &ctl->abort_flag)) { ok = false; break; }
                         const uint32_t own_bar = smem_addr(&ctl->full[stage]);
                         const uint32_t bar = PAIR ? map_to_cta(own_bar, 0) : own_bar;   // the leader's barrier
@@ -686,7 +716,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 if (!ACC2) buf ^= 1;
             }
             if (p.mode == kLse && row_ok && ok) {
-                const int sp = n0 / p.n_tiles_per_split;
+                // inverse of unit_range's n0(sp)
+                const int big = split_rem * (split_base + 1);
+                const int sp = n0 < big ? n0 / (split_base + 1) : split_rem + (n0 - big) / max(split_base, 1);
                 p.part[(long long)row * p.nsplit + sp] = make_float2(run_m, run_s);
                 if (p.part_u) p.part_u[(long long)row * p.nsplit + sp] = run_u;
             }
@@ -1087,6 +1119,7 @@ static std::atomic<int> g_pair{1};       // 1: cta_group::2 pair form, 0: single
 static std::atomic<int> g_m_block{0};    // row units per scheduling block of the sweep; 0: automatic
 static std::atomic<int> g_max_workers{0};   // persistent CTAs (or pairs) per launch; 0: one per SM (pair of SMs)
 static std::atomic<int> g_chunk_tiles{0};   // token tiles per backward chunk; 0: the most the workspace holds
+static std::atomic<int> g_pace{1};          // pacing of the workers' loads (see GemmParams::pace): 0 off, 1 gradient contractions, 2 all
 static std::atomic<int> g_row_ref{1};       // backward scratch: 1 exponentials against a per-row reference, 0 per-tile maxima
 
 template <bool PAIR, bool ACC2>
@@ -1141,6 +1174,19 @@ static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, co
     }
     if (g_m_block.load() > 0) q.m_block = g_m_block.load();
     if (workers > units) workers = units;
+    // The gradient contractions gain from it (cfg 3 at full size: grad_hidden 32 -> 10 GB of HBM reads and
+    // 9.6 -> 8.5 ms per launch, grad_W 35 -> 11 GB and 10.3 -> 9.1 ms).  The sweeps' reads fall as well
+    // (15 -> 3.5 GB), but their units differ in length (9 or 10 column tiles) and their drains jitter, and
+    // the time lost at the meeting points outweighs it (17.2 -> 18.7 ms): off for them unless asked for.
+    if (q.pace && (g_pace.load() == 2 || (g_pace.load() == 1 && !sweep))) {
+        // meeting points: every unit start plus interior points about 256 k-slabs apart
+        const long long unit_slabs = sweep ? (long long)((p.n_tiles + p.nsplit - 1) / p.nsplit) * p.k_slabs : p.k_slabs;
+        q.pace_parts = (int)((unit_slabs + 128) / 256);
+        if (q.pace_parts < 1) q.pace_parts = 1;
+        if (cudaMemsetAsync(q.pace, 0, sizeof(int), s) != cudaSuccess) return RLF_ERR_CUDA;
+    } else {
+        q.pace = nullptr;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(PAIR ? 2 * workers : workers);
     cfg.blockDim = dim3(kThreads);
@@ -1198,7 +1244,7 @@ static LmWs lm_workspace(int64_t T, int32_t V, int32_t D) {
     size_t o = 0;
     const size_t Tn = (size_t)(T > 0 ? T : 0);
     const size_t Tp = (Tn + 255) & ~(size_t)255;     // compact arrays are padded to whole tile pairs
-    w.n_count = o; o += 1024;                        // [0] mask count, [64] live / other row counts, [128] chunk flag
+    w.n_count = o; o += 1024;                        // [0] mask count, [64] live / other row counts, [128] chunk flag, [256] pacing counter
     w.partial = o; o += up1k(token_loss_partial_bytes());
     w.rec = o;     o += up1k(16 * Tn);
     w.zy = o;      o += up1k(4 * Tn);
@@ -1320,6 +1366,7 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
     g.k_slabs = D / BK;
     g.part = part;
     g.dev_status = dev_status;
+    g.pace = reinterpret_cast<int*>(ws + w.n_count + 256);
     auto set_rows = [&](GemmParams& q, int64_t rows) {
         q.M = (int)rows;
         q.m_tiles = (int)((rows + BM - 1) / BM);
@@ -1447,6 +1494,7 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
             h.live_off = (int)t0;
             h.row_index = idx_live;
             h.row_scale = row_ref ? scale_g + t0 : nullptr;
+            h.pace = g.pace;
             st = launch_gemm(mapDzK, mapWn, h, pair, s);
             if (st != RLF_OK) return st;
         }
@@ -1470,6 +1518,7 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
             q.dev_status = dev_status;
             q.live_count = counts;
             q.live_off = (int)t0;
+            q.pace = g.pace;
             st = launch_gemm(mapDzM, mapHn, q, pair, s);
             if (st != RLF_OK) return st;
         }
@@ -1572,6 +1621,8 @@ extern "C" rlf_status rlf_fused_lmhead_logp_entropy(const void* hidden, const vo
     g.part = part;
     g.part_u = entropy_out ? part_u : nullptr;
     g.dev_status = dev_status;
+    // the pacing counter sits in the kilobyte that closes the workspace
+    g.pace = reinterpret_cast<int*>(ws + up1k(4 * (size_t)T) + up1k(8 * (size_t)T * kMaxSplit) + up1k(4 * (size_t)T * kMaxSplit));
     st = launch_gemm(mapH, mapW, g, pair, s);
     if (st != RLF_OK) return st;
     combine_logp_entropy_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(part, g.part_u, g.nsplit, zy, T, logp_out,
@@ -1590,6 +1641,12 @@ extern "C" rlf_status rlf_tune_lmhead_backward(int row_reference, int two_accumu
     if ((row_reference != 0 && row_reference != 1) || (two_accumulators != 0 && two_accumulators != 1)) return RLF_ERR_SHAPE;
     rlf::lm::g_row_ref = row_reference;
     rlf::lm::g_acc2 = two_accumulators;
+    return RLF_OK;
+}
+
+extern "C" rlf_status rlf_tune_lmhead_pacing(int on) {
+    if (on < 0 || on > 2) return RLF_ERR_SHAPE;
+    rlf::lm::g_pace = on;
     return RLF_OK;
 }
 
