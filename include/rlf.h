@@ -439,14 +439,12 @@ rlf_status rlf_tune_lmhead_schedule(int m_block, int max_workers, int chunk_tile
  * pair with a double-buffered accumulator, as in the forward sweep.  Results are bit-identical. */
 rlf_status rlf_tune_lmhead_backward(int row_reference, int two_accumulators);
 
-/* Pacing of the fused contractions for later calls in this process.  The persistent CTAs (or pairs) of a
- * paced launch meet on a device counter at the start of each of their work units and at points about
- * 256 k-slabs apart inside it, so that workers which share operand slabs through L2 keep requesting
- * them at about the same time; without it they drift apart over a launch and each ends up streaming
- * its operands from HBM by itself.  Only loads are delayed, every wait is bounded, and a worker whose
- * wait runs out goes on unpaced.  0: no launch is paced; 1 (built-in): the two gradient contractions;
- * 2: the forward sweeps too (their units differ in length, so they lose more at the meeting points
- * than the saved HBM reads return).  Results do not depend on it. */
+/* Pacing of the fused contractions for later calls in this process.  1 (built-in): the persistent CTAs
+ * (or pairs) of a contraction launch meet on a device counter before each of their work units, so
+ * that workers which share operand slabs through L2 keep requesting them at about the same time;
+ * without it they drift apart over a launch and each ends up streaming its operands from HBM by
+ * itself.  Only loads are delayed, every wait is bounded, and a worker whose wait runs out goes on
+ * unpaced.  0: no meeting points.  Results do not depend on it. */
 rlf_status rlf_tune_lmhead_pacing(int on);
 
 /* Number of kernels this library has launched in this process (for accounting). */

@@ -98,13 +98,12 @@ struct GemmParams {
     const float* row_scale;   // kGradHidden (optional): fp32 factor of compact row r applied to its output row
     const int* run_flag;      // optional: the launch does nothing unless *run_flag == run_want
     int run_want;
-    // Pacing (optional): a counter, zero at launch, on which the load-issuing threads of all workers meet at
-    // the start of each of their units and at pace_parts - 1 evenly spaced points inside it.  Workers that
-    // share operand slabs through L2 then request them within a short time of each other; left alone they
-    // drift apart over a few thousand k-slabs until each fetches its slabs from HBM on its own.  Waits
-    // are bounded and only delay loads: a worker that gives up runs on unpaced.
+    // Pacing (optional): a counter, zero at launch, on which the load-issuing threads of all workers meet
+    // before each of their units but the first.  Workers that share operand slabs through L2 then
+    // request them within a short time of each other; left alone they drift apart over a launch until
+    // each fetches its slabs from HBM on its own.  Waits are bounded and only delay loads: a worker
+    // that gives up runs on unpaced.
     int* pace;
-    int pace_parts;
 };
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -126,6 +125,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 constexpr int kWaitPolls = 1 << 22;
 constexpr int kPacePolls = 1 << 14;          // a pacing wait gives up after about 10 ms and is not taken again
+// wait (bounded) until the pacing counter has reached `want`; `seen` is a value read earlier
+__device__ __forceinline__ void pace_settle(const int* counter, int seen, long long want, bool& keep_waiting) {
+    int polls = 0;
+    while ((long long)seen < want) {
+        if (++polls > kPacePolls) { keep_waiting = false; return; }
+        __nanosleep(64);
+        asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+    }
+}
 // bounded wait; on failure (or if another role already gave up) returns false
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     for (int i = 0; i < kWaitPolls; ++i) {
@@ -340,31 +348,32 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            // pacing: arrivals expected on the counter before this worker passes its next meeting point
-            long long pace_due = 0;
-            bool pace_wait = p.pace != nullptr;
+            long long pace_due = 0;       // arrivals expected on the counter before this worker goes on
+            bool pace_wait = p.pace != nullptr, pace_pending = false;
+            int pace_seen = 0;
             int iter = 0;
             for (int u = worker; u < units && ok && !no_k; u += workers, ++iter) {
                 int m, n0, n1;
                 unit_range(u, m, n0, n1);
                 const int with_me = min(workers, units - iter * workers);     // workers that have a unit number `iter`
-                const long long unit_slabs = (long long)(n1 - n0) * k_slabs;
                 long long pos = 0;
-                int next_meet = iter == 0 ? 1 : 0;                            // no meeting before the very first unit
                 for (int n = n0; n < n1 && ok; ++n) {
                     const int b_row0 = n * BN + rank * C::kBRows;      // this CTA's rows of the B tile
                     for (int kb = 0; kb < k_slabs; ++kb, ++pos) {
-                        while (p.pace && next_meet < p.pace_parts && pos == next_meet * unit_slabs / p.pace_parts) {
-                            ++next_meet;
+                        // the meeting point before a unit: announce the arrival and read the counter; the value
+                        // is looked at two k-slabs later, so its round trip to L2 overlaps the issue of those
+                        // slabs' loads instead of draining the ring
+                        if (p.pace && iter > 0 && pos == 0) {
                             pace_due += with_me;
-                            if (rank == 0) atomicAdd(p.pace, 1);
+                            if (rank == 0) asm volatile("red.relaxed.gpu.global.add.s32 [%0], 1;" :: "l"(p.pace) : "memory");
                             if (pace_wait) {
-                                int polls = 0;
-                                while ((long long)*reinterpret_cast<volatile int*>(p.pace) < pace_due) {
-                                    if (++polls > kPacePolls) { pace_wait = false; break; }
-                                    __nanosleep(64);
-                                }
+                                asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(pace_seen) : "l"(p.pace) : "memory");
+                                pace_pending = true;
                             }
+                        }
+                        if (pace_pending && pos >= 2) {
+                            pace_settle(p.pace, pace_seen, pace_due, pace_wait);
+                            pace_pending = false;
                         }
                         if (!mbar_wait(smem_addr(&ctl->empty[stage]), phase ^ 1u, &ctl->abort_flag)) { ok = false; break; }
                         const uint32_t own_bar = smem_addr(&ctl->full[stage]);
@@ -1119,7 +1128,7 @@ static std::atomic<int> g_pair{1};       // 1: cta_group::2 pair form, 0: single
 static std::atomic<int> g_m_block{0};    // row units per scheduling block of the sweep; 0: automatic
 static std::atomic<int> g_max_workers{0};   // persistent CTAs (or pairs) per launch; 0: one per SM (pair of SMs)
 static std::atomic<int> g_chunk_tiles{0};   // token tiles per backward chunk; 0: the most the workspace holds
-static std::atomic<int> g_pace{1};          // pacing of the workers' loads (see GemmParams::pace): 0 off, 1 gradient contractions, 2 all
+static std::atomic<int> g_pace{1};          // pacing of the workers' loads (see GemmParams::pace): 1 on, 0 off
 static std::atomic<int> g_row_ref{1};       // backward scratch: 1 exponentials against a per-row reference, 0 per-tile maxima
 
 template <bool PAIR, bool ACC2>
@@ -1174,15 +1183,10 @@ static rlf_status launch_gemm_t(const CUtensorMap& ma, const CUtensorMap& mb, co
     }
     if (g_m_block.load() > 0) q.m_block = g_m_block.load();
     if (workers > units) workers = units;
-    // The gradient contractions gain from it (cfg 3 at full size: grad_hidden 32 -> 10 GB of HBM reads and
-    // 9.6 -> 8.5 ms per launch, grad_W 35 -> 11 GB and 10.3 -> 9.1 ms).  The sweeps' reads fall as well
-    // (15 -> 3.5 GB), but their units differ in length (9 or 10 column tiles) and their drains jitter, and
-    // the time lost at the meeting points outweighs it (17.2 -> 18.7 ms): off for them unless asked for.
-    if (q.pace && (g_pace.load() == 2 || (g_pace.load() == 1 && !sweep))) {
-        // meeting points: every unit start plus interior points about 256 k-slabs apart
-        const long long unit_slabs = sweep ? (long long)((p.n_tiles + p.nsplit - 1) / p.nsplit) * p.k_slabs : p.k_slabs;
-        q.pace_parts = (int)((unit_slabs + 128) / 256);
-        if (q.pace_parts < 1) q.pace_parts = 1;
+    // Pacing, measured at full size with one-pass ncu counts: grad_hidden 32 -> 10 GB of HBM reads and
+    // 9.6 -> 8.5 ms per launch, grad_W 35 -> 11 GB and 10.3 -> 9.1 ms (D = 2560); the sweep at D = 4096
+    // 71 -> 61 ms.  Meeting points inside a unit were tried too and cost more than they return.
+    if (q.pace && g_pace.load() != 0) {
         if (cudaMemsetAsync(q.pace, 0, sizeof(int), s) != cudaSuccess) return RLF_ERR_CUDA;
     } else {
         q.pace = nullptr;
@@ -1645,7 +1649,7 @@ extern "C" rlf_status rlf_tune_lmhead_backward(int row_reference, int two_accumu
 }
 
 extern "C" rlf_status rlf_tune_lmhead_pacing(int on) {
-    if (on < 0 || on > 2) return RLF_ERR_SHAPE;
+    if (on != 0 && on != 1) return RLF_ERR_SHAPE;
     rlf::lm::g_pace = on;
     return RLF_OK;
 }
