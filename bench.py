@@ -36,9 +36,16 @@ METRIC = "GRPO loss fwd+bwd tokens/s at V=151936 bf16"
 UNIT = "tokens/s"
 WORKLOAD = "cfg1_qwen3_4b_microbatch: 16 responses x 2048 tokens, V=151936 bf16 logits"
 
-# DRAM bytes of one row-kernel launch from the ncu capture summarised under profiles/, as bytes per
-# token; valid only for the row kernel's source text it was taken from (else reported as null).
-NCU_TRAFFIC = {"logits_loss_cu_sha1": "beae1f6cbc292ea9da59db4c5f59b105793ed141", "dram_bytes_per_token": 594787.0}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised under
+# profiles/.  Each figure is valid only for the source text it was captured from: the key is the
+# hash that `python bench.py --source-keys` printed when the capture was taken, and a figure whose key
+# no longer matches the tree is reported as null.
+#   row kernel: one full-size launch (32768 rows; a one-pass capture), per token;
+#   streaming forward kernel: the T = 4096 capture, per token (traffic is proportional to rows);
+#   fused LM-head: every kernel of one forward / one forward + backward call at cfg 3 full size
+#   (one-pass capture of the whole call), per call.
+NCU_TRAFFIC = {"logits_loss_cu_sha1": "beae1f6cbc292ea9da59db4c5f59b105793ed141", "dram_bytes_per_token": 606029.0}
+NCU_TRAFFIC_FUSED = {"lmhead_cu_sha1": "", "fwd_bytes_per_call": None, "fwd_bwd_bytes_per_call": None}
 
 
 def _peaks():
@@ -99,7 +106,8 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3, responses=0
     # Tensor-core work is power-bound here: a kernel timed in the first second after an idle spell runs
     # at clocks it cannot hold.  Every variant is therefore looped for warm_s seconds before it is timed
     # (profiling captures at reduced size skip this: they take their figures from the counters).
-    warm_s = 0.0 if (tokens_per_response or responses) else 1.5
+    full_size = not (tokens_per_response or responses)
+    warm_s = 1.5 if full_size else 0.0
 
     def warm(fn):
         fn()
@@ -129,7 +137,9 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3, responses=0
                      "roofline": {"bound": "tensor", "achieved": useful, "peak": burst, "unit": "TFLOP/s",
                                   "frac": useful / burst, "peak_kind": "of " + kind + " (burst)",
                                   "frac_of_sustained": useful / sustained, "frac_of_nominal_2250": useful / 2250.0,
-                                  "traffic": None}}
+                                  "traffic": (NCU_TRAFFIC_FUSED["fwd_bwd_bytes_per_call" if bwd else "fwd_bytes_per_call"]
+                                              if full_size and cfg == 3 and NCU_TRAFFIC_FUSED["lmhead_cu_sha1"] == _lmhead_sha1()
+                                              else None)}}
     # the same call without multiplying the masked rows at all (their log-prob is not produced)
     def run_skip():
         rlf.rlf_fused_lmhead_grpo_obj(H, W, ids, seq, adv, old, ref, mask, synth.EPS_CLIP, synth.EPS_CLIP,
@@ -196,6 +206,12 @@ def _entropy_section_sha1():
     a = text.find(b"// Forward-only log-prob (+ entropy) of given target ids")
     b = text.find(b"// Skip-masked variant:")
     return hashlib.sha1(text[a:b] if 0 <= a < b else text).hexdigest()
+
+
+def _lmhead_sha1():
+    """Hash of the fused LM-head source file."""
+    with open(os.path.join(ROOT, "paper_2509_06980_b200", "csrc", "lmhead.cu"), "rb") as f:
+        return hashlib.sha1(f.read()).hexdigest()
 
 
 def _kernel_sha1():
@@ -914,7 +930,14 @@ def main():
                     help="with --fused-only: the Qwen3-4B head (3) or the Qwen3-8B head (4)")
     ap.add_argument("--responses", type=int, default=0,
                     help="with --fused-only: one group of this many full-length responses (profiling captures)")
+    ap.add_argument("--source-keys", action="store_true",
+                    help="print the source hashes that key the stored ncu traffic figures, and exit")
     args = ap.parse_args()
+    if args.source_keys:
+        print(json.dumps({"logits_loss_cu_sha1 (row kernel section)": _kernel_sha1(),
+                          "section_sha1 (forward-only section)": _entropy_section_sha1(),
+                          "lmhead_cu_sha1": _lmhead_sha1()}))
+        return
     if args.gpus < 1:
         raise SystemExit("--gpus must be at least 1")
     world_env = os.environ.get("WORLD_SIZE")

@@ -553,6 +553,12 @@ grpo_row_cluster_kernel(const FastParams p) {
         }
     }
     if (status && p.dev_status) atomicOr(p.dev_status, status);
+    // A warp that gave up has stopped waiting for its rows' exchanges, so peers' asynchronous stores
+    // of the last rows may still be on their way into this CTA's shared memory: give them two
+    // milliseconds (they take microseconds) before the CTA may be retired.  Every CTA still runs all
+    // its iterations and issues all its stores, so the barrier below is always reached by all.
+    if (gave_up)
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
     // no CTA leaves while a peer could still address its shared memory
     cluster_sync_all();
 }
@@ -779,51 +785,33 @@ static bool pick_shape(int nvec, FastShape* out) {
 
 typedef void (*FastKernel)(const FastParams);
 
-template <int THREADS, bool ONE_EXP>
-static FastKernel fast_kernel_for_nv(int nv) {
+// the row kernel's instantiation for a launch shape: vectors per thread (one of 1..6, 8, 10) and the
+// variant flags (one exponential per element, entropy output, skip-masked row list, per-token weights)
+template <int THREADS, bool ONE_EXP, bool ENT = false, bool SKIP = false, bool WT = false>
+static FastKernel row_kernel_for_nv(int nv) {
     switch (nv) {
-        case 1: return grpo_row_cluster_kernel<THREADS, 1, ONE_EXP>;
-        case 2: return grpo_row_cluster_kernel<THREADS, 2, ONE_EXP>;
-        case 3: return grpo_row_cluster_kernel<THREADS, 3, ONE_EXP>;
-        case 4: return grpo_row_cluster_kernel<THREADS, 4, ONE_EXP>;
-        case 5: return grpo_row_cluster_kernel<THREADS, 5, ONE_EXP>;
-        case 6: return grpo_row_cluster_kernel<THREADS, 6, ONE_EXP>;
-        case 8: return grpo_row_cluster_kernel<THREADS, 8, ONE_EXP>;
-        case 10: return grpo_row_cluster_kernel<THREADS, 10, ONE_EXP>;
+        case 1: return grpo_row_cluster_kernel<THREADS, 1, ONE_EXP, ENT, SKIP, WT>;
+        case 2: return grpo_row_cluster_kernel<THREADS, 2, ONE_EXP, ENT, SKIP, WT>;
+        case 3: return grpo_row_cluster_kernel<THREADS, 3, ONE_EXP, ENT, SKIP, WT>;
+        case 4: return grpo_row_cluster_kernel<THREADS, 4, ONE_EXP, ENT, SKIP, WT>;
+        case 5: return grpo_row_cluster_kernel<THREADS, 5, ONE_EXP, ENT, SKIP, WT>;
+        case 6: return grpo_row_cluster_kernel<THREADS, 6, ONE_EXP, ENT, SKIP, WT>;
+        case 8: return grpo_row_cluster_kernel<THREADS, 8, ONE_EXP, ENT, SKIP, WT>;
+        case 10: return grpo_row_cluster_kernel<THREADS, 10, ONE_EXP, ENT, SKIP, WT>;
     }
     return nullptr;
 }
-template <int THREADS>
-static FastKernel weighted_kernel_for_nv(int nv) {
-    switch (nv) {
-        case 1: return grpo_row_cluster_kernel<THREADS, 1, true, false, false, true>;
-        case 2: return grpo_row_cluster_kernel<THREADS, 2, true, false, false, true>;
-        case 3: return grpo_row_cluster_kernel<THREADS, 3, true, false, false, true>;
-        case 4: return grpo_row_cluster_kernel<THREADS, 4, true, false, false, true>;
-        case 5: return grpo_row_cluster_kernel<THREADS, 5, true, false, false, true>;
-        case 6: return grpo_row_cluster_kernel<THREADS, 6, true, false, false, true>;
-        case 8: return grpo_row_cluster_kernel<THREADS, 8, true, false, false, true>;
-        case 10: return grpo_row_cluster_kernel<THREADS, 10, true, false, false, true>;
-    }
+// ... for a thread count known at run time
+template <bool ONE_EXP, bool ENT = false, bool SKIP = false, bool WT = false>
+static FastKernel row_kernel_for(int threads, int nv) {
+    if (threads == 256) return row_kernel_for_nv<256, ONE_EXP, ENT, SKIP, WT>(nv);
+    if (threads == 512) return row_kernel_for_nv<512, ONE_EXP, ENT, SKIP, WT>(nv);
+    if (threads == 1024) return row_kernel_for_nv<1024, ONE_EXP, ENT, SKIP, WT>(nv);
     return nullptr;
 }
-static FastKernel weighted_kernel(const FastShape& sh) {
-    if (sh.threads == 256) return weighted_kernel_for_nv<256>(sh.nv);
-    if (sh.threads == 512) return weighted_kernel_for_nv<512>(sh.nv);
-    if (sh.threads == 1024) return weighted_kernel_for_nv<1024>(sh.nv);
-    return nullptr;
-}
+static FastKernel weighted_kernel(const FastShape& sh) { return row_kernel_for<true, false, false, true>(sh.threads, sh.nv); }
 static FastKernel fast_kernel(const FastShape& sh) {
-    if (sh.one_exp) {
-        if (sh.threads == 256) return fast_kernel_for_nv<256, true>(sh.nv);
-        if (sh.threads == 512) return fast_kernel_for_nv<512, true>(sh.nv);
-        if (sh.threads == 1024) return fast_kernel_for_nv<1024, true>(sh.nv);
-    } else {
-        if (sh.threads == 256) return fast_kernel_for_nv<256, false>(sh.nv);
-        if (sh.threads == 512) return fast_kernel_for_nv<512, false>(sh.nv);
-        if (sh.threads == 1024) return fast_kernel_for_nv<1024, false>(sh.nv);
-    }
-    return nullptr;
+    return sh.one_exp ? row_kernel_for<true>(sh.threads, sh.nv) : row_kernel_for<false>(sh.threads, sh.nv);
 }
 
 static int sm_count() {
@@ -1364,20 +1352,6 @@ size_t entropy_workspace_bytes(int64_t T, int32_t V) {
     return loss_workspace_bytes(T) + 16 * ws_tokens(T) * chunks * kStreamWarps + 256;
 }
 
-template <int THREADS>
-static FastKernel entropy_kernel_for_nv(int nv) {
-    switch (nv) {
-        case 1: return grpo_row_cluster_kernel<THREADS, 1, false, true>;
-        case 2: return grpo_row_cluster_kernel<THREADS, 2, false, true>;
-        case 3: return grpo_row_cluster_kernel<THREADS, 3, false, true>;
-        case 4: return grpo_row_cluster_kernel<THREADS, 4, false, true>;
-        case 5: return grpo_row_cluster_kernel<THREADS, 5, false, true>;
-        case 6: return grpo_row_cluster_kernel<THREADS, 6, false, true>;
-        case 8: return grpo_row_cluster_kernel<THREADS, 8, false, true>;
-        case 10: return grpo_row_cluster_kernel<THREADS, 10, false, true>;
-    }
-    return nullptr;
-}
 
 }  // namespace rlf
 
@@ -1442,9 +1416,7 @@ extern "C" rlf_status rlf_logp_entropy_fwd(const void* logits, rlf_dtype dt, int
 
     FastShape sh;
     if (fast_ok && pick_shape(V >> 3, &sh)) {
-        FastKernel k = sh.threads == 256 ? entropy_kernel_for_nv<256>(sh.nv)
-                     : sh.threads == 512 ? entropy_kernel_for_nv<512>(sh.nv)
-                                         : entropy_kernel_for_nv<1024>(sh.nv);
+        FastKernel k = row_kernel_for<false, true>(sh.threads, sh.nv);
         if (!k) return RLF_ERR_UNSUPPORTED;
         int nc = max_clusters(k, sh);
         if (nc <= 0) return RLF_ERR_UNSUPPORTED;
@@ -1539,20 +1511,6 @@ fill_dead_rows_kernel(const float4* __restrict__ rec, int64_t Tn, int32_t V, lon
     }
 }
 
-template <int THREADS>
-static FastKernel skip_kernel_for_nv(int nv) {
-    switch (nv) {
-        case 1: return grpo_row_cluster_kernel<THREADS, 1, true, false, true>;
-        case 2: return grpo_row_cluster_kernel<THREADS, 2, true, false, true>;
-        case 3: return grpo_row_cluster_kernel<THREADS, 3, true, false, true>;
-        case 4: return grpo_row_cluster_kernel<THREADS, 4, true, false, true>;
-        case 5: return grpo_row_cluster_kernel<THREADS, 5, true, false, true>;
-        case 6: return grpo_row_cluster_kernel<THREADS, 6, true, false, true>;
-        case 8: return grpo_row_cluster_kernel<THREADS, 8, true, false, true>;
-        case 10: return grpo_row_cluster_kernel<THREADS, 10, true, false, true>;
-    }
-    return nullptr;
-}
 
 }  // namespace rlf
 
@@ -1609,9 +1567,7 @@ extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd_skip_masked(
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
 
-    FastKernel k = sh.threads == 256 ? skip_kernel_for_nv<256>(sh.nv)
-                 : sh.threads == 512 ? skip_kernel_for_nv<512>(sh.nv)
-                                     : skip_kernel_for_nv<1024>(sh.nv);
+    FastKernel k = row_kernel_for<true, false, true>(sh.threads, sh.nv);
     if (!k) return RLF_ERR_UNSUPPORTED;
     int nc = max_clusters(k, sh);
     if (nc <= 0) return RLF_ERR_UNSUPPORTED;
