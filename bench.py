@@ -44,8 +44,9 @@ WORKLOAD = "cfg1_qwen3_4b_microbatch: 16 responses x 2048 tokens, V=151936 bf16 
 #   streaming forward kernel: the T = 4096 capture, per token (traffic is proportional to rows);
 #   fused LM-head: every kernel of one forward / one forward + backward call at cfg 3 full size
 #   (one-pass capture of the whole call), per call.
-NCU_TRAFFIC = {"logits_loss_cu_sha1": "beae1f6cbc292ea9da59db4c5f59b105793ed141", "dram_bytes_per_token": 606029.0}
-NCU_TRAFFIC_FUSED = {"lmhead_cu_sha1": "", "fwd_bytes_per_call": None, "fwd_bwd_bytes_per_call": None}
+NCU_TRAFFIC = {"logits_loss_cu_sha1": "e9eba217cbf85c3b6dfedb33354884a03d938b02", "dram_bytes_per_token": 606054.0}
+NCU_TRAFFIC_FUSED = {"lmhead_cu_sha1": "36d3dbaf7feb04b93e273de1ef1762bb222b4141",
+                     "fwd_bytes_per_call": 3925863680.0, "fwd_bwd_bytes_per_call": 32853937408.0}
 
 
 def _peaks():
@@ -195,7 +196,7 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3, responses=0
 
 
 # the same for the forward-only log-prob + entropy pass (profiles/logp_entropy_stream_kernel_T4096_ncu_full.md)
-NCU_TRAFFIC_ENTROPY = {"section_sha1": "301958076486f234067b1a04b5a95e4254d97c46", "dram_bytes_per_token": 305667.0}
+NCU_TRAFFIC_ENTROPY = {"section_sha1": "2ebec178e05253433bddc7e3733a94e8c4a2063e", "dram_bytes_per_token": 305838.0}
 
 
 def _entropy_section_sha1():

@@ -1028,8 +1028,9 @@ scale_rows_kernel(const __nv_bfloat16* __restrict__ Hl, int D, int rows_max, con
 
 // in place over one chunk of stored exponentials e = exp(z - tile max): dZ = coef (e exp(tile max - lse)
 // - [v == y]) as bf16; the target column takes the fp32 target logit.  Rows from the live extent up
-// to the next multiple of 256 become zeros.  One CTA per (token tile, 256-column tile): four adjacent
-// blocks of the scratch, 64 KB of contiguous memory.
+// to the next multiple of 256 become zeros.  A work item is one (token tile, 256-column tile): four adjacent
+// blocks of the scratch, 64 KB of contiguous memory; the CTAs stride over the items (the launch is
+// usually one that a device flag turns into a no-op, which a small grid makes cheap).
 __global__ void __launch_bounds__(256)
 dz_from_e_kernel(__nv_bfloat16* __restrict__ ebuf, int V, int n_tiles, const float* __restrict__ tmax, int rows_max,
                  const int* __restrict__ count, int off, const float* __restrict__ lse_g,
@@ -1039,9 +1040,11 @@ dz_from_e_kernel(__nv_bfloat16* __restrict__ ebuf, int V, int n_tiles, const flo
     if (run_flag && *run_flag != run_want) return;
     __shared__ int live_s[kDzBlockRows];
     const int n = max(0, min(*count - off, rows_max));
-    const int tt = blockIdx.x, jt = blockIdx.y;
-    if (tt * kDzBlockRows >= ((n + 255) & ~255)) return;
     const int nc = 4 * n_tiles;
+    const long long items = (long long)(((n + 255) & ~255) / kDzBlockRows) * n_tiles;
+    for (long long item = blockIdx.x; item < items; item += gridDim.x) {
+    const int tt = (int)(item / n_tiles), jt = (int)(item - (long long)tt * n_tiles);
+    __syncthreads();                             // the previous item's readers of f_s / live_s are done
     if (threadIdx.x < kDzBlockRows) {
         const int r = tt * kDzBlockRows + threadIdx.x;
         const float coef = r < n ? coef_g[off + r] : 0.0f;
@@ -1081,6 +1084,7 @@ dz_from_e_kernel(__nv_bfloat16* __restrict__ ebuf, int V, int n_tiles, const flo
             const float py = ex2_approx((zy[idx[off + r]] - lse_g[off + r]) * kLog2e);
             ebuf[dz_offset(r, y, nc)] = __float2bfloat16_rn(fmaf(coef, py, -coef));
         }
+    }
     }
 }
 
@@ -1446,7 +1450,8 @@ static rlf_status fused_lmhead_impl(const void* hidden, const void* W, int64_t T
         };
         const int64_t tcp = (tc + 255) & ~(int64_t)255;
         auto dz_pass = [&](const int* run_flag) {
-            dz_from_e_kernel<<<dim3((unsigned)(tcp / kDzBlockRows), (unsigned)z.n_tiles), 256, 0, s>>>(
+            const long long dz_items = (tcp / kDzBlockRows) * (long long)z.n_tiles;
+            dz_from_e_kernel<<<(unsigned)(dz_items < 148 * 8 ? dz_items : 148 * 8), 256, 0, s>>>(
                 dz, V, z.n_tiles, z.tmax, (int)tc, counts, (int)t0, lse_g, coef_g, y_g, idx_live, zy, run_flag, 1);
             count_launch();
         };
