@@ -17,7 +17,8 @@ MUTATIONS = [
     ("state_leaks_across_sequences", "        int inside = 0;\n        for (int64_t t = cu_seqlens[b]", "        static int inside = 0;\n        for (int64_t t = cu_seqlens[b]", "test_oracle_mask.py"),
     ("stray_close_opens_nothing_but_is_masked", "m = inside ? 0 : 1;", "m = (inside || ids[t] == close_id) ? 0 : 1;", "test_oracle_mask.py"),
     ("biased_std_always", "double div = unbiased ? (double)(n - 1) : (double)n;", "double div = (double)n;", "test_oracle_advantage.py"),
-    ("advantage_not_centred", "adv[i] = ((double)rewards[i] - mean) / (sd + eps);", "adv[i] = ((double)rewards[i]) / (sd + eps);", "test_oracle_advantage.py"),
+    ("advantage_not_centred", "? ((double)rewards[i] - mean) / (sd + eps) : 0.0;", "? ((double)rewards[i]) / (sd + eps) : 0.0;", "test_oracle_advantage.py"),
+    ("degenerate_group_divides_zero_by_zero", "adv[i] = (sd + eps > 0.0) ? ((double)rewards[i] - mean) / (sd + eps) : 0.0;", "adv[i] = ((double)rewards[i] - mean) / (sd + eps);", "test_oracle_advantage.py"),
     ("clip_uses_wrong_side", "*clipped = (A > 0.0 && rho > hi) || (A < 0.0 && rho < lo);", "*clipped = (A > 0.0 && rho < lo) || (A < 0.0 && rho > hi);", "test_oracle_loss.py"),
     ("kl_gradient_sign", "*dkl = 1.0 - exp(d);", "*dkl = exp(d) - 1.0;", "test_oracle_loss.py"),
     ("kl_direction", "double d = ref_lp - logp;", "double d = logp - ref_lp;", "test_oracle_loss.py"),
