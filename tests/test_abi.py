@@ -120,6 +120,9 @@ def test_host_validation_rejects_bad_arguments_before_touching_a_device(lib):
     bw = lib.rlf_tune_lmhead_backward
     bw.argtypes = [ctypes.c_int] * 2
     assert bw(2, 1) == -2 and bw(1, -1) == -2 and bw(0, 0) == 0 and bw(1, 1) == 0
+    pc = lib.rlf_tune_lmhead_pacing
+    pc.argtypes = [ctypes.c_int]
+    assert pc(2) == -2 and pc(-1) == -2 and pc(0) == 0 and pc(1) == 0
     t = lib.rlf_tune_logits_kernel
     t.argtypes = [ctypes.c_int] * 3
     assert t(3, 512, 0) == -2 and t(4, 500, 0) == -2 and t(0, 0, -1) == 0

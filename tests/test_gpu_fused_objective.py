@@ -125,6 +125,15 @@ def test_fused_results_do_not_depend_on_the_schedule():
             torch.cuda.synchronize()
     finally:
         b.tune_lmhead_schedule(0, 0, 0)
+    # pacing (the workers' meeting points before each unit) only delays loads
+    try:
+        b.tune_lmhead_pacing(0)
+        unpaced = b.rlf_fused_lmhead_grpo(*args, denom=n)
+        torch.cuda.synchronize()
+    finally:
+        b.tune_lmhead_pacing(1)
+    for got, want in zip(unpaced, outs[(0, 0, 0)]):
+        assert torch.equal(got, want)
     ref = outs[(0, 0, 0)]
     for key, o in outs.items():
         assert torch.equal(o[0], ref[0]) and torch.equal(o[1], ref[1]) and torch.equal(o[2], ref[2]), key
