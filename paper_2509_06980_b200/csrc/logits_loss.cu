@@ -312,11 +312,13 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t mbar, uint32_t parity
 // SKIP: the rows to process come from a compacted list (rows whose loss weight is zero are
 // neither read nor computed); token records are then indexed like the list.
 // WT: per-token loss weights from the caller replace the common 1 / N.
-template <int THREADS, int NV, bool ONE_EXP, bool ENT = false, bool SKIP = false, bool WT = false>
+// CMAX: the largest cluster the instantiation serves (8 is the portable limit; 16 for rows that 8 CTAs
+// of 256 threads cannot hold, e.g. a vocabulary of 262144, launched with the non-portable size allowed).
+template <int THREADS, int NV, bool ONE_EXP, bool ENT = false, bool SKIP = false, bool WT = false, int CMAX = 8>
 __global__ void __launch_bounds__(THREADS, ctas_per_sm(THREADS, NV))
 grpo_row_cluster_kernel(const FastParams p) {
     constexpr int NWARPS = THREADS / 32;
-    constexpr int MAXE = 8 * NWARPS;          // (max, sum) pairs per row: one per warp of the cluster
+    constexpr int MAXE = CMAX * NWARPS;       // (max, sum) pairs per row: one per warp of the cluster
     // staging: [NV][THREADS] 16-byte slots; a thread only ever touches its own slots, so its own
     // cp.async wait is all the synchronisation the logits data needs
     extern __shared__ __align__(16) uint4 stage[];
@@ -750,7 +752,7 @@ static std::atomic<int> g_units_per_cta{0};       // streaming forward pass; 0: 
 
 struct FastShape { int cluster, threads, nv, one_exp; };
 
-static const int kNvChoices[] = {1, 2, 3, 4, 5, 6, 8, 10};
+static const int kNvChoices[] = {1, 2, 3, 4, 5, 6, 7, 8, 9, 10};
 
 static int round_nv(int need) {
     for (int c : kNvChoices) if (c >= need) return c;
@@ -758,7 +760,7 @@ static int round_nv(int need) {
 }
 
 // launch shape that holds a row of nvec 16-byte vectors in registers
-static bool pick_shape(int nvec, FastShape* out) {
+static bool pick_shape(int nvec, FastShape* out, bool allow_wide_cluster = false) {
     const int tc = g_tune_cluster.load(), tt = g_tune_threads.load();
     const int oe = g_tune_one_exp.load() < 0 ? 1 : g_tune_one_exp.load();
     if (tc > 0 && tt > 0) {
@@ -779,13 +781,23 @@ static bool pick_shape(int nvec, FastShape* out) {
                 return true;
             }
         }
+        // rows beyond 8 x 256 x 10 vectors: a cluster of 16 such CTAs (four per SM, every register
+        // holding a piece of a row) before CTAs of 512 threads (two per SM): V = 262144 ran at 0.80 of
+        // the copy rate as 8 x 512 threads
+        if (th == 256 && allow_wide_cluster && oe) {
+            const int need = ((nvec + 15) / 16 + th - 1) / th;
+            if (need <= 10) {
+                *out = {16, th, round_nv(need), oe};
+                return true;
+            }
+        }
     }
     return false;
 }
 
 typedef void (*FastKernel)(const FastParams);
 
-// the row kernel's instantiation for a launch shape: vectors per thread (one of 1..6, 8, 10) and the
+// the row kernel's instantiation for a launch shape: vectors per thread (1 .. 10) and the
 // variant flags (one exponential per element, entropy output, skip-masked row list, per-token weights)
 template <int THREADS, bool ONE_EXP, bool ENT = false, bool SKIP = false, bool WT = false>
 static FastKernel row_kernel_for_nv(int nv) {
@@ -796,8 +808,21 @@ static FastKernel row_kernel_for_nv(int nv) {
         case 4: return grpo_row_cluster_kernel<THREADS, 4, ONE_EXP, ENT, SKIP, WT>;
         case 5: return grpo_row_cluster_kernel<THREADS, 5, ONE_EXP, ENT, SKIP, WT>;
         case 6: return grpo_row_cluster_kernel<THREADS, 6, ONE_EXP, ENT, SKIP, WT>;
+        case 7: return grpo_row_cluster_kernel<THREADS, 7, ONE_EXP, ENT, SKIP, WT>;
         case 8: return grpo_row_cluster_kernel<THREADS, 8, ONE_EXP, ENT, SKIP, WT>;
+        case 9: return grpo_row_cluster_kernel<THREADS, 9, ONE_EXP, ENT, SKIP, WT>;
         case 10: return grpo_row_cluster_kernel<THREADS, 10, ONE_EXP, ENT, SKIP, WT>;
+    }
+    return nullptr;
+}
+// the training kernel for a cluster of 16 CTAs of 256 threads (rows of 8 x 256 x 10 + 1 .. 16 x 256 x 10 vectors)
+static FastKernel wide_cluster_kernel(int nv) {
+    switch (nv) {
+        case 6: return grpo_row_cluster_kernel<256, 6, true, false, false, false, 16>;
+        case 7: return grpo_row_cluster_kernel<256, 7, true, false, false, false, 16>;
+        case 8: return grpo_row_cluster_kernel<256, 8, true, false, false, false, 16>;
+        case 9: return grpo_row_cluster_kernel<256, 9, true, false, false, false, 16>;
+        case 10: return grpo_row_cluster_kernel<256, 10, true, false, false, false, 16>;
     }
     return nullptr;
 }
@@ -811,6 +836,7 @@ static FastKernel row_kernel_for(int threads, int nv) {
 }
 static FastKernel weighted_kernel(const FastShape& sh) { return row_kernel_for<true, false, false, true>(sh.threads, sh.nv); }
 static FastKernel fast_kernel(const FastShape& sh) {
+    if (sh.cluster == 16) return wide_cluster_kernel(sh.nv);
     return sh.one_exp ? row_kernel_for<true>(sh.threads, sh.nv) : row_kernel_for<false>(sh.threads, sh.nv);
 }
 
@@ -853,6 +879,11 @@ static int max_clusters(FastKernel k, const FastShape& sh) {
         if (cache[i].dev == dev && cache[i].k == k && cache[i].cluster == sh.cluster) return cache[i].n;
     if (cudaFuncSetAttribute((const void*)k, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              stage_bytes(sh.threads, sh.nv)) != cudaSuccess) {
+        cudaGetLastError();
+        return -1;
+    }
+    if (sh.cluster > 8 &&
+        cudaFuncSetAttribute((const void*)k, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
         cudaGetLastError();
         return -1;
     }
@@ -990,10 +1021,15 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
 
         FastShape sh;
         const bool tuned = g_tune_cluster.load() > 0;
-        if (fast_ok && a.T < (1ll << 31) && pick_shape(a.V >> 3, &sh)) {
+        if (fast_ok && a.T < (1ll << 31) && pick_shape(a.V >> 3, &sh, /*allow_wide_cluster=*/wtok == nullptr)) {
             FastKernel k = wtok ? weighted_kernel(sh) : fast_kernel(sh);
+            int nc = k ? max_clusters(k, sh) : -1;
+            if (nc <= 0 && sh.cluster == 16 && pick_shape(a.V >> 3, &sh)) {
+                // the device does not take a cluster of 16: the portable shape instead
+                k = fast_kernel(sh);
+                nc = k ? max_clusters(k, sh) : -1;
+            }
             if (!k) return RLF_ERR_UNSUPPORTED;
-            int nc = max_clusters(k, sh);
             if (nc <= 0) return RLF_ERR_UNSUPPORTED;      // this shape does not fit on the device
             nc = clusters_for(nc, a.T);
             FastParams p;

@@ -101,7 +101,8 @@ def test_forward_only_and_run_to_run_determinism():
 
 
 @pytest.mark.parametrize("V,dtype", [(1000, "bf16"), (1001, "bf16"), (37, "f32"), (8, "bf16"), (4099, "f32"),
-                                     (8192, "bf16"), (12288 + 8, "bf16"), (1, "f32")])
+                                     (8192, "bf16"), (12288 + 8, "bf16"), (1, "f32"), (50304, "bf16"),
+                                     (262144, "bf16"), (200000, "bf16")])
 def test_odd_vocabularies_take_a_correct_path(V, dtype):
     spec = synth.scaled(synth.SPECS[0], V=V, logits_dtype=dtype, logits_std=3.0)
     batch = synth.make_batch(spec, DEV)
