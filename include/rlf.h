@@ -103,6 +103,18 @@ rlf_status rlf_build_loss_mask(const int32_t *ids, const int32_t *cu_seqlens, in
                                int32_t *dev_status, rlf_stream_t stream);
 
 /*
+ * Number of responses that carry loss: those with at least one token of mask 1.  (Paper Sec. 2.3.2:
+ * the loss is taken over the model's own tokens; a response that is all tool feedback, or cut to
+ * nothing, carries none.)  It is the denominator of the sequence-mean aggregation of the *_obj entry
+ * points (their `denom`), which a caller needs on its own when one batch is spread over several calls
+ * or several GPUs: each part counts its responses and the counts are added.
+ *   mask [T] uint8;  cu_seqlens [B+1] int32;  *count_out int64 on the device (overwritten)
+ * A malformed cu_seqlens sets RLF_DEV_BAD_SEQ and the response is clipped to [0, T).  B = 0 is valid.
+ */
+rlf_status rlf_count_live_responses(const uint8_t *mask, const int32_t *cu_seqlens, int32_t B, int64_t T,
+                                    int64_t *count_out, int32_t *dev_status, rlf_stream_t stream);
+
+/*
  * Group-relative outcome advantage.  (Paper Sec. 2.3.2 / Fig. 4 name GRPO as
  * the algorithm; the formula is the standard group normalisation.)
  *     A_i = (r_i - mean_g) / (std_g + eps),  g = group of response i

@@ -18,7 +18,7 @@ FN_LOGP_LOSS, FN_FUSED_LMHEAD, FN_LOGP_ENTROPY, FN_FUSED_LOGP_ENTROPY = 3, 4, 5,
 DEV_BAD_TARGET, DEV_BAD_SEQ, DEV_NONFINITE, DEV_TIMEOUT = 1, 2, 4, 8
 
 EXPORTS = [
-    "rlf_build_loss_mask", "rlf_group_advantage", "rlf_rule_reward", "rlf_kl_in_reward", "rlf_grpo_logp_loss_fwd_bwd",
+    "rlf_build_loss_mask", "rlf_count_live_responses", "rlf_group_advantage", "rlf_rule_reward", "rlf_kl_in_reward", "rlf_grpo_logp_loss_fwd_bwd",
     "rlf_grpo_logp_loss_fwd_bwd_static", "rlf_grpo_logp_loss_fwd_bwd_skip_masked", "rlf_grpo_logp_loss_fwd_bwd_obj", "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_fused_lmhead_grpo_obj", "rlf_fused_lmhead_logp_entropy", "rlf_workspace_bytes", "rlf_grpo_step_host", "rlf_step_arena_bytes",
     "rlf_tune_logits_kernel", "rlf_tune_logits_grid", "rlf_tune_lmhead", "rlf_tune_lmhead_schedule", "rlf_tune_lmhead_backward", "rlf_tune_lmhead_pacing", "rlf_launch_count", "rlf_status_string", "rlf_version",
 ]
@@ -33,6 +33,7 @@ _lib = ctypes.CDLL(_LIB_PATH)
 _vp, _i32, _i64, _f32, _sz, _int = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float,
                                     ctypes.c_size_t, ctypes.c_int)
 _lib.rlf_build_loss_mask.argtypes = [_vp, _vp, _i32, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]
+_lib.rlf_count_live_responses.argtypes = [_vp, _vp, _i32, _i64, _vp, _vp, _vp]
 _lib.rlf_group_advantage.argtypes = [_vp, _vp, _i32, _i32, _f32, _int, _vp, _vp, _vp]
 _lib.rlf_grpo_logp_loss_fwd_bwd.argtypes = [_vp, _int, _i64, _i32, _i64, _vp, _vp, _vp, _i32, _vp, _vp, _vp,
                                             _f32, _f32, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
@@ -68,7 +69,7 @@ _lib.rlf_fused_lmhead_grpo_obj.argtypes = [_vp, _vp, _i64, _i32, _i32, _vp, _vp,
                                            _f32, _int, _int, _vp, _vp, _vp, _vp, _vp, _int, _vp, _sz, _vp, _vp]
 _lib.rlf_fused_lmhead_logp_entropy.argtypes = [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]
 # every entry point that returns an rlf_status
-for _n in ("rlf_build_loss_mask", "rlf_group_advantage", "rlf_rule_reward", "rlf_kl_in_reward",
+for _n in ("rlf_build_loss_mask", "rlf_count_live_responses", "rlf_group_advantage", "rlf_rule_reward", "rlf_kl_in_reward",
            "rlf_grpo_logp_loss_fwd_bwd", "rlf_grpo_logp_loss_fwd_bwd_obj", "rlf_grpo_logp_loss_fwd_bwd_skip_masked",
            "rlf_logp_entropy_fwd", "rlf_fused_lmhead_grpo", "rlf_fused_lmhead_grpo_obj",
            "rlf_fused_lmhead_logp_entropy", "rlf_grpo_step_host", "rlf_tune_logits_kernel", "rlf_tune_logits_grid",
@@ -176,6 +177,18 @@ def rlf_build_loss_mask(ids, cu_seqlens, open_id, close_id, valid=None, mask_out
                                     _ptr(seq_id_out, torch.int32), _ptr(n_out, torch.int64),
                                     _ptr(dev_status, torch.int32), _stream()), "rlf_build_loss_mask")
     return mask_out, seq_id_out, n_out
+
+
+def rlf_count_live_responses(mask, cu_seqlens, count_out=None, dev_status=None):
+    """-> int64[1] on the device: responses with at least one token of mask 1."""
+    T = mask.shape[0]
+    B = cu_seqlens.shape[0] - 1
+    if count_out is None:
+        count_out = torch.zeros(1, dtype=torch.int64, device=mask.device)
+    _check(_lib.rlf_count_live_responses(_ptr(mask, torch.uint8), _ptr(cu_seqlens, torch.int32), B, T,
+                                         _ptr(count_out, torch.int64), _ptr(dev_status, torch.int32), _stream()),
+           "rlf_count_live_responses")
+    return count_out
 
 
 def rlf_group_advantage(rewards, group_size=None, group_id=None, num_groups=None, eps=1e-6,

@@ -104,3 +104,42 @@ extern "C" rlf_status rlf_build_loss_mask(const int32_t* ids, const int32_t* cu_
     }
     return RLF_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Number of responses that carry loss: those with at least one token of mask 1.  The denominator of
+// the sequence-mean aggregation; a rank of a sharded batch counts its own responses and the counts
+// are summed.  One CTA per response; integer atomics (exact).
+namespace rlf {
+__global__ void __launch_bounds__(256)
+count_live_responses_kernel(const uint8_t* __restrict__ mask, const int32_t* __restrict__ cu_seqlens, int64_t T,
+                            unsigned long long* __restrict__ count_out, int32_t* __restrict__ dev_status) {
+    long long lo = cu_seqlens[blockIdx.x], hi = cu_seqlens[blockIdx.x + 1];
+    if (lo < 0 || hi < lo || hi > T) {
+        if (threadIdx.x == 0 && dev_status) atomicOr(dev_status, RLF_DEV_BAD_SEQ);
+        lo = lo < 0 ? 0 : (lo > T ? T : lo);
+        hi = hi < lo ? lo : (hi > T ? T : hi);
+    }
+    int any = 0;
+    for (long long t = lo + threadIdx.x; t < hi; t += 256) any |= mask[t] != 0;
+    any = __syncthreads_or(any);
+    if (threadIdx.x == 0 && any) atomicAdd(count_out, 1ull);
+}
+}  // namespace rlf
+
+extern "C" rlf_status rlf_count_live_responses(const uint8_t* mask, const int32_t* cu_seqlens, int32_t B, int64_t T,
+                                               int64_t* count_out, int32_t* dev_status, rlf_stream_t stream) {
+    using namespace rlf;
+    if (B < 0 || T < 0) return RLF_ERR_SHAPE;
+    if (!count_out || (B > 0 && !cu_seqlens) || (T > 0 && B > 0 && !mask)) return RLF_ERR_NULL;
+    rlf_status st = check_arch();
+    if (st != RLF_OK) return st;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(count_out, 0, sizeof(int64_t), s) != cudaSuccess) return RLF_ERR_CUDA;
+    if (B > 0) {
+        count_live_responses_kernel<<<B, 256, 0, s>>>(mask, cu_seqlens, T, reinterpret_cast<unsigned long long*>(count_out),
+                                                      dev_status);
+        count_launch();
+        if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
+    }
+    return RLF_OK;
+}

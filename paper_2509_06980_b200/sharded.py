@@ -6,7 +6,9 @@ the rewards of its own GRPO group.  So a batch is cut between groups: every rank
 all-reduce sums over NCCL:
 
   1. the int64 count of loss-carrying tokens, before the loss kernel (its coefficients divide by the
-     global count);
+     global count); for the sequence-mean aggregation the count of loss-carrying RESPONSES instead
+     (rlf_count_live_responses on this rank's responses), the only thing that aggregation needs
+     from the other ranks;
   2. the four fp64 loss scalars, after it (each rank's are already divided by the global count, so
      they add up);
   3. for the fused LM-head path, grad_W [V, D] fp32 (the ordinary data-parallel weight-gradient
@@ -80,15 +82,32 @@ def count_phase(ids, cu_seqlens, open_id, close_id, ops=None):
 
 
 def loss_phase(n_global, mask, seq_id, ids, rewards, group_size, old_logp, ref_logp, eps_clip, beta_kl, logits=None,
-               hidden=None, W=None, grad_W=None, accumulate_grad_W=False, adv_eps=1e-6, ops=None):
-    """Phase 2 on this rank's tokens, against the batch's global token count: advantages of this rank's
-    groups, log-probs, this rank's share of the loss scalars (they add up over ranks) and gradients
-    (grad_W is this rank's contribution, still to be summed over the ranks)."""
+               hidden=None, W=None, grad_W=None, accumulate_grad_W=False, adv_eps=1e-6, ops=None, aggregation=0,
+               eps_clip_high=None):
+    """Phase 2 on this rank's tokens, against the batch's global count (tokens for the token mean,
+    loss-carrying responses for the sequence mean): advantages of this rank's groups, log-probs, this
+    rank's share of the loss scalars (they add up over ranks) and gradients (grad_W is this rank's
+    contribution, still to be summed over the ranks).  aggregation 1 or an upper clip width of its own
+    go through the *_obj entry points."""
     ops = _ops(ops)
     if (logits is None) == (hidden is None):
         raise ValueError("give either logits or hidden + W")
     adv = ops.rlf_group_advantage(rewards, group_size=group_size, eps=adv_eps)
     out = dict(adv=adv)
+    if aggregation != 0 or eps_clip_high is not None:
+        hi = eps_clip if eps_clip_high is None else eps_clip_high
+        if logits is not None:
+            logp, loss, grad = ops.rlf_grpo_logp_loss_fwd_bwd_obj(logits, ids, seq_id, adv, old_logp, ref_logp, mask,
+                                                                  eps_clip, hi, beta_kl, aggregation=aggregation,
+                                                                  denom=n_global)
+            out.update(logp=logp, loss=loss, grad_logits=grad)
+        else:
+            logp, loss, gh, gw = ops.rlf_fused_lmhead_grpo_obj(hidden, W, ids, seq_id, adv, old_logp, ref_logp, mask,
+                                                               eps_clip, hi, beta_kl, aggregation=aggregation,
+                                                               denom=n_global, grad_W=grad_W,
+                                                               accumulate_grad_W=accumulate_grad_W)
+            out.update(logp=logp, loss=loss, grad_hidden=gh, grad_W=gw)
+        return out
     if logits is not None:
         logp, loss, grad = ops.rlf_grpo_logp_loss_fwd_bwd(logits, ids, seq_id, adv, old_logp, ref_logp, mask, eps_clip,
                                                           beta_kl, denom=n_global)
@@ -103,7 +122,7 @@ def loss_phase(n_global, mask, seq_id, ids, rewards, group_size, old_logp, ref_l
 
 def sharded_grpo_step(ids, cu_seqlens, rewards, group_size, old_logp, ref_logp, open_id, close_id, eps_clip, beta_kl,
                       logits=None, hidden=None, W=None, grad_W=None, accumulate_grad_W=False, adv_eps=1e-6,
-                      group=None, ops=None, reduce_grad_W=True, n_global=None):
+                      group=None, ops=None, reduce_grad_W=True, n_global=None, aggregation=0, eps_clip_high=None):
     """This rank's part of one sharded step.  All tensors are this rank's own (whole groups).
 
     Give `logits` [T_local, V] for the logits path (returns grad_logits) or `hidden` [T_local, D] and
@@ -113,15 +132,19 @@ def sharded_grpo_step(ids, cu_seqlens, rewards, group_size, old_logp, ref_logp, 
     last one (a reduced buffer must not be reduced again), and pass the whole batch's token count as
     `n_global` (int64[1], e.g. the n_global a counting pass over the whole shard returned): a
     micro-batch's own count is not the batch's denominator.  With `n_global` given the count exchange
-    is skipped.
+    is skipped.  aggregation: 0 = masked token mean over the batch (the exchanged count is of tokens),
+    1 = mean over loss-carrying responses of each response's token mean (the exchanged count is of such
+    responses); eps_clip_high: upper clip width when it differs from eps_clip.
     -> dict(mask, seq_id, n_local, n_global, adv, logp, loss (global, fp64[4]), grad_logits | grad_hidden, grad_W)
     """
     mask, seq_id, n_local = count_phase(ids, cu_seqlens, open_id, close_id, ops)
+    if aggregation == 1:
+        n_local = _ops(ops).rlf_count_live_responses(mask, cu_seqlens)
     if n_global is None:
         n_global = _all_reduce_sum(n_local.clone(), group)
     out = loss_phase(n_global, mask, seq_id, ids, rewards, group_size, old_logp, ref_logp, eps_clip, beta_kl,
                      logits=logits, hidden=hidden, W=W, grad_W=grad_W, accumulate_grad_W=accumulate_grad_W,
-                     adv_eps=adv_eps, ops=ops)
+                     adv_eps=adv_eps, ops=ops, aggregation=aggregation, eps_clip_high=eps_clip_high)
     if "grad_W" in out and reduce_grad_W:
         _all_reduce_sum(out["grad_W"], group)
     out["loss"] = _all_reduce_sum(out["loss"].clone(), group)

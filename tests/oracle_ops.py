@@ -36,3 +36,16 @@ def rlf_fused_lmhead_grpo(hidden, W, ids, seq_id, adv, old_logp, ref_logp, mask,
             grad_W.copy_(gw)
         gw = grad_W
     return torch.from_numpy(r["logp"]), torch.from_numpy(r["loss"]), torch.from_numpy(r["grad_hidden"]), gw
+
+
+def rlf_count_live_responses(mask, cu_seqlens, **_):
+    m, cu = mask.numpy(), cu_seqlens.numpy()
+    return torch.tensor([sum(1 for b in range(len(cu) - 1) if m[cu[b]:cu[b + 1]].any())], dtype=torch.int64)
+
+
+def rlf_grpo_logp_loss_fwd_bwd_obj(logits, ids, seq_id, adv, old_logp, ref_logp, mask, eps_low, eps_high, beta_kl,
+                                   aggregation=0, denom=None, **_):
+    r = orc.grpo_loss_obj(logits.double().numpy(), ids.numpy(), seq_id.numpy(), adv.numpy(), old_logp.numpy(),
+                          ref_logp.numpy(), mask.numpy(), eps_low, eps_high, beta_kl, aggregation=aggregation,
+                          denom=None if denom is None else int(denom.item()))
+    return torch.from_numpy(r["logp"]), torch.from_numpy(r["loss"]), torch.from_numpy(r["grad"])

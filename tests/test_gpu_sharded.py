@@ -111,3 +111,47 @@ def test_fused_step_in_a_group_of_one_against_the_oracle():
     for name in ("grad_hidden", "grad_W"):
         got = out[name].float().cpu().numpy().astype(np.float64)
         assert np.abs(got - r[name]).max() <= 2.0 ** -7 * np.abs(r[name]).max(), name
+
+
+def test_live_response_count_and_sequence_mean_step_against_the_oracle():
+    """rlf_count_live_responses against a count made on the host (a response that is all tool feedback
+    carries no loss; a malformed boundary is clipped and flagged), then the sharded step with the
+    sequence-mean aggregation and an upper clip width of its own, in a group of one, against the
+    oracle's objective function."""
+    from oracle import rlf_oracle as orc
+    from util import loss_close
+    b = gc.binding()
+    spec = synth.scaled(synth.SPECS[2], V=4096, num_prompts=3, group_size=4, len_lo=12, len_hi=70, spans_lo=1,
+                        spans_hi=2, cover_lo=0.2, cover_hi=0.5)
+    batch = synth.make_batch(spec, DEV)
+    ora = gc.oracle_chain(batch)
+    cu = batch.cu_seqlens.cpu().numpy()
+    mask = torch.from_numpy(ora["mask"].copy()).to(DEV)
+    mask[cu[2]:cu[3]] = 0                                    # response 2: nothing but observations
+    mask[cu[7]:cu[8]] = 0
+    want = sum(1 for i in range(len(cu) - 1) if mask[cu[i]:cu[i + 1]].any().item())
+    assert want == len(cu) - 3
+    got = b.rlf_count_live_responses(mask, batch.cu_seqlens)
+    torch.cuda.synchronize()
+    assert got.item() == want
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    bad = batch.cu_seqlens.clone()
+    bad[-1] = batch.T + 5
+    assert b.rlf_count_live_responses(mask, bad, dev_status=st).item() == want and st.item() == 2
+    assert b.rlf_count_live_responses(mask[:0], batch.cu_seqlens[:1]).item() == 0
+
+    out = sharded.sharded_grpo_step(batch.ids, batch.cu_seqlens, batch.rewards, spec.group_size, batch.old_logp,
+                                    batch.ref_logp, spec.open_id, spec.close_id, 0.2, 0.02, logits=batch.logits,
+                                    aggregation=1, eps_clip_high=0.3)
+    torch.cuda.synchronize()
+    assert out["n_global"].item() == len(cu) - 1              # every response of the recipe carries loss
+    r = orc.grpo_loss_obj(gc.to_np(batch.logits), ora["ids"], ora["seq_id"], ora["adv"], batch.old_logp.cpu().numpy(),
+                          batch.ref_logp.cpu().numpy(), ora["mask"], 0.2, 0.3, 0.02, aggregation=1, want_coef=True)
+    assert np.abs(out["logp"].cpu().numpy() - r["logp"]).max() <= gc.LOGP_ATOL
+    lg = out["loss"].cpu().numpy()
+    for k in range(3):
+        assert loss_close(lg[k], r["loss"][k], 1e-6, gc.LOSS_RTOL), (k, lg, r["loss"])
+    guard = gc.near_clip_bound(r["logp"], batch.old_logp.cpu().numpy(), None, eps=0.2) | \
+        gc.near_clip_bound(r["logp"], batch.old_logp.cpu().numpy(), None, eps=0.3)
+    ulps = gc.grad_ulps(gc.grad_to_f64(out["grad_logits"])[~guard], r["grad"][~guard], ora["ids"][~guard], r["coef"][~guard])
+    assert ulps.max() <= gc.GRAD_ULPS

@@ -130,9 +130,13 @@ def _worker(rank, world, port, out):
                                       n_global=n_all, **common)
         assert o["grad_W"] is gw2 and o["n_global"] is n_all
         loss2 += o["loss"]
+    # sequence-mean aggregation with an upper clip width of its own: the exchanged count is of responses
+    sm = sharded.sharded_grpo_step(*args, old_logp=torch.from_numpy(t["old"]), ref_logp=torch.from_numpy(t["ref"]),
+                                   logits=P["logits"][rows], aggregation=1, eps_clip_high=0.3, **common)
     out.put((rank, t["rows"], a["n_local"].item(), a["n_global"].item(), a["loss"].numpy(), a["grad_logits"].numpy(),
              a["logp"].numpy(), b["loss"].numpy(), b["grad_hidden"].numpy(), b["grad_W"].numpy(), gw.numpy(),
-             gw2.numpy(), loss2.numpy()))
+             gw2.numpy(), loss2.numpy(), sm["loss"].numpy(), sm["grad_logits"].numpy(), sm["n_local"].item(),
+             sm["n_global"].item()))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -160,6 +164,8 @@ def test_two_ranks_add_up_to_the_unsharded_step():
     kw = dict(old_logp=torch.from_numpy(P["old"]), ref_logp=torch.from_numpy(P["ref"]))
     A = sharded.sharded_grpo_step(*args, logits=P["logits"], **kw, **common)
     Bf = sharded.sharded_grpo_step(*args, hidden=P["H"], W=P["W"], **kw, **common)
+    S = sharded.sharded_grpo_step(*args, logits=P["logits"], aggregation=1, eps_clip_high=0.3, **kw, **common)
+    assert S["n_global"].item() == 8 and not np.allclose(S["loss"].numpy(), A["loss"].numpy())
     n = A["n_global"].item()
     assert got[0][2] + got[1][2] == n and got[0][3] == got[1][3] == n and 0 < got[0][2] < n
     for g in got:
@@ -173,4 +179,7 @@ def test_two_ranks_add_up_to_the_unsharded_step():
         assert np.allclose(g[10], Bf["grad_W"].numpy(), rtol=1e-10, atol=1e-15)        # accumulated, reduced once
         assert np.allclose(g[11], Bf["grad_W"].numpy(), rtol=1e-10, atol=1e-15)        # ... by the step's own flags
         assert np.allclose(g[12], Bf["loss"].numpy(), rtol=1e-12, atol=1e-15)          # micro-batch losses add up
+        assert np.allclose(g[13], S["loss"].numpy(), rtol=1e-12, atol=1e-15)           # sequence mean: global loss
+        assert np.allclose(g[14], S["grad_logits"].numpy()[rows], rtol=1e-12, atol=1e-18)
+        assert g[15] == 4 and g[16] == 8                                              # responses: mine, everyone's
     assert sorted(np.concatenate([got[0][1], got[1][1]]).tolist()) == list(range(len(P["ids"])))
