@@ -56,7 +56,7 @@ typedef enum {
     RLF_ERR_WORKSPACE = -5, /* workspace NULL, misaligned or smaller than rlf_workspace_bytes() */
     RLF_ERR_ARCH = -6,      /* current device is not sm_100 */
     RLF_ERR_CUDA = -7,      /* a CUDA runtime call failed (launch, memset, copy) */
-    RLF_ERR_UNSUPPORTED = -8, /* valid request outside what this build implements */
+    RLF_ERR_UNSUPPORTED = -8, /* valid request outside what this library implements */
     RLF_ERR_TOO_LARGE = -9   /* more tokens than the built-in scratch of a *_static entry point holds */
 } rlf_status;
 

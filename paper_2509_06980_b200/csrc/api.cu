@@ -73,7 +73,7 @@ extern "C" const char* rlf_status_string(rlf_status s) {
         case RLF_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case RLF_ERR_ARCH: return "device is not sm_100";
         case RLF_ERR_CUDA: return "CUDA runtime error";
-        case RLF_ERR_UNSUPPORTED: return "request outside what this build implements";
+        case RLF_ERR_UNSUPPORTED: return "request outside what this library implements";
         case RLF_ERR_TOO_LARGE: return "more tokens than the built-in scratch holds (RLF_STATIC_MAX_TOKENS)";
     }
     return "unknown status";
