@@ -319,17 +319,23 @@ rlf_status rlf_grpo_logp_loss_fwd_bwd_static(const void *logits, rlf_dtype dt, i
  *   grad_hidden [T, D] bf16 or NULL;  grad_W [V, D] fp32 or NULL (both NULL: forward only)
  *   workspace   rlf_workspace_bytes(RLF_FN_FUSED_LMHEAD, T, V, D, RLF_BF16) bytes, 256-byte aligned.
  *               It holds per-token records and partial sums and, for the backward, a copy of hidden
- *               with the unmasked rows gathered first, and one chunk of min(T, 9472) rows by V
- *               (rounded up to whole 256-column tiles) of bf16, stored in blocks of 128 rows x 64
- *               columns (2.9 GB at V = 151936): the forward sweep of a chunk of unmasked rows leaves
- *               exp(z - max of the 256-column tile) there (never above 1, so no logit overflows
- *               it), an elementwise pass rescales it in place into dZ = grad_z once the row's
- *               log-sum-exp is known, and the two gradient contractions consume it.  The logits
- *               themselves are never stored.
- * Tensor-core contractions are bf16 x bf16 with fp32 accumulation in tensor memory; grad_z is
- * rounded to bf16 (twice: the stored exponential, then its product with the row's scale) before
- * the two gradient contractions.  Waits inside the kernels are bounded: if
- * one runs out, RLF_DEV_TIMEOUT is set in *dev_status and the outputs are not valid.
+ *               with the unmasked rows gathered first, one chunk of those rows times their row
+ *               factors, and one chunk of min(T, 18944) rows by V (rounded up to whole 256-column
+ *               tiles) of bf16, stored in blocks of 128 rows x 64 columns (5.8 GB at V = 151936,
+ *               T >= 18944): the forward sweep of a chunk of unmasked rows leaves exp(z - rho_t)
+ *               there, rho_t a per-row reference fixed before the sweep (the row's fp32 target logit
+ *               plus 32: bf16 has fp32's exponent range, so the entries that matter stay normal
+ *               numbers), and the two gradient contractions consume it with the per-row factor
+ *               c_t exp(rho_t - lse_t) applied in fp32 (grad_hidden) or to the hidden rows (grad_W).
+ *               A chunk with a row whose reference proves unusable (target log-prob below about -78)
+ *               is redone on the device with exponentials against per-tile maxima and one rescaling
+ *               pass over the scratch.  The logits themselves are never stored.
+ * Tensor-core contractions are bf16 x bf16 with fp32 accumulation in tensor memory; the stored
+ * exponentials are rounded to bf16 once, the scaled hidden rows of grad_W once more.  The contraction
+ * launches are persistent kernels of one CTA per SM whose workers meet on a counter in the workspace
+ * (see rlf_tune_lmhead_pacing); they are fastest with the GPU to themselves.  Waits inside the kernels
+ * are bounded: if one of the data waits runs out, RLF_DEV_TIMEOUT is set in *dev_status and the
+ * outputs are not valid.
  */
 rlf_status rlf_fused_lmhead_grpo(const void *hidden, const void *W, int64_t T, int32_t D, int32_t V,
                                  const int32_t *ids, const int32_t *seq_id, const float *adv,

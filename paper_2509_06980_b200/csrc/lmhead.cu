@@ -4,21 +4,26 @@
 //
 // One warp-specialised kernel template serves three contractions (all bf16 x bf16 -> fp32):
 //   LSE   z tile = H W^T, epilogue keeps a running (max, sum exp) per token      -> log-sum-exp;
-//         for rows that take part in the backward it also stores e = exp(z - tile max) as bf16
-//   GH    grad_hidden = dZ W      (A = dZ K-major, B = W vocabulary-major rows: N-major operand)
-//   GW    grad_W     += dZ^T H    (both operands token-major rows: M-/N-major operands)
+//         for rows that take part in the backward it also stores e = exp(z - rho_t) as bf16, rho_t a
+//         per-row reference known before the sweep (or exp(z - tile max) on the fallback path)
+//   GH    grad_hidden = f_t (e W)      (A = e K-major, B = W vocabulary-major rows: N-major operand;
+//                                       f_t = c_t exp(rho_t - lse_t) applied in the epilogue)
+//   GW    grad_W     += e^T (f_t H)    (both operands token-major rows: M-/N-major operands)
 // CTA = 192 threads: warp 0 issues TMA loads into a multi-stage ring, warp 1 issues the MMAs (one
-// thread) into a double-buffered 128 x 256 fp32 accumulator (all 512 TMEM columns),
-// warps 2..5 drain the accumulator with tcgen05.ld (one token row per thread) while the next tile
-// is being multiplied.  Every mbarrier wait is bounded; a wait that runs out raises a CTA-wide
-// abort flag, all roles leave their loops, tensor memory is released and RLF_DEV_TIMEOUT is set.
+// thread), warps 2..5 drain the accumulator with tcgen05.ld (one token row per thread).  The sweeps
+// use a double-buffered 128 x 256 fp32 accumulator (all 512 TMEM columns), so the drain of a tile
+// overlaps the multiplies of the next; the gradient contractions use both halves as two
+// accumulators that share every B slab.  Every mbarrier wait is bounded; a wait that runs out raises
+// a CTA-wide abort flag, all roles leave their loops, tensor memory is released and RLF_DEV_TIMEOUT
+// is set.  The persistent workers of a launch meet on a global counter before each of their units
+// (pacing), which keeps the operand slabs they share in L2.
 //
 // Forward + backward: the tokens are partitioned into unmasked rows and the others (only the first
 // carry gradient).  Unmasked rows go by chunks: LSE with the exponentials stored in a [chunk, V] bf16
-// scratch, an elementwise pass that rescales them in place into dZ = c_t (softmax - onehot) once the
-// row's log-sum-exp is known, then GH and GW read the scratch: three contractions per unmasked
-// row, one per masked row, no recomputation.  The logits themselves are never stored; the bf16
-// scratch is (stated in the entry point's contract).
+// scratch, per-row factors once the rows' log-sum-exp is known, then GH and GW read the scratch:
+// three contractions per unmasked row, one per masked row, no recomputation and no pass over the
+// scratch in between.  The logits themselves are never stored; the bf16 scratch is (stated in the
+// entry point's contract).
 #include <cuda.h>
 
 #include <atomic>
