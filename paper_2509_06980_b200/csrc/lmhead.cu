@@ -41,6 +41,7 @@ constexpr int BM = 128, BN = 256, BK = 64;
 // each CTA's tensor memory receives its own 128 rows of the accumulator.  Per flop the pair form
 // moves two thirds of the shared-memory bytes of the single form.
 constexpr int kABytes = BM * BK * 2;
+constexpr int kDrainPitch = 36;              // floats per row of a drain staging tile (32 + 4 of padding)
 // Two-accumulator pair form (ACC2, the two gradient contractions): a pair works on TWO 256-row tiles
 // against the same 256 columns, each CTA staging two A tiles beside its half of B (48 KB per stage, 4
 // stages), so every B slab that crosses L2 -> shared memory is used for 512 rows: three quarters of
@@ -55,7 +56,9 @@ template <bool PAIR, bool ACC2 = false> struct Cfg {
     static constexpr int kBRows = PAIR ? BN / 2 : BN;
     static constexpr int kBBytes = kBRows * BK * 2;
     static constexpr int kStageBytes = kAcc * kABytes + kBBytes;
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+    // + alignment slack, the barriers, and (two-accumulator form) a 32 x 32 fp32 staging tile per drain warp
+    static constexpr int kDrainBytes = ACC2 ? 4 * 32 * kDrainPitch * 4 : 0;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256 + kDrainBytes;
 };
 constexpr int kMaxStages = 6;
 constexpr int kThreads = 192;
@@ -255,6 +258,8 @@ struct SmemCtl {
     volatile int abort_flag;
 };
 
+static_assert(sizeof(SmemCtl) <= 256, "the barriers share a 256-byte slot behind the stage ring");
+
 // ---- the kernel -----------------------------------------------------------------------------
 template <bool PAIR, bool ACC2>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -270,6 +275,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const uint32_t raw = smem_addr(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     SmemCtl* ctl = reinterpret_cast<SmemCtl*>(smem_raw + (tiles - raw) + C::kStages * C::kStageBytes);
+    float* drain_stage = reinterpret_cast<float*>(smem_raw + (tiles - raw) + C::kStages * C::kStageBytes + 256);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool a_mn = p.mode == kGradW;
@@ -675,6 +681,37 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                                     if (i < nvalid) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]) * sc);
                             }
                         }
+                    } else if (ACC2 && nvalid == 32) {   // kGradW, two-accumulator form: the drain is not hidden
+                        // One accumulator row per thread means a warp's store touches 32 rows for 16 bytes
+                        // each.  The 32 x 32 chunk goes through a padded staging tile in shared memory
+                        // instead (rows of 144 bytes: conflict-free both ways), and comes back with eight
+                        // lanes along each row, so that a warp's store covers 4 rows x 128 contiguous bytes.
+                        float* stg = drain_stage + (warp - 2) * (32 * kDrainPitch);
+                        float4* w4 = reinterpret_cast<float4*>(stg + lane * kDrainPitch);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            w4[i] = make_float4(__uint_as_float(v[4 * i]), __uint_as_float(v[4 * i + 1]),
+                                                __uint_as_float(v[4 * i + 2]), __uint_as_float(v[4 * i + 3]));
+                        __syncwarp();
+                        const int piece = lane & 7, rq = lane >> 3;
+                        const int row_w0 = row_a - lane;                 // first row of this warp's 32
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const int r = rq + 4 * j;
+                            const float4 val = *reinterpret_cast<const float4*>(stg + r * kDrainPitch + piece * 4);
+                            if (row_w0 + r < M) {
+                                float4* d4 = reinterpret_cast<float4*>(p.out_f32 + (long long)(row_w0 + r) * p.out_stride + cb) + piece;
+                                // accumulation is a fire-and-forget vector reduction at the memory side (no
+                                // read round trip in the drain); each element gets exactly one addend per
+                                // launch, so the result does not depend on timing
+                                if (p.accumulate)
+                                    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
+                                                 :: "l"(d4), "f"(val.x), "f"(val.y), "f"(val.z), "f"(val.w) : "memory");
+                                else
+                                    *d4 = val;
+                            }
+                        }
+                        __syncwarp();                                    // the tile is free for the next chunk
                     } else {   // kGradW
                         if (row_ok_a) {
                             float* dst = p.out_f32 + (long long)row_a * p.out_stride + cb;
@@ -682,9 +719,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                                 float4* d4 = reinterpret_cast<float4*>(dst);
 #pragma unroll
                                 for (int i = 0; i < 8; ++i) {
-                                    // accumulation is a fire-and-forget vector reduction at the memory side (no
-                                    // read round trip in the drain); each element gets exactly one addend per
-                                    // launch, so the result does not depend on timing
                                     if (p.accumulate)
                                         asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
                                                      :: "l"(d4 + i), "r"(v[4 * i]), "r"(v[4 * i + 1]), "r"(v[4 * i + 2]),
