@@ -45,8 +45,8 @@ WORKLOAD = "cfg1_qwen3_4b_microbatch: 16 responses x 2048 tokens, V=151936 bf16 
 #   fused LM-head: every kernel of one forward / one forward + backward call at cfg 3 full size
 #   (one-pass capture of the whole call), per call.
 NCU_TRAFFIC = {"logits_loss_cu_sha1": "1adb1f55fa740cb18b27b090cc83c69d1d742942", "dram_bytes_per_token": 606039.0}
-NCU_TRAFFIC_FUSED = {"lmhead_cu_sha1": "6d2facbf9dbd0b6278fe8a2b382ec7645c6a84ea",
-                     "fwd_bytes_per_call": 3963365888.0, "fwd_bwd_bytes_per_call": 33498145024.0}
+NCU_TRAFFIC_FUSED = {"lmhead_cu_sha1": "23538aaabeed8d9a0c763b7f7e3bb6ee625b306d",
+                     "fwd_bytes_per_call": 3957591808.0, "fwd_bwd_bytes_per_call": 34875904256.0}
 
 
 def _peaks():
