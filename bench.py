@@ -285,6 +285,17 @@ class ClockSampler:
         return out
 
 
+def workload_config(world, tokens_per_response=0):
+    """The `config` object of the JSON line: the workload alone (the same for the CUDA arm and for the
+    oracle arm, which runs bounded samples of it), nothing about how an arm computes."""
+    spec = synth.SPECS[1]
+    tok = tokens_per_response or spec.len_hi
+    B = spec.num_prompts * spec.group_size
+    return {"workload": WORKLOAD if not tokens_per_response else "cfg1 recipe at %d tokens per response" % tokens_per_response,
+            "T": B * tok, "V": spec.V, "B": B, "G": spec.group_size, "eps_clip": synth.EPS_CLIP, "beta_kl": synth.BETA_KL,
+            "parallelism": "independent micro-batch per GPU" if world > 1 else "single GPU"}
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -379,8 +390,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * el / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD,
-                   "step": "fp64 CPU oracle on %d rows per step (bounded sample of the workload)" % rows},
+        "config": workload_config(max(1, args.gpus)),
+        "step": "fp64 CPU oracle on %d rows per step (bounded sample of the workload)" % rows,
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": "%d rows per step x %d steps, full vocabulary, forward + fp64 gradient"
                                    % (rows, args.steps)},
@@ -861,13 +872,10 @@ def run_cuda(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": ms_total_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": WORKLOAD if not args.tokens_per_response
-                   else "cfg1 recipe at %d tokens per response" % args.tokens_per_response,
-                   "T": T, "V": V, "B": B, "G": G, "eps_clip": synth.EPS_CLIP, "beta_kl": synth.BETA_KL,
-                   "arithmetic": "bf16 in/out, fp32 accumulate, fp64 loss sum",
-                   "l2": "inputs (%.1f GB per step) exceed L2; no flush needed" % (T * V * 2 / 1e9),
-                   "grad": "out of place",
-                   "parallelism": "independent micro-batch per GPU" if world > 1 else "single GPU"},
+        "config": workload_config(world, args.tokens_per_response),
+        "arithmetic": "bf16 in/out, fp32 accumulate, fp64 loss sum",
+        "l2": "inputs (%.1f GB per step) exceed L2; no flush needed" % (T * V * 2 / 1e9),
+        "grad": "out of place",
         "logits_gbs": achieved,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": "of " + peak_kind, "frac_of_nominal_8tbs": achieved / 8000.0, "traffic": traffic,
