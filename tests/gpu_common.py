@@ -45,28 +45,57 @@ def oracle_chain(batch, logits_np=None, want_grad=True, rows=None):
     return out
 
 
-def oracle_all_rows_through_fp64_head(hidden, W, ora, old, ref, row_chunk=2048):
+def oracle_all_rows_through_fp64_head(hidden, W, ora, old, ref, row_chunk=2048, want_coef=False):
     """Every row's log-prob and the scalar loss of the fused path from the oracle at full size.
     The head contraction z = H W^T is the one library step: torch.matmul in fp64 on the GPU (bf16
     inputs widened exactly), a chunk of rows at a time; each chunk's fp64 logits go to the host and
     through orc_grpo_loss (dtype f64) with the batch's token count as denominator, so the chunks'
     loss terms add up to the batch's.  Nothing of the library under test is involved.
-    -> (logp f64[T], loss f64[4])"""
+    -> (logp f64[T], loss f64[4]); with want_coef also the oracle's gradient coefficient c_t of every
+    row (grad_z[t, v] = c_t (p[t, v] - [v = y_t]))."""
     T = hidden.shape[0]
     W64 = W.double()
     logp = np.empty(T, np.float64)
+    coef = np.empty(T, np.float64)
     loss = np.zeros(4, np.float64)
     for r0 in range(0, T, row_chunk):
         sl = slice(r0, min(T, r0 + row_chunk))
         z = torch.matmul(hidden[sl].double(), W64.t()).cpu().numpy()
         r = orc.grpo_loss(z, ora["ids"][sl], ora["seq_id"][sl], ora["adv"], old[sl], ref[sl], ora["mask"][sl],
-                          synth.EPS_CLIP, synth.BETA_KL, denom=ora["n"], want_grad=False)
+                          synth.EPS_CLIP, synth.BETA_KL, denom=ora["n"], want_grad=False, want_coef=want_coef)
         logp[sl] = r["logp"]
+        if want_coef:
+            coef[sl] = r["coef"]
         loss += np.asarray(r["loss"], np.float64)
         del z
     del W64
     torch.cuda.empty_cache()
-    return logp, loss
+    return (logp, loss, coef) if want_coef else (logp, loss)
+
+
+def oracle_grad_W_rows(hidden, W, ids, logp_o, coef_o, vocab_rows, row_chunk=8192):
+    """Rows `vocab_rows` of grad_W at full size from the oracle's per-row outputs and the definition
+    grad_W[v, :] = sum_t c_t (p[t, v] - [v = y_t]) hidden[t, :], p[t, v] = exp(z[t, v] - lse_t), with
+    lse_t = z[t, y_t] - logp_t.  c_t and logp_t are the oracle's (fp64 logits route); the contractions
+    with hidden / W are the library's fp64 matmul on the GPU, a chunk of tokens at a time.
+    -> f64 [len(vocab_rows), D]"""
+    dev = hidden.device
+    vs = torch.as_tensor(np.asarray(vocab_rows), device=dev, dtype=torch.long)
+    Wv = W[vs].double()
+    T, D = hidden.shape
+    out = torch.zeros((len(vocab_rows), D), dtype=torch.float64, device=dev)
+    lp = torch.from_numpy(np.asarray(logp_o)).to(dev)
+    cf = torch.from_numpy(np.asarray(coef_o)).to(dev)
+    y = ids.to(device=dev, dtype=torch.long)
+    for r0 in range(0, T, row_chunk):
+        sl = slice(r0, min(T, r0 + row_chunk))
+        H = hidden[sl].double()
+        zy = (H * W[y[sl]].double()).sum(dim=1)
+        lse = zy - lp[sl]
+        p = torch.exp(H @ Wv.t() - lse[:, None])                   # [rows, len(vs)]
+        dz = cf[sl, None] * (p - (y[sl, None] == vs[None, :]).double())
+        out += dz.t() @ H
+    return out.cpu().numpy()
 
 
 def loss_floor(ora):

@@ -64,9 +64,14 @@ def test_cfg4_full_size_micro_batched():
 
     # every row of all eight micro-batches: log-prob and the summed scalar loss against the oracle
     # (fp64 logits from the library's fp64 contraction, then the oracle's loss)
-    logp_o, loss_o = gc.oracle_all_rows_through_fp64_head(batch.hidden, batch.W, ora, batch.old_logp.cpu().numpy(),
-                                                          batch.ref_logp.cpu().numpy(), row_chunk=2048)
+    logp_o, loss_o, coef_o = gc.oracle_all_rows_through_fp64_head(batch.hidden, batch.W, ora, batch.old_logp.cpu().numpy(),
+                                                                  batch.ref_logp.cpu().numpy(), row_chunk=2048,
+                                                                  want_coef=True)
     assert np.abs(logp.cpu().numpy() - logp_o).max() <= gc.LOGP_ATOL
+    # rows of the accumulated grad_W (a sum over all eight micro-batches) against the oracle's per-row outputs
+    vs = np.unique(np.concatenate([ora["ids"][live][:12], rng.integers(0, spec.V, size=12), [spec.V - 1]]))
+    gw_o = gc.oracle_grad_W_rows(batch.hidden, batch.W, batch.ids, logp_o, coef_o, vs)
+    _close_tensor(gw[torch.as_tensor(vs, device=DEV)].cpu().numpy(), gw_o, "grad_W rows")
     assert np.abs(logp_o[rows] - r["logp"]).max() <= 1e-9
     floor = gc.loss_floor(ora)
     ls = loss_sum.cpu().numpy()

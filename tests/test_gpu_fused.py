@@ -105,7 +105,7 @@ def test_cfg3_full_size_sampled_rows_and_invariants():
     """The launch configuration the benchmark times (T = 32768, D = 2560, V = 151936): log-probs and
     grad_hidden rows of sampled tokens against the oracle (a token's row depends only on that token
     and the batch's token count); every row's log-prob and the scalar loss against the oracle run on
-    fp64 logits of the whole batch; grad_W through the invariant that its columns sum to zero over the vocabulary."""
+    fp64 logits of the whole batch; sampled rows of grad_W rebuilt from the oracle's per-row outputs; grad_W also through the invariant that its columns sum to zero over the vocabulary."""
     b = gc.binding()
     spec = synth.SPECS[3]
     batch = synth.make_batch(spec, DEV)
@@ -137,9 +137,15 @@ def test_cfg3_full_size_sampled_rows_and_invariants():
 
     # every row's log-prob and the scalar loss against the oracle (fp64 logits from the library's
     # fp64 contraction, then the oracle's loss over all 32768 rows)
-    logp_o, loss_o = gc.oracle_all_rows_through_fp64_head(batch.hidden, batch.W, ora, batch.old_logp.cpu().numpy(),
-                                                          batch.ref_logp.cpu().numpy())
+    logp_o, loss_o, coef_o = gc.oracle_all_rows_through_fp64_head(batch.hidden, batch.W, ora, batch.old_logp.cpu().numpy(),
+                                                                  batch.ref_logp.cpu().numpy(), want_coef=True)
     assert np.abs(logp.cpu().numpy() - logp_o).max() <= gc.LOGP_ATOL
+    # rows of grad_W at full size: 16 vocabulary rows that are targets of unmasked tokens (their one-hot term
+    # matters), 16 random ones and the last row of the ragged last column tile
+    vs = np.unique(np.concatenate([ora["ids"][live][:16], rng.integers(0, spec.V, size=16), [spec.V - 1]]))
+    gw_o = gc.oracle_grad_W_rows(batch.hidden, batch.W, batch.ids, logp_o, coef_o, vs)
+    _close_tensor(gw[torch.as_tensor(vs, device=DEV)].cpu().numpy(), gw_o, "grad_W rows")
+    assert np.abs(gw_o).max() >= 0.05 * gw.abs().max().item()      # the sample reaches the tensor's scale
     assert np.abs(logp_o[rows] - r["logp"]).max() <= 1e-9      # the two oracle routes agree on the sampled rows
     lg = loss.cpu().numpy()
     floor = gc.loss_floor(ora)
