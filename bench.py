@@ -44,7 +44,7 @@ WORKLOAD = "cfg1_qwen3_4b_microbatch: 16 responses x 2048 tokens, V=151936 bf16 
 #   streaming forward kernel: the T = 4096 capture, per token (traffic is proportional to rows);
 #   fused LM-head: every kernel of one forward / one forward + backward call at cfg 3 full size
 #   (one-pass capture of the whole call), per call.
-NCU_TRAFFIC = {"logits_loss_cu_sha1": "1adb1f55fa740cb18b27b090cc83c69d1d742942", "dram_bytes_per_token": 606039.0}
+NCU_TRAFFIC = {"logits_loss_cu_sha1": "a4cf4f58a06c399db0363ce500787d9885a2893e", "dram_bytes_per_token": 606051.0}
 NCU_TRAFFIC_FUSED = {"lmhead_cu_sha1": "23538aaabeed8d9a0c763b7f7e3bb6ee625b306d",
                      "fwd_bytes_per_call": 3957591808.0, "fwd_bwd_bytes_per_call": 34875904256.0}
 

@@ -309,6 +309,8 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t mbar, uint32_t parity
     return false;
 }
 
+__device__ __forceinline__ int ring_read(const int* ring, int slot) { return reinterpret_cast<const volatile int*>(ring)[slot]; }
+
 // SKIP: the rows to process come from a compacted list (rows whose loss weight is zero are
 // neither read nor computed); token records are then indexed like the list.
 // WT: per-token loss weights from the caller replace the common 1 / N.
@@ -403,7 +405,11 @@ grpo_row_cluster_kernel(const FastParams p) {
     bool gave_up = false;                // a wait ran out: stop waiting, finish the loop, report
     for (int k = cluster_id; k < nrows; k += num_clusters, ++it) {
         const int parity = it & 1;
-        const int row = SKIP ? row_slot[it & RM] : k;
+        // the listed row's index is re-read from its ring slot where it is used (late in the iteration)
+        // instead of being held in a register across the passes: the skip variant is at its register
+        // budget, and a spill in this loop costs more than a few shared-memory reads
+        const int row = SKIP ? 0 : k;
+#define RLF_CUR_ROW() (SKIP ? ring_read(row_slot, it & RM) : row)
         const uint32_t bar = smem_u32(&row_bar[parity]);
         cp_async_wait_all();             // this thread's part of the row (and thread 0's metadata) has landed
         // an arrive releases what this thread did before it: the landed metadata becomes visible to
@@ -505,14 +511,14 @@ grpo_row_cluster_kernel(const FastParams p) {
         if (crank == 0 && tid == 0) {
             // forward-only variant: a row whose target id was out of range has no log-prob
             const bool has_logp = finite && (!ENT || __float_as_int(rec.w) < 0);
-            p.logp_out[row] = has_logp ? logp : __int_as_float(0x7fc00000);
+            p.logp_out[RLF_CUR_ROW()] = has_logp ? logp : __int_as_float(0x7fc00000);
             if (!finite) status |= RLF_DEV_NONFINITE;
             // H = ln S - ln2 * U / S  (= lse - E[z])
-            if (ENT && p.entropy_out) p.entropy_out[row] = finite ? (lg2s - U / S) * kLn2 : __int_as_float(0x7fc00000);
+            if (ENT && p.entropy_out) p.entropy_out[RLF_CUR_ROW()] = finite ? (lg2s - U / S) * kLn2 : __int_as_float(0x7fc00000);
         }
 
         if (!ENT && p.grad != nullptr) {
-            uint4* dst = reinterpret_cast<uint4*>(p.grad + (long long)row * p.stride) + vbeg;
+            uint4* dst = reinterpret_cast<uint4*>(p.grad + (long long)RLF_CUR_ROW() * p.stride) + vbeg;
             if (coef == 0.0f || !(fabsf(coef) < INFINITY)) {
                 const uint4 z4 = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
@@ -550,7 +556,7 @@ grpo_row_cluster_kernel(const FastParams p) {
                     }
                 }
                 // the owner overwrites the target column of the vector it has just stored
-                if (owner) p.grad[(long long)row * p.stride + y] = __float2bfloat16_rn(gy);
+                if (owner) p.grad[(long long)RLF_CUR_ROW() * p.stride + y] = __float2bfloat16_rn(gy);
             }
         }
     }
@@ -566,6 +572,8 @@ grpo_row_cluster_kernel(const FastParams p) {
 }
 
 // ---------------------------------------------------------------------------------------------
+#undef RLF_CUR_ROW
+
 // General row kernel: one CTA per row, scalar loads, any dtype / V / alignment.
 template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
