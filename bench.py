@@ -44,7 +44,7 @@ WORKLOAD = "cfg1_qwen3_4b_microbatch: 16 responses x 2048 tokens, V=151936 bf16 
 #   streaming forward kernel: the T = 4096 capture, per token (traffic is proportional to rows);
 #   fused LM-head: every kernel of one forward / one forward + backward call at cfg 3 full size
 #   (one-pass capture of the whole call), per call.
-NCU_TRAFFIC = {"logits_loss_cu_sha1": "a4cf4f58a06c399db0363ce500787d9885a2893e", "dram_bytes_per_token": 606051.0}
+NCU_TRAFFIC = {"logits_loss_cu_sha1": "373f8ff1bad542ed4ac3604f9ea1c3888ac745a5", "dram_bytes_per_token": 606041.0}
 NCU_TRAFFIC_FUSED = {"lmhead_cu_sha1": "23538aaabeed8d9a0c763b7f7e3bb6ee625b306d",
                      "fwd_bytes_per_call": 3957591808.0, "fwd_bwd_bytes_per_call": 34875904256.0}
 
@@ -196,7 +196,7 @@ def time_fused_lmhead(rlf, dev, steps, tokens_per_response=0, cfg=3, responses=0
 
 
 # the same for the forward-only log-prob + entropy pass (profiles/logp_entropy_stream_kernel_T4096_ncu_full.md)
-NCU_TRAFFIC_ENTROPY = {"section_sha1": "2ebec178e05253433bddc7e3733a94e8c4a2063e", "dram_bytes_per_token": 305838.0}
+NCU_TRAFFIC_ENTROPY = {"section_sha1": "cbd417db69ba91bea4be00d3c9c3cda5dee7abb9", "dram_bytes_per_token": 305813.0}
 
 
 def _entropy_section_sha1():
@@ -540,6 +540,39 @@ def run_other_configs(args):
     out["cfg0_tiny_step_latency"] = {"T": b0.T, "V": spec0.V, "launches_per_step": 6, "eager_us": eager_us,
                                      "cuda_graph_us": per_step_us(graph.replay)}
     del b0, o, graph
+
+    # the logits path at other vocabulary sizes (not stated configurations; about 4 GB of bf16 logits each,
+    # out of place, so 8 GB moved per call), as a fraction of the measured copy rate
+    peak_gbs, peak_kind = _peaks()
+    vocab = {}
+    g = torch.Generator(device=dev)
+    g.manual_seed(0)
+    for V_other in (32000, 50304, 128256, 200000, 262144):
+        Tv = int(4e9 // (2 * V_other)) // 16 * 16
+        z = torch.empty((Tv, V_other), dtype=torch.bfloat16, device=dev).normal_(0, 3, generator=g)
+        gz = torch.empty_like(z)
+        ids_v = torch.randint(0, V_other, (Tv,), device=dev, generator=g).to(torch.int32)
+        seq_v = (torch.arange(Tv, device=dev) * 16 // Tv).to(torch.int32)
+        adv_v = torch.randn(16, device=dev, generator=g)
+        mask_v = (torch.rand(Tv, device=dev, generator=g) < 0.55).to(torch.uint8)
+        old_v = torch.full((Tv,), -12.0, device=dev)
+        n_v = mask_v.sum().to(torch.int64).reshape(1)
+        ws_v = rlf.new_workspace(rlf.FN_LOGP_LOSS, Tv, V_other)
+        wse_v = rlf.new_workspace(rlf.FN_LOGP_ENTROPY, Tv, V_other)
+        lp_v = torch.empty(Tv, dtype=torch.float32, device=dev)
+        ent_v = torch.empty(Tv, dtype=torch.float32, device=dev)
+        ls_v = torch.empty(4, dtype=torch.float64, device=dev)
+        ms_t = timed(lambda: rlf.rlf_grpo_logp_loss_fwd_bwd(z, ids_v, seq_v, adv_v, old_v, old_v, mask_v, synth.EPS_CLIP,
+                                                            synth.BETA_KL, denom=n_v, grad_logits=gz, logp_out=lp_v,
+                                                            loss_out=ls_v, workspace=ws_v), 4 * steps)
+        ms_f = timed(lambda: rlf.rlf_logp_entropy_fwd(z, ids_v, logp_out=lp_v, entropy_out=ent_v, workspace=wse_v), 4 * steps)
+        gbs_t = Tv * V_other * 4 / ms_t / 1e6
+        gbs_f = Tv * V_other * 2 / ms_f / 1e6
+        vocab[str(V_other)] = {"T": Tv, "fwd_bwd_ms": ms_t, "fwd_bwd_gbs": gbs_t, "fwd_bwd_frac": gbs_t / peak_gbs,
+                               "logp_entropy_ms": ms_f, "logp_entropy_gbs": gbs_f, "logp_entropy_frac": gbs_f / peak_gbs}
+        del z, gz, ws_v, wse_v
+        torch.cuda.empty_cache()
+    out["logits_path_other_vocabularies"] = {"peak_gbs": peak_gbs, "peak_kind": "of " + peak_kind, "by_V": vocab}
 
     # cfg 2: in place over the whole packed batch (the gradient overwrites the logits, so every timed
     # call sees the previous call's output as its logits: same bytes moved, values irrelevant to time)

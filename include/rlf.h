@@ -412,8 +412,9 @@ rlf_status rlf_grpo_step_host(const void *h_logits, rlf_dtype dt, int64_t T, int
                               void *d_arena, size_t arena_bytes, rlf_stream_t stream);
 size_t rlf_step_arena_bytes(int64_t T, int32_t V, int32_t B, rlf_dtype dt);
 
-/* Launch shape of the fast logits kernel for later calls in this process: CTAs per cluster (1, 2,
- * 4 or 8), threads per CTA (256, 512 or 1024), and whether each element's exponential is taken once
+/* Launch shape of the fast logits kernel for later calls in this process: CTAs per cluster (1 to 16;
+ * above 8 only with 256 threads and one_exp, for the plain token-mean training call), threads per CTA
+ * (256, 512 or 1024), and whether each element's exponential is taken once
  * and kept as bf16 (one_exp = 1) or taken twice in fp32 (one_exp = 0; -1 = built-in choice).
  * cluster_ctas = 0 restores the built-in shape.  A shape that cannot hold a row in registers makes
  * rlf_grpo_logp_loss_fwd_bwd return RLF_ERR_UNSUPPORTED.  Results do not depend on the shape

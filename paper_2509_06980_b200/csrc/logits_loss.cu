@@ -26,6 +26,10 @@
 //   4. every warp merges all pairs of the row (lanes in parallel), forms lse, logp and the loss
 //      coefficient c_t, and writes grad = c_t (softmax - onehot) from the registers it still
 //      holds, either as exp2(z log2e + log2|c_t| - lse log2e) (two-exp) or as e * 2^(...) (one-exp).
+// In the training variants the target column stays out of the warps' (max, sum): its owner replaces
+// it by -inf in its staging slot before loading its registers, and every warp folds z_target back in
+// after the merge.  The sum over the other columns, S', gives the target's gradient as -c S' / S, which
+// keeps its digits when p_y rounds to one (c p_y - c does not).
 // Exponents are formed by one FFMA per element; rows whose maximum is huge in magnitude switch to
 // a subtract-first form so that the result stays accurate for any finite logits.
 // Token records ride the same cp.async groups two rows ahead, so no scalar input costs a register
@@ -415,6 +419,23 @@ grpo_row_cluster_kernel(const FastParams p) {
         // an arrive releases what this thread did before it: the landed metadata becomes visible to
         // every thread that later sees this barrier's phase complete
         if (tid == 0) mbar_arrive_expect_tx(bar, row_bytes);
+        // the owner of the target column sends z_target to every CTA of the cluster; the target id is
+        // re-read from its ring slot where the gradient needs it again, not held across the passes
+#define RLF_TARGET_ID() (ring_read(reinterpret_cast<const int*>(rec_slot), 4 * (it & RM) + 3) & 0x7fffffff)
+#define RLF_OWNS(yrel) ((yrel) >= 0 && ((yrel) & (THREADS - 1)) == 0 && ((yrel) / THREADS) < nvalid)
+        const int y = RLF_TARGET_ID();
+        const int yrel = (y >> 3) - vbeg;             // owner iff a multiple of THREADS below nvalid * THREADS
+        if (RLF_OWNS(yrel)) {
+            // the target logit sits in this thread's own staging slot
+            __nv_bfloat16* sv = reinterpret_cast<__nv_bfloat16*>(&stage[yrel + tid]);
+            const float zt = __bfloat162float(sv[y & 7]);
+            for (int r = 0; r < csize; ++r) st_async_f1(smem_u32(&zy_slot[parity]), bar, (uint32_t)r, zt);
+            // The training variants sum over the OTHER columns: the target becomes -inf in the slot
+            // before the registers are loaded, so it drops out of (max, sum) here and comes back in
+            // once per row from z_target.  S' = S - 2^(z_y - M) is what the target column's gradient
+            // needs, -c S' / S, and summing it directly avoids the cancellation of c (p_y - 1).
+            if (!ENT) sv[y & 7] = __ushort_as_bfloat16((unsigned short)0xff80u);
+        }
         uint4 d[NV];
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
@@ -422,21 +443,11 @@ grpo_row_cluster_kernel(const FastParams p) {
             else d[i] = make_uint4(kNegInfPair, kNegInfPair, kNegInfPair, kNegInfPair);
         }
 
-        // max over the registers (packed), then over the warp; the owner of the target column
-        // sends z_target to every CTA of the cluster
-        const int y = __float_as_int(rec_slot[it & RM].w) & 0x7fffffff;
-        const int yrel = (y >> 3) - vbeg;             // owner iff a multiple of THREADS below nvalid * THREADS
-        const bool owner = yrel >= 0 && (yrel & (THREADS - 1)) == 0 && (yrel / THREADS) < nvalid;
+        // max over the registers (packed), then over the warp
         uint32_t mx = kNegInfPair;
 #pragma unroll
         for (int i = 0; i < NV; ++i)
             mx = max_bf16x2(mx, max_bf16x2(max_bf16x2(d[i].x, d[i].y), max_bf16x2(d[i].z, d[i].w)));
-        if (owner) {
-            // the target logit still sits in this thread's staging slot
-            const __nv_bfloat16* sv = reinterpret_cast<const __nv_bfloat16*>(&stage[yrel + tid]);
-            const float zt = __bfloat162float(sv[y & 7]);
-            for (int r = 0; r < csize; ++r) st_async_f1(smem_u32(&zy_slot[parity]), bar, (uint32_t)r, zt);
-        }
         // the staging slots have been consumed (the max needed every register): refill them with
         // the cluster's next row while this one is processed
         {
@@ -482,6 +493,8 @@ grpo_row_cluster_kernel(const FastParams p) {
             M = fmaxf(M, e[j].x);
         }
         M = ord2f(__reduce_max_sync(0xffffffffu, f2ord(M)));
+        const float zy = zy_slot[parity];
+        if (!ENT) M = fmaxf(M, zy);                  // the pairs of the training variants leave the target out
         float S = 0.0f, U = 0.0f;
 #pragma unroll
         for (int j = 0; j < (MAXE + 31) / 32; ++j) {
@@ -499,8 +512,14 @@ grpo_row_cluster_kernel(const FastParams p) {
         }
         S = warp_sum(S);
         if (ENT) U = warp_sum(U);
-        const float zy = zy_slot[parity];
         const float4 rec = rec_slot[it & RM];
+        // the training variants summed without the target column: S' = S here, S = S' + 2^((z_y - M) log2e)
+        float others = 0.0f;                         // S' / S = 1 - p_y
+        if (!ENT) {
+            const float s_all = S + ex2_approx((zy - M) * kLog2e);
+            others = __fdividef(S, s_all);
+            S = s_all;
+        }
         const float lg2s = lg2_approx(S);
         const float logp = (zy - M) - lg2s * kLn2;
         const bool finite = (M > -INFINITY) && (M < INFINITY) && (S > 0.0f) && (S < INFINITY) &&
@@ -525,9 +544,9 @@ grpo_row_cluster_kernel(const FastParams p) {
                 for (int i = 0; i < NV; ++i)
                     if (i < nvalid) st_stream(dst + i * THREADS, z4);
             } else {
-                // grad = sign(c) 2^((z - M) log2e + lc), lc = log2|c| - log2 S; the target column gets -c on top
+                // grad = sign(c) 2^((z - M) log2e + lc), lc = log2|c| - log2 S; the target column is written apart
                 const float lc = lg2_approx(fabsf(coef)) - lg2s;
-                const float gy = fmaf(coef, ex2_approx(fmaf(zy - M, kLog2e, -lg2s)), -coef);   // c (p_y - 1)
+                const float gy = -coef * others;                                    // c (p_y - 1) = -c S' / S
                 if (ONE_EXP) {
                     // the registers hold 2^((z - m_w) log2e): rescale from the warp's base to the row's
                     const float scale = copysignf(ex2_approx(fmaf(m_ws - M, kLog2e, lc)), coef);
@@ -556,7 +575,8 @@ grpo_row_cluster_kernel(const FastParams p) {
                     }
                 }
                 // the owner overwrites the target column of the vector it has just stored
-                if (owner) p.grad[(long long)RLF_CUR_ROW() * p.stride + y] = __float2bfloat16_rn(gy);
+                const int yg = RLF_TARGET_ID();
+                if (RLF_OWNS((yg >> 3) - vbeg)) p.grad[(long long)RLF_CUR_ROW() * p.stride + yg] = __float2bfloat16_rn(gy);
             }
         }
     }
@@ -573,6 +593,8 @@ grpo_row_cluster_kernel(const FastParams p) {
 
 // ---------------------------------------------------------------------------------------------
 #undef RLF_CUR_ROW
+#undef RLF_TARGET_ID
+#undef RLF_OWNS
 
 // General row kernel: one CTA per row, scalar loads, any dtype / V / alignment.
 template <typename T> __device__ __forceinline__ float to_f32(T v);
@@ -631,9 +653,11 @@ grpo_row_general_kernel(const GenParams p) {
         const float M = bcast;
         const float Ms = (M == -INFINITY) ? 0.0f : M;
         float s = 0.0f, u = 0.0f;
+        // the sums leave the target column out; it comes back in once per row below.  S' = sum over the
+        // other columns gives the target's gradient as -c S' / S without the cancellation of c (p_y - 1)
         for (int v = tid; v < p.V; v += kGenThreads) {
             const float x = fmaxf((to_f32<T>(z[v]) - Ms) * kLog2e, -1e30f);
-            const float e = ex2_approx(x);
+            const float e = (v == y) ? 0.0f : ex2_approx(x);
             s += e;
             u = fmaf(e, x, u);                 // for the entropy: sum 2^x * x
         }
@@ -649,8 +673,11 @@ grpo_row_general_kernel(const GenParams p) {
             bcast_u = uu;
         }
         __syncthreads();
-        const float S = bcast;
-        const float U = bcast_u;
+        const float S_others = bcast;
+        const float x_y = fmaxf((zy - Ms) * kLog2e, -1e30f);
+        const float e_y = ex2_approx(x_y);
+        const float S = S_others + e_y;
+        const float U = fmaf(e_y, x_y, bcast_u);
         __syncthreads();
 
         const float lg2s = lg2_approx(S);
@@ -673,7 +700,7 @@ grpo_row_general_kernel(const GenParams p) {
             } else {
                 for (int v = tid; v < p.V; v += kGenThreads) {
                     const float pv = ex2_approx(fmaf(to_f32<T>(z[v]) - M, kLog2e, -lg2s));
-                    const float gv = (v == y) ? fmaf(coef, pv, -coef) : coef * pv;
+                    const float gv = (v == y) ? -coef * (S_others / S) : coef * pv;
                     g[v] = from_f32<T>(gv);
                 }
             }
@@ -767,14 +794,24 @@ static int round_nv(int need) {
     return 0;
 }
 
+// 16-byte vectors of a row per CTA of a cluster: an even split rounded up to whole 128-byte lines, so
+// that every CTA's piece of a (line-aligned) row starts on a line.  Pieces that start in the middle of
+// a 32-byte sector cost 10 - 20 % of the bandwidth (V = 200000 over 16 CTAs: 1563 vectors each).
+static int per_cta_vectors(int nvec, int cluster) {
+    return (((nvec + cluster - 1) / cluster) + 7) & ~7;
+}
+
 // launch shape that holds a row of nvec 16-byte vectors in registers
 static bool pick_shape(int nvec, FastShape* out, bool allow_wide_cluster = false) {
     const int tc = g_tune_cluster.load(), tt = g_tune_threads.load();
     const int oe = g_tune_one_exp.load() < 0 ? 1 : g_tune_one_exp.load();
     if (tc > 0 && tt > 0) {
-        const int per = (nvec + tc - 1) / tc;
-        const int nv = round_nv((per + tt - 1) / tt);
+        // clusters beyond the portable 8 exist for the plain training kernel with 256-thread CTAs only
+        if (tc > 8 && (!allow_wide_cluster || tt != 256 || !oe)) return false;
+        const int per = per_cta_vectors(nvec, tc);
+        int nv = round_nv((per + tt - 1) / tt);
         if (nv == 0) return false;
+        if (tc > 8 && nv < 6) nv = 6;                 // the smallest instantiation for those clusters
         *out = {tc, tt, nv, oe};
         return true;
     }
@@ -782,7 +819,7 @@ static bool pick_shape(int nvec, FastShape* out, bool allow_wide_cluster = false
     // the smallest cluster that covers the row; wider CTAs only for rows beyond 8 x 256 x 10 vectors
     for (int th = 256; th <= 1024; th *= 2) {
         for (int c = 1; c <= 8; c *= 2) {
-            const int per = (nvec + c - 1) / c;
+            const int per = per_cta_vectors(nvec, c);
             const int need = (per + th - 1) / th;
             if (need <= 10 && stage_bytes(th, round_nv(need)) <= kSmemBudget) {
                 *out = {c, th, round_nv(need), oe};
@@ -792,11 +829,15 @@ static bool pick_shape(int nvec, FastShape* out, bool allow_wide_cluster = false
         // rows beyond 8 x 256 x 10 vectors: a cluster of 16 such CTAs (four per SM, every register
         // holding a piece of a row) before CTAs of 512 threads (two per SM): V = 262144 ran at 0.80 of
         // the copy rate as 8 x 512 threads
+        // (10 CTAs where they hold the row, V <= 204800, else 16: V = 200000 runs at 6.09 TB/s over 10 CTAs
+        // with 10 vectors per thread, 5.51 over 16 with 7; between 10 and 16 nothing beat 16 where 10 is too few)
         if (th == 256 && allow_wide_cluster && oe) {
-            const int need = ((nvec + 15) / 16 + th - 1) / th;
-            if (need <= 10) {
-                *out = {16, th, round_nv(need), oe};
-                return true;
+            for (int c = 10; c <= 16; c += 6) {
+                const int need = (per_cta_vectors(nvec, c) + th - 1) / th;
+                if (need <= 10) {
+                    *out = {c, th, round_nv(need), oe};
+                    return true;
+                }
             }
         }
     }
@@ -844,7 +885,7 @@ static FastKernel row_kernel_for(int threads, int nv) {
 }
 static FastKernel weighted_kernel(const FastShape& sh) { return row_kernel_for<true, false, false, true>(sh.threads, sh.nv); }
 static FastKernel fast_kernel(const FastShape& sh) {
-    if (sh.cluster == 16) return wide_cluster_kernel(sh.nv);
+    if (sh.cluster > 8) return wide_cluster_kernel(sh.nv);
     return sh.one_exp ? row_kernel_for<true>(sh.threads, sh.nv) : row_kernel_for<false>(sh.threads, sh.nv);
 }
 
@@ -1032,7 +1073,7 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
         if (fast_ok && a.T < (1ll << 31) && pick_shape(a.V >> 3, &sh, /*allow_wide_cluster=*/wtok == nullptr)) {
             FastKernel k = wtok ? weighted_kernel(sh) : fast_kernel(sh);
             int nc = k ? max_clusters(k, sh) : -1;
-            if (nc <= 0 && sh.cluster == 16 && pick_shape(a.V >> 3, &sh)) {
+            if (nc <= 0 && sh.cluster > 8 && !tuned && pick_shape(a.V >> 3, &sh)) {
                 // the device does not take a cluster of 16: the portable shape instead
                 k = fast_kernel(sh);
                 nc = k ? max_clusters(k, sh) : -1;
@@ -1046,7 +1087,7 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
             p.stride = a.stride;
             p.T = (int)a.T;
             p.nvec = a.V >> 3;
-            p.per_cta_vec = (p.nvec + sh.cluster - 1) / sh.cluster;
+            p.per_cta_vec = per_cta_vectors(p.nvec, sh.cluster);
             p.rec = rec;
             p.denom = denom;
             p.logp_out = a.logp_out;
@@ -1100,7 +1141,7 @@ extern "C" rlf_status rlf_tune_logits_kernel(int cluster_ctas, int threads_per_c
         rlf::g_tune_threads = 0;
         return RLF_OK;
     }
-    const bool c_ok = cluster_ctas == 1 || cluster_ctas == 2 || cluster_ctas == 4 || cluster_ctas == 8;
+    const bool c_ok = cluster_ctas >= 1 && cluster_ctas <= 16;
     const bool t_ok = threads_per_cta == 256 || threads_per_cta == 512 || threads_per_cta == 1024;
     if (!c_ok || !t_ok) return RLF_ERR_SHAPE;
     rlf::g_tune_cluster = cluster_ctas;
@@ -1471,7 +1512,7 @@ extern "C" rlf_status rlf_logp_entropy_fwd(const void* logits, rlf_dtype dt, int
         p.stride = row_stride;
         p.T = (int)T;
         p.nvec = V >> 3;
-        p.per_cta_vec = (p.nvec + sh.cluster - 1) / sh.cluster;
+        p.per_cta_vec = per_cta_vectors(p.nvec, sh.cluster);
         p.rec = rec;
         p.denom = one;
         p.logp_out = logp_out;
@@ -1622,7 +1663,7 @@ extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd_skip_masked(
     p.stride = row_stride;
     p.T = (int)T;
     p.nvec = V >> 3;
-    p.per_cta_vec = (p.nvec + sh.cluster - 1) / sh.cluster;
+    p.per_cta_vec = per_cta_vectors(p.nvec, sh.cluster);
     p.rec = rec_c;
     p.denom = dn;
     p.logp_out = logp_out;

@@ -125,7 +125,7 @@ def test_host_validation_rejects_bad_arguments_before_touching_a_device(lib):
     assert pc(2) == -2 and pc(-1) == -2 and pc(0) == 0 and pc(1) == 0
     t = lib.rlf_tune_logits_kernel
     t.argtypes = [ctypes.c_int] * 3
-    assert t(3, 512, 0) == -2 and t(4, 500, 0) == -2 and t(0, 0, -1) == 0
+    assert t(17, 256, 0) == -2 and t(-1, 256, 0) == -2 and t(4, 500, 0) == -2 and t(3, 512, 0) == 0 and t(0, 0, -1) == 0
 
 
 def test_product_package_does_not_import_the_oracle():

@@ -53,7 +53,8 @@ def test_degenerate_groups_get_exactly_zero_advantage(eps):
 
 
 @pytest.mark.parametrize("shape", [(1, 512, -1), (2, 512, -1), (4, 512, 0), (8, 512, 1), (4, 256, 1),
-                                   (2, 1024, 0), (0, 0, 0), (0, 0, 1)])
+                                   (2, 1024, 0), (0, 0, 0), (0, 0, 1), (3, 256, 1), (6, 512, 1), (7, 512, 0),
+                                   (10, 256, 1), (12, 256, 1), (13, 256, 1), (16, 256, 1)])
 def test_cfg1_shape_reduced_T_bf16(shape):
     """Qwen3 vocabulary (151936 = 18 x 8192 + 4480: ragged tail in every launch shape) at 16 x 24
     tokens; every launch shape of the fast kernel, both exponential variants."""
@@ -167,6 +168,59 @@ def test_extreme_logits_and_targets_at_the_ends():
         from util import ulp_error_bf16, loss_close
         assert gc.grad_ulps(gc.grad_to_f64(grad), r["grad"], ids.cpu().numpy(), r["coef"]).max() <= gc.GRAD_ULPS
         assert loss_close(loss[0].item(), r["loss"][0], 1e-6, 1e-4)
+
+
+@pytest.mark.parametrize("V,dtype", [(4096, torch.bfloat16), (151936, torch.bfloat16), (1001, torch.float32)])
+def test_target_gradient_keeps_its_digits_when_p_y_rounds_to_one(V, dtype):
+    """Rows whose target leads the other logits by 4 ... 72: 1 - p_y runs from 1e-1 down to 1e-27, far
+    below what p_y - 1 can hold in fp32 (and still inside the fp32 exponent range: past a lead of
+    about 85 the other columns' weights underflow in fp32 and the kernels return zero where the exact
+    value is some 1e-37 |c|).  The target column of grad_logits = c (p_y - 1) must still
+    agree with the fp64 oracle to the same number of ulps as every other column."""
+    b = gc.binding()
+    gaps = [4.0, 8.0, 12.0, 16.0, 20.0, 24.0, 32.0, 48.0, 60.0, 72.0]
+    T = len(gaps)
+    g = torch.Generator(device="cpu").manual_seed(77)
+    z = torch.randn((T, V), generator=g).to(dtype).to(DEV)
+    ids_list = [0, V - 1, 7, V // 2, 8, V - 9, 255, 256, 1, V // 3]
+    for t, gap in enumerate(gaps):
+        z[t, ids_list[t]] = float(z[t].float().max().item()) + gap
+    ids = torch.tensor(ids_list, dtype=torch.int32, device=DEV)
+    seq = torch.zeros(T, dtype=torch.int32, device=DEV)
+    adv = torch.tensor([-0.9], device=DEV)
+    mask = torch.ones(T, dtype=torch.uint8, device=DEV)
+    zn = gc.to_np(z)
+    new = orc.grpo_loss(zn, ids.cpu().numpy(), [0] * T, [-0.9], np.zeros(T), np.zeros(T), [1] * T, 0.2, 0.0,
+                        want_grad=False)["logp"]
+    old = torch.tensor(new + 0.03, dtype=torch.float32, device=DEV)
+    ref = torch.tensor(new - 0.02, dtype=torch.float32, device=DEV)
+    st = _status()
+    logp, loss, grad = b.rlf_grpo_logp_loss_fwd_bwd(z, ids, seq, adv, old, ref, mask, 0.2, 0.01, dev_status=st)
+    torch.cuda.synchronize()
+    assert st.item() == 0
+    r = orc.grpo_loss(zn, ids.cpu().numpy(), seq.cpu().numpy(), adv.cpu().numpy(), old.cpu().numpy(),
+                      ref.cpu().numpy(), mask.cpu().numpy(), 0.2, 0.01, want_coef=True)
+    assert np.all(r["coef"] != 0)
+    gq = gc.grad_to_f64(grad)
+    rows = np.arange(T)
+    # The oracle's own target column is c (p_y - 1) in fp64 and is zero or digit-free on most of these
+    # rows.  A softmax gradient row sums to zero, so minus the sum of the oracle's other columns (each
+    # c p_v, accurate to fp64 rounding at any magnitude) is the value the target column must have.
+    others = r["grad"].copy()
+    others[rows, ids_list] = 0.0
+    want_y = -others.sum(axis=1)
+    assert np.all(want_y != 0) and np.abs(want_y / r["coef"]).min() < 1e-20
+    assert np.all(np.abs(want_y - r["grad"][rows, ids_list]) <= 2.0 ** -35 * np.abs(r["coef"]))
+    want = r["grad"].copy()
+    want[rows, ids_list] = want_y
+    if dtype == torch.bfloat16:
+        from util import bf16_ulp
+        ulps = np.abs(gq - want) / bf16_ulp(want)
+        assert ulps.max() <= gc.GRAD_ULPS, ulps[rows, ids_list]
+    else:
+        rel = np.abs(gq[rows, ids_list] - want_y) / np.abs(want_y)
+        assert rel.max() <= 2e-5, rel
+    assert np.abs(logp.cpu().numpy() - r["logp"]).max() <= gc.LOGP_ATOL
 
 
 def test_bad_rows_are_neutralised_and_flagged():
