@@ -64,7 +64,8 @@ def take_shard(responses, cu_seqlens, per_token, per_response):
 
 
 def _all_reduce_sum(t, group):
-    if group is not None and dist.is_initialized() and dist.get_world_size(group) > 1:
+    # issued whenever a group is given, a group of one included: the call is the same for any size
+    if group is not None and dist.is_initialized():
         dist.all_reduce(t, op=dist.ReduceOp.SUM, group=group)
     return t
 
@@ -127,7 +128,7 @@ def sharded_grpo_step(ids, cu_seqlens, rewards, group_size, old_logp, ref_logp, 
 
     Give `logits` [T_local, V] for the logits path (returns grad_logits) or `hidden` [T_local, D] and
     `W` [V, D] for the fused LM-head path (returns grad_hidden and the all-reduced grad_W).
-    `group`: the process group of the ranks that share the batch (None or a group of one: no exchange).
+    `group`: the process group of the ranks that share the batch (None: no exchange, a single-rank step).
     When grad_W is accumulated over several micro-batches, pass reduce_grad_W=False on all but the
     last one (a reduced buffer must not be reduced again), and pass the whole batch's token count as
     `n_global` (int64[1], e.g. the n_global a counting pass over the whole shard returned): a

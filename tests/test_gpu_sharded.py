@@ -155,3 +155,22 @@ def test_live_response_count_and_sequence_mean_step_against_the_oracle():
         gc.near_clip_bound(r["logp"], batch.old_logp.cpu().numpy(), None, eps=0.3)
     ulps = gc.grad_ulps(gc.grad_to_f64(out["grad_logits"])[~guard], r["grad"][~guard], ora["ids"][~guard], r["coef"][~guard])
     assert ulps.max() <= gc.GRAD_ULPS
+
+
+def test_step_with_its_all_reduces_through_nccl_in_a_group_of_one():
+    """The three exchanges of sharded_grpo_step issued through torch.distributed's NCCL backend on CUDA
+    tensors (one rank: one GPU is all a test gets), in a child process so that the process group, its
+    environment and NCCL's state stay out of this one.  The child checks every output against the CPU
+    oracle, including a grad_W accumulated over two micro-batches and reduced once."""
+    import json
+    import os
+    import subprocess
+    import sys
+    child = os.path.join(os.path.dirname(os.path.abspath(__file__)), "nccl_single_rank_child.py")
+    env = dict(os.environ, NCCL_NVLS_ENABLE="0")
+    p = subprocess.run([sys.executable, child], capture_output=True, text=True, timeout=600, env=env)
+    assert p.returncode == 0, p.stdout[-2000:] + p.stderr[-4000:]
+    line = [l for l in p.stdout.splitlines() if l.startswith("{")][-1]
+    res = json.loads(line)
+    assert res["ok"] and res["backend"] == "nccl" and res["world_size"] == 1
+    assert len(res["all_reduce_calls"]) == 5
