@@ -134,6 +134,8 @@ rlf_status rlf_group_advantage(const float *rewards, const int32_t *group_id, in
 /*
  * Rule reward.  (Paper Eq. 1: R_rule = sum_i w_i r_i over the n rule dimensions, e.g. call-format
  * validity, task completion, efficiency.)  The result feeds rlf_group_advantage as `rewards`.
+ * Scores that a judge model (Eq. 2) or a verification tool (Eq. 3) produced elsewhere enter the same
+ * way, as further columns with weights of their own.
  *   scores [B, n] fp32 row-major;  weights [n] fp32;  reward_out [B] fp32 (fp64 accumulation)
  */
 rlf_status rlf_rule_reward(const float *scores, const float *weights, int32_t B, int32_t n,
