@@ -11,6 +11,7 @@ import socket
 import sys
 
 os.environ.setdefault("NCCL_NVLS_ENABLE", "0")
+os.environ.setdefault("NCCL_SOCKET_IFNAME", "lo")        # one rank on this host: the loopback interface will do
 HERE = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, HERE)
 sys.path.insert(0, os.path.dirname(HERE))
