@@ -169,6 +169,8 @@ def test_step_with_its_all_reduces_through_nccl_in_a_group_of_one():
     child = os.path.join(os.path.dirname(os.path.abspath(__file__)), "nccl_single_rank_child.py")
     env = dict(os.environ, NCCL_NVLS_ENABLE="0")
     p = subprocess.run([sys.executable, child], capture_output=True, text=True, timeout=600, env=env)
+    if p.returncode == 77:
+        pytest.skip("the NCCL process group could not be created here: " + p.stdout[-300:])
     assert p.returncode == 0, p.stdout[-2000:] + p.stderr[-4000:]
     line = [l for l in p.stdout.splitlines() if l.startswith("{")][-1]
     res = json.loads(line)
