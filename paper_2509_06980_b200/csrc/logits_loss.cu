@@ -864,14 +864,16 @@ static FastKernel row_kernel_for_nv(int nv) {
     }
     return nullptr;
 }
-// the training kernel for a cluster of 16 CTAs of 256 threads (rows of 8 x 256 x 10 + 1 .. 16 x 256 x 10 vectors)
+// the training kernels for clusters of 9 to 16 CTAs of 256 threads (rows beyond 8 x 256 x 10 vectors):
+// plain, skip-masked and weighted variants, one exponential per element
+template <bool SKIP = false, bool WT = false>
 static FastKernel wide_cluster_kernel(int nv) {
     switch (nv) {
-        case 6: return grpo_row_cluster_kernel<256, 6, true, false, false, false, 16>;
-        case 7: return grpo_row_cluster_kernel<256, 7, true, false, false, false, 16>;
-        case 8: return grpo_row_cluster_kernel<256, 8, true, false, false, false, 16>;
-        case 9: return grpo_row_cluster_kernel<256, 9, true, false, false, false, 16>;
-        case 10: return grpo_row_cluster_kernel<256, 10, true, false, false, false, 16>;
+        case 6: return grpo_row_cluster_kernel<256, 6, true, false, SKIP, WT, 16>;
+        case 7: return grpo_row_cluster_kernel<256, 7, true, false, SKIP, WT, 16>;
+        case 8: return grpo_row_cluster_kernel<256, 8, true, false, SKIP, WT, 16>;
+        case 9: return grpo_row_cluster_kernel<256, 9, true, false, SKIP, WT, 16>;
+        case 10: return grpo_row_cluster_kernel<256, 10, true, false, SKIP, WT, 16>;
     }
     return nullptr;
 }
@@ -883,9 +885,16 @@ static FastKernel row_kernel_for(int threads, int nv) {
     if (threads == 1024) return row_kernel_for_nv<1024, ONE_EXP, ENT, SKIP, WT>(nv);
     return nullptr;
 }
-static FastKernel weighted_kernel(const FastShape& sh) { return row_kernel_for<true, false, false, true>(sh.threads, sh.nv); }
+static FastKernel weighted_kernel(const FastShape& sh) {
+    if (sh.cluster > 8) return wide_cluster_kernel<false, true>(sh.nv);
+    return row_kernel_for<true, false, false, true>(sh.threads, sh.nv);
+}
+static FastKernel skip_kernel(const FastShape& sh) {
+    if (sh.cluster > 8) return wide_cluster_kernel<true, false>(sh.nv);
+    return row_kernel_for<true, false, true>(sh.threads, sh.nv);
+}
 static FastKernel fast_kernel(const FastShape& sh) {
-    if (sh.cluster > 8) return wide_cluster_kernel(sh.nv);
+    if (sh.cluster > 8) return wide_cluster_kernel<>(sh.nv);
     return sh.one_exp ? row_kernel_for<true>(sh.threads, sh.nv) : row_kernel_for<false>(sh.threads, sh.nv);
 }
 
@@ -1070,12 +1079,12 @@ static rlf_status launch_logits_loss(const LossArgs& a, bool fast_ok, void* work
 
         FastShape sh;
         const bool tuned = g_tune_cluster.load() > 0;
-        if (fast_ok && a.T < (1ll << 31) && pick_shape(a.V >> 3, &sh, /*allow_wide_cluster=*/wtok == nullptr)) {
+        if (fast_ok && a.T < (1ll << 31) && pick_shape(a.V >> 3, &sh, /*allow_wide_cluster=*/true)) {
             FastKernel k = wtok ? weighted_kernel(sh) : fast_kernel(sh);
             int nc = k ? max_clusters(k, sh) : -1;
             if (nc <= 0 && sh.cluster > 8 && !tuned && pick_shape(a.V >> 3, &sh)) {
                 // the device does not take a cluster of 16: the portable shape instead
-                k = fast_kernel(sh);
+                k = wtok ? weighted_kernel(sh) : fast_kernel(sh);
                 nc = k ? max_clusters(k, sh) : -1;
             }
             if (!k) return RLF_ERR_UNSUPPORTED;
@@ -1618,7 +1627,7 @@ extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd_skip_masked(
     const bool fast_ok = dt == RLF_BF16 && (V % 8 == 0) && (row_stride % 8 == 0) && aligned(logits, 16) &&
                          aligned(grad_logits, 16) && T < (1ll << 30);
     FastShape sh;
-    if (T == 0 || !fast_ok || !pick_shape(V >> 3, &sh)) {
+    if (T == 0 || !fast_ok || !pick_shape(V >> 3, &sh, /*allow_wide_cluster=*/true)) {
         // nothing to gain on the general path: process every row, then mark the dead rows' log-probs
         rlf_status st0 = rlf_grpo_logp_loss_fwd_bwd(logits, dt, T, V, row_stride, ids, seq_id, adv, B, old_logp, ref_logp,
                                                     mask, eps_clip, beta_kl, denom, logp_out, loss_out, grad_logits,
@@ -1652,10 +1661,13 @@ extern "C" rlf_status rlf_grpo_logp_loss_fwd_bwd_skip_masked(
     count_launch();
     if (cudaGetLastError() != cudaSuccess) return RLF_ERR_CUDA;
 
-    FastKernel k = row_kernel_for<true, false, true>(sh.threads, sh.nv);
-    if (!k) return RLF_ERR_UNSUPPORTED;
-    int nc = max_clusters(k, sh);
-    if (nc <= 0) return RLF_ERR_UNSUPPORTED;
+    FastKernel k = skip_kernel(sh);
+    int nc = k ? max_clusters(k, sh) : -1;
+    if (nc <= 0 && sh.cluster > 8 && g_tune_cluster.load() == 0 && pick_shape(V >> 3, &sh)) {
+        k = skip_kernel(sh);             // the device does not take the wide cluster: the portable shape
+        nc = k ? max_clusters(k, sh) : -1;
+    }
+    if (!k || nc <= 0) return RLF_ERR_UNSUPPORTED;
     nc = clusters_for(nc, T);            // T bounds the listed rows, whose number is only known on the device
     FastParams p;
     p.logits = static_cast<const __nv_bfloat16*>(logits);

@@ -158,7 +158,10 @@ def make_tokens(spec: Spec) -> Tokens:
         else:
             obs = [int(x) for x in rng.integers(spec.obs_lo, spec.obs_hi + 1, size=k)]
             while sum(obs) + 2 * k + (k + 1) > L:        # reduced-size cases: shrink to fit
-                obs = [max(1, x // 2) for x in obs]
+                if all(x == 1 for x in obs):             # even one-token spans do not fit: one span fewer
+                    obs, k = obs[:-1], k - 1
+                else:
+                    obs = [max(1, x // 2) for x in obs]
         starts = place_spans(rng, L, obs)
         for s, n in zip(starts, obs):
             a = int(cu[b]) + s

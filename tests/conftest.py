@@ -13,6 +13,12 @@ def pytest_configure(config):
 
 
 def pytest_collection_modifyitems(config, items):
+    # no single test of this suite needs more than two minutes: a test that runs for a quarter of an hour
+    # is stuck (an input generator that cannot satisfy its recipe, a child process), so it fails instead
+    if config.pluginmanager.hasplugin("timeout"):
+        for it in items:
+            if it.get_closest_marker("timeout") is None:
+                it.add_marker(pytest.mark.timeout(900))
     import torch
     if torch.cuda.is_available():
         return

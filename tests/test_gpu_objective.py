@@ -15,7 +15,8 @@ DEV = "cuda"
 
 @pytest.mark.parametrize("V,dtype,lo,hi,agg", [(151936, "bf16", 0.2, 0.28, 0), (151936, "bf16", 0.2, 0.28, 1),
                                                  (4096, "bf16", 0.05, 0.1, 1), (1024, "f32", 0.2, 0.3, 1),
-                                                 (1001, "bf16", 0.1, 0.1, 1)])
+                                                 (1001, "bf16", 0.1, 0.1, 1), (200000, "bf16", 0.2, 0.28, 1),
+                                                 (262144, "bf16", 0.2, 0.2, 1)])
 def test_objective_variants_match_oracle(V, dtype, lo, hi, agg):
     b = gc.binding()
     spec = synth.scaled(synth.SPECS[2], V=V, logits_dtype=dtype, num_prompts=2, group_size=4, len_lo=10, len_hi=60,

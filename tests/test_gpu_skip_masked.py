@@ -20,7 +20,8 @@ def _inputs(spec):
     return b, batch, mask, seq, n, adv
 
 
-@pytest.mark.parametrize("V,dtype,L", [(151936, "bf16", 40), (32768, "bf16", 300), (1001, "bf16", 30), (1024, "f32", 30)])
+@pytest.mark.parametrize("V,dtype,L", [(151936, "bf16", 40), (32768, "bf16", 300), (1001, "bf16", 30), (1024, "f32", 30),
+                                       (200000, "bf16", 24), (262144, "bf16", 24)])
 def test_skip_masked_equals_full_processing_on_live_rows(V, dtype, L):
     spec = synth.scaled(synth.SPECS[1], V=V, logits_dtype=dtype, len_lo=L, len_hi=L, spans_lo=1, spans_hi=3,
                         obs_lo=3, obs_hi=max(4, L // 6))
