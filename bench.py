@@ -44,7 +44,7 @@ WORKLOAD = "cfg1_qwen3_4b_microbatch: 16 responses x 2048 tokens, V=151936 bf16 
 #   streaming forward kernel: the T = 4096 capture, per token (traffic is proportional to rows);
 #   fused LM-head: every kernel of one forward / one forward + backward call at cfg 3 full size
 #   (one-pass capture of the whole call), per call.
-NCU_TRAFFIC = {"logits_loss_cu_sha1": "373f8ff1bad542ed4ac3604f9ea1c3888ac745a5", "dram_bytes_per_token": 606041.0}
+NCU_TRAFFIC = {"logits_loss_cu_sha1": "ee482c3f18de39e50fed56d917e964b8673b1d59", "dram_bytes_per_token": 606028.0}
 NCU_TRAFFIC_FUSED = {"lmhead_cu_sha1": "23538aaabeed8d9a0c763b7f7e3bb6ee625b306d",
                      "fwd_bytes_per_call": 3957591808.0, "fwd_bwd_bytes_per_call": 34875904256.0}
 

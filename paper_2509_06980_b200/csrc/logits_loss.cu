@@ -434,7 +434,10 @@ grpo_row_cluster_kernel(const FastParams p) {
             // before the registers are loaded, so it drops out of (max, sum) here and comes back in
             // once per row from z_target.  S' = S - 2^(z_y - M) is what the target column's gradient
             // needs, -c S' / S, and summing it directly avoids the cancellation of c (p_y - 1).
-            if (!ENT) sv[y & 7] = __ushort_as_bfloat16((unsigned short)0xff80u);
+            // (stored by an asm statement with a memory clobber: the loads below read the same bytes through
+            // another type, and nothing may move them above this store)
+            if (!ENT)
+                asm volatile("st.shared.b16 [%0], %1;" :: "r"(smem_u32(sv + (y & 7))), "h"((unsigned short)0xff80u) : "memory");
         }
         uint4 d[NV];
 #pragma unroll
