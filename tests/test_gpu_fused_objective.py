@@ -174,3 +174,25 @@ def test_two_accumulator_gradient_contractions_are_bit_identical_to_the_one_accu
         ref = outs[(0, chunk, accumulate)]
         for got, want in zip(o, ref):
             assert torch.equal(got, want), (acc2, chunk, accumulate)
+
+
+def test_fused_repeated_calls_reproduce_the_first_bit_for_bit():
+    """Twenty calls over the same inputs on the Qwen3-4B head shape (full V and D, 1536 tokens: several
+    token tiles, all 74 CTA pairs busy, workers paced by a device counter): log-probs, loss, grad_hidden
+    and, within one backward chunk, grad_W come out with the same bits every time."""
+    b = gc.binding()
+    spec = synth.scaled(synth.SPECS[3], len_lo=96, len_hi=96, spans_lo=1, spans_hi=2, obs_lo=4, obs_hi=12)
+    batch = synth.make_batch(spec, DEV)
+    mask, seq, n = b.rlf_build_loss_mask(batch.ids, batch.cu_seqlens, spec.open_id, spec.close_id)
+    adv = b.rlf_group_advantage(batch.rewards, group_size=batch.tokens.group_size)
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    first = None
+    for _ in range(20):
+        out = b.rlf_fused_lmhead_grpo(batch.hidden, batch.W, batch.ids, seq, adv, batch.old_logp, batch.ref_logp, mask,
+                                      synth.EPS_CLIP, synth.BETA_KL, denom=n, dev_status=st)
+        cur = [o.clone() for o in out]
+        if first is None:
+            first = cur
+        else:
+            assert all(torch.equal(x, y) for x, y in zip(cur, first))
+    assert st.item() == 0
