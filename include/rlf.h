@@ -179,6 +179,8 @@ rlf_status rlf_kl_in_reward(const float *rewards, const float *old_logp, const f
  *     grad_logits[t,v] = d loss_out[0] / d z[t,v] = c_t (softmax(z[t,:])[v] - 1[v = y]),
  *         c_t = -(mask[t]/Nd) (dpg/dlogp + beta (1 - exp d)),
  *         dpg/dlogp = 0 where the clipped branch is active (A>0, rho>1+eps or A<0, rho<1-eps), else -A rho.
+ *     The target column is formed as -c_t S'/S, S' the row's exponential sum over the other columns,
+ *     so it keeps its relative accuracy when softmax[y] rounds to one.
  * Each logits row is read from HBM once and grad written once; max / sum are
  * accumulated in fp32, the token-level loss terms are summed in fp64 in a fixed order
  * (results are run-to-run identical).
